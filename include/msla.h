@@ -1,0 +1,154 @@
+/*
+ * libmsla -- forward pass of the multi-scale ReLU linear attention module of
+ * EfficientViT (arXiv 2205.14756, Section 3.1) for NVIDIA B200 (sm_100a).
+ *
+ * Conventions shared by every entry point
+ *   - Plain C ABI.  Pointers named q, k, v, x, out, weights' members and
+ *     workspaces are DEVICE pointers; desc / weights structs are HOST memory and
+ *     are read only during the call.  `stream` is a cudaStream_t passed as
+ *     void* (NULL = the legacy default stream).
+ *   - Calls validate on the host, enqueue kernels on `stream` and return; they
+ *     never synchronise, print, throw or abort.  A non-zero status means no
+ *     kernel was launched by that call (except MSLA_ERR_CUDA raised by a launch
+ *     in the middle of a multi-kernel call).  msla_last_error() gives a
+ *     thread-local detail string for the most recent failure on this thread.
+ *   - All buffers are caller-owned.  The library keeps no pointer past the
+ *     completion of the work it enqueued.  Outputs must not overlap inputs or
+ *     the workspace (overlap is reported as MSLA_ERR_INVALID_ARG).
+ *   - Device pointers must be 16-byte aligned (MSLA_ERR_ALIGNMENT otherwise).
+ *   - Accumulation is always fp32; bf16 conversions round to nearest even.
+ *   - Results are bitwise reproducible for a given shape and dtype: no
+ *     floating-point atomics, and the split of the token reduction depends on
+ *     the shape only.
+ *   - There is no CPU fallback: on a device that is not compute capability
+ *     10.x every compute call returns MSLA_ERR_ARCH.
+ */
+#ifndef MSLA_H_
+#define MSLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MSLA_OK = 0,
+  MSLA_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, inconsistent descriptor, overlap */
+  MSLA_ERR_UNSUPPORTED = 2, /* a shape or option this build has no kernel for */
+  MSLA_ERR_ALIGNMENT = 3,   /* a device pointer is not 16-byte aligned */
+  MSLA_ERR_WORKSPACE = 4,   /* workspace missing or smaller than the *_workspace_bytes() answer */
+  MSLA_ERR_ARCH = 5,        /* current device is not sm_100 */
+  MSLA_ERR_CUDA = 6         /* a CUDA runtime call or launch failed; see msla_last_error() */
+} msla_status_t;
+
+typedef enum { MSLA_F32 = 0, MSLA_BF16 = 1 } msla_dtype_t;
+
+/* ------------------------------------------------------------------------- *
+ * Attention core: ReLU linear attention, Eq. 3 of the paper (the linear-time
+ * re-association of Eq. 1 under the similarity of Eq. 2), per (batch, head):
+ *
+ *   KV[a,c] = sum_j relu(k[j,a]) * v[j,c]        ks[a] = sum_j relu(k[j,a])
+ *   out[i,c] = sum_a relu(q[i,a]) * KV[a,c] / (sum_a relu(q[i,a]) * ks[a] + eps)
+ *
+ * q, k, v, out: device, dense [B, heads, N, d] with d innermost; bf16 for
+ * msla_linattn_relu, fp32 for msla_linattn_relu_f32.  d must be 16 or 32
+ * (MSLA_ERR_UNSUPPORTED otherwise); B, heads, N >= 1.  eps is added once to the
+ * denominator, so a query row with no positive entry gives an all-zero output
+ * row rather than 0/0.  There is no 1/sqrt(d) scaling (that belongs to the
+ * softmax similarity only).
+ *
+ * The reduction over tokens is split into chunks whose fp32 partial states
+ * live in scratch memory.  These two calls take that scratch from the stream's
+ * memory pool (cudaMallocAsync / cudaFreeAsync on `stream`); use
+ * msla_linattn_relu_ws to supply it yourself.
+ * ------------------------------------------------------------------------- */
+msla_status_t msla_linattn_relu(const void* q, const void* k, const void* v, void* out,
+                                int B, int heads, int N, int d, float eps, void* stream);
+msla_status_t msla_linattn_relu_f32(const float* q, const float* k, const float* v, float* out,
+                                    int B, int heads, int N, int d, float eps, void* stream);
+
+/* Scratch bytes the core needs for this shape (0 if the shape is invalid). */
+size_t msla_linattn_relu_workspace_bytes(int B, int heads, int N, int d);
+
+/* Same operation (Eq. 3) with caller-owned scratch: `workspace` is device
+ * memory of at least msla_linattn_relu_workspace_bytes() bytes, 16-byte
+ * aligned, contents irrelevant on entry and undefined on exit.  Two calls that
+ * may run concurrently must not share a workspace. */
+msla_status_t msla_linattn_relu_ws(msla_dtype_t dtype, const void* q, const void* k, const void* v,
+                                   void* out, int B, int heads, int N, int d, float eps,
+                                   void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------- *
+ * Whole module (Section 3.1, Figure 2 right) on an NCHW feature map:
+ *
+ *   1. qkv = 1x1 conv (x, w_qkv)                    C  -> 3C'   (Q = xW_Q, K = xW_K, V = xW_V)
+ *   2. agg = grouped 1x1 (depthwise kxk (qkv))      3C' -> 3C'  multi-scale token aggregation:
+ *            one depthwise conv, stride 1, zero padding k/2, cross-correlation,
+ *            then one 1x1 group convolution with 3*heads groups of d channels
+ *   3. multi-scale tokens = {qkv, agg}: 2*heads heads; in each head the 3d
+ *      channels are [q | k | v]; token n = row*W + col
+ *   4. ReLU linear attention (Eq. 3) per (batch, head) over all N = H*W tokens
+ *   5. head outputs concatenated along channels (all heads of the original
+ *      scale first, then the aggregated scale), then
+ *      out = 1x1 conv (att, w_proj) (+ b_proj)      2C' -> C_out
+ *
+ * with C' = heads*d.  Section 4.1 fixes two branches and 5x5 aggregation;
+ * n_scales must be 2 and agg_kernel must be 5.  No bias, normalisation or
+ * activation sits between the stages; the residual connection around the
+ * module is the caller's.
+ * ------------------------------------------------------------------------- */
+typedef struct {
+  uint32_t struct_size;   /* sizeof(msla_desc), for versioning */
+  int B, C, H, W;         /* input x is [B, C, H, W] */
+  int heads, d;           /* heads per scale and channels per head; d in {16, 32} */
+  int n_scales;           /* 2 */
+  int agg_kernel;         /* 5 */
+  int C_out;              /* output channels */
+  msla_dtype_t dtype;     /* type of x, out and all weights */
+  float eps;              /* added to the attention denominator */
+  void* workspace;        /* device scratch, >= msla_forward_workspace_bytes(desc) */
+  size_t workspace_bytes;
+} msla_desc;
+
+typedef struct {
+  const void* w_qkv;  /* [3C', C]     row o = output channel (h*3 + t)*d + i, t: 0 q, 1 k, 2 v */
+  const void* w_dw;   /* [3C', k, k]  taps [dy][dx]; tap reads pixel (row+dy-k/2, col+dx-k/2) */
+  const void* w_pw;   /* [3C', d]     out channel o reads in channels (o/d)*d .. (o/d)*d + d-1 */
+  const void* w_proj; /* [C_out, 2C'] column j = att channel head*d + c */
+  const void* b_proj; /* [C_out] or NULL */
+} msla_weights;
+
+/* Scratch bytes msla_forward needs for this descriptor (workspace fields are
+ * ignored); 0 if the descriptor is invalid or unsupported. */
+size_t msla_forward_workspace_bytes(const msla_desc* desc);
+
+/* x: device [B, C, H, W]; out: device [B, C_out, H, W]; both of desc->dtype.
+ * C, 3C' and 2C' must be multiples of 8 so that every row of the internal
+ * token-major buffers starts on a 16-byte boundary. */
+msla_status_t msla_forward(const msla_desc* desc, const void* x, const msla_weights* weights,
+                           void* out, void* stream);
+
+/* Stage entry points (the module's steps 1, 2 and 5 on their own), exposed so
+ * that each kernel can be checked and timed in isolation.  Internal
+ * activations are token-major: act[b][n][channel].
+ *   msla_project_in : x [B, C, N] (NCHW) , w [Cout, C]        -> y [B, N, Cout]
+ *   msla_aggregate  : t [B, H*W, Ch], w_dw [Ch,5,5], w_pw [Ch,d] -> y [B, H*W, Ch]
+ *   msla_project_out: a [B, N, Cin], w [Cout, Cin], bias|NULL  -> y [B, Cout, N] (NCHW)
+ */
+msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y,
+                              int B, int C, int Cout, int N, void* stream);
+msla_status_t msla_aggregate(msla_dtype_t dtype, const void* t, const void* w_dw, const void* w_pw,
+                             void* y, int B, int H, int W, int Ch, int d, void* stream);
+msla_status_t msla_project_out(msla_dtype_t dtype, const void* a, const void* w, const void* bias,
+                               void* y, int B, int Cin, int Cout, int N, void* stream);
+
+const char* msla_status_string(msla_status_t status);
+const char* msla_last_error(void); /* thread-local; empty string if none */
+int msla_version(void);            /* major*10000 + minor*100 + patch */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MSLA_H_ */

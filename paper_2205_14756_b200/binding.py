@@ -1,0 +1,159 @@
+"""ctypes binding of libmsla: argument marshalling only.
+
+Every function has the name and argument order of its C entry point in
+``include/msla.h``; tensors are torch CUDA tensors whose ``data_ptr()`` is
+passed through.  PyTorch supplies device memory and streams, nothing else.
+There is no fallback: if ``libmsla.so`` is missing the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libmsla.so")
+
+MSLA_F32, MSLA_BF16 = 0, 1
+_DTYPES = {torch.float32: MSLA_F32, torch.bfloat16: MSLA_BF16}
+
+c_int, c_float, c_size_t, c_void_p = ctypes.c_int, ctypes.c_float, ctypes.c_size_t, ctypes.c_void_p
+
+
+class MslaError(RuntimeError):
+    def __init__(self, status: int, name: str, detail: str):
+        super().__init__(f"libmsla status {status} ({name}): {detail}")
+        self.status = status
+
+
+class msla_desc(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("B", c_int), ("C", c_int), ("H", c_int), ("W", c_int),
+                ("heads", c_int), ("d", c_int), ("n_scales", c_int), ("agg_kernel", c_int),
+                ("C_out", c_int), ("dtype", c_int), ("eps", c_float), ("workspace", c_void_p),
+                ("workspace_bytes", c_size_t)]
+
+
+class msla_weights(ctypes.Structure):
+    _fields_ = [("w_qkv", c_void_p), ("w_dw", c_void_p), ("w_pw", c_void_p), ("w_proj", c_void_p),
+                ("b_proj", c_void_p)]
+
+
+EXPORTS = {
+    "msla_linattn_relu": (c_int, [c_void_p] * 4 + [c_int] * 4 + [c_float, c_void_p]),
+    "msla_linattn_relu_f32": (c_int, [c_void_p] * 4 + [c_int] * 4 + [c_float, c_void_p]),
+    "msla_linattn_relu_workspace_bytes": (c_size_t, [c_int] * 4),
+    "msla_linattn_relu_ws": (c_int, [c_int] + [c_void_p] * 4 + [c_int] * 4 + [c_float, c_void_p, c_size_t, c_void_p]),
+    "msla_forward_workspace_bytes": (c_size_t, [ctypes.POINTER(msla_desc)]),
+    "msla_forward": (c_int, [ctypes.POINTER(msla_desc), c_void_p, ctypes.POINTER(msla_weights), c_void_p, c_void_p]),
+    "msla_project_in": (c_int, [c_int] + [c_void_p] * 3 + [c_int] * 4 + [c_void_p]),
+    "msla_aggregate": (c_int, [c_int] + [c_void_p] * 4 + [c_int] * 5 + [c_void_p]),
+    "msla_project_out": (c_int, [c_int] + [c_void_p] * 4 + [c_int] * 4 + [c_void_p]),
+    "msla_status_string": (ctypes.c_char_p, [c_int]),
+    "msla_last_error": (ctypes.c_char_p, []),
+    "msla_version": (c_int, []),
+}
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2205_14756_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        handle = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in EXPORTS.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+def _check(status: int) -> None:
+    if status != 0:
+        handle = lib()
+        raise MslaError(status, handle.msla_status_string(status).decode(), handle.msla_last_error().decode())
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("libmsla takes contiguous CUDA tensors")
+    return t.data_ptr()
+
+
+def msla_version() -> int:
+    return lib().msla_version()
+
+
+def msla_linattn_relu_workspace_bytes(B: int, heads: int, N: int, d: int) -> int:
+    return lib().msla_linattn_relu_workspace_bytes(B, heads, N, d)
+
+
+def msla_linattn_relu(q, k, v, out, B, heads, N, d, eps=1e-15, stream=None) -> None:
+    """bf16 attention core on [B, heads, N, d] tensors (scratch from the stream's pool)."""
+    _check(lib().msla_linattn_relu(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, heads, N, d, eps, _stream(stream)))
+
+
+def msla_linattn_relu_f32(q, k, v, out, B, heads, N, d, eps=1e-15, stream=None) -> None:
+    _check(lib().msla_linattn_relu_f32(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, heads, N, d, eps, _stream(stream)))
+
+
+def msla_linattn_relu_ws(dtype, q, k, v, out, B, heads, N, d, eps, workspace, workspace_bytes, stream=None) -> None:
+    _check(lib().msla_linattn_relu_ws(dtype, _ptr(q), _ptr(k), _ptr(v), _ptr(out), B, heads, N, d, eps,
+                                      _ptr(workspace), workspace_bytes, _stream(stream)))
+
+
+def make_desc(B, C, H, W, heads, d, C_out, dtype, eps=1e-15, n_scales=2, agg_kernel=5,
+              workspace: Optional[torch.Tensor] = None) -> msla_desc:
+    desc = msla_desc()
+    desc.struct_size = ctypes.sizeof(msla_desc)
+    desc.B, desc.C, desc.H, desc.W = B, C, H, W
+    desc.heads, desc.d, desc.n_scales, desc.agg_kernel, desc.C_out = heads, d, n_scales, agg_kernel, C_out
+    desc.dtype = dtype
+    desc.eps = eps
+    desc.workspace = _ptr(workspace) if workspace is not None else None
+    desc.workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    return desc
+
+
+def msla_forward_workspace_bytes(desc: msla_desc) -> int:
+    return lib().msla_forward_workspace_bytes(ctypes.byref(desc))
+
+
+def msla_forward(desc: msla_desc, x, weights: msla_weights, out, stream=None) -> None:
+    _check(lib().msla_forward(ctypes.byref(desc), _ptr(x), ctypes.byref(weights), _ptr(out), _stream(stream)))
+
+
+def make_weights(w_qkv, w_dw, w_pw, w_proj, b_proj=None) -> msla_weights:
+    w = msla_weights()
+    w.w_qkv, w.w_dw, w.w_pw, w.w_proj, w.b_proj = _ptr(w_qkv), _ptr(w_dw), _ptr(w_pw), _ptr(w_proj), _ptr(b_proj)
+    return w
+
+
+def msla_project_in(dtype, x, w, y, B, C, Cout, N, stream=None) -> None:
+    _check(lib().msla_project_in(dtype, _ptr(x), _ptr(w), _ptr(y), B, C, Cout, N, _stream(stream)))
+
+
+def msla_aggregate(dtype, t, w_dw, w_pw, y, B, H, W, Ch, d, stream=None) -> None:
+    _check(lib().msla_aggregate(dtype, _ptr(t), _ptr(w_dw), _ptr(w_pw), _ptr(y), B, H, W, Ch, d, _stream(stream)))
+
+
+def msla_project_out(dtype, a, w, bias, y, B, Cin, Cout, N, stream=None) -> None:
+    _check(lib().msla_project_out(dtype, _ptr(a), _ptr(w), _ptr(bias), _ptr(y), B, Cin, Cout, N, _stream(stream)))
+
+
+def dtype_code(t: torch.dtype) -> int:
+    return _DTYPES[t]

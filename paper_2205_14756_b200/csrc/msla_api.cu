@@ -1,0 +1,349 @@
+// C ABI of libmsla: host-side validation, workspace carving and kernel dispatch.
+#include "../../include/msla.h"
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "generic_kernels.cuh"
+#include "msla_common.cuh"
+#include "msla_host.h"
+
+namespace msla {
+
+static thread_local char g_last_error[512] = "";
+
+msla_status_t fail(msla_status_t st, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_last_error, sizeof(g_last_error), fmt, ap);
+  va_end(ap);
+  return st;
+}
+
+msla_status_t check_launch(const char* what) {
+  const cudaError_t e = cudaPeekAtLastError();
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return fail(MSLA_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+  }
+  return MSLA_OK;
+}
+
+static msla_status_t check_arch() {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return fail(MSLA_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+  }
+  static int cached_major[64];  // 0 = unknown
+  int major = (dev >= 0 && dev < 64) ? cached_major[dev] : 0;
+  if (major == 0) {
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      return fail(MSLA_ERR_CUDA, "cudaDeviceGetAttribute: %s", cudaGetErrorString(e));
+    }
+    if (dev >= 0 && dev < 64) cached_major[dev] = major;
+  }
+  if (major != 10) return fail(MSLA_ERR_ARCH, "device %d has compute capability %d.x; sm_100 is required", dev, major);
+  return MSLA_OK;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+  return a0 < b0 + nb && b0 < a0 + na;
+}
+
+static size_t elem_size(msla_dtype_t t) { return t == MSLA_F32 ? 4 : 2; }
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ----------------------------------------------------------------- core plan
+// The split of the token reduction is a function of the shape only.
+CorePlan make_core_plan(long long BH, int N, int d) {
+  CorePlan p;
+  p.ne = d * (d + 1);
+  const long long s_max = ceil_div_ll(N, 256);
+  const long long s_want = ceil_div_ll(592, BH);
+  long long S = s_max < s_want ? s_max : s_want;
+  if (S > 64) S = 64;
+  if (S < 1) S = 1;
+  long long chunk = ceil_div_ll(N, S);
+  chunk = ceil_div_ll(chunk, 64) * 64;
+  p.chunk = (int)chunk;
+  p.S = (int)ceil_div_ll(N, chunk);
+  p.partial_off = 0;
+  p.state_off = align_up((size_t)BH * p.S * p.ne * sizeof(float), 256);
+  p.bytes = p.state_off + align_up((size_t)BH * p.ne * sizeof(float), 256);
+  return p;
+}
+
+static bool core_shape_ok(int B, int heads, int N, int d) {
+  return B >= 1 && heads >= 1 && N >= 1 && (d == 16 || d == 32) && (long long)B * heads <= 65535;
+}
+
+template <typename T>
+static msla_status_t run_core_generic(const T* q, const T* k, const T* v, T* out, HeadView in,
+                                      HeadView ov, int B, int heads, int N, int d, float eps,
+                                      const CorePlan& p, char* ws, cudaStream_t st) {
+  const long long BH = (long long)B * heads;
+  float* partial = reinterpret_cast<float*>(ws + p.partial_off);
+  float* state = reinterpret_cast<float*>(ws + p.state_off);
+  generic::kv_partial_kernel<T><<<dim3((unsigned)BH, p.S), 256, 0, st>>>(k, v, partial, in, heads, N, d, p.S, p.chunk);
+  const long long total = BH * p.ne;
+  generic::kv_combine_kernel<<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>(partial, state, p.S, p.ne, total);
+  generic::apply_kernel<T><<<dim3((unsigned)ceil_div_ll(N, 128), (unsigned)BH), 128, 0, st>>>(
+      q, state, out, in, ov, heads, N, d, eps);
+  return check_launch("attention core kernels");
+}
+
+// q/k/v views share strides; k = q + d and v = q + 2d in the module layout,
+// separate tensors in the dense layout, so three pointers are passed.
+static msla_status_t run_core(msla_dtype_t dtype, const void* q, const void* k, const void* v,
+                              void* out, HeadView in, HeadView ov, int B, int heads, int N, int d,
+                              float eps, const CorePlan& p, void* ws, cudaStream_t st) {
+  if (dtype == MSLA_F32)
+    return run_core_generic<float>((const float*)q, (const float*)k, (const float*)v, (float*)out,
+                                   in, ov, B, heads, N, d, eps, p, (char*)ws, st);
+  return run_core_generic<__nv_bfloat16>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
+                                         (const __nv_bfloat16*)v, (__nv_bfloat16*)out, in, ov, B,
+                                         heads, N, d, eps, p, (char*)ws, st);
+}
+
+static msla_status_t core_entry(msla_dtype_t dtype, const void* q, const void* k, const void* v,
+                                void* out, int B, int heads, int N, int d, float eps, void* ws,
+                                size_t ws_bytes, bool own_ws, cudaStream_t st) {
+  if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype %d", (int)dtype);
+  if (!q || !k || !v || !out) return fail(MSLA_ERR_INVALID_ARG, "null tensor pointer");
+  if (B < 1 || heads < 1 || N < 1 || d < 1) return fail(MSLA_ERR_INVALID_ARG, "B, heads, N, d must be positive (got %d, %d, %d, %d)", B, heads, N, d);
+  if (!(eps >= 0.f)) return fail(MSLA_ERR_INVALID_ARG, "eps must be >= 0");
+  if (d != 16 && d != 32) return fail(MSLA_ERR_UNSUPPORTED, "d = %d; only 16 and 32 are supported", d);
+  if ((long long)B * heads > 65535) return fail(MSLA_ERR_UNSUPPORTED, "B*heads = %lld exceeds 65535", (long long)B * heads);
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return fail(MSLA_ERR_ALIGNMENT, "q, k, v, out must be 16-byte aligned");
+  const size_t bytes = (size_t)B * heads * N * d * elem_size(dtype);
+  if (overlaps(out, bytes, q, bytes) || overlaps(out, bytes, k, bytes) || overlaps(out, bytes, v, bytes))
+    return fail(MSLA_ERR_INVALID_ARG, "out overlaps an input");
+  const CorePlan p = make_core_plan((long long)B * heads, N, d);
+  if (!own_ws) {
+    if (!ws || ws_bytes < p.bytes) return fail(MSLA_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", p.bytes, ws ? ws_bytes : (size_t)0);
+    if (!aligned16(ws)) return fail(MSLA_ERR_ALIGNMENT, "workspace must be 16-byte aligned");
+    if (overlaps(out, bytes, ws, p.bytes) || overlaps(q, bytes, ws, p.bytes) ||
+        overlaps(k, bytes, ws, p.bytes) || overlaps(v, bytes, ws, p.bytes))
+      return fail(MSLA_ERR_INVALID_ARG, "workspace overlaps a tensor");
+  }
+  msla_status_t s = check_arch();
+  if (s != MSLA_OK) return s;
+  if (own_ws) {
+    const cudaError_t e = cudaMallocAsync(&ws, p.bytes, st);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      return fail(MSLA_ERR_CUDA, "cudaMallocAsync(%zu): %s", p.bytes, cudaGetErrorString(e));
+    }
+  }
+  const HeadView in{(long long)heads * N * d, (long long)N * d, d};
+  s = run_core(dtype, q, k, v, out, in, in, B, heads, N, d, eps, p, ws, st);
+  if (own_ws) cudaFreeAsync(ws, st);
+  return s;
+}
+
+// ------------------------------------------------------------- module plan
+struct ForwardPlan {
+  size_t ms_off, att_off, core_off, bytes;
+  CorePlan core;
+  int Cp, N;
+};
+
+static msla_status_t validate_desc(const msla_desc* d, ForwardPlan* plan) {
+  if (!d) return fail(MSLA_ERR_INVALID_ARG, "null descriptor");
+  if (d->struct_size != sizeof(msla_desc)) return fail(MSLA_ERR_INVALID_ARG, "desc.struct_size = %u, expected %zu", d->struct_size, sizeof(msla_desc));
+  if (d->dtype != MSLA_F32 && d->dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype %d", (int)d->dtype);
+  if (d->B < 1 || d->C < 1 || d->H < 1 || d->W < 1 || d->heads < 1 || d->d < 1 || d->C_out < 1)
+    return fail(MSLA_ERR_INVALID_ARG, "B, C, H, W, heads, d, C_out must be positive");
+  if (!(d->eps >= 0.f)) return fail(MSLA_ERR_INVALID_ARG, "eps must be >= 0");
+  if (d->n_scales != 2) return fail(MSLA_ERR_UNSUPPORTED, "n_scales = %d; the module has two branches", d->n_scales);
+  if (d->agg_kernel != 5) return fail(MSLA_ERR_UNSUPPORTED, "agg_kernel = %d; only 5x5 aggregation is supported", d->agg_kernel);
+  if (d->d != 16 && d->d != 32) return fail(MSLA_ERR_UNSUPPORTED, "d = %d; only 16 and 32 are supported", d->d);
+  if ((long long)d->H * d->W > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "H*W exceeds 2^31-1");
+  if (d->C % 8 != 0 || d->C_out % 8 != 0) return fail(MSLA_ERR_UNSUPPORTED, "C and C_out must be multiples of 8");
+  if ((long long)d->B * 2 * d->heads > 65535 || d->B > 65535) return fail(MSLA_ERR_UNSUPPORTED, "B*2*heads exceeds 65535");
+  plan->Cp = d->heads * d->d;
+  plan->N = d->H * d->W;
+  const size_t e = elem_size(d->dtype);
+  const size_t tokens = (size_t)d->B * plan->N;
+  plan->core = make_core_plan((long long)d->B * 2 * d->heads, plan->N, d->d);
+  plan->ms_off = 0;
+  plan->att_off = align_up(tokens * 6 * plan->Cp * e, 256);
+  plan->core_off = plan->att_off + align_up(tokens * 2 * plan->Cp * e, 256);
+  plan->bytes = plan->core_off + plan->core.bytes;
+  return MSLA_OK;
+}
+
+template <typename T>
+static void launch_gemm(const T* A, const T* W, const T* bias, T* D, generic::GemmArgs g, int B, cudaStream_t st) {
+  dim3 grid((unsigned)ceil_div_ll(g.M, 64), (unsigned)ceil_div_ll(g.Nc, 64), (unsigned)B);
+  generic::gemm_kernel<T><<<grid, 256, 0, st>>>(A, W, bias, D, g);
+}
+
+static msla_status_t run_project_in(msla_dtype_t dt, const void* x, const void* w, void* y, int B,
+                                    int C, int Cout, int N, long long ldy, cudaStream_t st) {
+  generic::GemmArgs g{(long long)C * N, 1, N, (long long)N * ldy, ldy, 1, N, Cout, C};
+  if (dt == MSLA_F32) launch_gemm<float>((const float*)x, (const float*)w, nullptr, (float*)y, g, B, st);
+  else launch_gemm<__nv_bfloat16>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w, nullptr, (__nv_bfloat16*)y, g, B, st);
+  return check_launch("input projection");
+}
+
+static msla_status_t run_project_out(msla_dtype_t dt, const void* a, const void* w, const void* bias,
+                                     void* y, int B, int Cin, int Cout, int N, cudaStream_t st) {
+  generic::GemmArgs g{(long long)N * Cin, Cin, 1, (long long)Cout * N, 1, N, N, Cout, Cin};
+  if (dt == MSLA_F32) launch_gemm<float>((const float*)a, (const float*)w, (const float*)bias, (float*)y, g, B, st);
+  else launch_gemm<__nv_bfloat16>((const __nv_bfloat16*)a, (const __nv_bfloat16*)w, (const __nv_bfloat16*)bias, (__nv_bfloat16*)y, g, B, st);
+  return check_launch("output projection");
+}
+
+static msla_status_t run_aggregate(msla_dtype_t dt, const void* src, const void* w_dw, const void* w_pw,
+                                   void* dst, int B, int H, int W, int Ch, int d, long long src_ld,
+                                   long long dst_ld, cudaStream_t st) {
+  const long long N = (long long)H * W;
+  dim3 grid((unsigned)(ceil_div_ll(W, 8) * ceil_div_ll(H, 8)), (unsigned)(Ch / d), (unsigned)B);
+  if (dt == MSLA_F32)
+    generic::aggregate_kernel<float><<<grid, 256, 0, st>>>((const float*)src, (const float*)w_dw, (const float*)w_pw,
+                                                           (float*)dst, H, W, d, N * src_ld, src_ld, N * dst_ld, dst_ld);
+  else
+    generic::aggregate_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)src, (const __nv_bfloat16*)w_dw,
+                                                                   (const __nv_bfloat16*)w_pw, (__nv_bfloat16*)dst, H, W, d,
+                                                                   N * src_ld, src_ld, N * dst_ld, dst_ld);
+  return check_launch("token aggregation");
+}
+
+}  // namespace msla
+
+using namespace msla;
+
+extern "C" {
+
+msla_status_t msla_linattn_relu(const void* q, const void* k, const void* v, void* out, int B,
+                                int heads, int N, int d, float eps, void* stream) {
+  return core_entry(MSLA_BF16, q, k, v, out, B, heads, N, d, eps, nullptr, 0, true, (cudaStream_t)stream);
+}
+
+msla_status_t msla_linattn_relu_f32(const float* q, const float* k, const float* v, float* out,
+                                    int B, int heads, int N, int d, float eps, void* stream) {
+  return core_entry(MSLA_F32, q, k, v, out, B, heads, N, d, eps, nullptr, 0, true, (cudaStream_t)stream);
+}
+
+size_t msla_linattn_relu_workspace_bytes(int B, int heads, int N, int d) {
+  if (!core_shape_ok(B, heads, N, d)) return 0;
+  return make_core_plan((long long)B * heads, N, d).bytes;
+}
+
+msla_status_t msla_linattn_relu_ws(msla_dtype_t dtype, const void* q, const void* k, const void* v,
+                                   void* out, int B, int heads, int N, int d, float eps,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+  return core_entry(dtype, q, k, v, out, B, heads, N, d, eps, workspace, workspace_bytes, false, (cudaStream_t)stream);
+}
+
+size_t msla_forward_workspace_bytes(const msla_desc* desc) {
+  ForwardPlan p;
+  if (validate_desc(desc, &p) != MSLA_OK) return 0;
+  return p.bytes;
+}
+
+msla_status_t msla_forward(const msla_desc* desc, const void* x, const msla_weights* w, void* out, void* stream) {
+  ForwardPlan p;
+  msla_status_t s = validate_desc(desc, &p);
+  if (s != MSLA_OK) return s;
+  if (!x || !out || !w) return fail(MSLA_ERR_INVALID_ARG, "null x, out or weights");
+  if (!w->w_qkv || !w->w_dw || !w->w_pw || !w->w_proj) return fail(MSLA_ERR_INVALID_ARG, "null weight pointer");
+  const void* ptrs[] = {x, out, w->w_qkv, w->w_dw, w->w_pw, w->w_proj, w->b_proj, desc->workspace};
+  for (const void* ptr : ptrs)
+    if (ptr && !aligned16(ptr)) return fail(MSLA_ERR_ALIGNMENT, "all device pointers must be 16-byte aligned");
+  if (!desc->workspace || desc->workspace_bytes < p.bytes)
+    return fail(MSLA_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", p.bytes, desc->workspace ? desc->workspace_bytes : (size_t)0);
+  const size_t e = elem_size(desc->dtype);
+  const size_t xb = (size_t)desc->B * desc->C * p.N * e, ob = (size_t)desc->B * desc->C_out * p.N * e;
+  if (overlaps(out, ob, x, xb)) return fail(MSLA_ERR_INVALID_ARG, "out overlaps x");
+  if (overlaps(out, ob, desc->workspace, p.bytes) || overlaps(x, xb, desc->workspace, p.bytes))
+    return fail(MSLA_ERR_INVALID_ARG, "workspace overlaps x or out");
+  s = check_arch();
+  if (s != MSLA_OK) return s;
+
+  cudaStream_t st = (cudaStream_t)stream;
+  char* ws = (char*)desc->workspace;
+  const int Cp = p.Cp, N = p.N, d = desc->d, heads = desc->heads;
+  const long long ld_ms = 6LL * Cp, ld_att = 2LL * Cp;
+  char* ms = ws + p.ms_off;    // [B, N, 6C']: channels [0,3C') = qkv, [3C',6C') = aggregated
+  char* att = ws + p.att_off;  // [B, N, 2C']
+  // 1. QKV projection into the first half of every multi-scale row
+  s = run_project_in(desc->dtype, x, w->w_qkv, ms, desc->B, desc->C, 3 * Cp, N, ld_ms, st);
+  if (s != MSLA_OK) return s;
+  // 2. aggregation into the second half
+  s = run_aggregate(desc->dtype, ms, w->w_dw, w->w_pw, ms + 3 * Cp * e, desc->B, desc->H, desc->W, 3 * Cp, d, ld_ms, ld_ms, st);
+  if (s != MSLA_OK) return s;
+  // 3+4. attention over 2*heads heads of [q|k|v]; outputs land at channel head*d (concat)
+  const HeadView in{(long long)N * ld_ms, 3LL * d, ld_ms};
+  const HeadView ov{(long long)N * ld_att, d, ld_att};
+  s = run_core(desc->dtype, ms, ms + d * e, ms + 2 * d * e, att, in, ov, desc->B, 2 * heads, N, d, desc->eps, p.core, ws + p.core_off, st);
+  if (s != MSLA_OK) return s;
+  // 5. output projection back to NCHW
+  return run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out, desc->B, 2 * Cp, desc->C_out, N, st);
+}
+
+msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y, int B, int C, int Cout, int N, void* stream) {
+  if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");
+  if (!x || !w || !y) return fail(MSLA_ERR_INVALID_ARG, "null pointer");
+  if (B < 1 || C < 1 || Cout < 1 || N < 1 || B > 65535) return fail(MSLA_ERR_INVALID_ARG, "sizes must be positive (B <= 65535)");
+  if (C % 8 || Cout % 8) return fail(MSLA_ERR_UNSUPPORTED, "C and Cout must be multiples of 8");
+  if (!aligned16(x) || !aligned16(w) || !aligned16(y)) return fail(MSLA_ERR_ALIGNMENT, "pointers must be 16-byte aligned");
+  msla_status_t s = check_arch();
+  if (s != MSLA_OK) return s;
+  return run_project_in(dtype, x, w, y, B, C, Cout, N, Cout, (cudaStream_t)stream);
+}
+
+msla_status_t msla_aggregate(msla_dtype_t dtype, const void* t, const void* w_dw, const void* w_pw, void* y, int B, int H, int W, int Ch, int d, void* stream) {
+  if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");
+  if (!t || !w_dw || !w_pw || !y) return fail(MSLA_ERR_INVALID_ARG, "null pointer");
+  if (B < 1 || H < 1 || W < 1 || Ch < 1 || d < 1 || B > 65535) return fail(MSLA_ERR_INVALID_ARG, "sizes must be positive (B <= 65535)");
+  if ((long long)H * W > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "H*W exceeds 2^31-1");
+  if (d != 16 && d != 32) return fail(MSLA_ERR_UNSUPPORTED, "d = %d; only 16 and 32 are supported", d);
+  if (Ch % d) return fail(MSLA_ERR_INVALID_ARG, "Ch must be a multiple of d");
+  if (Ch / d > 65535) return fail(MSLA_ERR_UNSUPPORTED, "more than 65535 groups");
+  if (!aligned16(t) || !aligned16(w_dw) || !aligned16(w_pw) || !aligned16(y)) return fail(MSLA_ERR_ALIGNMENT, "pointers must be 16-byte aligned");
+  const size_t bytes = (size_t)B * H * W * Ch * elem_size(dtype);
+  if (overlaps(t, bytes, y, bytes)) return fail(MSLA_ERR_INVALID_ARG, "y overlaps t");
+  msla_status_t s = check_arch();
+  if (s != MSLA_OK) return s;
+  return run_aggregate(dtype, t, w_dw, w_pw, y, B, H, W, Ch, d, Ch, Ch, (cudaStream_t)stream);
+}
+
+msla_status_t msla_project_out(msla_dtype_t dtype, const void* a, const void* w, const void* bias, void* y, int B, int Cin, int Cout, int N, void* stream) {
+  if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");
+  if (!a || !w || !y) return fail(MSLA_ERR_INVALID_ARG, "null pointer");
+  if (B < 1 || Cin < 1 || Cout < 1 || N < 1 || B > 65535) return fail(MSLA_ERR_INVALID_ARG, "sizes must be positive (B <= 65535)");
+  if (Cin % 8 || Cout % 8) return fail(MSLA_ERR_UNSUPPORTED, "Cin and Cout must be multiples of 8");
+  if (!aligned16(a) || !aligned16(w) || !aligned16(y) || (bias && !aligned16(bias))) return fail(MSLA_ERR_ALIGNMENT, "pointers must be 16-byte aligned");
+  msla_status_t s = check_arch();
+  if (s != MSLA_OK) return s;
+  return run_project_out(dtype, a, w, bias, y, B, Cin, Cout, N, (cudaStream_t)stream);
+}
+
+const char* msla_status_string(msla_status_t s) {
+  switch (s) {
+    case MSLA_OK: return "ok";
+    case MSLA_ERR_INVALID_ARG: return "invalid argument";
+    case MSLA_ERR_UNSUPPORTED: return "unsupported shape or option";
+    case MSLA_ERR_ALIGNMENT: return "misaligned pointer";
+    case MSLA_ERR_WORKSPACE: return "workspace missing or too small";
+    case MSLA_ERR_ARCH: return "device is not sm_100";
+    case MSLA_ERR_CUDA: return "CUDA error";
+  }
+  return "unknown status";
+}
+
+const char* msla_last_error(void) { return g_last_error; }
+
+int msla_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,34 @@
+// Shared device/host helpers for libmsla kernels (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace msla {
+
+// Strided view of per-head token matrices: element (b, h, n, i) of tensor t is
+//   t[b * batch + h * head + n * ld + i].
+// Dense [B, heads, N, d] input:        batch = heads*N*d, head = N*d, ld = d.
+// Token-major multi-scale buffer
+// [B, N, 6C'] with [q|k|v] per head:   batch = N*6C',  head = 3d,  ld = 6C'.
+struct HeadView {
+  long long batch;
+  long long head;
+  long long ld;
+};
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) {
+  return __float2bfloat16_rn(v);
+}
+
+__host__ __device__ __forceinline__ long long ceil_div_ll(long long a, long long b) {
+  return (a + b - 1) / b;
+}
+
+}  // namespace msla

@@ -1,0 +1,27 @@
+// Host-side declarations shared by the translation units of libmsla.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+
+#include "../../include/msla.h"
+
+namespace msla {
+
+// Carving of the attention core's scratch: fp32 partial states
+// [BH][S][d*(d+1)] at partial_off, combined states [BH][d*(d+1)] at state_off.
+struct CorePlan {
+  int S;       // number of token chunks per (batch, head)
+  int chunk;   // tokens per chunk (multiple of 64)
+  int ne;      // d*(d+1) state entries
+  size_t partial_off, state_off, bytes;
+};
+
+CorePlan make_core_plan(long long BH, int N, int d);
+
+// Records a thread-local message and returns `st`.
+msla_status_t fail(msla_status_t st, const char* fmt, ...);
+// MSLA_OK, or MSLA_ERR_CUDA if a launch since the last check failed.
+msla_status_t check_launch(const char* what);
+
+}  // namespace msla

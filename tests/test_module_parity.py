@@ -1,0 +1,125 @@
+"""GPU module forward and its stages (through the C ABI) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import __graft_entry__  # noqa: F401
+import oracle
+import util
+from paper_2205_14756_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _ref(s, t, bias=None):
+    return oracle.msla_forward(t["x"], t["w_qkv"], t["w_dw"], t["w_pw"], t["w_proj"], bias,
+                               heads=s.heads, d=s.d, eps=s.eps)
+
+
+def test_config1_fp32():
+    s = inputs.CONFIG1
+    t = inputs.module_inputs(s)
+    util.assert_close(util.run_module(s, t), _ref(s, t), "f32", "config 1")
+
+
+SMALL = [
+    # name, dtype, B, C, H, W, heads, d: ragged tiles, images narrower than a tile, H=1
+    ("r1", "f32", 2, 32, 5, 7, 2, 16),
+    ("r2", "bf16", 1, 64, 9, 33, 2, 32),
+    ("r3", "bf16", 2, 32, 1, 40, 1, 32),
+    ("r4", "f32", 1, 64, 3, 3, 2, 32),
+    ("r5", "bf16", 1, 96, 24, 20, 3, 32),
+    ("r6", "bf16", 3, 64, 17, 16, 4, 16),
+    ("r7", "f32", 1, 16, 1, 1, 1, 16),
+]
+
+
+@pytest.mark.parametrize("name,dtype,B,C,H,W,heads,d", SMALL)
+def test_small_modules(name, dtype, B, C, H, W, heads, d):
+    s = inputs.ModuleShape(name, dtype, B, C, H, W, heads, d, seed=40 + H)
+    t = inputs.module_inputs(s)
+    util.assert_close(util.run_module(s, t), _ref(s, t), dtype, name)
+
+
+def test_module_with_bias_and_different_c_out():
+    s = inputs.ModuleShape("bias", "bf16", 1, 64, 8, 8, 2, 32, seed=77)
+    t = inputs.module_inputs(s)
+    t["w_proj"] = inputs.quantise(inputs.normal(77, 9, 40 * 128, 128 ** -0.5).reshape(40, 128), "bf16")
+    bias = inputs.quantise(inputs.normal(77, 10, 40), "bf16")
+    dt = s.dtype
+    x, w_qkv, w_dw, w_pw, w_proj, b = (util.dev(a, dt) for a in (t["x"], t["w_qkv"], t["w_dw"], t["w_pw"], t["w_proj"], bias))
+    desc = binding.make_desc(1, 64, 8, 8, 2, 32, 40, binding.MSLA_BF16)
+    ws = torch.empty(binding.msla_forward_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+    desc = binding.make_desc(1, 64, 8, 8, 2, 32, 40, binding.MSLA_BF16, workspace=ws)
+    out = torch.empty(1, 40, 8, 8, dtype=torch.bfloat16, device="cuda")
+    binding.msla_forward(desc, x, binding.make_weights(w_qkv, w_dw, w_pw, w_proj, b), out)
+    torch.cuda.synchronize()
+    util.assert_close(util.host(out), _ref(s, t, bias), "bf16", "bias + C_out=40")
+
+
+def test_config3_bf16():
+    s = inputs.CONFIG3
+    t = inputs.module_inputs(s)
+    util.assert_close(util.run_module(s, t), _ref(s, t), "bf16", "config 3")
+
+
+def test_config4_bf16():
+    s = inputs.CONFIG4
+    t = inputs.module_inputs(s)
+    util.assert_close(util.run_module(s, t), _ref(s, t), "bf16", "config 4")
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 3])
+def test_config5_sweep_bf16(idx):
+    s = inputs.CONFIG5[idx]
+    t = inputs.module_inputs(s)
+    util.assert_close(util.run_module(s, t), _ref(s, t), "bf16", s.name)
+
+
+def test_module_is_bitwise_reproducible():
+    s = inputs.ModuleShape("det", "bf16", 2, 64, 20, 24, 2, 32, seed=8)
+    t = inputs.module_inputs(s)
+    a = util.run_module(s, t)
+    assert np.array_equal(a, util.run_module(s, t))
+
+
+# ------------------------------------------------------------------ stages
+def _tok_major(a):      # [B, C, H, W] -> [B, H*W, C]
+    B, C = a.shape[:2]
+    return np.ascontiguousarray(a.reshape(B, C, -1).transpose(0, 2, 1))
+
+
+@pytest.mark.parametrize("dtype,B,C,Cout,N", [("f32", 2, 24, 40, 100), ("bf16", 1, 64, 192, 333), ("bf16", 2, 256, 768, 4096)])
+def test_stage_project_in(dtype, B, C, Cout, N):
+    x = inputs.quantise(inputs.normal(1, 0, B * C * N).reshape(B, C, N), dtype)
+    w = inputs.quantise(inputs.normal(1, 1, Cout * C, C ** -0.5).reshape(Cout, C), dtype)
+    y = torch.empty(B, N, Cout, dtype=util.TORCH_DTYPE[dtype], device="cuda")
+    binding.msla_project_in(util.CODE[dtype], util.dev(x, dtype), util.dev(w, dtype), y, B, C, Cout, N)
+    torch.cuda.synchronize()
+    ref = _tok_major(oracle.conv1x1(x[..., None], w))
+    util.assert_close(util.host(y), ref, dtype, "project_in")
+
+
+@pytest.mark.parametrize("dtype,B,Cin,Cout,N", [("f32", 2, 24, 40, 100), ("bf16", 1, 128, 64, 333), ("bf16", 2, 512, 256, 4096)])
+def test_stage_project_out(dtype, B, Cin, Cout, N):
+    a = inputs.quantise(inputs.normal(2, 0, B * N * Cin).reshape(B, N, Cin), dtype)
+    w = inputs.quantise(inputs.normal(2, 1, Cout * Cin, Cin ** -0.5).reshape(Cout, Cin), dtype)
+    bias = inputs.quantise(inputs.normal(2, 2, Cout), dtype)
+    y = torch.empty(B, Cout, N, dtype=util.TORCH_DTYPE[dtype], device="cuda")
+    binding.msla_project_out(util.CODE[dtype], util.dev(a, dtype), util.dev(w, dtype), util.dev(bias, dtype), y, B, Cin, Cout, N)
+    torch.cuda.synchronize()
+    ref = oracle.conv1x1(np.ascontiguousarray(a.transpose(0, 2, 1)), w, bias)
+    util.assert_close(util.host(y), ref, dtype, "project_out")
+
+
+@pytest.mark.parametrize("dtype,B,H,W,Ch,d", [("f32", 1, 6, 9, 48, 16), ("bf16", 2, 13, 21, 96, 32), ("bf16", 1, 1, 5, 32, 32),
+                                              ("bf16", 1, 64, 64, 192, 32), ("bf16", 1, 3, 70, 64, 16)])
+def test_stage_aggregate(dtype, B, H, W, Ch, d):
+    t = inputs.quantise(inputs.normal(3, 0, B * Ch * H * W).reshape(B, Ch, H, W), dtype)
+    w_dw = inputs.quantise(inputs.normal(3, 1, Ch * 25, 0.2).reshape(Ch, 5, 5), dtype)
+    w_pw = inputs.quantise(inputs.normal(3, 2, Ch * d, d ** -0.5).reshape(Ch, d), dtype)
+    y = torch.empty(B, H * W, Ch, dtype=util.TORCH_DTYPE[dtype], device="cuda")
+    binding.msla_aggregate(util.CODE[dtype], util.dev(_tok_major(t), dtype), util.dev(w_dw, dtype), util.dev(w_pw, dtype), y, B, H, W, Ch, d)
+    torch.cuda.synchronize()
+    ref = _tok_major(oracle.group1x1(oracle.dwconv(t, w_dw), w_pw))
+    util.assert_close(util.host(y), ref, dtype, "aggregate")
