@@ -130,6 +130,31 @@ size_t msla_forward_workspace_bytes(const msla_desc* desc);
 msla_status_t msla_forward(const msla_desc* desc, const void* x, const msla_weights* weights,
                            void* out, void* stream);
 
+/* msla_forward with CUDA events recorded between the module's five steps, so
+ * that each step can be timed inside a real forward pass.  `events` is a host
+ * array of n_events = 6 cudaEvent_t handles (as void*): events[0] is recorded
+ * on `stream` before step 1 and events[i] after step i (1 projection, 2
+ * aggregation, 3 KV-state reduction, 4 apply, 5 output projection; Section
+ * 3.1).  Everything else is as for msla_forward. */
+msla_status_t msla_forward_profiled(const msla_desc* desc, const void* x, const msla_weights* weights,
+                                    void* out, void* stream, void* const* events, int n_events);
+
+/* msla_forward for callers whose activations live in HOST memory (the paper's
+ * latency protocol, Section 4.1, includes the data transfer).  x_host and
+ * out_host are host pointers (pinned memory if the copies are to be
+ * asynchronous); weights stay device pointers.  The call enqueues a
+ * host-to-device copy of x, the five steps and a device-to-host copy of the
+ * result on `stream`.  desc->workspace must hold
+ * msla_forward_host_workspace_bytes(desc) bytes: the forward scratch plus
+ * device staging for x and out. */
+size_t msla_forward_host_workspace_bytes(const msla_desc* desc);
+msla_status_t msla_forward_host(const msla_desc* desc, const void* x_host, const msla_weights* weights,
+                                void* out_host, void* stream);
+
+/* Number of kernels this library has launched from the calling thread since it
+ * was loaded (a bookkeeping counter for benchmarks; no paper counterpart). */
+unsigned long long msla_kernel_launches(void);
+
 /* Stage entry points (the module's steps 1, 2 and 5 on their own), exposed so
  * that each kernel can be checked and timed in isolation.  Internal
  * activations are token-major: act[b][n][channel].

@@ -47,6 +47,11 @@ EXPORTS = {
     "msla_linattn_relu_ws": (c_int, [c_int] + [c_void_p] * 4 + [c_int] * 4 + [c_float, c_void_p, c_size_t, c_void_p]),
     "msla_forward_workspace_bytes": (c_size_t, [ctypes.POINTER(msla_desc)]),
     "msla_forward": (c_int, [ctypes.POINTER(msla_desc), c_void_p, ctypes.POINTER(msla_weights), c_void_p, c_void_p]),
+    "msla_forward_profiled": (c_int, [ctypes.POINTER(msla_desc), c_void_p, ctypes.POINTER(msla_weights), c_void_p, c_void_p,
+                                      ctypes.POINTER(c_void_p), c_int]),
+    "msla_forward_host_workspace_bytes": (c_size_t, [ctypes.POINTER(msla_desc)]),
+    "msla_forward_host": (c_int, [ctypes.POINTER(msla_desc), c_void_p, ctypes.POINTER(msla_weights), c_void_p, c_void_p]),
+    "msla_kernel_launches": (ctypes.c_ulonglong, []),
     "msla_project_in": (c_int, [c_int] + [c_void_p] * 3 + [c_int] * 4 + [c_void_p]),
     "msla_aggregate": (c_int, [c_int] + [c_void_p] * 4 + [c_int] * 5 + [c_void_p]),
     "msla_project_out": (c_int, [c_int] + [c_void_p] * 4 + [c_int] * 4 + [c_void_p]),
@@ -135,6 +140,30 @@ def msla_forward_workspace_bytes(desc: msla_desc) -> int:
 
 def msla_forward(desc: msla_desc, x, weights: msla_weights, out, stream=None) -> None:
     _check(lib().msla_forward(ctypes.byref(desc), _ptr(x), ctypes.byref(weights), _ptr(out), _stream(stream)))
+
+
+def msla_forward_profiled(desc: msla_desc, x, weights: msla_weights, out, stream, events) -> None:
+    """`events`: six torch.cuda.Event(enable_timing=True) objects (created, i.e. recorded once)."""
+    handles = (c_void_p * 6)(*[e.cuda_event for e in events])
+    _check(lib().msla_forward_profiled(ctypes.byref(desc), _ptr(x), ctypes.byref(weights), _ptr(out), _stream(stream),
+                                       handles, 6))
+
+
+def msla_forward_host_workspace_bytes(desc: msla_desc) -> int:
+    return lib().msla_forward_host_workspace_bytes(ctypes.byref(desc))
+
+
+def msla_forward_host(desc: msla_desc, x_host, weights: msla_weights, out_host, stream=None) -> None:
+    """x_host / out_host: contiguous CPU tensors (pinned for asynchronous copies)."""
+    for t in (x_host, out_host):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("msla_forward_host takes contiguous host tensors")
+    _check(lib().msla_forward_host(ctypes.byref(desc), x_host.data_ptr(), ctypes.byref(weights), out_host.data_ptr(),
+                                   _stream(stream)))
+
+
+def msla_kernel_launches() -> int:
+    return lib().msla_kernel_launches()
 
 
 def make_weights(w_qkv, w_dw, w_pw, w_proj, b_proj=None) -> msla_weights:

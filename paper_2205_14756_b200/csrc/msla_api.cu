@@ -21,6 +21,9 @@ msla_status_t fail(msla_status_t st, const char* fmt, ...) {
   return st;
 }
 
+static thread_local unsigned long long g_launches = 0;
+void count_launches(int n) { g_launches += (unsigned long long)n; }
+
 msla_status_t check_launch(const char* what) {
   const cudaError_t e = cudaPeekAtLastError();
   if (e != cudaSuccess) {
@@ -88,15 +91,17 @@ static bool core_shape_ok(int B, int heads, int N, int d) {
 template <typename T>
 static msla_status_t run_core_generic(const T* q, const T* k, const T* v, T* out, HeadView in,
                                       HeadView ov, int B, int heads, int N, int d, float eps,
-                                      const CorePlan& p, char* ws, cudaStream_t st) {
+                                      const CorePlan& p, char* ws, cudaStream_t st, cudaEvent_t mid) {
   const long long BH = (long long)B * heads;
   float* partial = reinterpret_cast<float*>(ws + p.partial_off);
   float* state = reinterpret_cast<float*>(ws + p.state_off);
   generic::kv_partial_kernel<T><<<dim3((unsigned)BH, p.S), 256, 0, st>>>(k, v, partial, in, heads, N, d, p.S, p.chunk);
   const long long total = BH * p.ne;
   generic::kv_combine_kernel<<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>(partial, state, p.S, p.ne, total);
+  if (mid) cudaEventRecord(mid, st);
   generic::apply_kernel<T><<<dim3((unsigned)ceil_div_ll(N, 128), (unsigned)BH), 128, 0, st>>>(
       q, state, out, in, ov, heads, N, d, eps);
+  count_launches(3);
   return check_launch("attention core kernels");
 }
 
@@ -104,13 +109,14 @@ static msla_status_t run_core_generic(const T* q, const T* k, const T* v, T* out
 // separate tensors in the dense layout, so three pointers are passed.
 static msla_status_t run_core(msla_dtype_t dtype, const void* q, const void* k, const void* v,
                               void* out, HeadView in, HeadView ov, int B, int heads, int N, int d,
-                              float eps, const CorePlan& p, void* ws, cudaStream_t st) {
+                              float eps, const CorePlan& p, void* ws, cudaStream_t st,
+                              cudaEvent_t mid = nullptr) {
   if (dtype == MSLA_F32)
     return run_core_generic<float>((const float*)q, (const float*)k, (const float*)v, (float*)out,
-                                   in, ov, B, heads, N, d, eps, p, (char*)ws, st);
+                                   in, ov, B, heads, N, d, eps, p, (char*)ws, st, mid);
   return run_core_generic<__nv_bfloat16>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
                                          (const __nv_bfloat16*)v, (__nv_bfloat16*)out, in, ov, B,
-                                         heads, N, d, eps, p, (char*)ws, st);
+                                         heads, N, d, eps, p, (char*)ws, st, mid);
 }
 
 static msla_status_t core_entry(msla_dtype_t dtype, const void* q, const void* k, const void* v,
@@ -185,6 +191,7 @@ template <typename T>
 static void launch_gemm(const T* A, const T* W, const T* bias, T* D, generic::GemmArgs g, int B, cudaStream_t st) {
   dim3 grid((unsigned)ceil_div_ll(g.M, 64), (unsigned)ceil_div_ll(g.Nc, 64), (unsigned)B);
   generic::gemm_kernel<T><<<grid, 256, 0, st>>>(A, W, bias, D, g);
+  count_launches(1);
 }
 
 static msla_status_t run_project_in(msla_dtype_t dt, const void* x, const void* w, void* y, int B,
@@ -215,7 +222,86 @@ static msla_status_t run_aggregate(msla_dtype_t dt, const void* src, const void*
     generic::aggregate_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)src, (const __nv_bfloat16*)w_dw,
                                                                    (const __nv_bfloat16*)w_pw, (__nv_bfloat16*)dst, H, W, d,
                                                                    N * src_ld, src_ld, N * dst_ld, dst_ld);
+  count_launches(1);
   return check_launch("token aggregation");
+}
+
+static msla_status_t record(void* const* events, int i, cudaStream_t st) {
+  if (!events) return MSLA_OK;
+  const cudaError_t e = cudaEventRecord((cudaEvent_t)events[i], st);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return fail(MSLA_ERR_CUDA, "cudaEventRecord: %s", cudaGetErrorString(e));
+  }
+  return MSLA_OK;
+}
+
+// host_io: x and out are host pointers staged through the tail of the workspace.
+static msla_status_t forward_impl(const msla_desc* desc, const void* x, const msla_weights* w, void* out,
+                                  cudaStream_t st, void* const* events, bool host_io) {
+  ForwardPlan p;
+  msla_status_t s = validate_desc(desc, &p);
+  if (s != MSLA_OK) return s;
+  if (!x || !out || !w) return fail(MSLA_ERR_INVALID_ARG, "null x, out or weights");
+  if (!w->w_qkv || !w->w_dw || !w->w_pw || !w->w_proj) return fail(MSLA_ERR_INVALID_ARG, "null weight pointer");
+  const void* ptrs[] = {host_io ? nullptr : x, host_io ? nullptr : out, w->w_qkv, w->w_dw, w->w_pw, w->w_proj, w->b_proj, desc->workspace};
+  for (const void* ptr : ptrs)
+    if (ptr && !aligned16(ptr)) return fail(MSLA_ERR_ALIGNMENT, "all device pointers must be 16-byte aligned");
+  const size_t e = elem_size(desc->dtype);
+  const size_t xb = (size_t)desc->B * desc->C * p.N * e, ob = (size_t)desc->B * desc->C_out * p.N * e;
+  const size_t need = p.bytes + (host_io ? align_up(xb, 256) + align_up(ob, 256) : 0);
+  if (!desc->workspace || desc->workspace_bytes < need)
+    return fail(MSLA_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, desc->workspace ? desc->workspace_bytes : (size_t)0);
+  if (overlaps(out, ob, x, xb)) return fail(MSLA_ERR_INVALID_ARG, "out overlaps x");
+  if (!host_io && (overlaps(out, ob, desc->workspace, need) || overlaps(x, xb, desc->workspace, need)))
+    return fail(MSLA_ERR_INVALID_ARG, "workspace overlaps x or out");
+  s = check_arch();
+  if (s != MSLA_OK) return s;
+
+  char* ws = (char*)desc->workspace;
+  const void* x_dev = x;
+  void* out_dev = out;
+  if (host_io) {
+    x_dev = ws + p.bytes;
+    out_dev = ws + p.bytes + align_up(xb, 256);
+    const cudaError_t ce = cudaMemcpyAsync((void*)x_dev, x, xb, cudaMemcpyHostToDevice, st);
+    if (ce != cudaSuccess) {
+      cudaGetLastError();
+      return fail(MSLA_ERR_CUDA, "host-to-device copy of x: %s", cudaGetErrorString(ce));
+    }
+  }
+  const int Cp = p.Cp, N = p.N, d = desc->d, heads = desc->heads;
+  const long long ld_ms = 6LL * Cp, ld_att = 2LL * Cp;
+  char* ms = ws + p.ms_off;    // [B, N, 6C']: channels [0,3C') = qkv, [3C',6C') = aggregated
+  char* att = ws + p.att_off;  // [B, N, 2C']
+  if ((s = record(events, 0, st)) != MSLA_OK) return s;
+  // 1. QKV projection into the first half of every multi-scale row
+  s = run_project_in(desc->dtype, x_dev, w->w_qkv, ms, desc->B, desc->C, 3 * Cp, N, ld_ms, st);
+  if (s != MSLA_OK) return s;
+  if ((s = record(events, 1, st)) != MSLA_OK) return s;
+  // 2. aggregation into the second half
+  s = run_aggregate(desc->dtype, ms, w->w_dw, w->w_pw, ms + 3 * Cp * e, desc->B, desc->H, desc->W, 3 * Cp, d, ld_ms, ld_ms, st);
+  if (s != MSLA_OK) return s;
+  if ((s = record(events, 2, st)) != MSLA_OK) return s;
+  // 3+4. attention over 2*heads heads of [q|k|v]; outputs land at channel head*d (concat)
+  const HeadView in{(long long)N * ld_ms, 3LL * d, ld_ms};
+  const HeadView ov{(long long)N * ld_att, d, ld_att};
+  s = run_core(desc->dtype, ms, ms + d * e, ms + 2 * d * e, att, in, ov, desc->B, 2 * heads, N, d, desc->eps, p.core,
+               ws + p.core_off, st, events ? (cudaEvent_t)events[3] : nullptr);
+  if (s != MSLA_OK) return s;
+  if ((s = record(events, 4, st)) != MSLA_OK) return s;
+  // 5. output projection back to NCHW
+  s = run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st);
+  if (s != MSLA_OK) return s;
+  if ((s = record(events, 5, st)) != MSLA_OK) return s;
+  if (host_io) {
+    const cudaError_t ce = cudaMemcpyAsync(out, out_dev, ob, cudaMemcpyDeviceToHost, st);
+    if (ce != cudaSuccess) {
+      cudaGetLastError();
+      return fail(MSLA_ERR_CUDA, "device-to-host copy of out: %s", cudaGetErrorString(ce));
+    }
+  }
+  return MSLA_OK;
 }
 
 }  // namespace msla
@@ -252,44 +338,29 @@ size_t msla_forward_workspace_bytes(const msla_desc* desc) {
 }
 
 msla_status_t msla_forward(const msla_desc* desc, const void* x, const msla_weights* w, void* out, void* stream) {
-  ForwardPlan p;
-  msla_status_t s = validate_desc(desc, &p);
-  if (s != MSLA_OK) return s;
-  if (!x || !out || !w) return fail(MSLA_ERR_INVALID_ARG, "null x, out or weights");
-  if (!w->w_qkv || !w->w_dw || !w->w_pw || !w->w_proj) return fail(MSLA_ERR_INVALID_ARG, "null weight pointer");
-  const void* ptrs[] = {x, out, w->w_qkv, w->w_dw, w->w_pw, w->w_proj, w->b_proj, desc->workspace};
-  for (const void* ptr : ptrs)
-    if (ptr && !aligned16(ptr)) return fail(MSLA_ERR_ALIGNMENT, "all device pointers must be 16-byte aligned");
-  if (!desc->workspace || desc->workspace_bytes < p.bytes)
-    return fail(MSLA_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", p.bytes, desc->workspace ? desc->workspace_bytes : (size_t)0);
-  const size_t e = elem_size(desc->dtype);
-  const size_t xb = (size_t)desc->B * desc->C * p.N * e, ob = (size_t)desc->B * desc->C_out * p.N * e;
-  if (overlaps(out, ob, x, xb)) return fail(MSLA_ERR_INVALID_ARG, "out overlaps x");
-  if (overlaps(out, ob, desc->workspace, p.bytes) || overlaps(x, xb, desc->workspace, p.bytes))
-    return fail(MSLA_ERR_INVALID_ARG, "workspace overlaps x or out");
-  s = check_arch();
-  if (s != MSLA_OK) return s;
-
-  cudaStream_t st = (cudaStream_t)stream;
-  char* ws = (char*)desc->workspace;
-  const int Cp = p.Cp, N = p.N, d = desc->d, heads = desc->heads;
-  const long long ld_ms = 6LL * Cp, ld_att = 2LL * Cp;
-  char* ms = ws + p.ms_off;    // [B, N, 6C']: channels [0,3C') = qkv, [3C',6C') = aggregated
-  char* att = ws + p.att_off;  // [B, N, 2C']
-  // 1. QKV projection into the first half of every multi-scale row
-  s = run_project_in(desc->dtype, x, w->w_qkv, ms, desc->B, desc->C, 3 * Cp, N, ld_ms, st);
-  if (s != MSLA_OK) return s;
-  // 2. aggregation into the second half
-  s = run_aggregate(desc->dtype, ms, w->w_dw, w->w_pw, ms + 3 * Cp * e, desc->B, desc->H, desc->W, 3 * Cp, d, ld_ms, ld_ms, st);
-  if (s != MSLA_OK) return s;
-  // 3+4. attention over 2*heads heads of [q|k|v]; outputs land at channel head*d (concat)
-  const HeadView in{(long long)N * ld_ms, 3LL * d, ld_ms};
-  const HeadView ov{(long long)N * ld_att, d, ld_att};
-  s = run_core(desc->dtype, ms, ms + d * e, ms + 2 * d * e, att, in, ov, desc->B, 2 * heads, N, d, desc->eps, p.core, ws + p.core_off, st);
-  if (s != MSLA_OK) return s;
-  // 5. output projection back to NCHW
-  return run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out, desc->B, 2 * Cp, desc->C_out, N, st);
+  return forward_impl(desc, x, w, out, (cudaStream_t)stream, nullptr, false);
 }
+
+msla_status_t msla_forward_profiled(const msla_desc* desc, const void* x, const msla_weights* w, void* out,
+                                    void* stream, void* const* events, int n_events) {
+  if (!events || n_events != 6) return fail(MSLA_ERR_INVALID_ARG, "events must hold exactly 6 cudaEvent_t handles");
+  for (int i = 0; i < 6; ++i)
+    if (!events[i]) return fail(MSLA_ERR_INVALID_ARG, "events[%d] is null", i);
+  return forward_impl(desc, x, w, out, (cudaStream_t)stream, events, false);
+}
+
+size_t msla_forward_host_workspace_bytes(const msla_desc* desc) {
+  ForwardPlan p;
+  if (validate_desc(desc, &p) != MSLA_OK) return 0;
+  const size_t e = elem_size(desc->dtype);
+  return p.bytes + align_up((size_t)desc->B * desc->C * p.N * e, 256) + align_up((size_t)desc->B * desc->C_out * p.N * e, 256);
+}
+
+msla_status_t msla_forward_host(const msla_desc* desc, const void* x_host, const msla_weights* w, void* out_host, void* stream) {
+  return forward_impl(desc, x_host, w, out_host, (cudaStream_t)stream, nullptr, true);
+}
+
+unsigned long long msla_kernel_launches(void) { return g_launches; }
 
 msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y, int B, int C, int Cout, int N, void* stream) {
   if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");
