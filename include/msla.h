@@ -80,6 +80,34 @@ msla_status_t msla_linattn_relu_ws(msla_dtype_t dtype, const void* q, const void
                                    void* out, int B, int heads, int N, int d, float eps,
                                    void* workspace, size_t workspace_bytes, void* stream);
 
+/* Attention core for callers that must not allocate.  (The paper has no
+ * counterpart to this entry point; it exists for deployment reasons only.)
+ *
+ * Some hosts of this library cannot call cudaMalloc or its stream-ordered
+ * relatives when they need the result: control loops with a hard deadline
+ * that forbid allocation after start-up (an allocation may block, synchronise
+ * the device or fail), and plug-ins living inside a runtime that owns every
+ * byte of device memory and hands none out at call time.  For them the
+ * scratch of the token reduction comes from a fixed array that is part of the
+ * library image: MSLA_NOALLOC_SCRATCH_BYTES of device memory, reserved on
+ * every GPU that loads the library for as long as the process lives.
+ *
+ * Same arguments and result as msla_linattn_relu_ws without the workspace.
+ * Shapes whose scratch need (msla_linattn_relu_workspace_bytes) exceeds
+ * MSLA_NOALLOC_SCRATCH_BYTES are refused with MSLA_ERR_WORKSPACE and nothing
+ * is launched.  The call never allocates or frees memory, on host or device.
+ *
+ * The first call on each device looks up the array's device address (a
+ * symbol query, not an allocation); make that first call outside any stream
+ * capture.  All calls on a device share the one array, and its contents
+ * persist from call to call, so two calls whose kernels may overlap on the GPU
+ * (different streams, no ordering between them) race; order them on one stream
+ * or with events. */
+#define MSLA_NOALLOC_SCRATCH_BYTES (4u << 20)
+msla_status_t msla_linattn_relu_noalloc(msla_dtype_t dtype, const void* q, const void* k, const void* v,
+                                        void* out, int B, int heads, int N, int d, float eps,
+                                        void* stream);
+
 /* ------------------------------------------------------------------------- *
  * Whole module (Section 3.1, Figure 2 right) on an NCHW feature map:
  *

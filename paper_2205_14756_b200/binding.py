@@ -45,6 +45,7 @@ EXPORTS = {
     "msla_linattn_relu_f32": (c_int, [c_void_p] * 4 + [c_int] * 4 + [c_float, c_void_p]),
     "msla_linattn_relu_workspace_bytes": (c_size_t, [c_int] * 4),
     "msla_linattn_relu_ws": (c_int, [c_int] + [c_void_p] * 4 + [c_int] * 4 + [c_float, c_void_p, c_size_t, c_void_p]),
+    "msla_linattn_relu_noalloc": (c_int, [c_int] + [c_void_p] * 4 + [c_int] * 4 + [c_float, c_void_p]),
     "msla_forward_workspace_bytes": (c_size_t, [ctypes.POINTER(msla_desc)]),
     "msla_forward": (c_int, [ctypes.POINTER(msla_desc), c_void_p, ctypes.POINTER(msla_weights), c_void_p, c_void_p]),
     "msla_forward_profiled": (c_int, [ctypes.POINTER(msla_desc), c_void_p, ctypes.POINTER(msla_weights), c_void_p, c_void_p,
@@ -119,6 +120,19 @@ def msla_linattn_relu_f32(q, k, v, out, B, heads, N, d, eps=1e-15, stream=None) 
 def msla_linattn_relu_ws(dtype, q, k, v, out, B, heads, N, d, eps, workspace, workspace_bytes, stream=None) -> None:
     _check(lib().msla_linattn_relu_ws(dtype, _ptr(q), _ptr(k), _ptr(v), _ptr(out), B, heads, N, d, eps,
                                       _ptr(workspace), workspace_bytes, _stream(stream)))
+
+
+MSLA_NOALLOC_SCRATCH_BYTES = 4 << 20
+
+
+def msla_linattn_relu_noalloc(dtype, q, k, v, out, B, heads, N, d, eps=1e-15, stream=None) -> None:
+    """Attention core that takes its scratch from the library's built-in device
+    array instead of allocating: for callers that may not allocate (deadline
+    loops that forbid allocation after start-up, runtimes that own all memory).
+    Shapes needing more than MSLA_NOALLOC_SCRATCH_BYTES raise MslaError(4).
+    Calls on one device share the array: keep them ordered on the GPU."""
+    _check(lib().msla_linattn_relu_noalloc(dtype, _ptr(q), _ptr(k), _ptr(v), _ptr(out), B, heads, N, d, eps,
+                                           _stream(stream)))
 
 
 def make_desc(B, C, H, W, heads, d, C_out, dtype, eps=1e-15, n_scales=2, agg_kernel=5,

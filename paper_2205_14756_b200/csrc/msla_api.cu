@@ -4,6 +4,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "generic_kernels.cuh"
 #include "msla_common.cuh"
@@ -153,6 +154,62 @@ static msla_status_t core_entry(msla_dtype_t dtype, const void* q, const void* k
   s = run_core(dtype, q, k, v, out, in, in, B, heads, N, d, eps, p, ws, st);
   if (own_ws) cudaFreeAsync(ws, st);
   return s;
+}
+
+// ------------------------------------------------ allocation-free variant
+// Scratch for msla_linattn_relu_noalloc.  In host code this name is only a
+// handle for the symbol; the address kernels can use comes from
+// cudaGetSymbolAddress, queried once per device with that device current.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[MSLA_NOALLOC_SCRATCH_BYTES];
+
+static msla_status_t noalloc_scratch(void** out_ptr) {
+  static std::mutex mu;
+  static void* per_device[64];  // nullptr = not looked up yet
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return fail(MSLA_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+  }
+  if (dev < 0 || dev >= 64) return fail(MSLA_ERR_UNSUPPORTED, "device ordinal %d is beyond the 64 this entry point tracks", dev);
+  std::lock_guard<std::mutex> lock(mu);
+  if (!per_device[dev]) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+    if (e != cudaSuccess || !ptr) {
+      cudaGetLastError();
+      return fail(MSLA_ERR_CUDA, "cudaGetSymbolAddress(scratch): %s", cudaGetErrorString(e));
+    }
+    per_device[dev] = ptr;
+  }
+  *out_ptr = per_device[dev];
+  return MSLA_OK;
+}
+
+static msla_status_t core_entry_noalloc(msla_dtype_t dtype, const void* q, const void* k, const void* v,
+                                        void* out, int B, int heads, int N, int d, float eps, cudaStream_t st) {
+  if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype %d", (int)dtype);
+  if (!q || !k || !v || !out) return fail(MSLA_ERR_INVALID_ARG, "null tensor pointer");
+  if (B < 1 || heads < 1 || N < 1 || d < 1) return fail(MSLA_ERR_INVALID_ARG, "B, heads, N, d must be positive (got %d, %d, %d, %d)", B, heads, N, d);
+  if (!(eps >= 0.f)) return fail(MSLA_ERR_INVALID_ARG, "eps must be >= 0");
+  if (d != 16 && d != 32) return fail(MSLA_ERR_UNSUPPORTED, "d = %d; only 16 and 32 are supported", d);
+  if ((long long)B * heads > 65535) return fail(MSLA_ERR_UNSUPPORTED, "B*heads = %lld exceeds 65535", (long long)B * heads);
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return fail(MSLA_ERR_ALIGNMENT, "q, k, v, out must be 16-byte aligned");
+  const size_t bytes = (size_t)B * heads * N * d * elem_size(dtype);
+  if (overlaps(out, bytes, q, bytes) || overlaps(out, bytes, k, bytes) || overlaps(out, bytes, v, bytes))
+    return fail(MSLA_ERR_INVALID_ARG, "out overlaps an input");
+  const CorePlan p = make_core_plan((long long)B * heads, N, d);
+  if (p.bytes > (size_t)MSLA_NOALLOC_SCRATCH_BYTES)
+    return fail(MSLA_ERR_WORKSPACE, "this shape needs %zu bytes of scratch; the built-in array holds %u (use msla_linattn_relu_ws)",
+                p.bytes, (unsigned)MSLA_NOALLOC_SCRATCH_BYTES);
+  msla_status_t s = check_arch();
+  if (s != MSLA_OK) return s;
+  void* ws = nullptr;
+  if ((s = noalloc_scratch(&ws)) != MSLA_OK) return s;
+  // Every partial and state entry the apply step reads is written earlier in
+  // this same call, so nothing left over from a previous call needs clearing.
+  const HeadView in{(long long)heads * N * d, (long long)N * d, d};
+  return run_core(dtype, q, k, v, out, in, in, B, heads, N, d, eps, p, ws, st);
 }
 
 // ------------------------------------------------------------- module plan
@@ -329,6 +386,11 @@ msla_status_t msla_linattn_relu_ws(msla_dtype_t dtype, const void* q, const void
                                    void* out, int B, int heads, int N, int d, float eps,
                                    void* workspace, size_t workspace_bytes, void* stream) {
   return core_entry(dtype, q, k, v, out, B, heads, N, d, eps, workspace, workspace_bytes, false, (cudaStream_t)stream);
+}
+
+msla_status_t msla_linattn_relu_noalloc(msla_dtype_t dtype, const void* q, const void* k, const void* v,
+                                        void* out, int B, int heads, int N, int d, float eps, void* stream) {
+  return core_entry_noalloc(dtype, q, k, v, out, B, heads, N, d, eps, (cudaStream_t)stream);
 }
 
 size_t msla_forward_workspace_bytes(const msla_desc* desc) {
