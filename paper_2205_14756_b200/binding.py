@@ -14,7 +14,7 @@ from typing import Optional
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libmsla.so")
+LIB_PATH = os.environ.get("MSLA_LIBRARY_PATH") or os.path.join(_PKG, "libmsla.so")
 
 MSLA_F32, MSLA_BF16 = 0, 1
 _DTYPES = {torch.float32: MSLA_F32, torch.bfloat16: MSLA_BF16}

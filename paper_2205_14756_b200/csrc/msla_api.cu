@@ -79,6 +79,8 @@ CorePlan make_core_plan(long long BH, int N, int d) {
   chunk = ceil_div_ll(chunk, 64) * 64;
   p.chunk = (int)chunk;
   p.S = (int)ceil_div_ll(N, chunk);
+  long long at = ceil_div_ll(ceil_div_ll((long long)N * BH, 1184), 256) * 256;
+  p.apply_tokens = (int)(at < 256 ? 256 : (at > 2048 ? 2048 : at));
   p.partial_off = 0;
   p.state_off = align_up((size_t)BH * p.S * p.ne * sizeof(float), 256);
   p.bytes = p.state_off + align_up((size_t)BH * p.ne * sizeof(float), 256);
@@ -115,6 +117,9 @@ static msla_status_t run_core(msla_dtype_t dtype, const void* q, const void* k, 
   if (dtype == MSLA_F32)
     return run_core_generic<float>((const float*)q, (const float*)k, (const float*)v, (float*)out,
                                    in, ov, B, heads, N, d, eps, p, (char*)ws, st, mid);
+  const bool strides_ok = in.batch % 8 == 0 && in.head % 8 == 0 && in.ld % 8 == 0 && ov.batch % 8 == 0 &&
+                          ov.head % 8 == 0 && ov.ld % 8 == 0;
+  if (strides_ok) return run_core_bf16(q, k, v, out, in, ov, B, heads, N, d, eps, p, ws, st, mid);
   return run_core_generic<__nv_bfloat16>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
                                          (const __nv_bfloat16*)v, (__nv_bfloat16*)out, in, ov, B,
                                          heads, N, d, eps, p, (char*)ws, st, mid);

@@ -14,6 +14,7 @@ struct CorePlan {
   int S;       // number of token chunks per (batch, head)
   int chunk;   // tokens per chunk (multiple of 64)
   int ne;      // d*(d+1) state entries
+  int apply_tokens;  // tokens per CTA of the tuned apply kernel (multiple of 256)
   size_t partial_off, state_off, bytes;
 };
 
@@ -23,5 +24,13 @@ CorePlan make_core_plan(long long BH, int N, int d);
 msla_status_t fail(msla_status_t st, const char* fmt, ...);
 // MSLA_OK, or MSLA_ERR_CUDA if a launch since the last check failed.
 msla_status_t check_launch(const char* what);
+
+void count_launches(int n);
+
+struct HeadView;
+// Tuned bf16 attention core (d in {16, 32}); all view strides must be multiples of 8 elements.
+msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* out, HeadView in, HeadView ov, int B,
+                            int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st,
+                            cudaEvent_t mid);
 
 }  // namespace msla
