@@ -12,16 +12,19 @@
 
 // Launch shapes (overridable at build time for tuning sweeps).
 #ifndef MSLA_KV_WARPS
-#define MSLA_KV_WARPS 8
+#define MSLA_KV_WARPS 4
 #endif
-#ifndef MSLA_KV_U
-#define MSLA_KV_U 4
+#ifndef MSLA_KV_STAGES
+#define MSLA_KV_STAGES 4
 #endif
 #ifndef MSLA_AP_WARPS
 #define MSLA_AP_WARPS 4
 #endif
+#ifndef MSLA_AP_STAGES
+#define MSLA_AP_STAGES 4
+#endif
 #ifndef MSLA_AP_U
-#define MSLA_AP_U 4
+#define MSLA_AP_U 2
 #endif
 
 namespace msla {
@@ -41,20 +44,7 @@ __device__ __forceinline__ uint32_t relu2(uint32_t x) {  // packed bf16x2 max(x,
   return r;
 }
 
-__device__ __forceinline__ uint32_t lo_pair(uint32_t a, uint32_t b) { return __byte_perm(a, b, 0x5410); }
-__device__ __forceinline__ uint32_t hi_pair(uint32_t a, uint32_t b) { return __byte_perm(a, b, 0x7632); }
 
-// Streaming loads: every byte is used once, keep it out of L1.
-__device__ __forceinline__ void ldg_stream(const void* p, uint32_t (&r)[1]) {
-  asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(r[0]) : "l"(p));
-}
-__device__ __forceinline__ void ldg_stream(const void* p, uint32_t (&r)[2]) {
-  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "l"(p));
-}
-__device__ __forceinline__ void ldg_stream(const void* p, uint32_t (&r)[4]) {
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "l"(p));
-}
 __device__ __forceinline__ void stg(void* p, const uint32_t (&r)[2]) {
   asm volatile("st.global.v2.u32 [%0], {%1,%2};" ::"l"(p), "r"(r[0]), "r"(r[1]) : "memory");
 }
@@ -68,39 +58,89 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// 16-byte asynchronous global->shared copy; src_bytes = 0 writes zeros instead.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void lds128(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void lds64(uint32_t (&r)[2], uint32_t addr) {
+  asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
+}
+
 // ---------------------------------------------------------------------------
-// KV-state reduction, first level.  One CTA = one (batch, head, token chunk);
-// each warp owns 16-token MMA steps, U of them per loop trip.
+// KV-state reduction, first level.  One CTA = one (batch, head, token chunk).
 //
 // MMA view: state[a][c] += sum over 16 tokens of relu(k[n][a]) * v[n][c],
 // A = relu(K)^T (rows = channel a, contraction = token), B = [V | 1].
-// Lane (g = lane/4, t = lane%4) loads, for the four tokens {t, t+4, t+8, t+12}
-// of a step, the D/8 consecutive channels starting at g*D/8 of K and of V
-// (8 bytes for D = 32).  Those tokens sit in contraction slots {2t, 2t+1,
-// 2t+8, 2t+9}: exactly the slots this lane must supply for both operands.
-// Word w of a load holds channels (2w, 2w+1) of the lane's group:
-//   A tile w   : row g = channel g*D/8 + 2w, row g+8 = channel g*D/8 + 2w + 1
-//   B tile 2w+p: column g = channel g*D/8 + 2w + p
-// An extra B tile of ones yields sum relu(k).
+//
+// Every warp runs its own STAGES-deep ring of cp.async groups: a stage holds TS
+// tokens of K and of V as [token][channel] rows in shared memory (16-byte
+// chunks XOR-swizzled by row so that ldmatrix is bank-conflict free).  Both
+// operands want the token index along the contraction, i.e. the transpose of
+// how the rows lie in memory, which is exactly ldmatrix.trans.  Memory latency
+// is covered by the ring (bytes in flight do not depend on registers or
+// occupancy); no block-wide barrier is taken inside the loop.  An extra B tile
+// of bf16 ones yields sum relu(k).
 // ---------------------------------------------------------------------------
-template <int D, int NWARPS, int U>
+template <int D, int NWARPS, int STAGES>
 __global__ void __launch_bounds__(NWARPS * 32)
 kv_state_mma_kernel(const bf16* __restrict__ k, const bf16* __restrict__ v, float* __restrict__ partial,
                     HeadView kv, int heads, int N, int S, int chunk) {
-  constexpr int W = D / 16;   // 32-bit words per lane per token
-  constexpr int MT = D / 16;  // A tiles (16 channels each)
-  constexpr int NT = D / 8;   // B tiles (8 channels each), + 1 tile of ones
-  constexpr int CG = D / 8;   // channels per lane group
+  constexpr int TS = 32;            // tokens per stage
+  constexpr int MT = D / 16;        // A tiles (16 channels each)
+  constexpr int NT = D / 8;         // B tiles (8 channels each), + 1 tile of ones
+  constexpr int CH = D / 8;         // 16-byte chunks per token row
+  constexpr int ROWB = D * 2;       // bytes per token row
+  constexpr int TILEB = TS * ROWB;  // bytes of one K (or V) tile
+  constexpr int SW_SHIFT = CH == 4 ? 1 : 2;
   constexpr int NE = D * (D + 1);
-  __shared__ float red[NWARPS][NE];
+  constexpr int CPL = TS * CH / 32;  // cp.async per lane per tile
+  constexpr int RPI = 32 / CH;       // token rows covered by one warp-wide cp.async
+  extern __shared__ __align__(128) unsigned char smem[];
+  static_assert(NWARPS * STAGES * 2 * TILEB >= NWARPS * NE * 4, "reduction buffer must fit in the stage ring");
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int bh = blockIdx.x, s = blockIdx.y;
   const int b = bh / heads, h = bh % heads;
-  const long long base = (long long)b * kv.batch + (long long)h * kv.head + g * CG;
+  const long long base = (long long)b * kv.batch + (long long)h * kv.head;
   const int n_begin = s * chunk;
   const int n_end = min(N, n_begin + chunk);
+  const int groups = (n_end - n_begin + TS - 1) / TS;           // TS-token groups in this chunk
+  const int my_groups = groups > warp ? (groups - warp + NWARPS - 1) / NWARPS : 0;
+
+  const uint32_t ring = smem_u32(smem) + warp * (STAGES * 2 * TILEB);
+  // this lane's slot in a warp-wide copy: row r_cp (+ RPI per copy), chunk c_cp
+  const int r_cp = lane / CH, c_cp = lane % CH;
+  const bf16* ksrc = k + base + c_cp * 8;
+  const bf16* vsrc = v + base + c_cp * 8;
+
+  auto issue = [&](int it) {  // it-th group of this warp -> stage it % STAGES
+    const uint32_t dstK = ring + (it % STAGES) * (2 * TILEB), dstV = dstK + TILEB;
+    const int n0 = n_begin + (warp + it * NWARPS) * TS;
+#pragma unroll
+    for (int i = 0; i < CPL; ++i) {
+      const int r = r_cp + i * RPI;
+      const int n = n0 + r;
+      const bool ok = n < n_end;
+      const long long off = (long long)(ok ? n : n_begin) * kv.ld;
+      const uint32_t d = r * ROWB + ((c_cp ^ ((r >> SW_SHIFT) & (CH - 1))) << 4);
+      cp_async16(dstK + d, ksrc + off, ok ? 16 : 0);
+      cp_async16(dstV + d, vsrc + off, ok ? 16 : 0);
+    }
+  };
 
   float acc[MT][NT + 1][4];
 #pragma unroll
@@ -110,35 +150,39 @@ kv_state_mma_kernel(const bf16* __restrict__ k, const bf16* __restrict__ v, floa
 #pragma unroll
       for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
 
-  for (int n0 = n_begin + warp * (16 * U); n0 < n_end; n0 += NWARPS * 16 * U) {
-    uint32_t kr[U][4][W], vr[U][4][W];
 #pragma unroll
-    for (int u = 0; u < U; ++u)
+  for (int p = 0; p < STAGES - 1; ++p) {
+    if (p < my_groups) issue(p);
+    cp_async_commit();
+  }
+  // ldmatrix row address pieces for this lane: matrix m = lane/8, row lane%8
+  const int lm = lane >> 3, lr = lane & 7;
+  for (int it = 0; it < my_groups; ++it) {
+    if (it + STAGES - 1 < my_groups) issue(it + STAGES - 1);
+    cp_async_commit();
+    cp_async_wait<STAGES - 1>();
+    __syncwarp();
+    const uint32_t tK = ring + (it % STAGES) * (2 * TILEB), tV = tK + TILEB;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int n = n0 + u * 16 + t + 4 * j;
-        if (n < n_end) {
-          const long long off = base + (long long)n * kv.ld;
-          ldg_stream(k + off, kr[u][j]);
-          ldg_stream(v + off, vr[u][j]);
-        } else {
-#pragma unroll
-          for (int w = 0; w < W; ++w) kr[u][j][w] = vr[u][j][w] = 0u;
-        }
-      }
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
+    for (int ks = 0; ks < TS / 16; ++ks) {
       uint32_t A[MT][4], Bt[NT][2];
 #pragma unroll
-      for (int w = 0; w < W; ++w) {
-        const uint32_t k0 = relu2(kr[u][0][w]), k1 = relu2(kr[u][1][w]);
-        const uint32_t k2 = relu2(kr[u][2][w]), k3 = relu2(kr[u][3][w]);
-        A[w][0] = lo_pair(k0, k1); A[w][1] = hi_pair(k0, k1);
-        A[w][2] = lo_pair(k2, k3); A[w][3] = hi_pair(k2, k3);
-        Bt[2 * w][0] = lo_pair(vr[u][0][w], vr[u][1][w]);
-        Bt[2 * w][1] = lo_pair(vr[u][2][w], vr[u][3][w]);
-        Bt[2 * w + 1][0] = hi_pair(vr[u][0][w], vr[u][1][w]);
-        Bt[2 * w + 1][1] = hi_pair(vr[u][2][w], vr[u][3][w]);
+      for (int i = 0; i < MT; ++i) {
+        // matrices: (tok 0-7, ch chunk 2i) (tok 0-7, chunk 2i+1) (tok 8-15, chunk 2i) (tok 8-15, chunk 2i+1)
+        const int r = ks * 16 + lr + ((lm >> 1) << 3);
+        const int c = 2 * i + (lm & 1);
+        ldsm_x4_trans(A[i], tK + r * ROWB + ((c ^ ((r >> SW_SHIFT) & (CH - 1))) << 4));
+#pragma unroll
+        for (int e = 0; e < 4; ++e) A[i][e] = relu2(A[i][e]);
+      }
+#pragma unroll
+      for (int j = 0; j < NT; j += 2) {
+        // matrices: (tok 0-7, chunk j) (tok 8-15, chunk j) (tok 0-7, chunk j+1) (tok 8-15, chunk j+1)
+        const int r = ks * 16 + lr + ((lm & 1) << 3);
+        const int c = j + (lm >> 1);
+        uint32_t x[4];
+        ldsm_x4_trans(x, tV + r * ROWB + ((c ^ ((r >> SW_SHIFT) & (CH - 1))) << 4));
+        Bt[j][0] = x[0]; Bt[j][1] = x[1]; Bt[j + 1][0] = x[2]; Bt[j + 1][1] = x[3];
       }
 #pragma unroll
       for (int i = 0; i < MT; ++i) {
@@ -147,26 +191,30 @@ kv_state_mma_kernel(const bf16* __restrict__ k, const bf16* __restrict__ v, floa
         mma_bf16(acc[i][NT], A[i], 0x3F803F80u, 0x3F803F80u);  // bf16 ones
       }
     }
+    __syncwarp();  // all lanes done with this stage before a later issue() overwrites it
   }
+  cp_async_wait<0>();
+  __syncthreads();  // every warp has left its ring: reuse it for the reduction
 
   // fixed-order combine of the warps' accumulators (level one of two)
+  float* red = reinterpret_cast<float*>(smem);
 #pragma unroll
   for (int i = 0; i < MT; ++i)
 #pragma unroll
     for (int j = 0; j <= NT; ++j)
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const int a = g * CG + 2 * i + (e >> 1);
+        const int a = 16 * i + g + 8 * (e >> 1);
         const int col = 2 * t + (e & 1);
-        if (j < NT) red[warp][a * (D + 1) + col * CG + j] = acc[i][j][e];
-        else if (col == 0) red[warp][a * (D + 1) + D] = acc[i][j][e];
+        if (j < NT) red[warp * NE + a * (D + 1) + 8 * j + col] = acc[i][j][e];
+        else if (col == 0) red[warp * NE + a * (D + 1) + D] = acc[i][j][e];
       }
   __syncthreads();
   float* out = partial + ((long long)bh * S + s) * NE;
   for (int e = threadIdx.x; e < NE; e += NWARPS * 32) {
-    float sum = red[0][e];
+    float sum = red[e];
 #pragma unroll
-    for (int w = 1; w < NWARPS; ++w) sum += red[w][e];
+    for (int w = 1; w < NWARPS; ++w) sum += red[w * NE + e];
     out[e] = sum;
   }
 }
@@ -197,19 +245,54 @@ kv_combine_bf16path_kernel(const float* __restrict__ partial, float* __restrict_
 // The fp32 state is fed as bf16 hi + bf16 lo (two MMAs) to keep ~16 mantissa
 // bits; one extra tile whose columns all hold ks gives the denominator.
 // ---------------------------------------------------------------------------
-template <int D, int NWARPS, int U>
+template <int D, int NWARPS, int STAGES, int U>
 __global__ void __launch_bounds__(NWARPS * 32)
 apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf16* __restrict__ out,
                  HeadView qv, HeadView ov, int heads, int N, float eps, int tok_per_cta) {
-  constexpr int KS = D / 16;  // MMA steps over the channel contraction
-  constexpr int NT = D / 8;   // output tiles, + 1 for the denominator
-  constexpr int CPT = D / 4;  // channels per lane per token
-  constexpr int WQ = D / 8;   // 32-bit words per lane per token
+  constexpr int KS = D / 16;   // MMA steps over the channel contraction
+  constexpr int NT = D / 8;    // output tiles, + 1 for the denominator
+  constexpr int CPT = D / 4;   // channels per lane per token
+  constexpr int WQ = D / 8;    // 32-bit words per lane per token
+  constexpr int LB = CPT * 2;  // bytes per lane per token (16 or 8)
+  constexpr int STAGEB = U * 2 * 32 * LB;
+  // Each lane streams its own query bytes through a private FIFO in shared
+  // memory (cp.async in, plain load out), so loads run STAGES groups ahead of
+  // the MMAs without holding registers and without any cross-lane hand-off.
+  __shared__ __align__(16) unsigned char fifo[NWARPS * STAGES * STAGEB];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int bh = blockIdx.y;
   const int b = bh / heads, h = bh % heads;
+  const long long qbase = (long long)b * qv.batch + (long long)h * qv.head + t * CPT;
+  const long long obase = (long long)b * ov.batch + (long long)h * ov.head + t * CPT;
+  const int n_begin = blockIdx.x * tok_per_cta;
+  const int n_end = min(N, n_begin + tok_per_cta);
+  constexpr int TS = 16 * U;
+  const int groups = (n_end - n_begin + TS - 1) / TS;
+  const int my_groups = groups > warp ? (groups - warp + NWARPS - 1) / NWARPS : 0;
+  const uint32_t ring = smem_u32(fifo) + warp * (STAGES * STAGEB) + lane * LB;
 
+  auto issue = [&](int it) {
+    const uint32_t dst = ring + (it % STAGES) * STAGEB;
+    const int n0 = n_begin + (warp + it * NWARPS) * TS + g;
+#pragma unroll
+    for (int u = 0; u < 2 * U; ++u) {  // u even: token g of tile u/2, odd: token g+8
+      const int n = n0 + u * 8;
+      const bool ok = n < n_end;
+      const bf16* src = q + qbase + (long long)(ok ? n : n_begin) * qv.ld;
+      if constexpr (LB == 16)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + u * 32 * LB), "l"(src), "r"(ok ? 16 : 0) : "memory");
+      else
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst + u * 32 * LB), "l"(src), "r"(ok ? 8 : 0) : "memory");
+    }
+  };
+#pragma unroll
+  for (int p = 0; p < STAGES - 1; ++p) {
+    if (p < my_groups) issue(p);
+    cp_async_commit();
+  }
+
+  // state -> B fragments (bf16 hi + lo), overlapping the first copies
   uint32_t bhi[KS][NT + 1][2], blo[KS][NT + 1][2];
   {
     const float* st = state + (long long)bh * D * (D + 1);
@@ -228,70 +311,83 @@ apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf
         }
   }
 
-  const long long qbase = (long long)b * qv.batch + (long long)h * qv.head + t * CPT;
-  const long long obase = (long long)b * ov.batch + (long long)h * ov.head + t * CPT;
-  const int n_begin = blockIdx.x * tok_per_cta;
-  const int n_end = min(N, n_begin + tok_per_cta);
-
-  for (int n0 = n_begin + warp * (16 * U); n0 < n_end; n0 += NWARPS * 16 * U) {
+  for (int it = 0; it < my_groups; ++it) {
+    if (it + STAGES - 1 < my_groups) issue(it + STAGES - 1);
+    cp_async_commit();
+    cp_async_wait<STAGES - 1>();
+    const uint32_t src = ring + (it % STAGES) * STAGEB;
+    const int n0 = n_begin + (warp + it * NWARPS) * TS;
     uint32_t qa[U][WQ], qb[U][WQ];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const int na = n0 + u * 16 + g, nb = na + 8;
-      if (na < n_end) ldg_stream(q + qbase + (long long)na * qv.ld, qa[u]);
-      else {
-#pragma unroll
-        for (int w = 0; w < WQ; ++w) qa[u][w] = 0u;
-      }
-      if (nb < n_end) ldg_stream(q + qbase + (long long)nb * qv.ld, qb[u]);
-      else {
-#pragma unroll
-        for (int w = 0; w < WQ; ++w) qb[u][w] = 0u;
+      if constexpr (LB == 16) {
+        lds128(qa[u], src + (2 * u) * 32 * LB);
+        lds128(qb[u], src + (2 * u + 1) * 32 * LB);
+      } else {
+        lds64(qa[u], src + (2 * u) * 32 * LB);
+        lds64(qb[u], src + (2 * u + 1) * 32 * LB);
       }
     }
+    float acc[U][NT + 1][4];
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      float acc[NT + 1][4];
+    for (int u = 0; u < U; ++u)
 #pragma unroll
       for (int j = 0; j <= NT; ++j)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) acc[j][e] = 0.f;
+        for (int e = 0; e < 4; ++e) acc[u][j][e] = 0.f;
 #pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
-        const uint32_t A[4] = {relu2(qa[u][2 * ks]), relu2(qb[u][2 * ks]), relu2(qa[u][2 * ks + 1]), relu2(qb[u][2 * ks + 1])};
+    for (int ks = 0; ks < KS; ++ks) {
+      uint32_t A[U][4];
 #pragma unroll
-        for (int j = 0; j <= NT; ++j) {
-          mma_bf16(acc[j], A, bhi[ks][j][0], bhi[ks][j][1]);
-          mma_bf16(acc[j], A, blo[ks][j][0], blo[ks][j][1]);
-        }
+      for (int u = 0; u < U; ++u) {
+        A[u][0] = relu2(qa[u][2 * ks]); A[u][1] = relu2(qb[u][2 * ks]);
+        A[u][2] = relu2(qa[u][2 * ks + 1]); A[u][3] = relu2(qb[u][2 * ks + 1]);
       }
-      const float inv_a = 1.f / (acc[NT][0] + eps), inv_b = 1.f / (acc[NT][2] + eps);
+#pragma unroll
+      for (int j = 0; j <= NT; ++j)
+#pragma unroll
+        for (int u = 0; u < U; ++u) mma_bf16(acc[u][j], A[u], bhi[ks][j][0], bhi[ks][j][1]);
+#pragma unroll
+      for (int j = 0; j <= NT; ++j)
+#pragma unroll
+        for (int u = 0; u < U; ++u) mma_bf16(acc[u][j], A[u], blo[ks][j][0], blo[ks][j][1]);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const float inv_a = 1.f / (acc[u][NT][0] + eps), inv_b = 1.f / (acc[u][NT][2] + eps);
       uint32_t oa[WQ], ob[WQ];
 #pragma unroll
       for (int j = 0; j < NT; ++j) {
-        oa[j] = pack_bf16(acc[j][0] * inv_a, acc[j][1] * inv_a);
-        ob[j] = pack_bf16(acc[j][2] * inv_b, acc[j][3] * inv_b);
+        oa[j] = pack_bf16(acc[u][j][0] * inv_a, acc[u][j][1] * inv_a);
+        ob[j] = pack_bf16(acc[u][j][2] * inv_b, acc[u][j][3] * inv_b);
       }
       const int na = n0 + u * 16 + g, nb = na + 8;
       if (na < n_end) stg(out + obase + (long long)na * ov.ld, oa);
       if (nb < n_end) stg(out + obase + (long long)nb * ov.ld, ob);
     }
   }
+  cp_async_wait<0>();
 }
 
 template <int D>
 msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out, HeadView in, HeadView ov, int B,
                           int heads, int N, float eps, const CorePlan& p, char* ws, cudaStream_t st, cudaEvent_t mid) {
-  constexpr int KV_WARPS = MSLA_KV_WARPS, KV_U = MSLA_KV_U, AP_WARPS = MSLA_AP_WARPS, AP_U = MSLA_AP_U;
+  constexpr int KV_WARPS = MSLA_KV_WARPS, KV_STAGES = MSLA_KV_STAGES, AP_WARPS = MSLA_AP_WARPS, AP_STAGES = MSLA_AP_STAGES, AP_U = MSLA_AP_U;
   const long long BH = (long long)B * heads;
   float* partial = reinterpret_cast<float*>(ws + p.partial_off);
   float* state = reinterpret_cast<float*>(ws + p.state_off);
-  kv_state_mma_kernel<D, KV_WARPS, KV_U><<<dim3((unsigned)BH, p.S), KV_WARPS * 32, 0, st>>>(k, v, partial, in, heads, N, p.S, p.chunk);
+  constexpr int kv_smem = KV_WARPS * KV_STAGES * 2 * 32 * D * 2;
+  static bool attr_done = false;  // idempotent; a race only repeats the call
+  if (!attr_done) {
+    cudaFuncSetAttribute(kv_state_mma_kernel<D, KV_WARPS, KV_STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, kv_smem);
+    attr_done = true;
+  }
+  kv_state_mma_kernel<D, KV_WARPS, KV_STAGES><<<dim3((unsigned)BH, p.S), KV_WARPS * 32, kv_smem, st>>>(k, v, partial, in, heads, N, p.S, p.chunk);
   const long long total = BH * p.ne;
   kv_combine_bf16path_kernel<<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>(partial, state, p.S, p.ne, total);
   if (mid) cudaEventRecord(mid, st);
   const int tok_per_cta = p.apply_tokens;
-  apply_mma_kernel<D, AP_WARPS, AP_U><<<dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)BH), AP_WARPS * 32, 0, st>>>(
+  apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U><<<dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)BH), AP_WARPS * 32, 0, st>>>(
       q, state, out, in, ov, heads, N, eps, tok_per_cta);
   count_launches(3);
   return check_launch("attention core kernels (bf16)");
