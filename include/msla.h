@@ -183,6 +183,13 @@ msla_status_t msla_forward_host(const msla_desc* desc, const void* x_host, const
  * was loaded (a bookkeeping counter for benchmarks; no paper counterpart). */
 unsigned long long msla_kernel_launches(void);
 
+/* Diagnostic (no paper counterpart): every wait inside the library's kernels
+ * is bounded; a kernel whose wait ran out raises a sticky device flag, releases
+ * what it holds and returns, leaving its output undefined.  This call
+ * SYNCHRONISES the device and returns 1 if that ever happened in this process,
+ * 0 if not, -1 if the flag could not be read. */
+int msla_debug_wait_timeouts(void);
+
 /* Stage entry points (the module's steps 1, 2 and 5 on their own), exposed so
  * that each kernel can be checked and timed in isolation.  Internal
  * activations are token-major: act[b][n][channel].

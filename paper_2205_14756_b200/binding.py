@@ -53,6 +53,7 @@ EXPORTS = {
     "msla_forward_host_workspace_bytes": (c_size_t, [ctypes.POINTER(msla_desc)]),
     "msla_forward_host": (c_int, [ctypes.POINTER(msla_desc), c_void_p, ctypes.POINTER(msla_weights), c_void_p, c_void_p]),
     "msla_kernel_launches": (ctypes.c_ulonglong, []),
+    "msla_debug_wait_timeouts": (c_int, []),
     "msla_project_in": (c_int, [c_int] + [c_void_p] * 3 + [c_int] * 4 + [c_void_p]),
     "msla_aggregate": (c_int, [c_int] + [c_void_p] * 4 + [c_int] * 5 + [c_void_p]),
     "msla_project_out": (c_int, [c_int] + [c_void_p] * 4 + [c_int] * 4 + [c_void_p]),
@@ -174,6 +175,10 @@ def msla_forward_host(desc: msla_desc, x_host, weights: msla_weights, out_host, 
             raise ValueError("msla_forward_host takes contiguous host tensors")
     _check(lib().msla_forward_host(ctypes.byref(desc), x_host.data_ptr(), ctypes.byref(weights), out_host.data_ptr(),
                                    _stream(stream)))
+
+
+def msla_debug_wait_timeouts() -> int:
+    return lib().msla_debug_wait_timeouts()
 
 
 def msla_kernel_launches() -> int:

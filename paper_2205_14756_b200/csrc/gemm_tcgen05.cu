@@ -1,0 +1,414 @@
+// bf16 GEMM for the module's two 1x1 projections (Section 3.1: Q = xW_Q,
+// K = xW_K, V = xW_V, and the final linear projection) on the 5th-generation
+// tensor cores: TMA loads into 128B-swizzled shared memory, tcgen05.mma with
+// fp32 accumulators in tensor memory, tcgen05.ld epilogue.
+//
+//   D[m][n] = sum_k A[m][k] * B[n][k] (+ bias),   fp32 accumulate, bf16 out,
+//   out[(batch * rows_per_batch + m) * ld_out + n]   (n contiguous)
+//
+// Input projection : m = token, n = output channel; A = x taken straight from
+//                    NCHW (the token index is contiguous: an "MN-major" operand),
+//                    B = w_qkv (K-major).
+// Output projection: m = output channel, n = token; A = w_proj (K-major),
+//                    B = attention output, token-major (K-major); D rows are
+//                    NCHW planes, so each thread stores runs of tokens.
+//
+// One persistent CTA per SM, warp-specialised: warp 0 issues TMA, warp 1
+// issues MMAs (and owns the tensor-memory allocation), warps 2-5 drain the
+// accumulators.  Two 128x256 fp32 accumulators (all 512 TMEM columns) let the
+// epilogue of one tile overlap the MMAs of the next.  Every mbarrier wait is
+// bounded: on time-out the CTA raises a flag, all roles leave their loops, the
+// tensor memory is released and the kernel returns.
+#include <cuda.h>
+
+#include "msla_common.cuh"
+#include "msla_host.h"
+
+namespace msla {
+namespace {
+
+using bf16 = __nv_bfloat16;
+
+constexpr int BM = 128, BN = 256, BK = 64;  // CTA tile; BK = one 128-byte swizzle span of bf16
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * BK * 2;  // 16 KB
+constexpr int B_STAGE_BYTES = BN * BK * 2;  // 32 KB
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int NUM_THREADS = 192;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 256 + 1024;  // ring + barriers + alignment slack
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;          // ~2 s at 2 GHz
+
+// Sticky: set when any wait in any GEMM launch of this process timed out.
+__device__ int g_gemm_timeout_flag = 0;
+
+struct GemmParams {
+  int M, N, K;            // per batch
+  int batches;
+  int m_tiles, n_tiles;   // per batch
+  int rows_per_batch;     // output rows between consecutive batches
+  long long ld_out;       // output row stride (elements)
+  int bias_per_row;       // 1: bias[m], 0: bias[n] (ignored when bias == nullptr)
+  int n_fastest;          // tile order: 1 = consecutive tiles share the A tile, 0 = share the B tile
+  const bf16* bias;
+  bf16* out;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred P1;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, P1;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (and raises *abort_flag) if the phase did not
+// complete within the cycle limit, or if another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  Offsets are in 16-byte
+// units: lbo = distance between 64-element blocks along M/N (MN-major only),
+// sbo = distance between groups of 8 rows (K-major) or 8 k-slices (MN-major).
+__device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo16, uint32_t sbo16) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)lbo16 << 16) | ((uint64_t)sbo16 << 32) |
+         (1ull << 46) /* descriptor version */ | (2ull << 61) /* SWIZZLE_128B */;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+__device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& b, int& mt, int& nt) {
+  const int per_batch = p.m_tiles * p.n_tiles;
+  b = tile / per_batch;
+  const int r = tile % per_batch;
+  if (p.n_fastest) { mt = r / p.n_tiles; nt = r % p.n_tiles; }
+  else             { nt = r / p.m_tiles; mt = r % p.m_tiles; }
+}
+
+template <bool A_MN_MAJOR>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
+  const uint32_t bars = smem_base + STAGES * STAGE_BYTES;
+  const uint32_t full_bar = bars, empty_bar = bars + 8 * STAGES;
+  const uint32_t tfull_bar = bars + 16 * STAGES, tempty_bar = tfull_bar + 16;
+  const uint32_t tmem_slot = tempty_bar + 16;
+  __shared__ int abort_flag;
+  __shared__ uint32_t tmem_base_sh;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_tiles = p.batches * p.m_tiles * p.n_tiles;
+  const int k_iters = (p.K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar + 8 * a, 1); mbar_init(tempty_bar + 8 * a, 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // whole warp: allocate all 512 tensor-memory columns (one CTA per SM)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (threadIdx.x == 0) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(tmem_slot));
+    tmem_base_sh = v;
+  }
+  __syncthreads();
+  const uint32_t tmem_base = tmem_base_sh;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        int b, mt, nt;
+        tile_coords(p, tile, b, mt, nt);
+        for (int kb = 0; ok && kb < k_iters; ++kb, ++it) {
+          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+          ok = mbar_wait(empty_bar + 8 * s, ph ^ 1, &abort_flag);
+          if (!ok) break;
+          const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+          mbar_expect_tx(full_bar + 8 * s, STAGE_BYTES);
+          if (A_MN_MAJOR) {  // two boxes of 64 tokens x 64 k
+            tma_load_3d(sa, &tmA, full_bar + 8 * s, mt * BM, kb * BK, b);
+            tma_load_3d(sa + A_STAGE_BYTES / 2, &tmA, full_bar + 8 * s, mt * BM + 64, kb * BK, b);
+          } else {           // one box of 64 k x 128 rows
+            tma_load_3d(sa, &tmA, full_bar + 8 * s, kb * BK, mt * BM, 0);
+          }
+          tma_load_3d(sb, &tmB, full_bar + 8 * s, kb * BK, nt * BN, A_MN_MAJOR ? 0 : b);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // -------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      // instruction descriptor: D = f32, A = B = bf16, A major, B K-major, N = 256, M = 128
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN_MAJOR ? 1u : 0u) << 15) |
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      uint32_t it = 0, local = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++local) {
+        const uint32_t acc = local & 1, acc_ph = (local >> 1) & 1;
+        ok = mbar_wait(tempty_bar + 8 * acc, acc_ph ^ 1, &abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; ok && kb < k_iters; ++kb, ++it) {
+          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+          ok = mbar_wait(full_bar + 8 * s, ph, &abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < BK / 16; ++kk) {
+            // MN-major A: 16 k-slices of 128 B further on; K-major: 32 B along the swizzled row
+            const uint64_t ad = A_MN_MAJOR ? make_desc(sa + kk * 2048, (A_STAGE_BYTES / 2) >> 4, 1024 >> 4)
+                                           : make_desc(sa + kk * 32, 1, 1024 >> 4);
+            const uint64_t bd = make_desc(sb + kk * 32, 1, 1024 >> 4);
+            umma_bf16(d_tmem, ad, bd, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+          }
+          umma_commit(empty_bar + 8 * s);  // stage reusable once these MMAs have read it
+        }
+        if (ok) umma_commit(tfull_bar + 8 * acc);  // accumulator complete
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int quarter = warp & 3;  // a warp may only touch TMEM lanes 32*(warp%4) .. +31
+    uint32_t local = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++local) {
+      int b, mt, nt;
+      tile_coords(p, tile, b, mt, nt);
+      const uint32_t acc = local & 1, acc_ph = (local >> 1) & 1;
+      ok = mbar_wait(tfull_bar + 8 * acc, acc_ph, &abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int m = mt * BM + quarter * 32 + lane;
+      const bool row_ok = m < p.M;
+      bf16* orow = p.out + ((long long)b * p.rows_per_batch + m) * p.ld_out + (long long)nt * BN;
+      const float bias_row = (p.bias && p.bias_per_row && row_ok) ? __bfloat162float(p.bias[m]) : 0.f;
+      const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld32(taddr + c * 32, r);
+        tmem_ld_wait();
+        const int n0 = nt * BN + c * 32;
+        if (row_ok && n0 < p.N) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {  // 4 x (8 columns = 16 bytes)
+            if (n0 + v * 8 < p.N) {      // N is a multiple of 8
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                float f0 = __uint_as_float(r[v * 8 + 2 * e]) + bias_row;
+                float f1 = __uint_as_float(r[v * 8 + 2 * e + 1]) + bias_row;
+                if (p.bias && !p.bias_per_row) {
+                  f0 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e]);
+                  f1 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e + 1]);
+                }
+                w[e] = pack2(f0, f1);
+              }
+              asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(orow + c * 32 + v * 8), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);  // accumulator drained by this warp
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
+    // give copies and MMAs still in flight time to land before memory is released
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    if (threadIdx.x == 0) atomicExch(&g_gemm_timeout_flag, 1);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+    else
+      cudaGetLastError();
+  }
+  return fn;
+}
+
+// 3-D bf16 tensor map, 128-byte swizzle, zero fill outside the tensor.
+// dims/box are innermost first; strides (bytes) are for dims 1 and 2.
+bool make_map(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t s1, uint64_t s2,
+              uint32_t b0, uint32_t b1) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {d0, d1, d2};
+  const cuuint64_t strides[2] = {s1, s2};
+  const cuuint32_t box[3] = {b0, b1, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+template <bool A_MN>
+msla_status_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, cudaStream_t st) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel<A_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
+      cudaGetLastError();
+      return fail(MSLA_ERR_CUDA, "cannot reserve %d bytes of shared memory for the projection GEMM", SMEM_BYTES);
+    }
+    attr_done = true;
+  }
+  const long long tiles = (long long)p.batches * p.m_tiles * p.n_tiles;
+  const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+  gemm_bf16_tcgen05_kernel<A_MN><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tmA, tmB, p);
+  count_launches(1);
+  return check_launch("projection GEMM (tcgen05)");
+}
+
+}  // namespace
+
+bool project_in_bf16_supported(int C, int Cout, int N, long long ldy) {
+  return C % 8 == 0 && Cout % 8 == 0 && N % 8 == 0 && ldy % 8 == 0;
+}
+
+// y[b][n][o] = sum_c w[o][c] * x[b][c][n];  x NCHW [B, C, N], y token-major with row stride ldy.
+msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, int C, int Cout, int N, long long ldy,
+                                  cudaStream_t st) {
+  CUtensorMap tmA, tmB;
+  if (!make_map(&tmA, x, (uint64_t)N, (uint64_t)C, (uint64_t)B, (uint64_t)N * 2, (uint64_t)C * N * 2, 64, BK) ||
+      !make_map(&tmB, w, (uint64_t)C, (uint64_t)Cout, 1, (uint64_t)C * 2, (uint64_t)C * Cout * 2, BK, BN))
+    return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the input projection");
+  GemmParams p{};
+  p.M = N; p.N = Cout; p.K = C; p.batches = B;
+  p.m_tiles = (N + BM - 1) / BM; p.n_tiles = (Cout + BN - 1) / BN;
+  p.rows_per_batch = N; p.ld_out = ldy; p.bias_per_row = 0; p.n_fastest = 1;
+  p.bias = nullptr; p.out = (bf16*)y;
+  return launch<true>(tmA, tmB, p, st);
+}
+
+bool project_out_bf16_supported(int Cin, int Cout, int N) { return Cin % 8 == 0 && N % 8 == 0 && Cout >= 1; }
+
+// y[b][m][n] = sum_j w[m][j] * a[b][n][j] + bias[m];  a token-major [B, N, Cin], y NCHW [B, Cout, N].
+msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin, int Cout,
+                                   int N, cudaStream_t st) {
+  CUtensorMap tmA, tmB;
+  if (!make_map(&tmA, w, (uint64_t)Cin, (uint64_t)Cout, 1, (uint64_t)Cin * 2, (uint64_t)Cin * Cout * 2, BK, BM) ||
+      !make_map(&tmB, a, (uint64_t)Cin, (uint64_t)N, (uint64_t)B, (uint64_t)Cin * 2, (uint64_t)N * Cin * 2, BK, BN))
+    return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the output projection");
+  GemmParams p{};
+  p.M = Cout; p.N = N; p.K = Cin; p.batches = B;
+  p.m_tiles = (Cout + BM - 1) / BM; p.n_tiles = (N + BN - 1) / BN;
+  p.rows_per_batch = Cout; p.ld_out = N; p.bias_per_row = 1; p.n_fastest = 0;
+  p.bias = (const bf16*)bias; p.out = (bf16*)y;
+  return launch<false>(tmA, tmB, p, st);
+}
+
+// Non-zero once any projection GEMM of this process hit a wait time-out (synchronises the device).
+int gemm_timeout_flag() {
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, g_gemm_timeout_flag, sizeof(int)) != cudaSuccess) {
+    cudaGetLastError();
+    return -1;
+  }
+  return v;
+}
+
+}  // namespace msla

@@ -258,6 +258,7 @@ static void launch_gemm(const T* A, const T* W, const T* bias, T* D, generic::Ge
 
 static msla_status_t run_project_in(msla_dtype_t dt, const void* x, const void* w, void* y, int B,
                                     int C, int Cout, int N, long long ldy, cudaStream_t st) {
+  if (dt == MSLA_BF16 && project_in_bf16_supported(C, Cout, N, ldy)) return run_project_in_bf16(x, w, y, B, C, Cout, N, ldy, st);
   generic::GemmArgs g{(long long)C * N, 1, N, (long long)N * ldy, ldy, 1, N, Cout, C};
   if (dt == MSLA_F32) launch_gemm<float>((const float*)x, (const float*)w, nullptr, (float*)y, g, B, st);
   else launch_gemm<__nv_bfloat16>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w, nullptr, (__nv_bfloat16*)y, g, B, st);
@@ -266,6 +267,7 @@ static msla_status_t run_project_in(msla_dtype_t dt, const void* x, const void* 
 
 static msla_status_t run_project_out(msla_dtype_t dt, const void* a, const void* w, const void* bias,
                                      void* y, int B, int Cin, int Cout, int N, cudaStream_t st) {
+  if (dt == MSLA_BF16 && project_out_bf16_supported(Cin, Cout, N)) return run_project_out_bf16(a, w, bias, y, B, Cin, Cout, N, st);
   generic::GemmArgs g{(long long)N * Cin, Cin, 1, (long long)Cout * N, 1, N, N, Cout, Cin};
   if (dt == MSLA_F32) launch_gemm<float>((const float*)a, (const float*)w, (const float*)bias, (float*)y, g, B, st);
   else launch_gemm<__nv_bfloat16>((const __nv_bfloat16*)a, (const __nv_bfloat16*)w, (const __nv_bfloat16*)bias, (__nv_bfloat16*)y, g, B, st);
@@ -428,6 +430,8 @@ msla_status_t msla_forward_host(const msla_desc* desc, const void* x_host, const
 }
 
 unsigned long long msla_kernel_launches(void) { return g_launches; }
+
+int msla_debug_wait_timeouts(void) { return gemm_timeout_flag(); }
 
 msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y, int B, int C, int Cout, int N, void* stream) {
   if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");

@@ -89,7 +89,9 @@ def _tok_major(a):      # [B, C, H, W] -> [B, H*W, C]
     return np.ascontiguousarray(a.reshape(B, C, -1).transpose(0, 2, 1))
 
 
-@pytest.mark.parametrize("dtype,B,C,Cout,N", [("f32", 2, 24, 40, 100), ("bf16", 1, 64, 192, 333), ("bf16", 2, 256, 768, 4096)])
+@pytest.mark.parametrize("dtype,B,C,Cout,N", [("f32", 2, 24, 40, 100), ("bf16", 1, 64, 192, 333), ("bf16", 2, 256, 768, 4096),
+                                              ("bf16", 1, 64, 192, 128), ("bf16", 3, 72, 200, 1000), ("bf16", 1, 192, 576, 8192),
+                                              ("bf16", 2, 8, 8, 8)])
 def test_stage_project_in(dtype, B, C, Cout, N):
     x = inputs.quantise(inputs.normal(1, 0, B * C * N).reshape(B, C, N), dtype)
     w = inputs.quantise(inputs.normal(1, 1, Cout * C, C ** -0.5).reshape(Cout, C), dtype)
@@ -98,9 +100,12 @@ def test_stage_project_in(dtype, B, C, Cout, N):
     torch.cuda.synchronize()
     ref = _tok_major(oracle.conv1x1(x[..., None], w))
     util.assert_close(util.host(y), ref, dtype, "project_in")
+    assert binding.msla_debug_wait_timeouts() == 0
 
 
-@pytest.mark.parametrize("dtype,B,Cin,Cout,N", [("f32", 2, 24, 40, 100), ("bf16", 1, 128, 64, 333), ("bf16", 2, 512, 256, 4096)])
+@pytest.mark.parametrize("dtype,B,Cin,Cout,N", [("f32", 2, 24, 40, 100), ("bf16", 1, 128, 64, 333), ("bf16", 2, 512, 256, 4096),
+                                                ("bf16", 1, 128, 64, 256), ("bf16", 3, 136, 200, 1000), ("bf16", 1, 384, 192, 8192),
+                                                ("bf16", 2, 8, 8, 8)])
 def test_stage_project_out(dtype, B, Cin, Cout, N):
     a = inputs.quantise(inputs.normal(2, 0, B * N * Cin).reshape(B, N, Cin), dtype)
     w = inputs.quantise(inputs.normal(2, 1, Cout * Cin, Cin ** -0.5).reshape(Cout, Cin), dtype)
@@ -110,6 +115,7 @@ def test_stage_project_out(dtype, B, Cin, Cout, N):
     torch.cuda.synchronize()
     ref = oracle.conv1x1(np.ascontiguousarray(a.transpose(0, 2, 1)), w, bias)
     util.assert_close(util.host(y), ref, dtype, "project_out")
+    assert binding.msla_debug_wait_timeouts() == 0
 
 
 @pytest.mark.parametrize("dtype,B,H,W,Ch,d", [("f32", 1, 6, 9, 48, 16), ("bf16", 2, 13, 21, 96, 32), ("bf16", 1, 1, 5, 32, 32),
