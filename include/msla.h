@@ -153,8 +153,7 @@ typedef struct {
 size_t msla_forward_workspace_bytes(const msla_desc* desc);
 
 /* x: device [B, C, H, W]; out: device [B, C_out, H, W]; both of desc->dtype.
- * C, 3C' and 2C' must be multiples of 8 so that every row of the internal
- * token-major buffers starts on a 16-byte boundary. */
+ * C and C_out must be multiples of 8. */
 msla_status_t msla_forward(const msla_desc* desc, const void* x, const msla_weights* weights,
                            void* out, void* stream);
 
@@ -190,15 +189,19 @@ unsigned long long msla_kernel_launches(void);
  * 0 if not, -1 if the flag could not be read. */
 int msla_debug_wait_timeouts(void);
 
-/* Stage entry points (the module's steps 1, 2 and 5 on their own), exposed so
- * that each kernel can be checked and timed in isolation.  Internal
- * activations are token-major: act[b][n][channel].
- *   msla_project_in : x [B, C, N] (NCHW) , w [Cout, C]        -> y [B, N, Cout]
- *   msla_aggregate  : t [B, H*W, Ch], w_dw [Ch,5,5], w_pw [Ch,d] -> y [B, H*W, Ch]
- *   msla_project_out: a [B, N, Cin], w [Cout, Cin], bias|NULL  -> y [B, Cout, N] (NCHW)
+/* Stage entry points (the module's steps 1, 2 and 5 of Section 3.1 on their
+ * own), exposed so that each kernel can be checked and timed in isolation.
+ * Between the steps the library keeps activations "planar": channels are cut
+ * into groups of d (one group = the q, k or v of one head, which is also one
+ * group of the aggregation's 1x1 group convolution), each group a dense
+ * [N][d] matrix: act[b][group][n][i], channel = group*d + i.
+ *   msla_project_in : x [B, C, N] (NCHW), w [Cout, C]              -> y [B, Cout/d, N, d]
+ *   msla_aggregate  : t [B, Ch/d, H*W, d], w_dw [Ch,5,5], w_pw [Ch,d] -> y [B, Ch/d, H*W, d]
+ *   msla_project_out: a [B, N, Cin] (token-major), w [Cout, Cin], bias [Cout]|NULL -> y [B, Cout, N] (NCHW)
+ * d must be 16 or 32 and divide Cout / Ch.
  */
 msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y,
-                              int B, int C, int Cout, int N, void* stream);
+                              int B, int C, int Cout, int N, int d, void* stream);
 msla_status_t msla_aggregate(msla_dtype_t dtype, const void* t, const void* w_dw, const void* w_pw,
                              void* y, int B, int H, int W, int Ch, int d, void* stream);
 msla_status_t msla_project_out(msla_dtype_t dtype, const void* a, const void* w, const void* bias,

@@ -4,7 +4,9 @@
 // fp32 accumulators in tensor memory, tcgen05.ld epilogue.
 //
 //   D[m][n] = sum_k A[m][k] * B[n][k] (+ bias),   fp32 accumulate, bf16 out,
-//   out[(batch * rows_per_batch + m) * ld_out + n]   (n contiguous)
+//   out[batch * out_batch_stride + m * ld_out + n]                     (group == 0), or
+//   out[batch * out_batch_stride + ((n / group) * M + m) * group + n % group]
+//   (columns split into planes of `group` channels, each plane [M][group])
 //
 // Input projection : m = token, n = output channel; A = x taken straight from
 //                    NCHW (the token index is contiguous: an "MN-major" operand),
@@ -45,8 +47,9 @@ struct GemmParams {
   int M, N, K;            // per batch
   int batches;
   int m_tiles, n_tiles;   // per batch
-  int rows_per_batch;     // output rows between consecutive batches
-  long long ld_out;       // output row stride (elements)
+  long long out_batch_stride;  // elements between consecutive batches of the output
+  long long ld_out;       // output row stride (elements) when group == 0
+  int group;              // 0, or channels per output plane (16 or 32)
   int bias_per_row;       // 1: bias[m], 0: bias[n] (ignored when bias == nullptr)
   int n_fastest;          // tile order: 1 = consecutive tiles share the A tile, 0 = share the B tile
   const bf16* bias;
@@ -252,7 +255,8 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
       tc_fence_after();
       const int m = mt * BM + quarter * 32 + lane;
       const bool row_ok = m < p.M;
-      bf16* orow = p.out + ((long long)b * p.rows_per_batch + m) * p.ld_out + (long long)nt * BN;
+      bf16* obase = p.out + (long long)b * p.out_batch_stride;
+      bf16* orow = obase + (long long)m * p.ld_out + (long long)nt * BN;  // group == 0
       const float bias_row = (p.bias && p.bias_per_row && row_ok) ? __bfloat162float(p.bias[m]) : 0.f;
       const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll 1
@@ -276,7 +280,10 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 }
                 w[e] = pack2(f0, f1);
               }
-              asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(orow + c * 32 + v * 8), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+              const int n = n0 + v * 8;
+              bf16* dst = p.group ? obase + ((long long)(n / p.group) * p.M + m) * p.group + n % p.group
+                                  : orow + c * 32 + v * 8;
+              asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
             }
           }
         }
@@ -365,13 +372,13 @@ msla_status_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmP
 
 }  // namespace
 
-bool project_in_bf16_supported(int C, int Cout, int N, long long ldy) {
-  return C % 8 == 0 && Cout % 8 == 0 && N % 8 == 0 && ldy % 8 == 0;
+bool project_in_bf16_supported(int C, int Cout, int N, int d) {
+  return C % 8 == 0 && Cout % 8 == 0 && N % 8 == 0 && (d == 16 || d == 32) && Cout % d == 0;
 }
 
-// y[b][n][o] = sum_c w[o][c] * x[b][c][n];  x NCHW [B, C, N], y token-major with row stride ldy.
-msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, int C, int Cout, int N, long long ldy,
-                                  cudaStream_t st) {
+// y[b][o / d][n][o % d] = sum_c w[o][c] * x[b][c][n];  x NCHW [B, C, N], y planar with batch stride y_sb.
+msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d,
+                                  long long y_sb, cudaStream_t st) {
   CUtensorMap tmA, tmB;
   if (!make_map(&tmA, x, (uint64_t)N, (uint64_t)C, (uint64_t)B, (uint64_t)N * 2, (uint64_t)C * N * 2, 64, BK) ||
       !make_map(&tmB, w, (uint64_t)C, (uint64_t)Cout, 1, (uint64_t)C * 2, (uint64_t)C * Cout * 2, BK, BN))
@@ -379,7 +386,7 @@ msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, 
   GemmParams p{};
   p.M = N; p.N = Cout; p.K = C; p.batches = B;
   p.m_tiles = (N + BM - 1) / BM; p.n_tiles = (Cout + BN - 1) / BN;
-  p.rows_per_batch = N; p.ld_out = ldy; p.bias_per_row = 0; p.n_fastest = 1;
+  p.out_batch_stride = y_sb; p.ld_out = 0; p.group = d; p.bias_per_row = 0; p.n_fastest = 1;
   p.bias = nullptr; p.out = (bf16*)y;
   return launch<true>(tmA, tmB, p, st);
 }
@@ -396,7 +403,7 @@ msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bia
   GemmParams p{};
   p.M = Cout; p.N = N; p.K = Cin; p.batches = B;
   p.m_tiles = (Cout + BM - 1) / BM; p.n_tiles = (N + BN - 1) / BN;
-  p.rows_per_batch = Cout; p.ld_out = N; p.bias_per_row = 1; p.n_fastest = 0;
+  p.out_batch_stride = (long long)Cout * N; p.ld_out = N; p.group = 0; p.bias_per_row = 1; p.n_fastest = 0;
   p.bias = (const bf16*)bias; p.out = (bf16*)y;
   return launch<false>(tmA, tmB, p, st);
 }

@@ -13,12 +13,15 @@ namespace generic {
 // Strided GEMM for the two 1x1 projections (Section 3.1: Q = xW_Q, K = xW_K,
 // V = xW_V; final linear projection):
 //   D(m, n) = sum_k A(m, k) * W[n, k] (+ bias[n]),   m = token, n = out channel
-// A(m, k) = A[b*sAb + m*sAm + k*sAk];  D(m, n) = D[b*sDb + m*sDm + n*sDn].
+// A(m, k) = A[b*sAb + m*sAm + k*sAk];
+// D(m, n) = D[b*sDb + (n / group)*sDg + m*sDm + (n % group)*sDn]: out channels
+// may be split into groups of `group` that live in separate planes.
 // ---------------------------------------------------------------------------
 struct GemmArgs {
   long long sAb, sAm, sAk;
-  long long sDb, sDm, sDn;
+  long long sDb, sDm, sDn, sDg;
   int M, Nc, K;  // tokens, out channels, in channels
+  int group;     // out channels per plane (>= Nc: one plane)
 };
 
 template <typename T>
@@ -80,7 +83,7 @@ gemm_kernel(const T* __restrict__ A, const T* __restrict__ Wt, const T* __restri
       const int n = n0 + ni + j;
       if (n >= g.Nc) continue;
       const float r = acc[i][j] + (bias ? to_f32(bias[n]) : 0.f);
-      Db[m * g.sDm + (long long)n * g.sDn] = from_f32<T>(r);
+      Db[(long long)(n / g.group) * g.sDg + m * g.sDm + (long long)(n % g.group) * g.sDn] = from_f32<T>(r);
     }
   }
 }
@@ -88,14 +91,14 @@ gemm_kernel(const T* __restrict__ A, const T* __restrict__ Wt, const T* __restri
 // ---------------------------------------------------------------------------
 // Multi-scale token aggregation (Section 3.1): 5x5 depthwise convolution
 // (cross-correlation, zero padding 2) followed by the grouped 1x1 convolution,
-// on token-major activations.  One CTA = one 8x8 pixel tile of one group of d
-// channels.  src(b, n, ch) = src[b*sb + n*ld + ch]; dst likewise.
+// on planar activations [B, groups, H*W, d].  One CTA = one 8x8 pixel tile of
+// one group of d channels.  src(b, g, n, i) = src[b*src_sb + (g*H*W + n)*d + i];
+// dst likewise with dst_sb.
 // ---------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256)
 aggregate_kernel(const T* __restrict__ src, const T* __restrict__ w_dw, const T* __restrict__ w_pw,
-                 T* __restrict__ dst, int H, int W, int d, long long src_sb, long long src_ld,
-                 long long dst_sb, long long dst_ld) {
+                 T* __restrict__ dst, int H, int W, int d, long long src_sb, long long dst_sb) {
   constexpr int TS = 8, HALO = TS + 4, DMAX = 32;
   __shared__ float tile[HALO * HALO][DMAX + 1];
   __shared__ float dwo[TS * TS][DMAX + 1];
@@ -106,14 +109,14 @@ aggregate_kernel(const T* __restrict__ src, const T* __restrict__ w_dw, const T*
   const int x0 = (blockIdx.x % tiles_x) * TS, y0 = (blockIdx.x / tiles_x) * TS;
   const int ch0 = blockIdx.y * d;
   const int b = blockIdx.z;
-  const T* sb = src + (long long)b * src_sb;
+  const T* sb = src + (long long)b * src_sb + (long long)blockIdx.y * H * W * d;
   for (int e = tid; e < d * 25; e += 256) wdw[e / 25][e % 25] = to_f32(w_dw[(long long)ch0 * 25 + e]);
   for (int e = tid; e < d * d; e += 256) wpw[e / d][e % d] = to_f32(w_pw[(long long)ch0 * d + e]);
   for (int e = tid; e < HALO * HALO * d; e += 256) {
     const int c = e % d, p = e / d;
     const int yy = y0 + p / HALO - 2, xx = x0 + p % HALO - 2;
     float v = 0.f;
-    if (yy >= 0 && yy < H && xx >= 0 && xx < W) v = to_f32(sb[((long long)yy * W + xx) * src_ld + ch0 + c]);
+    if (yy >= 0 && yy < H && xx >= 0 && xx < W) v = to_f32(sb[((long long)yy * W + xx) * d + c]);
     tile[p][c] = v;
   }
   __syncthreads();
@@ -129,14 +132,14 @@ aggregate_kernel(const T* __restrict__ src, const T* __restrict__ w_dw, const T*
     dwo[p][c] = acc;
   }
   __syncthreads();
-  T* db = dst + (long long)b * dst_sb;
+  T* db = dst + (long long)b * dst_sb + (long long)blockIdx.y * H * W * d;
   for (int e = tid; e < TS * TS * d; e += 256) {
     const int o = e % d, p = e / d;
     const int yy = y0 + p / TS, xx = x0 + p % TS;
     if (yy >= H || xx >= W) continue;
     float acc = 0.f;
     for (int i = 0; i < d; ++i) acc = fmaf(wpw[o][i], dwo[p][i], acc);
-    db[((long long)yy * W + xx) * dst_ld + ch0 + o] = from_f32<T>(acc);
+    db[((long long)yy * W + xx) * d + o] = from_f32<T>(acc);
   }
 }
 

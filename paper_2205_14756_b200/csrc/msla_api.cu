@@ -256,10 +256,11 @@ static void launch_gemm(const T* A, const T* W, const T* bias, T* D, generic::Ge
   count_launches(1);
 }
 
+// y planar: y[b*y_sb + ((o/d)*N + n)*d + o%d]
 static msla_status_t run_project_in(msla_dtype_t dt, const void* x, const void* w, void* y, int B,
-                                    int C, int Cout, int N, long long ldy, cudaStream_t st) {
-  if (dt == MSLA_BF16 && project_in_bf16_supported(C, Cout, N, ldy)) return run_project_in_bf16(x, w, y, B, C, Cout, N, ldy, st);
-  generic::GemmArgs g{(long long)C * N, 1, N, (long long)N * ldy, ldy, 1, N, Cout, C};
+                                    int C, int Cout, int N, int d, long long y_sb, cudaStream_t st) {
+  if (dt == MSLA_BF16 && project_in_bf16_supported(C, Cout, N, d)) return run_project_in_bf16(x, w, y, B, C, Cout, N, d, y_sb, st);
+  generic::GemmArgs g{(long long)C * N, 1, N, y_sb, d, 1, (long long)N * d, N, Cout, C, d};
   if (dt == MSLA_F32) launch_gemm<float>((const float*)x, (const float*)w, nullptr, (float*)y, g, B, st);
   else launch_gemm<__nv_bfloat16>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w, nullptr, (__nv_bfloat16*)y, g, B, st);
   return check_launch("input projection");
@@ -268,24 +269,24 @@ static msla_status_t run_project_in(msla_dtype_t dt, const void* x, const void* 
 static msla_status_t run_project_out(msla_dtype_t dt, const void* a, const void* w, const void* bias,
                                      void* y, int B, int Cin, int Cout, int N, cudaStream_t st) {
   if (dt == MSLA_BF16 && project_out_bf16_supported(Cin, Cout, N)) return run_project_out_bf16(a, w, bias, y, B, Cin, Cout, N, st);
-  generic::GemmArgs g{(long long)N * Cin, Cin, 1, (long long)Cout * N, 1, N, N, Cout, Cin};
+  generic::GemmArgs g{(long long)N * Cin, Cin, 1, (long long)Cout * N, 1, N, 0, N, Cout, Cin, Cout};
   if (dt == MSLA_F32) launch_gemm<float>((const float*)a, (const float*)w, (const float*)bias, (float*)y, g, B, st);
   else launch_gemm<__nv_bfloat16>((const __nv_bfloat16*)a, (const __nv_bfloat16*)w, (const __nv_bfloat16*)bias, (__nv_bfloat16*)y, g, B, st);
   return check_launch("output projection");
 }
 
+// src, dst planar [B, Ch/d, H*W, d] with batch strides src_sb, dst_sb (elements)
 static msla_status_t run_aggregate(msla_dtype_t dt, const void* src, const void* w_dw, const void* w_pw,
-                                   void* dst, int B, int H, int W, int Ch, int d, long long src_ld,
-                                   long long dst_ld, cudaStream_t st) {
-  const long long N = (long long)H * W;
+                                   void* dst, int B, int H, int W, int Ch, int d, long long src_sb,
+                                   long long dst_sb, cudaStream_t st) {
   dim3 grid((unsigned)(ceil_div_ll(W, 8) * ceil_div_ll(H, 8)), (unsigned)(Ch / d), (unsigned)B);
   if (dt == MSLA_F32)
     generic::aggregate_kernel<float><<<grid, 256, 0, st>>>((const float*)src, (const float*)w_dw, (const float*)w_pw,
-                                                           (float*)dst, H, W, d, N * src_ld, src_ld, N * dst_ld, dst_ld);
+                                                           (float*)dst, H, W, d, src_sb, dst_sb);
   else
     generic::aggregate_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)src, (const __nv_bfloat16*)w_dw,
                                                                    (const __nv_bfloat16*)w_pw, (__nv_bfloat16*)dst, H, W, d,
-                                                                   N * src_ld, src_ld, N * dst_ld, dst_ld);
+                                                                   src_sb, dst_sb);
   count_launches(1);
   return check_launch("token aggregation");
 }
@@ -335,22 +336,25 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
     }
   }
   const int Cp = p.Cp, N = p.N, d = desc->d, heads = desc->heads;
-  const long long ld_ms = 6LL * Cp, ld_att = 2LL * Cp;
-  char* ms = ws + p.ms_off;    // [B, N, 6C']: channels [0,3C') = qkv, [3C',6C') = aggregated
-  char* att = ws + p.att_off;  // [B, N, 2C']
+  const long long ld_att = 2LL * Cp;
+  const long long ms_sb = 6LL * Cp * N;  // elements per image of the multi-scale buffer
+  // ms: planar [B][6*heads planes][N][d]; plane (s*heads + h)*3 + t holds q (t=0), k (1) or v (2)
+  // of head h at scale s (0: projected tokens, 1: aggregated tokens).
+  char* ms = ws + p.ms_off;
+  char* att = ws + p.att_off;  // [B, N, 2C'] token-major head concat
   if ((s = record(events, 0, st)) != MSLA_OK) return s;
-  // 1. QKV projection into the first half of every multi-scale row
-  s = run_project_in(desc->dtype, x_dev, w->w_qkv, ms, desc->B, desc->C, 3 * Cp, N, ld_ms, st);
+  // 1. QKV projection into the scale-0 planes
+  s = run_project_in(desc->dtype, x_dev, w->w_qkv, ms, desc->B, desc->C, 3 * Cp, N, d, ms_sb, st);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 1, st)) != MSLA_OK) return s;
-  // 2. aggregation into the second half
-  s = run_aggregate(desc->dtype, ms, w->w_dw, w->w_pw, ms + 3 * Cp * e, desc->B, desc->H, desc->W, 3 * Cp, d, ld_ms, ld_ms, st);
+  // 2. aggregation of every scale-0 plane into the matching scale-1 plane
+  s = run_aggregate(desc->dtype, ms, w->w_dw, w->w_pw, ms + (size_t)3 * Cp * N * e, desc->B, desc->H, desc->W, 3 * Cp, d, ms_sb, ms_sb, st);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 2, st)) != MSLA_OK) return s;
   // 3+4. attention over 2*heads heads of [q|k|v]; outputs land at channel head*d (concat)
-  const HeadView in{(long long)N * ld_ms, 3LL * d, ld_ms};
+  const HeadView in{ms_sb, 3LL * N * d, d};
   const HeadView ov{(long long)N * ld_att, d, ld_att};
-  s = run_core(desc->dtype, ms, ms + d * e, ms + 2 * d * e, att, in, ov, desc->B, 2 * heads, N, d, desc->eps, p.core,
+  s = run_core(desc->dtype, ms, ms + (size_t)N * d * e, ms + (size_t)2 * N * d * e, att, in, ov, desc->B, 2 * heads, N, d, desc->eps, p.core,
                ws + p.core_off, st, events ? (cudaEvent_t)events[3] : nullptr);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 4, st)) != MSLA_OK) return s;
@@ -433,15 +437,17 @@ unsigned long long msla_kernel_launches(void) { return g_launches; }
 
 int msla_debug_wait_timeouts(void) { return gemm_timeout_flag(); }
 
-msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y, int B, int C, int Cout, int N, void* stream) {
+msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d, void* stream) {
   if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");
   if (!x || !w || !y) return fail(MSLA_ERR_INVALID_ARG, "null pointer");
   if (B < 1 || C < 1 || Cout < 1 || N < 1 || B > 65535) return fail(MSLA_ERR_INVALID_ARG, "sizes must be positive (B <= 65535)");
   if (C % 8 || Cout % 8) return fail(MSLA_ERR_UNSUPPORTED, "C and Cout must be multiples of 8");
+  if (d != 16 && d != 32) return fail(MSLA_ERR_UNSUPPORTED, "d = %d; only 16 and 32 are supported", d);
+  if (Cout % d) return fail(MSLA_ERR_INVALID_ARG, "Cout must be a multiple of d");
   if (!aligned16(x) || !aligned16(w) || !aligned16(y)) return fail(MSLA_ERR_ALIGNMENT, "pointers must be 16-byte aligned");
   msla_status_t s = check_arch();
   if (s != MSLA_OK) return s;
-  return run_project_in(dtype, x, w, y, B, C, Cout, N, Cout, (cudaStream_t)stream);
+  return run_project_in(dtype, x, w, y, B, C, Cout, N, d, (long long)Cout * N, (cudaStream_t)stream);
 }
 
 msla_status_t msla_aggregate(msla_dtype_t dtype, const void* t, const void* w_dw, const void* w_pw, void* y, int B, int H, int W, int Ch, int d, void* stream) {
@@ -457,7 +463,7 @@ msla_status_t msla_aggregate(msla_dtype_t dtype, const void* t, const void* w_dw
   if (overlaps(t, bytes, y, bytes)) return fail(MSLA_ERR_INVALID_ARG, "y overlaps t");
   msla_status_t s = check_arch();
   if (s != MSLA_OK) return s;
-  return run_aggregate(dtype, t, w_dw, w_pw, y, B, H, W, Ch, d, Ch, Ch, (cudaStream_t)stream);
+  return run_aggregate(dtype, t, w_dw, w_pw, y, B, H, W, Ch, d, (long long)Ch * H * W, (long long)Ch * H * W, (cudaStream_t)stream);
 }
 
 msla_status_t msla_project_out(msla_dtype_t dtype, const void* a, const void* w, const void* bias, void* y, int B, int Cin, int Cout, int N, void* stream) {

@@ -34,9 +34,9 @@ msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* o
                             cudaEvent_t mid);
 
 // bf16 projections on tcgen05 tensor cores (gemm_tcgen05.cu).
-bool project_in_bf16_supported(int C, int Cout, int N, long long ldy);
-msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, int C, int Cout, int N, long long ldy,
-                                  cudaStream_t st);
+bool project_in_bf16_supported(int C, int Cout, int N, int d);
+msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d,
+                                  long long y_batch_stride, cudaStream_t st);
 bool project_out_bf16_supported(int Cin, int Cout, int N);
 msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin, int Cout,
                                    int N, cudaStream_t st);

@@ -89,16 +89,22 @@ def _tok_major(a):      # [B, C, H, W] -> [B, H*W, C]
     return np.ascontiguousarray(a.reshape(B, C, -1).transpose(0, 2, 1))
 
 
-@pytest.mark.parametrize("dtype,B,C,Cout,N", [("f32", 2, 24, 40, 100), ("bf16", 1, 64, 192, 333), ("bf16", 2, 256, 768, 4096),
-                                              ("bf16", 1, 64, 192, 128), ("bf16", 3, 72, 200, 1000), ("bf16", 1, 192, 576, 8192),
-                                              ("bf16", 2, 8, 8, 8)])
+def _planar(a, d):      # [B, C, H, W] -> [B, C/d, H*W, d]
+    B, C = a.shape[:2]
+    return np.ascontiguousarray(a.reshape(B, C // d, d, -1).transpose(0, 1, 3, 2))
+
+
+@pytest.mark.parametrize("dtype,B,C,Cout,N", [("f32", 2, 24, 48, 100), ("bf16", 1, 64, 192, 333), ("bf16", 2, 256, 768, 4096),
+                                              ("bf16", 1, 64, 192, 128), ("bf16", 3, 72, 208, 1000), ("bf16", 1, 192, 576, 8192),
+                                              ("bf16", 2, 8, 16, 8)])
 def test_stage_project_in(dtype, B, C, Cout, N):
+    d = 32 if Cout % 32 == 0 else 16 if Cout % 16 == 0 else 8
     x = inputs.quantise(inputs.normal(1, 0, B * C * N).reshape(B, C, N), dtype)
     w = inputs.quantise(inputs.normal(1, 1, Cout * C, C ** -0.5).reshape(Cout, C), dtype)
-    y = torch.empty(B, N, Cout, dtype=util.TORCH_DTYPE[dtype], device="cuda")
-    binding.msla_project_in(util.CODE[dtype], util.dev(x, dtype), util.dev(w, dtype), y, B, C, Cout, N)
+    y = torch.empty(B, Cout // d, N, d, dtype=util.TORCH_DTYPE[dtype], device="cuda")
+    binding.msla_project_in(util.CODE[dtype], util.dev(x, dtype), util.dev(w, dtype), y, B, C, Cout, N, d)
     torch.cuda.synchronize()
-    ref = _tok_major(oracle.conv1x1(x[..., None], w))
+    ref = _planar(oracle.conv1x1(x[..., None], w), d)
     util.assert_close(util.host(y), ref, dtype, "project_in")
     assert binding.msla_debug_wait_timeouts() == 0
 
@@ -124,8 +130,8 @@ def test_stage_aggregate(dtype, B, H, W, Ch, d):
     t = inputs.quantise(inputs.normal(3, 0, B * Ch * H * W).reshape(B, Ch, H, W), dtype)
     w_dw = inputs.quantise(inputs.normal(3, 1, Ch * 25, 0.2).reshape(Ch, 5, 5), dtype)
     w_pw = inputs.quantise(inputs.normal(3, 2, Ch * d, d ** -0.5).reshape(Ch, d), dtype)
-    y = torch.empty(B, H * W, Ch, dtype=util.TORCH_DTYPE[dtype], device="cuda")
-    binding.msla_aggregate(util.CODE[dtype], util.dev(_tok_major(t), dtype), util.dev(w_dw, dtype), util.dev(w_pw, dtype), y, B, H, W, Ch, d)
+    y = torch.empty(B, Ch // d, H * W, d, dtype=util.TORCH_DTYPE[dtype], device="cuda")
+    binding.msla_aggregate(util.CODE[dtype], util.dev(_planar(t, d), dtype), util.dev(w_dw, dtype), util.dev(w_pw, dtype), y, B, H, W, Ch, d)
     torch.cuda.synchronize()
-    ref = _tok_major(oracle.group1x1(oracle.dwconv(t, w_dw), w_pw))
+    ref = _planar(oracle.group1x1(oracle.dwconv(t, w_dw), w_pw), d)
     util.assert_close(util.host(y), ref, dtype, "aggregate")
