@@ -1,0 +1,241 @@
+// Fused multi-scale token aggregation for bf16, d = 32 (Section 3.1): the 5x5
+// depthwise convolution and the grouped 1x1 convolution of one group of 32
+// channels in one kernel, on planar activations [planes][H*W][32].
+//
+// One CTA = one TW x TH pixel tile of one group.  A single TMA copy stages the
+// (TW+4) x (TH+4) halo tile in shared memory; coordinates outside the image are
+// zero-filled by the TMA unit, which is exactly the convolution's zero padding.
+// Each warp owns an 8x8 pixel block: lane (g = lane/4, t = lane%4) computes the
+// depthwise result of the 8 pixels of column g for channels 8t..8t+7 in fp32
+// registers (packed two-wide FMAs, sliding the 5-tap window down the column),
+// rounds it once to bf16 and uses it, in place, as the A operand of
+// mma.sync.m16n8k16 against the group's 32x32 pointwise weights: the grouped
+// 1x1 is fed from registers, with no shared-memory round trip in between.
+#include <cuda.h>
+
+#include "msla_common.cuh"
+#include "msla_host.h"
+#include "tma_host.h"
+
+#ifndef MSLA_AGG_WX
+#define MSLA_AGG_WX 2  // warps along x (8 pixels each)
+#endif
+#ifndef MSLA_AGG_WY
+#define MSLA_AGG_WY 2  // warps along y
+#endif
+
+namespace msla {
+namespace {
+
+using bf16 = __nv_bfloat16;
+constexpr int D = 32;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;
+
+__device__ int g_agg_timeout_flag = 0;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void fma2(float2& acc, const float2& a, const float2& b) {
+  unsigned long long& c = reinterpret_cast<unsigned long long&>(acc);
+  asm("fma.rn.f32x2 %0, %1, %2, %0;"
+      : "+l"(c)
+      : "l"(reinterpret_cast<const unsigned long long&>(a)), "l"(reinterpret_cast<const unsigned long long&>(b)));
+}
+__device__ __forceinline__ float2 unpack_bf16x2(uint32_t v) {  // exact widening
+  return make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+struct AggParams {
+  const bf16* w_dw;  // [Ch][5][5]
+  const bf16* w_pw;  // [Ch][32]
+  bf16* dst;         // planar output
+  long long dst_batch_stride;  // elements
+  int src_planes_per_batch;    // plane index of (b, group) in the tensor map = b * this + group
+  int H, W;
+  int tiles_x;
+};
+
+template <int WX, int WY>
+__global__ void __launch_bounds__(WX * WY * 32)
+aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
+  constexpr int TW = 8 * WX, TH = 8 * WY, HW_ = TW + 4, HH = TH + 4;
+  constexpr int TILE_BYTES = HW_ * HH * D * 2;
+  __shared__ __align__(128) unsigned char tile[TILE_BYTES];
+  __shared__ __align__(16) float wdw_s[5][5][D];  // [dx][dy][channel]
+  __shared__ __align__(8) unsigned long long bar_storage;
+  __shared__ int timed_out;
+
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  const int wx = warp % WX, wy = warp / WX;
+  const int x0 = (blockIdx.x % p.tiles_x) * TW, y0 = (blockIdx.x / p.tiles_x) * TH;
+  const int group = blockIdx.y, b = blockIdx.z;
+  const int ch0 = group * D;
+  const uint32_t bar = smem_u32(&bar_storage);
+
+  if (threadIdx.x == 0) {
+    timed_out = 0;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(TILE_BYTES) : "memory");
+    // x and y may start at -2 (and run past W, H): those pixels read as zero.
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(tile)), "l"(&tm_src), "r"(bar), "r"(0), "r"(x0 - 2), "r"(y0 - 2),
+          "r"(b * p.src_planes_per_batch + group) : "memory");
+  }
+  // depthwise taps -> fp32 [dx][dy][c] while the copy is in flight
+  for (int e = threadIdx.x; e < 25 * D; e += WX * WY * 32) {
+    const int c = e / 25, tap = e % 25;
+    wdw_s[tap % 5][tap / 5][c] = __bfloat162float(p.w_dw[(long long)(ch0 + c) * 25 + tap]);
+  }
+  // pointwise weights as B fragments: slots (2t,2t+1)+8r <-> in channels 8t+4ks+2r,+1; column g <-> out channel oc(jn)
+  uint32_t bw[2][4][2];
+#pragma unroll
+  for (int ks = 0; ks < 2; ++ks)
+#pragma unroll
+    for (int jn = 0; jn < 4; ++jn)
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int oc = 8 * (g >> 1) + 2 * jn + (g & 1);
+        bw[ks][jn][r] = *reinterpret_cast<const uint32_t*>(p.w_pw + (long long)(ch0 + oc) * D + 8 * t + 4 * ks + 2 * r);
+      }
+  __syncthreads();  // barrier initialised and taps staged before anyone proceeds
+
+  {  // bounded wait for the halo tile
+    uint32_t ok = 0;
+    const long long t_start = clock64();
+    while (true) {
+      asm volatile(
+          "{\n\t.reg .pred P1;\n\tmbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\tselp.b32 %0, 1, 0, P1;\n\t}"
+          : "=r"(ok) : "r"(bar), "r"(0) : "memory");
+      if (ok) break;
+      if (clock64() - t_start > WAIT_LIMIT_CYCLES) { timed_out = 1; break; }
+    }
+  }
+  __syncthreads();
+  if (timed_out) {  // leave without touching the output; the copy had two seconds to land
+    if (threadIdx.x == 0) atomicExch(&g_agg_timeout_flag, 1);
+    return;
+  }
+
+  // ---- depthwise 5x5: column (wx*8 + g), rows wy*8 .. +7, channels 8t .. 8t+7
+  float2 acc[8][4];
+#pragma unroll
+  for (int r = 0; r < 8; ++r)
+#pragma unroll
+    for (int q = 0; q < 4; ++q) acc[r][q] = make_float2(0.f, 0.f);
+  const uint32_t col_base = smem_u32(tile) + (uint32_t)(((wy * 8) * HW_ + wx * 8 + g) * (D * 2) + t * 16);
+#pragma unroll 1
+  for (int dx = 0; dx < 5; ++dx) {
+    float2 w[5][4];
+#pragma unroll
+    for (int dy = 0; dy < 5; ++dy) {
+      const float4 lo = *reinterpret_cast<const float4*>(&wdw_s[dx][dy][8 * t]);
+      const float4 hi = *reinterpret_cast<const float4*>(&wdw_s[dx][dy][8 * t + 4]);
+      w[dy][0] = make_float2(lo.x, lo.y); w[dy][1] = make_float2(lo.z, lo.w);
+      w[dy][2] = make_float2(hi.x, hi.y); w[dy][3] = make_float2(hi.z, hi.w);
+    }
+#pragma unroll
+    for (int i = 0; i < 12; ++i) {  // input row i of the column feeds output rows i-4 .. i
+      uint32_t raw[4];
+      asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                   : "=r"(raw[0]), "=r"(raw[1]), "=r"(raw[2]), "=r"(raw[3])
+                   : "r"(col_base + (uint32_t)((i * HW_ + dx) * (D * 2))));
+      float2 in[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) in[q] = unpack_bf16x2(raw[q]);
+#pragma unroll
+      for (int dy = 0; dy < 5; ++dy) {
+        const int r = i - dy;
+        if (r >= 0 && r < 8) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) fma2(acc[r][q], w[dy][q], in[q]);
+        }
+      }
+    }
+  }
+
+  // ---- grouped 1x1 on tensor cores, straight from the accumulators
+  const int x = x0 + wx * 8 + g;
+  bf16* plane = p.dst + (long long)b * p.dst_batch_stride + (long long)group * p.H * p.W * D;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {  // MMA rows g / g+8 = pixels (x, 2j) / (x, 2j+1) of the warp block
+    float c[4][4];
+#pragma unroll
+    for (int jn = 0; jn < 4; ++jn)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) c[jn][e] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < 2; ++ks) {
+      const uint32_t A[4] = {pack_bf16(acc[2 * j][2 * ks].x, acc[2 * j][2 * ks].y),
+                             pack_bf16(acc[2 * j + 1][2 * ks].x, acc[2 * j + 1][2 * ks].y),
+                             pack_bf16(acc[2 * j][2 * ks + 1].x, acc[2 * j][2 * ks + 1].y),
+                             pack_bf16(acc[2 * j + 1][2 * ks + 1].x, acc[2 * j + 1][2 * ks + 1].y)};
+#pragma unroll
+      for (int jn = 0; jn < 4; ++jn) mma_bf16(c[jn], A, bw[ks][jn][0], bw[ks][jn][1]);
+    }
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const int y = y0 + wy * 8 + 2 * j + half;
+      if (x < p.W && y < p.H) {
+        bf16* dst = plane + ((long long)y * p.W + x) * D + 8 * t;
+        asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(dst),
+                     "r"(pack_bf16(c[0][2 * half], c[0][2 * half + 1])), "r"(pack_bf16(c[1][2 * half], c[1][2 * half + 1])),
+                     "r"(pack_bf16(c[2][2 * half], c[2][2 * half + 1])), "r"(pack_bf16(c[3][2 * half], c[3][2 * half + 1]))
+                     : "memory");
+      }
+    }
+  }
+}
+
+}  // namespace
+
+bool aggregate_bf16_supported(int H, int W, int Ch, int d) {
+  return d == 32 && Ch % 32 == 0 && H >= 1 && W >= 1;
+}
+
+// src, dst: planar bf16 [.., planes, H*W, 32]; group g of image b is plane b*src_ppb + g of src
+// (src_planes_total planes in all) and lives at dst + b*dst_sb + g*H*W*32.
+msla_status_t run_aggregate_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
+                                 const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch,
+                                 cudaStream_t st) {
+  constexpr int WX = MSLA_AGG_WX, WY = MSLA_AGG_WY, TW = 8 * WX, TH = 8 * WY;
+  CUtensorMap tm;
+  const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)src_planes_total};
+  const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)W * D * 2, (cuuint64_t)H * W * D * 2};
+  const cuuint32_t box[4] = {(cuuint32_t)D, (cuuint32_t)(TW + 4), (cuuint32_t)(TH + 4), 1};
+  if (!tma_make_map_bf16(&tm, src, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
+    return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the aggregation input");
+  AggParams p;
+  p.w_dw = (const bf16*)w_dw; p.w_pw = (const bf16*)w_pw; p.dst = (bf16*)dst;
+  p.dst_batch_stride = dst_sb; p.src_planes_per_batch = src_ppb; p.H = H; p.W = W;
+  p.tiles_x = (W + TW - 1) / TW;
+  const long long tiles = (long long)p.tiles_x * ((H + TH - 1) / TH);
+  if (tiles > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many aggregation tiles");
+  dim3 grid((unsigned)tiles, (unsigned)(Ch / D), (unsigned)B);
+  aggregate_bf16_kernel<WX, WY><<<grid, WX * WY * 32, 0, st>>>(tm, p);
+  count_launches(1);
+  return check_launch("token aggregation (bf16)");
+}
+
+int agg_timeout_flag() {
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, g_agg_timeout_flag, sizeof(int)) != cudaSuccess) {
+    cudaGetLastError();
+    return -1;
+  }
+  return v;
+}
+
+}  // namespace msla

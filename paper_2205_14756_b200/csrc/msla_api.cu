@@ -279,6 +279,9 @@ static msla_status_t run_project_out(msla_dtype_t dt, const void* a, const void*
 static msla_status_t run_aggregate(msla_dtype_t dt, const void* src, const void* w_dw, const void* w_pw,
                                    void* dst, int B, int H, int W, int Ch, int d, long long src_sb,
                                    long long dst_sb, cudaStream_t st) {
+  const long long plane = (long long)H * W * d;
+  if (dt == MSLA_BF16 && aggregate_bf16_supported(H, W, Ch, d) && src_sb % plane == 0)
+    return run_aggregate_bf16(src, (long long)B * (src_sb / plane), (int)(src_sb / plane), w_dw, w_pw, dst, dst_sb, B, H, W, Ch, st);
   dim3 grid((unsigned)(ceil_div_ll(W, 8) * ceil_div_ll(H, 8)), (unsigned)(Ch / d), (unsigned)B);
   if (dt == MSLA_F32)
     generic::aggregate_kernel<float><<<grid, 256, 0, st>>>((const float*)src, (const float*)w_dw, (const float*)w_pw,
@@ -435,7 +438,10 @@ msla_status_t msla_forward_host(const msla_desc* desc, const void* x_host, const
 
 unsigned long long msla_kernel_launches(void) { return g_launches; }
 
-int msla_debug_wait_timeouts(void) { return gemm_timeout_flag(); }
+int msla_debug_wait_timeouts(void) {
+  const int a = gemm_timeout_flag(), b = agg_timeout_flag();
+  return (a < 0 || b < 0) ? -1 : (a | b);
+}
 
 msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d, void* stream) {
   if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");

@@ -42,4 +42,11 @@ msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bia
                                    int N, cudaStream_t st);
 int gemm_timeout_flag();
 
+// bf16, d = 32 aggregation with TMA halo tiles (agg_bf16.cu).
+bool aggregate_bf16_supported(int H, int W, int Ch, int d);
+msla_status_t run_aggregate_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
+                                 const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch,
+                                 cudaStream_t st);
+int agg_timeout_flag();
+
 }  // namespace msla

@@ -125,7 +125,8 @@ def test_stage_project_out(dtype, B, Cin, Cout, N):
 
 
 @pytest.mark.parametrize("dtype,B,H,W,Ch,d", [("f32", 1, 6, 9, 48, 16), ("bf16", 2, 13, 21, 96, 32), ("bf16", 1, 1, 5, 32, 32),
-                                              ("bf16", 1, 64, 64, 192, 32), ("bf16", 1, 3, 70, 64, 16)])
+                                              ("bf16", 1, 64, 64, 192, 32), ("bf16", 1, 3, 70, 64, 16), ("bf16", 2, 16, 16, 32, 32),
+                                              ("bf16", 1, 17, 35, 64, 32), ("bf16", 1, 5, 3, 32, 32), ("bf16", 1, 40, 7, 32, 32)])
 def test_stage_aggregate(dtype, B, H, W, Ch, d):
     t = inputs.quantise(inputs.normal(3, 0, B * Ch * H * W).reshape(B, Ch, H, W), dtype)
     w_dw = inputs.quantise(inputs.normal(3, 1, Ch * 25, 0.2).reshape(Ch, 5, 5), dtype)
@@ -135,3 +136,4 @@ def test_stage_aggregate(dtype, B, H, W, Ch, d):
     torch.cuda.synchronize()
     ref = _planar(oracle.group1x1(oracle.dwconv(t, w_dw), w_pw), d)
     util.assert_close(util.host(y), ref, dtype, "aggregate")
+    assert binding.msla_debug_wait_timeouts() == 0
