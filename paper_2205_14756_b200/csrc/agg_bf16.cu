@@ -96,7 +96,7 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
   }
   // depthwise taps -> fp32 [dx][dy][c] while the copy is in flight
   for (int e = threadIdx.x; e < 25 * D; e += WX * WY * 32) {
-    const int c = e / 25, tap = e % 25;
+    const int c = e % D, tap = e / D;  // consecutive threads -> consecutive channels: conflict-free stores
     wdw_s[tap % 5][tap / 5][c] = __bfloat162float(p.w_dw[(long long)(ch0 + c) * 25 + tap]);
   }
   // pointwise weights as B fragments: slots (2t,2t+1)+8r <-> in channels 8t+4ks+2r,+1; column g <-> out channel oc(jn)

@@ -16,7 +16,7 @@
 //                    NCHW planes, so each thread stores runs of tokens.
 //
 // One persistent CTA per SM, warp-specialised: warp 0 issues TMA, warp 1
-// issues MMAs (and owns the tensor-memory allocation), warps 2-5 drain the
+// issues MMAs (and owns the tensor-memory allocation), warps 2-9 drain the
 // accumulators.  Two 128x256 fp32 accumulators (all 512 TMEM columns) let the
 // epilogue of one tile overlap the MMAs of the next.  Every mbarrier wait is
 // bounded: on time-out the CTA raises a flag, all roles leave their loops, the
@@ -37,7 +37,7 @@ constexpr int STAGES = 4;
 constexpr int A_STAGE_BYTES = BM * BK * 2;  // 16 KB
 constexpr int B_STAGE_BYTES = BN * BK * 2;  // 32 KB
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;  // TMA warp, MMA warp, 8 epilogue warps
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 256 + 1024;  // ring + barriers + alignment slack
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;          // ~2 s at 2 GHz
 
@@ -164,7 +164,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar + 8 * a, 1); mbar_init(tempty_bar + 8 * a, 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar + 8 * a, 1); mbar_init(tempty_bar + 8 * a, 8); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {  // whole warp: allocate all 512 tensor-memory columns (one CTA per SM)
@@ -243,7 +243,11 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     }
   } else {
     // ---------------------------------------------------------------- epilogue
-    const int quarter = warp & 3;  // a warp may only touch TMEM lanes 32*(warp%4) .. +31
+    // Eight warps: warp%4 selects the TMEM lane quarter (a hardware rule), the
+    // other bit selects which 128 of the tile's 256 columns the warp drains.
+    const int quarter = warp & 3;
+    const int col_half = (warp - 2) >> 2;
+    const int gs = p.group == 32 ? 5 : 4;  // log2(group) when the output is planar
     uint32_t local = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++local) {
@@ -257,33 +261,36 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
       const int m = mt * BM + quarter * 32 + lane;
       const bool row_ok = m < p.M;
       bf16* obase = p.out + (long long)b * p.out_batch_stride;
-      bf16* orow = obase + (long long)m * p.ld_out + (long long)nt * BN;  // group == 0
       const float bias_row = (p.bias && p.bias_per_row && row_ok) ? __bfloat162float(p.bias[m]) : 0.f;
-      const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(taddr + c * 32, r);
+      const bool bias_col = p.bias && !p.bias_per_row;
+      const int ncol0 = nt * BN + col_half * 128;
+      const uint32_t taddr = tmem_base + acc * BN + col_half * 128 + ((uint32_t)(quarter * 32) << 16);
+      uint32_t r[2][32];
+      tmem_ld32(taddr, r[0]);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
         tmem_ld_wait();
-        const int n0 = nt * BN + c * 32;
+        if (c + 1 < 4) tmem_ld32(taddr + (c + 1) * 32, r[(c + 1) & 1]);  // next chunk streams in while this one is stored
+        const uint32_t(&rc)[32] = r[c & 1];
+        const int n0 = ncol0 + c * 32;
         if (row_ok && n0 < p.N) {
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {  // 4 x (8 columns = 16 bytes)
-            if (n0 + v * 8 < p.N) {      // N is a multiple of 8
+          for (int v = 0; v < 4; ++v) {  // 4 x (8 columns = 16 bytes); N is a multiple of 8
+            const int n = n0 + v * 8;
+            if (n < p.N) {
               uint32_t w[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
-                float f0 = __uint_as_float(r[v * 8 + 2 * e]) + bias_row;
-                float f1 = __uint_as_float(r[v * 8 + 2 * e + 1]) + bias_row;
-                if (p.bias && !p.bias_per_row) {
-                  f0 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e]);
-                  f1 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e + 1]);
+                float f0 = __uint_as_float(rc[v * 8 + 2 * e]) + bias_row;
+                float f1 = __uint_as_float(rc[v * 8 + 2 * e + 1]) + bias_row;
+                if (bias_col) {
+                  f0 += __bfloat162float(p.bias[n + 2 * e]);
+                  f1 += __bfloat162float(p.bias[n + 2 * e + 1]);
                 }
                 w[e] = pack2(f0, f1);
               }
-              const int n = n0 + v * 8;
-              bf16* dst = p.group ? obase + ((long long)(n / p.group) * p.M + m) * p.group + n % p.group
-                                  : orow + c * 32 + v * 8;
+              bf16* dst = p.group ? obase + (((long long)(n >> gs) * p.M + m) << gs) + (n & (p.group - 1))
+                                  : obase + (long long)m * p.ld_out + n;
               asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
             }
           }
@@ -291,7 +298,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);  // accumulator drained by this warp
+      if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);  // this warp's share of the accumulator is drained
     }
   }
 
