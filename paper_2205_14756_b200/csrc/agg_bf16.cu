@@ -24,6 +24,10 @@
 #define MSLA_AGG_WY 2  // warps along y
 #endif
 
+#ifndef MSLA_AGG_MIN_BLOCKS
+#define MSLA_AGG_MIN_BLOCKS 3
+#endif
+
 namespace msla {
 namespace {
 
@@ -36,6 +40,9 @@ __device__ int g_agg_timeout_flag = 0;
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void fma2(float2& acc, const float2& a, const float2& b) {
+#ifdef MSLA_AGG_SCALAR_FMA
+  acc.x = fmaf(a.x, b.x, acc.x); acc.y = fmaf(a.y, b.y, acc.y); return;
+#endif
   unsigned long long& c = reinterpret_cast<unsigned long long&>(acc);
   asm("fma.rn.f32x2 %0, %1, %2, %0;"
       : "+l"(c)
@@ -62,39 +69,53 @@ struct AggParams {
   long long dst_batch_stride;  // elements
   int src_planes_per_batch;    // plane index of (b, group) in the tensor map = b * this + group
   int H, W;
-  int tiles_x;
+  int tiles_x, tiles_total;    // tiles per plane
+  int tiles_per_cta;           // consecutive tiles of one plane handled by one CTA
 };
 
 template <int WX, int WY>
-__global__ void __launch_bounds__(WX * WY * 32)
+__global__ void __launch_bounds__(WX * WY * 32, MSLA_AGG_MIN_BLOCKS)
 aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
   constexpr int TW = 8 * WX, TH = 8 * WY, HW_ = TW + 4, HH = TH + 4;
   constexpr int TILE_BYTES = HW_ * HH * D * 2;
-  __shared__ __align__(128) unsigned char tile[TILE_BYTES];
-  __shared__ __align__(16) float wdw_s[5][5][D];  // [dx][dy][channel]
-  __shared__ __align__(8) unsigned long long bar_storage;
+  constexpr int TILE_PITCH = (TILE_BYTES + 127) / 128 * 128;
+  extern __shared__ __align__(128) unsigned char tiles[];  // two halo tiles (double buffer), dynamic
+  __shared__ __align__(16) float wdw_s[5][5][D];           // [dx][dy][channel]
+  __shared__ __align__(8) unsigned long long bar_storage[2];
   __shared__ int timed_out;
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int wx = warp % WX, wy = warp / WX;
-  const int x0 = (blockIdx.x % p.tiles_x) * TW, y0 = (blockIdx.x / p.tiles_x) * TH;
   const int group = blockIdx.y, b = blockIdx.z;
   const int ch0 = group * D;
-  const uint32_t bar = smem_u32(&bar_storage);
+  const int tile_first = blockIdx.x * p.tiles_per_cta;
+  const int tile_count = min(p.tiles_per_cta, p.tiles_total - tile_first);
+  const int plane_idx = b * p.src_planes_per_batch + group;
+  const uint32_t bar0 = smem_u32(&bar_storage[0]);
+  const uint32_t tiles0 = smem_u32(tiles);
+
+  // One elected thread feeds the two-deep ring.  x and y may start at -2 (and
+  // run past W, H): the TMA unit returns zeros there, i.e. the zero padding.
+  auto issue = [&](int k) {
+    const int tile = tile_first + k;
+    const int tx0 = (tile % p.tiles_x) * TW, ty0 = (tile / p.tiles_x) * TH;
+    const uint32_t bar = bar0 + 8 * (k & 1);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(TILE_BYTES) : "memory");
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(tiles0 + (k & 1) * TILE_PITCH), "l"(&tm_src), "r"(bar), "r"(0), "r"(tx0 - 2), "r"(ty0 - 2), "r"(plane_idx)
+        : "memory");
+  };
 
   if (threadIdx.x == 0) {
     timed_out = 0;
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(TILE_BYTES) : "memory");
-    // x and y may start at -2 (and run past W, H): those pixels read as zero.
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(smem_u32(tile)), "l"(&tm_src), "r"(bar), "r"(0), "r"(x0 - 2), "r"(y0 - 2),
-          "r"(b * p.src_planes_per_batch + group) : "memory");
+    issue(0);
   }
-  // depthwise taps -> fp32 [dx][dy][c] while the copy is in flight
+  // depthwise taps -> fp32 [dx][dy][c] while the first copy is in flight
   for (int e = threadIdx.x; e < 25 * D; e += WX * WY * 32) {
     const int c = e % D, tap = e / D;  // consecutive threads -> consecutive channels: conflict-free stores
     wdw_s[tap % 5][tap / 5][c] = __bfloat162float(p.w_dw[(long long)(ch0 + c) * 25 + tap]);
@@ -110,92 +131,103 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
         const int oc = 8 * (g >> 1) + 2 * jn + (g & 1);
         bw[ks][jn][r] = *reinterpret_cast<const uint32_t*>(p.w_pw + (long long)(ch0 + oc) * D + 8 * t + 4 * ks + 2 * r);
       }
-  __syncthreads();  // barrier initialised and taps staged before anyone proceeds
+  __syncthreads();  // barriers initialised and taps staged before anyone proceeds
 
-  {  // bounded wait for the halo tile
-    uint32_t ok = 0;
-    const long long t_start = clock64();
-    while (true) {
-      asm volatile(
-          "{\n\t.reg .pred P1;\n\tmbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\tselp.b32 %0, 1, 0, P1;\n\t}"
-          : "=r"(ok) : "r"(bar), "r"(0) : "memory");
-      if (ok) break;
-      if (clock64() - t_start > WAIT_LIMIT_CYCLES) { timed_out = 1; break; }
-    }
-  }
-  __syncthreads();
-  if (timed_out) {  // leave without touching the output; the copy had two seconds to land
-    if (threadIdx.x == 0) atomicExch(&g_agg_timeout_flag, 1);
-    return;
-  }
-
-  // ---- depthwise 5x5: column (wx*8 + g), rows wy*8 .. +7, channels 8t .. 8t+7
-  float2 acc[8][4];
-#pragma unroll
-  for (int r = 0; r < 8; ++r)
-#pragma unroll
-    for (int q = 0; q < 4; ++q) acc[r][q] = make_float2(0.f, 0.f);
-  const uint32_t col_base = smem_u32(tile) + (uint32_t)(((wy * 8) * HW_ + wx * 8 + g) * (D * 2) + t * 16);
+  bf16* plane = p.dst + (long long)b * p.dst_batch_stride + (long long)group * p.H * p.W * D;
 #pragma unroll 1
-  for (int dx = 0; dx < 5; ++dx) {
-    float2 w[5][4];
-#pragma unroll
-    for (int dy = 0; dy < 5; ++dy) {
-      const float4 lo = *reinterpret_cast<const float4*>(&wdw_s[dx][dy][8 * t]);
-      const float4 hi = *reinterpret_cast<const float4*>(&wdw_s[dx][dy][8 * t + 4]);
-      w[dy][0] = make_float2(lo.x, lo.y); w[dy][1] = make_float2(lo.z, lo.w);
-      w[dy][2] = make_float2(hi.x, hi.y); w[dy][3] = make_float2(hi.z, hi.w);
+  for (int k = 0; k < tile_count; ++k) {
+    // prefetch the next tile into the buffer everyone left at the end of iteration k-1
+    if (threadIdx.x == 0 && k + 1 < tile_count) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // order the earlier generic reads before the async write
+      issue(k + 1);
     }
+    {  // bounded wait for this tile
+      const uint32_t bar = bar0 + 8 * (k & 1), parity = (k >> 1) & 1;
+      uint32_t ok = 0;
+      const long long t_start = clock64();
+      while (true) {
+        asm volatile(
+            "{\n\t.reg .pred P1;\n\tmbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\tselp.b32 %0, 1, 0, P1;\n\t}"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) break;
+        if (timed_out || clock64() - t_start > WAIT_LIMIT_CYCLES) { timed_out = 1; break; }
+      }
+    }
+    if (__syncthreads_or(timed_out)) {  // leave without touching this tile; the copy had two seconds to land
+      if (threadIdx.x == 0) atomicExch(&g_agg_timeout_flag, 1);
+      return;
+    }
+    const int tile = tile_first + k;
+    const int x0 = (tile % p.tiles_x) * TW, y0 = (tile / p.tiles_x) * TH;
+
+    // ---- depthwise 5x5: column (wx*8 + g), rows wy*8 .. +7, channels 8t .. 8t+7
+    float2 acc[8][4];
 #pragma unroll
-    for (int i = 0; i < 12; ++i) {  // input row i of the column feeds output rows i-4 .. i
-      uint32_t raw[4];
-      asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                   : "=r"(raw[0]), "=r"(raw[1]), "=r"(raw[2]), "=r"(raw[3])
-                   : "r"(col_base + (uint32_t)((i * HW_ + dx) * (D * 2))));
-      float2 in[4];
+    for (int r = 0; r < 8; ++r)
 #pragma unroll
-      for (int q = 0; q < 4; ++q) in[q] = unpack_bf16x2(raw[q]);
+      for (int q = 0; q < 4; ++q) acc[r][q] = make_float2(0.f, 0.f);
+    const uint32_t col_base = tiles0 + (k & 1) * TILE_PITCH + (uint32_t)(((wy * 8) * HW_ + wx * 8 + g) * (D * 2) + t * 16);
+#pragma unroll 1
+    for (int dx = 0; dx < 5; ++dx) {
+      float2 w[5][4];
 #pragma unroll
       for (int dy = 0; dy < 5; ++dy) {
-        const int r = i - dy;
-        if (r >= 0 && r < 8) {
+        const float4 lo = *reinterpret_cast<const float4*>(&wdw_s[dx][dy][8 * t]);
+        const float4 hi = *reinterpret_cast<const float4*>(&wdw_s[dx][dy][8 * t + 4]);
+        w[dy][0] = make_float2(lo.x, lo.y); w[dy][1] = make_float2(lo.z, lo.w);
+        w[dy][2] = make_float2(hi.x, hi.y); w[dy][3] = make_float2(hi.z, hi.w);
+      }
 #pragma unroll
-          for (int q = 0; q < 4; ++q) fma2(acc[r][q], w[dy][q], in[q]);
+      for (int i = 0; i < 12; ++i) {  // input row i of the column feeds output rows i-4 .. i
+        uint32_t raw[4];
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(raw[0]), "=r"(raw[1]), "=r"(raw[2]), "=r"(raw[3])
+                     : "r"(col_base + (uint32_t)((i * HW_ + dx) * (D * 2))));
+        float2 in[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) in[q] = unpack_bf16x2(raw[q]);
+#pragma unroll
+        for (int dy = 0; dy < 5; ++dy) {
+          const int r = i - dy;
+          if (r >= 0 && r < 8) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) fma2(acc[r][q], w[dy][q], in[q]);
+          }
         }
       }
     }
-  }
 
-  // ---- grouped 1x1 on tensor cores, straight from the accumulators
-  const int x = x0 + wx * 8 + g;
-  bf16* plane = p.dst + (long long)b * p.dst_batch_stride + (long long)group * p.H * p.W * D;
+    // ---- grouped 1x1 on tensor cores, straight from the accumulators
+    const int x = x0 + wx * 8 + g;
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {  // MMA rows g / g+8 = pixels (x, 2j) / (x, 2j+1) of the warp block
-    float c[4][4];
+    for (int j = 0; j < 4; ++j) {  // MMA rows g / g+8 = pixels (x, 2j) / (x, 2j+1) of the warp block
+      float c[4][4];
 #pragma unroll
-    for (int jn = 0; jn < 4; ++jn)
+      for (int jn = 0; jn < 4; ++jn)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) c[jn][e] = 0.f;
+        for (int e = 0; e < 4; ++e) c[jn][e] = 0.f;
 #pragma unroll
-    for (int ks = 0; ks < 2; ++ks) {
-      const uint32_t A[4] = {pack_bf16(acc[2 * j][2 * ks].x, acc[2 * j][2 * ks].y),
-                             pack_bf16(acc[2 * j + 1][2 * ks].x, acc[2 * j + 1][2 * ks].y),
-                             pack_bf16(acc[2 * j][2 * ks + 1].x, acc[2 * j][2 * ks + 1].y),
-                             pack_bf16(acc[2 * j + 1][2 * ks + 1].x, acc[2 * j + 1][2 * ks + 1].y)};
+      for (int ks = 0; ks < 2; ++ks) {
+        const uint32_t A[4] = {pack_bf16(acc[2 * j][2 * ks].x, acc[2 * j][2 * ks].y),
+                               pack_bf16(acc[2 * j + 1][2 * ks].x, acc[2 * j + 1][2 * ks].y),
+                               pack_bf16(acc[2 * j][2 * ks + 1].x, acc[2 * j][2 * ks + 1].y),
+                               pack_bf16(acc[2 * j + 1][2 * ks + 1].x, acc[2 * j + 1][2 * ks + 1].y)};
 #pragma unroll
-      for (int jn = 0; jn < 4; ++jn) mma_bf16(c[jn], A, bw[ks][jn][0], bw[ks][jn][1]);
-    }
+        for (int jn = 0; jn < 4; ++jn) mma_bf16(c[jn], A, bw[ks][jn][0], bw[ks][jn][1]);
+      }
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      const int y = y0 + wy * 8 + 2 * j + half;
-      if (x < p.W && y < p.H) {
-        bf16* dst = plane + ((long long)y * p.W + x) * D + 8 * t;
-        asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(dst),
-                     "r"(pack_bf16(c[0][2 * half], c[0][2 * half + 1])), "r"(pack_bf16(c[1][2 * half], c[1][2 * half + 1])),
-                     "r"(pack_bf16(c[2][2 * half], c[2][2 * half + 1])), "r"(pack_bf16(c[3][2 * half], c[3][2 * half + 1]))
-                     : "memory");
+      for (int half = 0; half < 2; ++half) {
+        const int y = y0 + wy * 8 + 2 * j + half;
+        if (x < p.W && y < p.H) {
+          bf16* dst = plane + ((long long)y * p.W + x) * D + 8 * t;
+          asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(dst),
+                       "r"(pack_bf16(c[0][2 * half], c[0][2 * half + 1])), "r"(pack_bf16(c[1][2 * half], c[1][2 * half + 1])),
+                       "r"(pack_bf16(c[2][2 * half], c[2][2 * half + 1])), "r"(pack_bf16(c[3][2 * half], c[3][2 * half + 1]))
+                       : "memory");
+        }
       }
     }
+    __syncthreads();  // every warp is done with buffer k&1 before iteration k+1 refills it (for tile k+2)
   }
 }
 
@@ -223,8 +255,18 @@ msla_status_t run_aggregate_bf16(const void* src, long long src_planes_total, in
   p.tiles_x = (W + TW - 1) / TW;
   const long long tiles = (long long)p.tiles_x * ((H + TH - 1) / TH);
   if (tiles > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many aggregation tiles");
-  dim3 grid((unsigned)tiles, (unsigned)(Ch / D), (unsigned)B);
-  aggregate_bf16_kernel<WX, WY><<<grid, WX * WY * 32, 0, st>>>(tm, p);
+  p.tiles_total = (int)tiles;
+  // enough CTAs for a few waves over the GPU, otherwise as many tiles per CTA as possible (up to 8)
+  const long long units = tiles * (Ch / D) * B;
+  p.tiles_per_cta = units >= 8 * 2400 ? 8 : units >= 4 * 2400 ? 4 : units >= 2 * 2400 ? 2 : 1;
+  dim3 grid((unsigned)((tiles + p.tiles_per_cta - 1) / p.tiles_per_cta), (unsigned)(Ch / D), (unsigned)B);
+  constexpr int tile_bytes = 2 * (((TW + 4) * (TH + 4) * D * 2 + 127) / 128 * 128);
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaFuncSetAttribute(aggregate_bf16_kernel<WX, WY>, cudaFuncAttributeMaxDynamicSharedMemorySize, tile_bytes);
+    attr_done = true;
+  }
+  aggregate_bf16_kernel<WX, WY><<<grid, WX * WY * 32, tile_bytes, st>>>(tm, p);
   count_launches(1);
   return check_launch("token aggregation (bf16)");
 }
