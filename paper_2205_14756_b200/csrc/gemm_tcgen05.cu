@@ -145,6 +145,52 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& 
   else             { nt = r / p.m_tiles; mt = r % p.m_tiles; }
 }
 
+// One epilogue warp's share of a finished 128x256 accumulator: TMEM lanes
+// 32*quarter .. +31 (= tile rows), columns col_half*128 .. +127, converted to
+// bf16 (+ bias) and stored with 16-byte vectors.
+__device__ __forceinline__ void drain_accumulator(const GemmParams& p, int b, int mt, int nt, uint32_t tmem_acc,
+                                                  int quarter, int col_half, int lane) {
+  const int gs = p.group == 32 ? 5 : 4;  // log2(group) when the output is planar
+  const int m = mt * BM + quarter * 32 + lane;
+  const bool row_ok = m < p.M;
+  bf16* obase = p.out + (long long)b * p.out_batch_stride;
+  const float bias_row = (p.bias && p.bias_per_row && row_ok) ? __bfloat162float(p.bias[m]) : 0.f;
+  const bool bias_col = p.bias && !p.bias_per_row;
+  const int ncol0 = nt * BN + col_half * 128;
+  const uint32_t taddr = tmem_acc + col_half * 128 + ((uint32_t)(quarter * 32) << 16);
+  uint32_t r[2][32];
+  tmem_ld32(taddr, r[0]);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    tmem_ld_wait();
+    if (c + 1 < 4) tmem_ld32(taddr + (c + 1) * 32, r[(c + 1) & 1]);  // next chunk streams in while this one is stored
+    const uint32_t(&rc)[32] = r[c & 1];
+    const int n0 = ncol0 + c * 32;
+    if (row_ok && n0 < p.N) {
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {  // 4 x (8 columns = 16 bytes); N is a multiple of 8
+        const int n = n0 + v * 8;
+        if (n < p.N) {
+          uint32_t w[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float f0 = __uint_as_float(rc[v * 8 + 2 * e]) + bias_row;
+            float f1 = __uint_as_float(rc[v * 8 + 2 * e + 1]) + bias_row;
+            if (bias_col) {
+              f0 += __bfloat162float(p.bias[n + 2 * e]);
+              f1 += __bfloat162float(p.bias[n + 2 * e + 1]);
+            }
+            w[e] = pack2(f0, f1);
+          }
+          bf16* dst = p.group ? obase + (((long long)(n >> gs) * p.M + m) << gs) + (n & (p.group - 1))
+                              : obase + (long long)m * p.ld_out + n;
+          asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+        }
+      }
+    }
+  }
+}
+
 template <bool A_MN_MAJOR>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
@@ -247,7 +293,6 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     // other bit selects which 128 of the tile's 256 columns the warp drains.
     const int quarter = warp & 3;
     const int col_half = (warp - 2) >> 2;
-    const int gs = p.group == 32 ? 5 : 4;  // log2(group) when the output is planar
     uint32_t local = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++local) {
@@ -258,44 +303,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const int m = mt * BM + quarter * 32 + lane;
-      const bool row_ok = m < p.M;
-      bf16* obase = p.out + (long long)b * p.out_batch_stride;
-      const float bias_row = (p.bias && p.bias_per_row && row_ok) ? __bfloat162float(p.bias[m]) : 0.f;
-      const bool bias_col = p.bias && !p.bias_per_row;
-      const int ncol0 = nt * BN + col_half * 128;
-      const uint32_t taddr = tmem_base + acc * BN + col_half * 128 + ((uint32_t)(quarter * 32) << 16);
-      uint32_t r[2][32];
-      tmem_ld32(taddr, r[0]);
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        tmem_ld_wait();
-        if (c + 1 < 4) tmem_ld32(taddr + (c + 1) * 32, r[(c + 1) & 1]);  // next chunk streams in while this one is stored
-        const uint32_t(&rc)[32] = r[c & 1];
-        const int n0 = ncol0 + c * 32;
-        if (row_ok && n0 < p.N) {
-#pragma unroll
-          for (int v = 0; v < 4; ++v) {  // 4 x (8 columns = 16 bytes); N is a multiple of 8
-            const int n = n0 + v * 8;
-            if (n < p.N) {
-              uint32_t w[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                float f0 = __uint_as_float(rc[v * 8 + 2 * e]) + bias_row;
-                float f1 = __uint_as_float(rc[v * 8 + 2 * e + 1]) + bias_row;
-                if (bias_col) {
-                  f0 += __bfloat162float(p.bias[n + 2 * e]);
-                  f1 += __bfloat162float(p.bias[n + 2 * e + 1]);
-                }
-                w[e] = pack2(f0, f1);
-              }
-              bf16* dst = p.group ? obase + (((long long)(n >> gs) * p.M + m) << gs) + (n & (p.group - 1))
-                                  : obase + (long long)m * p.ld_out + n;
-              asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
-            }
-          }
-        }
-      }
+      drain_accumulator(p, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);  // this warp's share of the accumulator is drained
@@ -307,6 +315,170 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
   __syncthreads();
   if (abort_flag) {
     // give copies and MMAs still in flight time to land before memory is released
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    if (threadIdx.x == 0) atomicExch(&g_gemm_timeout_flag, 1);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
+
+// ---------------------------------------------------------------------------
+// Weight-stationary variant.  Every CTA of the streaming kernel above re-reads
+// the same weight slices from L2 at the same time, and those few hot lines
+// serialise in their L2 slices.  Here a CTA owns one block of output channels
+// for its whole life: that block of the weight matrix (<= 128 KB) is loaded
+// into shared memory once, and only activation tiles stream through a ring.
+//   RES_IS_B = true  (input projection) : B = 256 weight rows resident (K <= 256),
+//                                         A = 128-token x tiles, MN-major, 16 KB stages
+//   RES_IS_B = false (output projection): A = 128 weight rows resident (K <= 512),
+//                                         B = 256-token attention tiles, 32 KB stages
+// CTA c serves weight block c % blocks and the activation tiles c / blocks,
+// c / blocks + workers, ...  Barriers, TMEM use and epilogue are as above.
+// ---------------------------------------------------------------------------
+constexpr int RES_BYTES = 128 * 1024;
+constexpr int WS_RING_BYTES = 96 * 1024;
+constexpr int WS_SMEM_BYTES = RES_BYTES + WS_RING_BYTES + 256 + 1024;
+constexpr int WS_MAX_STAGES = 6;
+
+template <bool RES_IS_B>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p,
+                            int blocks, int workers) {
+  constexpr int STREAM_BYTES = RES_IS_B ? A_STAGE_BYTES : B_STAGE_BYTES;  // one k-slice of the streamed operand
+  constexpr int NSTAGE = WS_RING_BYTES / STREAM_BYTES;                     // 6 or 3
+  constexpr int RES_SLICE = RES_IS_B ? B_STAGE_BYTES : A_STAGE_BYTES;      // one k-slice of the resident operand
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t res_base = smem_base, ring_base = smem_base + RES_BYTES;
+  const uint32_t bars = ring_base + WS_RING_BYTES;
+  const uint32_t full_bar = bars, empty_bar = bars + 8 * WS_MAX_STAGES;
+  const uint32_t tfull_bar = bars + 16 * WS_MAX_STAGES, tempty_bar = tfull_bar + 16;
+  const uint32_t res_bar = tempty_bar + 16, tmem_slot = res_bar + 8;
+  __shared__ int abort_flag;
+  __shared__ uint32_t tmem_base_sh;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int k_iters = (p.K + BK - 1) / BK;
+  const int blk = blockIdx.x % blocks, worker = blockIdx.x / blocks;
+  const int stream_per_batch = RES_IS_B ? p.m_tiles : p.n_tiles;
+  const int stream_total = p.batches * stream_per_batch;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < NSTAGE; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar + 8 * a, 1); mbar_init(tempty_bar + 8 * a, 8); }
+    mbar_init(res_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (threadIdx.x == 0) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(tmem_slot));
+    tmem_base_sh = v;
+  }
+  __syncthreads();
+  const uint32_t tmem_base = tmem_base_sh;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+      // the resident weight block: all k-slices on one barrier
+      mbar_expect_tx(res_bar, (uint32_t)(k_iters * RES_SLICE));
+      for (int kb = 0; kb < k_iters; ++kb) {
+        if (RES_IS_B) tma_load_3d(res_base + kb * RES_SLICE, &tmB, res_bar, kb * BK, blk * BN, 0);
+        else          tma_load_3d(res_base + kb * RES_SLICE, &tmA, res_bar, kb * BK, blk * BM, 0);
+      }
+      uint32_t it = 0;
+      bool ok = true;
+      for (int si = worker; ok && si < stream_total; si += workers) {
+        const int b = si / stream_per_batch, st = si % stream_per_batch;
+        for (int kb = 0; ok && kb < k_iters; ++kb, ++it) {
+          const uint32_t s = it % NSTAGE, ph = (it / NSTAGE) & 1;
+          ok = mbar_wait(empty_bar + 8 * s, ph ^ 1, &abort_flag);
+          if (!ok) break;
+          const uint32_t dst = ring_base + s * STREAM_BYTES;
+          mbar_expect_tx(full_bar + 8 * s, STREAM_BYTES);
+          if (RES_IS_B) {  // x tile: two boxes of 64 tokens x 64 k
+            tma_load_3d(dst, &tmA, full_bar + 8 * s, st * BM, kb * BK, b);
+            tma_load_3d(dst + STREAM_BYTES / 2, &tmA, full_bar + 8 * s, st * BM + 64, kb * BK, b);
+          } else {         // attention tile: one box of 64 k x 256 tokens
+            tma_load_3d(dst, &tmB, full_bar + 8 * s, kb * BK, st * BN, b);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // -------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((RES_IS_B ? 1u : 0u) << 15) |
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      uint32_t it = 0, local = 0;
+      bool ok = mbar_wait(res_bar, 0, &abort_flag);
+      for (int si = worker; ok && si < stream_total; si += workers, ++local) {
+        const uint32_t acc = local & 1, acc_ph = (local >> 1) & 1;
+        ok = mbar_wait(tempty_bar + 8 * acc, acc_ph ^ 1, &abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; ok && kb < k_iters; ++kb, ++it) {
+          const uint32_t s = it % NSTAGE, ph = (it / NSTAGE) & 1;
+          ok = mbar_wait(full_bar + 8 * s, ph, &abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t stream = ring_base + s * STREAM_BYTES, res = res_base + kb * RES_SLICE;
+#pragma unroll
+          for (int kk = 0; kk < BK / 16; ++kk) {
+            uint64_t ad, bd;
+            if (RES_IS_B) {
+              ad = make_desc(stream + kk * 2048, (A_STAGE_BYTES / 2) >> 4, 1024 >> 4);  // MN-major x tile
+              bd = make_desc(res + kk * 32, 1, 1024 >> 4);
+            } else {
+              ad = make_desc(res + kk * 32, 1, 1024 >> 4);
+              bd = make_desc(stream + kk * 32, 1, 1024 >> 4);
+            }
+            umma_bf16(d_tmem, ad, bd, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+          }
+          umma_commit(empty_bar + 8 * s);
+        }
+        if (ok) umma_commit(tfull_bar + 8 * acc);
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int quarter = warp & 3;
+    const int col_half = (warp - 2) >> 2;
+    uint32_t local = 0;
+    bool ok = true;
+    for (int si = worker; ok && si < stream_total; si += workers, ++local) {
+      const int b = si / stream_per_batch, st = si % stream_per_batch;
+      const int mt = RES_IS_B ? st : blk, nt = RES_IS_B ? blk : st;
+      const uint32_t acc = local & 1, acc_ph = (local >> 1) & 1;
+      ok = mbar_wait(tfull_bar + 8 * acc, acc_ph, &abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      drain_accumulator(p, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
     if (threadIdx.x == 0) atomicExch(&g_gemm_timeout_flag, 1);
     __syncthreads();
@@ -339,7 +511,30 @@ int sm_count() {
 }
 
 template <bool A_MN>
+msla_status_t launch_stationary(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, int blocks, cudaStream_t st) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(gemm_bf16_stationary_kernel<A_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, WS_SMEM_BYTES) != cudaSuccess) {
+      cudaGetLastError();
+      return fail(MSLA_ERR_CUDA, "cannot reserve %d bytes of shared memory for the projection GEMM", WS_SMEM_BYTES);
+    }
+    attr_done = true;
+  }
+  const long long stream_total = (long long)p.batches * (A_MN ? p.m_tiles : p.n_tiles);
+  long long workers = sm_count() / blocks;
+  if (workers > stream_total) workers = stream_total;
+  gemm_bf16_stationary_kernel<A_MN><<<(unsigned)(workers * blocks), NUM_THREADS, WS_SMEM_BYTES, st>>>(tmA, tmB, p, blocks, (int)workers);
+  count_launches(1);
+  return check_launch("projection GEMM (tcgen05, stationary weights)");
+}
+
+template <bool A_MN>
 msla_status_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, cudaStream_t st) {
+  // weight-stationary kernel when the CTA's weight block fits its 128 KB of shared memory
+  const int blocks = A_MN ? p.n_tiles : p.m_tiles;
+  const int k_iters = (p.K + BK - 1) / BK;
+  if (k_iters * (A_MN ? B_STAGE_BYTES : A_STAGE_BYTES) <= RES_BYTES && blocks <= 16 && blocks <= sm_count())
+    return launch_stationary<A_MN>(tmA, tmB, p, blocks, st);
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel<A_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
