@@ -38,7 +38,7 @@ constexpr int A_STAGE_BYTES = BM * BK * 2;  // 16 KB
 constexpr int B_STAGE_BYTES = BN * BK * 2;  // 32 KB
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int NUM_THREADS = 320;  // TMA warp, MMA warp, 8 epilogue warps
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 256 + 1024;  // ring + barriers + alignment slack
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 8 * 2048 + 256 + 1024;  // ring + epilogue staging + barriers + alignment slack
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;          // ~2 s at 2 GHz
 
 // Sticky: set when any wait in any GEMM launch of this process timed out.
@@ -55,6 +55,8 @@ struct GemmParams {
   int n_fastest;          // tile order: 1 = consecutive tiles share the A tile, 0 = share the B tile
   const bf16* bias;
   bf16* out;
+  int tma_store;          // 1: epilogue stages 32x32 blocks in shared memory and writes them with TMA (tmO)
+  int planes_per_batch;   // planar output: plane coordinate of (batch, n) = batch*planes_per_batch + n/32
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -98,6 +100,11 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 
 // Shared-memory matrix descriptor, 128-byte swizzle.  Offsets are in 16-byte
@@ -145,19 +152,28 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& 
   else             { nt = r / p.m_tiles; mt = r % p.m_tiles; }
 }
 
+constexpr int STAGING_BYTES = 8 * 2048;  // one 32-row x 64-byte block per epilogue warp
+
 // One epilogue warp's share of a finished 128x256 accumulator: TMEM lanes
 // 32*quarter .. +31 (= tile rows), columns col_half*128 .. +127, converted to
-// bf16 (+ bias) and stored with 16-byte vectors.
-__device__ __forceinline__ void drain_accumulator(const GemmParams& p, int b, int mt, int nt, uint32_t tmem_acc,
-                                                  int quarter, int col_half, int lane) {
+// bf16 (+ bias).  A lane owns one row, so storing straight from registers
+// scatters 16-byte pieces over 32 rows per instruction; instead each 32x32
+// block is laid out in shared memory (64-byte rows, 16-byte chunks XOR-swizzled
+// as the TMA unit's 64B mode expects) and written by one TMA store, which
+// emits whole lines and clips rows and columns outside the tensor.  Without a
+// store map (planes of 16 channels) the lane stores its vectors directly.
+__device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUtensorMap* tmO, uint32_t stage, int b,
+                                                  int mt, int nt, uint32_t tmem_acc, int quarter, int col_half, int lane) {
   const int gs = p.group == 32 ? 5 : 4;  // log2(group) when the output is planar
-  const int m = mt * BM + quarter * 32 + lane;
+  const int row0 = mt * BM + quarter * 32;
+  const int m = row0 + lane;
   const bool row_ok = m < p.M;
   bf16* obase = p.out + (long long)b * p.out_batch_stride;
   const float bias_row = (p.bias && p.bias_per_row && row_ok) ? __bfloat162float(p.bias[m]) : 0.f;
   const bool bias_col = p.bias && !p.bias_per_row;
   const int ncol0 = nt * BN + col_half * 128;
   const uint32_t taddr = tmem_acc + col_half * 128 + ((uint32_t)(quarter * 32) << 16);
+  const uint32_t my_row = stage + lane * 64, sw = (uint32_t)((lane >> 1) & 3);
   uint32_t r[2][32];
   tmem_ld32(taddr, r[0]);
 #pragma unroll
@@ -166,25 +182,43 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, int b, in
     if (c + 1 < 4) tmem_ld32(taddr + (c + 1) * 32, r[(c + 1) & 1]);  // next chunk streams in while this one is stored
     const uint32_t(&rc)[32] = r[c & 1];
     const int n0 = ncol0 + c * 32;
-    if (row_ok && n0 < p.N) {
+    if (n0 >= p.N) continue;  // warp-uniform
+    uint32_t w[4][4];
+#pragma unroll
+    for (int v = 0; v < 4; ++v)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float f0 = __uint_as_float(rc[v * 8 + 2 * e]) + bias_row;
+        float f1 = __uint_as_float(rc[v * 8 + 2 * e + 1]) + bias_row;
+        if (bias_col && n0 + v * 8 < p.N) {
+          f0 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e]);
+          f1 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e + 1]);
+        }
+        w[v][e] = pack2(f0, f1);
+      }
+    if (p.tma_store) {
+      // the previous block must have been read out of the staging buffer
+      if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      __syncwarp();
+#pragma unroll
+      for (int v = 0; v < 4; ++v)
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(my_row + (((uint32_t)v ^ sw) << 4)), "r"(w[v][0]),
+                     "r"(w[v][1]), "r"(w[v][2]), "r"(w[v][3]) : "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) {
+        if (p.group) tma_store_3d(tmO, stage, 0, row0, b * p.planes_per_batch + (n0 >> 5));
+        else         tma_store_3d(tmO, stage, n0, row0, b);
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      }
+    } else if (row_ok) {
 #pragma unroll
       for (int v = 0; v < 4; ++v) {  // 4 x (8 columns = 16 bytes); N is a multiple of 8
         const int n = n0 + v * 8;
         if (n < p.N) {
-          uint32_t w[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            float f0 = __uint_as_float(rc[v * 8 + 2 * e]) + bias_row;
-            float f1 = __uint_as_float(rc[v * 8 + 2 * e + 1]) + bias_row;
-            if (bias_col) {
-              f0 += __bfloat162float(p.bias[n + 2 * e]);
-              f1 += __bfloat162float(p.bias[n + 2 * e + 1]);
-            }
-            w[e] = pack2(f0, f1);
-          }
           bf16* dst = p.group ? obase + (((long long)(n >> gs) * p.M + m) << gs) + (n & (p.group - 1))
                               : obase + (long long)m * p.ld_out + n;
-          asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+          asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(dst), "r"(w[v][0]), "r"(w[v][1]), "r"(w[v][2]), "r"(w[v][3]) : "memory");
         }
       }
     }
@@ -193,10 +227,12 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, int b, in
 
 template <bool A_MN_MAJOR>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
+gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                         const __grid_constant__ CUtensorMap tmO, GemmParams p) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
-  const uint32_t bars = smem_base + STAGES * STAGE_BYTES;
+  const uint32_t staging = smem_base + STAGES * STAGE_BYTES;
+  const uint32_t bars = staging + STAGING_BYTES;
   const uint32_t full_bar = bars, empty_bar = bars + 8 * STAGES;
   const uint32_t tfull_bar = bars + 16 * STAGES, tempty_bar = tfull_bar + 16;
   const uint32_t tmem_slot = tempty_bar + 16;
@@ -303,11 +339,12 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      drain_accumulator(p, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
+      drain_accumulator(p, &tmO, staging + (warp - 2) * 2048, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);  // this warp's share of the accumulator is drained
     }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // TMA stores done before the CTA retires
   }
 
   // ------------------------------------------------------------------ teardown
@@ -333,28 +370,29 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
 // for its whole life: that block of the weight matrix (<= 128 KB) is loaded
 // into shared memory once, and only activation tiles stream through a ring.
 //   RES_IS_B = true  (input projection) : B = 256 weight rows resident (K <= 256),
-//                                         A = 128-token x tiles, MN-major, 16 KB stages
+//                                         A = 128-token x tiles, MN-major, 16 KB stages (5 deep)
 //   RES_IS_B = false (output projection): A = 128 weight rows resident (K <= 512),
-//                                         B = 256-token attention tiles, 32 KB stages
+//                                         B = 256-token attention tiles, 32 KB stages (2 deep)
 // CTA c serves weight block c % blocks and the activation tiles c / blocks,
 // c / blocks + workers, ...  Barriers, TMEM use and epilogue are as above.
 // ---------------------------------------------------------------------------
 constexpr int RES_BYTES = 128 * 1024;
-constexpr int WS_RING_BYTES = 96 * 1024;
-constexpr int WS_SMEM_BYTES = RES_BYTES + WS_RING_BYTES + 256 + 1024;
+constexpr int WS_RING_BYTES = 80 * 1024;
+constexpr int WS_SMEM_BYTES = RES_BYTES + WS_RING_BYTES + STAGING_BYTES + 256 + 1024;
 constexpr int WS_MAX_STAGES = 6;
 
 template <bool RES_IS_B>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p,
-                            int blocks, int workers) {
+gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                            const __grid_constant__ CUtensorMap tmO, GemmParams p, int blocks, int workers) {
   constexpr int STREAM_BYTES = RES_IS_B ? A_STAGE_BYTES : B_STAGE_BYTES;  // one k-slice of the streamed operand
-  constexpr int NSTAGE = WS_RING_BYTES / STREAM_BYTES;                     // 6 or 3
+  constexpr int NSTAGE = WS_RING_BYTES / STREAM_BYTES;                     // 5 or 2
   constexpr int RES_SLICE = RES_IS_B ? B_STAGE_BYTES : A_STAGE_BYTES;      // one k-slice of the resident operand
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t res_base = smem_base, ring_base = smem_base + RES_BYTES;
-  const uint32_t bars = ring_base + WS_RING_BYTES;
+  const uint32_t staging = ring_base + WS_RING_BYTES;
+  const uint32_t bars = staging + STAGING_BYTES;
   const uint32_t full_bar = bars, empty_bar = bars + 8 * WS_MAX_STAGES;
   const uint32_t tfull_bar = bars + 16 * WS_MAX_STAGES, tempty_bar = tfull_bar + 16;
   const uint32_t res_bar = tempty_bar + 16, tmem_slot = res_bar + 8;
@@ -469,11 +507,12 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      drain_accumulator(p, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
+      drain_accumulator(p, &tmO, staging + (warp - 2) * 2048, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);
     }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   tc_fence_before();
@@ -511,7 +550,8 @@ int sm_count() {
 }
 
 template <bool A_MN>
-msla_status_t launch_stationary(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, int blocks, cudaStream_t st) {
+msla_status_t launch_stationary(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO, const GemmParams& p,
+                                int blocks, cudaStream_t st) {
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(gemm_bf16_stationary_kernel<A_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, WS_SMEM_BYTES) != cudaSuccess) {
@@ -523,18 +563,18 @@ msla_status_t launch_stationary(const CUtensorMap& tmA, const CUtensorMap& tmB, 
   const long long stream_total = (long long)p.batches * (A_MN ? p.m_tiles : p.n_tiles);
   long long workers = sm_count() / blocks;
   if (workers > stream_total) workers = stream_total;
-  gemm_bf16_stationary_kernel<A_MN><<<(unsigned)(workers * blocks), NUM_THREADS, WS_SMEM_BYTES, st>>>(tmA, tmB, p, blocks, (int)workers);
+  gemm_bf16_stationary_kernel<A_MN><<<(unsigned)(workers * blocks), NUM_THREADS, WS_SMEM_BYTES, st>>>(tmA, tmB, tmO, p, blocks, (int)workers);
   count_launches(1);
   return check_launch("projection GEMM (tcgen05, stationary weights)");
 }
 
 template <bool A_MN>
-msla_status_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, cudaStream_t st) {
+msla_status_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO, const GemmParams& p, cudaStream_t st) {
   // weight-stationary kernel when the CTA's weight block fits its 128 KB of shared memory
   const int blocks = A_MN ? p.n_tiles : p.m_tiles;
   const int k_iters = (p.K + BK - 1) / BK;
-  if (k_iters * (A_MN ? B_STAGE_BYTES : A_STAGE_BYTES) <= RES_BYTES && blocks <= 16 && blocks <= sm_count())
-    return launch_stationary<A_MN>(tmA, tmB, p, blocks, st);
+  if (A_MN && k_iters * B_STAGE_BYTES <= RES_BYTES && blocks <= 16 && blocks <= sm_count())
+    return launch_stationary<A_MN>(tmA, tmB, tmO, p, blocks, st);
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel<A_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
@@ -545,7 +585,7 @@ msla_status_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmP
   }
   const long long tiles = (long long)p.batches * p.m_tiles * p.n_tiles;
   const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-  gemm_bf16_tcgen05_kernel<A_MN><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tmA, tmB, p);
+  gemm_bf16_tcgen05_kernel<A_MN><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tmA, tmB, tmO, p);
   count_launches(1);
   return check_launch("projection GEMM (tcgen05)");
 }
@@ -568,7 +608,19 @@ msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, 
   p.m_tiles = (N + BM - 1) / BM; p.n_tiles = (Cout + BN - 1) / BN;
   p.out_batch_stride = y_sb; p.ld_out = 0; p.group = d; p.bias_per_row = 0; p.n_fastest = 1;
   p.bias = nullptr; p.out = (bf16*)y;
-  return launch<true>(tmA, tmB, p, st);
+  // planes of 32 channels are written as 32-token x 32-channel blocks by TMA
+  CUtensorMap tmO = tmA;  // placeholder when the direct-store epilogue is used
+  const long long plane_elems = (long long)N * 32;
+  if (d == 32 && y_sb % plane_elems == 0) {
+    p.tma_store = 1;
+    p.planes_per_batch = (int)(y_sb / plane_elems);
+    const cuuint64_t dims[3] = {32, (cuuint64_t)N, (cuuint64_t)B * p.planes_per_batch};
+    const cuuint64_t strides[2] = {64, (cuuint64_t)N * 64};
+    const cuuint32_t box[3] = {32, 32, 1};
+    if (!tma_make_map_bf16(&tmO, y, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B))
+      return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the input projection's output");
+  }
+  return launch<true>(tmA, tmB, tmO, p, st);
 }
 
 bool project_out_bf16_supported(int Cin, int Cout, int N) { return Cin % 8 == 0 && N % 8 == 0 && Cout >= 1; }
@@ -585,7 +637,16 @@ msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bia
   p.m_tiles = (Cout + BM - 1) / BM; p.n_tiles = (N + BN - 1) / BN;
   p.out_batch_stride = (long long)Cout * N; p.ld_out = N; p.group = 0; p.bias_per_row = 1; p.n_fastest = 0;
   p.bias = (const bf16*)bias; p.out = (bf16*)y;
-  return launch<false>(tmA, tmB, p, st);
+  CUtensorMap tmO;  // NCHW output as [batch][channel][token]; blocks of 32 channels x 32 tokens
+  {
+    p.tma_store = 1;
+    const cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)Cout, (cuuint64_t)B};
+    const cuuint64_t strides[2] = {(cuuint64_t)N * 2, (cuuint64_t)Cout * N * 2};
+    const cuuint32_t box[3] = {32, 32, 1};
+    if (!tma_make_map_bf16(&tmO, y, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B))
+      return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the output projection's output");
+  }
+  return launch<false>(tmA, tmB, tmO, p, st);
 }
 
 // Non-zero once any projection GEMM of this process hit a wait time-out (synchronises the device).
