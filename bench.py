@@ -30,6 +30,8 @@ METRIC = "msla_fwd_tokens_per_s"
 UNIT = "tokens/s"
 STAGES = ("project_in", "aggregate", "kv_state", "apply", "project_out")
 FALLBACK_HBM_GBS = 6650.0
+# Plain fp32 pipes of a B200: 148 SMs x 128 FMA lanes x 1.965 GHz (max SM clock), 2 flop per FMA.
+FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 
 
 def workload_by_name(name: str) -> inputs.ModuleShape:
@@ -345,6 +347,23 @@ def main() -> None:
         core_ms = stage_ms["kv_state"] + stage_ms["apply"]
         core_gbps = (bpt["kv_state"] + bpt["apply"]) * s.B * s.N / (core_ms * 1e-3) / 1e9
         e = 4 if s.dtype == "f32" else 2
+        roofline = {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                    "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}",
+                    "traffic": recorded_traffic(dom, s.name),
+                    "algorithmic_bytes_per_launch": bpt[dom] * s.B * s.N}
+        if dom == "aggregate":
+            # The 25-tap depthwise filter runs on the plain fp32 pipes (its grouped 1x1 is on tensor
+            # cores): 25 FMA per channel and token.  At C = 256 that takes longer at the fp32 peak than
+            # the kernel's bytes take at the HBM peak, so the fp32 pipes are the binding roof.
+            dw_flops = 2 * 25 * 3 * s.Cp * s.B * s.N
+            t_alu, t_hbm = dw_flops / (FP32_PEAK_TFLOPS * 1e12), bpt[dom] * s.B * s.N / (peak * 1e9)
+            if t_alu >= t_hbm:
+                tf = dw_flops / (stage_ms[dom] * 1e-3) / 1e12
+                roofline.update({"bound": "alu", "achieved": round(tf, 2), "peak": round(FP32_PEAK_TFLOPS, 2),
+                                 "unit": "TFLOP/s", "frac": round(tf / FP32_PEAK_TFLOPS, 4),
+                                 "peak_kind": "fp32 FMA lanes x max SM clock (derived)",
+                                 "algorithmic_flops_per_launch": dw_flops,
+                                 "hbm_frac": round(achieved / peak, 4), "hbm_GBps": round(achieved, 1)})
         result = {
             "metric": METRIC, "value": whole_job_value(s.B * s.N, world, ms_total, K), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": W, "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -359,10 +378,7 @@ def main() -> None:
                     "ms_per_step": ms_e2e / K, "calls_in_flight": 3,
                     "single_stream_ms_per_step": ms_e2e_serial / K},
             "gpu_launches": int(launches),
-            "roofline": {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
-                         "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}",
-                         "traffic": recorded_traffic(dom, s.name),
-                         "algorithmic_bytes_per_launch": bpt[dom] * s.B * s.N},
+            "roofline": roofline,
             "attention_core": {"ms": round(core_ms, 5), "GBps": round(core_gbps, 1),
                                "frac_of_%s_hbm" % peak_kind: round(core_gbps / peak, 4),
                                "frac_of_8TBps": round(core_gbps / 8000.0, 4)},
