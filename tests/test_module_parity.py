@@ -69,8 +69,10 @@ def test_config4_bf16():
     util.assert_close(util.run_module(s, t), _ref(s, t), "bf16", "config 4")
 
 
-@pytest.mark.parametrize("idx", [0, 1, 2, 3])
+@pytest.mark.parametrize("idx", [0, 1, 2, 3, 4])
 def test_config5_sweep_bf16(idx):
+    """The resolution sweep, element by element against the oracle; idx 4 (512x512,
+    262144 tokens) is the shape and launch configuration the benchmark times."""
     s = inputs.CONFIG5[idx]
     t = inputs.module_inputs(s)
     util.assert_close(util.run_module(s, t), _ref(s, t), "bf16", s.name)
