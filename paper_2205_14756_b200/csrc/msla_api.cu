@@ -356,13 +356,18 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   if ((s = record(events, 2, st)) != MSLA_OK) return s;
   // 3+4. attention over 2*heads heads of [q|k|v]; outputs land at channel head*d (concat)
   const HeadView in{ms_sb, 3LL * N * d, d};
-  const HeadView ov{(long long)N * ld_att, d, ld_att};
+  // Attention output: one [N][d] plane per head when the tcgen05 output projection can take it
+  // (dense 64-byte rows for the apply kernel's stores), otherwise token-major [N][2C'].
+  const bool att_planar = desc->dtype == MSLA_BF16 && d == 32 && project_out_planar_bf16_supported(2 * Cp, desc->C_out, N);
+  const HeadView ov = att_planar ? HeadView{(long long)N * ld_att, (long long)N * d, d}
+                                 : HeadView{(long long)N * ld_att, d, ld_att};
   s = run_core(desc->dtype, ms, ms + (size_t)N * d * e, ms + (size_t)2 * N * d * e, att, in, ov, desc->B, 2 * heads, N, d, desc->eps, p.core,
                ws + p.core_off, st, events ? (cudaEvent_t)events[3] : nullptr);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 4, st)) != MSLA_OK) return s;
   // 5. output projection back to NCHW
-  s = run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st);
+  s = att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st)
+                 : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 5, st)) != MSLA_OK) return s;
   if (host_io) {

@@ -40,6 +40,9 @@ msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, 
 bool project_out_bf16_supported(int Cin, int Cout, int N);
 msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin, int Cout,
                                    int N, cudaStream_t st);
+bool project_out_planar_bf16_supported(int Cin, int Cout, int N);
+msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin,
+                                          int Cout, int N, cudaStream_t st);
 int gemm_timeout_flag();
 
 // bf16, d = 32 aggregation with TMA halo tiles (agg_bf16.cu).
