@@ -24,6 +24,9 @@
 #define MSLA_AGG_WY 2  // warps along y
 #endif
 
+#ifndef MSLA_AGG_TC_COLS
+#define MSLA_AGG_TC_COLS 4  // tap columns (dx) of the depthwise filter evaluated on tensor cores: 0, 2 or 4
+#endif
 #ifndef MSLA_AGG_MIN_BLOCKS
 #define MSLA_AGG_MIN_BLOCKS 3
 #endif
@@ -79,8 +82,12 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
   constexpr int TW = 8 * WX, TH = 8 * WY, HW_ = TW + 4, HH = TH + 4;
   constexpr int TILE_BYTES = HW_ * HH * D * 2;
   constexpr int TILE_PITCH = (TILE_BYTES + 127) / 128 * 128;
+  constexpr int TC_COLS = MSLA_AGG_TC_COLS;
   extern __shared__ __align__(128) unsigned char tiles[];  // two halo tiles (double buffer), dynamic
   __shared__ __align__(16) float wdw_s[5][5][D];           // [dx][dy][channel]
+  // Depthwise taps of the first TC_COLS tap columns as per-lane B fragments of 8x8 diagonal
+  // matrices (see below): [dx][dy][channel-pair block jn][lane].
+  __shared__ uint32_t bdiag[TC_COLS > 0 ? TC_COLS : 1][5][4][32];
   __shared__ __align__(8) unsigned long long bar_storage[2];
   __shared__ int timed_out;
 
@@ -119,6 +126,19 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
   for (int e = threadIdx.x; e < 25 * D; e += WX * WY * 32) {
     const int c = e % D, tap = e / D;  // consecutive threads -> consecutive channels: conflict-free stores
     wdw_s[tap % 5][tap / 5][c] = __bfloat162float(p.w_dw[(long long)(ch0 + c) * 25 + tap]);
+  }
+  // B fragment of diag(w[ch]) over the channel set {8t'+2jn+e}: lane (g, t) holds rows k = 2t, 2t+1 of
+  // column n = g, so only lanes with g/2 == t hold a non-zero: the tap of channel 8t+2jn+(g&1), in the
+  // low (g even) or high (g odd) half of the register.
+  for (int e = threadIdx.x; e < TC_COLS * 5 * 4 * 32; e += WX * WY * 32) {
+    const int ln = e & 31, jn = (e >> 5) & 3, dy = (e >> 7) % 5, dx = (e >> 7) / 5;
+    const int lg = ln >> 2, lt = ln & 3;
+    uint32_t v = 0;
+    if ((lg >> 1) == lt) {
+      const bf16 wv = p.w_dw[(long long)(ch0 + 8 * lt + 2 * jn + (lg & 1)) * 25 + dy * 5 + dx];
+      v = (uint32_t)__bfloat16_as_ushort(wv) << (16 * (lg & 1));
+    }
+    bdiag[dx][dy][jn][ln] = v;
   }
   // pointwise weights as B fragments: slots (2t,2t+1)+8r <-> in channels 8t+4ks+2r,+1; column g <-> out channel oc(jn)
   uint32_t bw[2][4][2];
@@ -167,8 +187,56 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) acc[r][q] = make_float2(0.f, 0.f);
     const uint32_t col_base = tiles0 + (k & 1) * TILE_PITCH + (uint32_t)(((wy * 8) * HW_ + wx * 8 + g) * (D * 2) + t * 16);
+    // Tap columns 0 .. TC_COLS-1 on tensor cores, two columns per MMA.  For one tap (dy, dx) and one
+    // block jn of 8 channels, out[pixel][ch] += in[pixel + (dy, dx)][ch] * w[ch] is the product of a
+    // 16x8 pixel-by-channel matrix with the 8x8 matrix diag(w); m16n8k16 takes the taps (dy, dx) and
+    // (dy, dx+1) at once (contraction slots 0-7 and 8-15).  With MMA rows g / g+8 = pixels (x, 2j) /
+    // (x, 2j+1) and the channel set {8t'+2jn+e}, the A fragment of lane (g, t) is word jn of the very
+    // 16 bytes it loads for the fp32 path (input rows 2j+dy, 2j+dy+1 of columns dx, dx+1), untouched,
+    // and the accumulator fragment is acc[2j][jn], acc[2j+1][jn].  Products of bf16 values are exact
+    // and accumulation is fp32: the same arithmetic as the FMA path, on a pipe that is idle here.
 #pragma unroll 1
-    for (int dx = 0; dx < 5; ++dx) {
+    for (int dx = 0; dx < TC_COLS; dx += 2) {
+      uint32_t bd0[5][4], bd1[5][4];
+#pragma unroll
+      for (int dy = 0; dy < 5; ++dy)
+#pragma unroll
+        for (int jn = 0; jn < 4; ++jn) { bd0[dy][jn] = bdiag[dx][dy][jn][lane]; bd1[dy][jn] = bdiag[dx + 1][dy][jn][lane]; }
+      uint32_t A[4][4];  // [jn][a0: row i col dx, a1: row i+1 col dx, a2: row i col dx+1, a3: row i+1 col dx+1]
+      {
+        uint32_t r0[4], r1[4];
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r0[0]), "=r"(r0[1]), "=r"(r0[2]), "=r"(r0[3])
+                     : "r"(col_base + (uint32_t)(dx * (D * 2))));
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r1[0]), "=r"(r1[1]), "=r"(r1[2]), "=r"(r1[3])
+                     : "r"(col_base + (uint32_t)((dx + 1) * (D * 2))));
+#pragma unroll
+        for (int jn = 0; jn < 4; ++jn) { A[jn][1] = r0[jn]; A[jn][3] = r1[jn]; }
+      }
+#pragma unroll
+      for (int i = 0; i < 11; ++i) {  // input rows i and i+1 feed output rows (i-dy, i-dy+1)
+        uint32_t r0[4], r1[4];
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r0[0]), "=r"(r0[1]), "=r"(r0[2]), "=r"(r0[3])
+                     : "r"(col_base + (uint32_t)(((i + 1) * HW_ + dx) * (D * 2))));
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r1[0]), "=r"(r1[1]), "=r"(r1[2]), "=r"(r1[3])
+                     : "r"(col_base + (uint32_t)(((i + 1) * HW_ + dx + 1) * (D * 2))));
+#pragma unroll
+        for (int jn = 0; jn < 4; ++jn) { A[jn][0] = A[jn][1]; A[jn][2] = A[jn][3]; A[jn][1] = r0[jn]; A[jn][3] = r1[jn]; }
+#pragma unroll
+        for (int dy = 0; dy < 5; ++dy) {
+          const int r = i - dy;
+          if (r >= 0 && r < 8 && (r & 1) == 0) {
+#pragma unroll
+            for (int jn = 0; jn < 4; ++jn) {
+              float c[4] = {acc[r][jn].x, acc[r][jn].y, acc[r + 1][jn].x, acc[r + 1][jn].y};
+              mma_bf16(c, A[jn], bd0[dy][jn], bd1[dy][jn]);
+              acc[r][jn] = make_float2(c[0], c[1]); acc[r + 1][jn] = make_float2(c[2], c[3]);
+            }
+          }
+        }
+      }
+    }
+#pragma unroll 1
+    for (int dx = TC_COLS; dx < 5; ++dx) {
       float2 w[5][4];
 #pragma unroll
       for (int dy = 0; dy < 5; ++dy) {
