@@ -139,3 +139,71 @@ def test_stage_aggregate(dtype, B, H, W, Ch, d):
     ref = _planar(oracle.group1x1(oracle.dwconv(t, w_dw), w_pw), d)
     util.assert_close(util.host(y), ref, dtype, "aggregate")
     assert binding.msla_debug_wait_timeouts() == 0
+
+
+# ------------------------------------------------- other entry points of the module
+def test_forward_host_and_profiled_match_forward():
+    """msla_forward_host (host buffers, copies inside the call) and msla_forward_profiled
+    (events between the steps) run the same kernels as msla_forward: bitwise equal output."""
+    s = inputs.ModuleShape("entry", "bf16", 2, 64, 24, 40, 2, 32, seed=31)
+    t = inputs.module_inputs(s)
+    ref = util.run_module(s, t)
+    dt = torch.bfloat16
+    x, w_qkv, w_dw, w_pw, w_proj = (util.dev(t[n], "bf16") for n in ("x", "w_qkv", "w_dw", "w_pw", "w_proj"))
+    weights = binding.make_weights(w_qkv, w_dw, w_pw, w_proj)
+    d0 = binding.make_desc(s.B, s.C, s.H, s.W, s.heads, s.d, s.C_out, binding.MSLA_BF16, s.eps)
+    nbytes = binding.msla_forward_host_workspace_bytes(d0)
+    assert nbytes > binding.msla_forward_workspace_bytes(d0)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    desc = binding.make_desc(s.B, s.C, s.H, s.W, s.heads, s.d, s.C_out, binding.MSLA_BF16, s.eps, workspace=ws)
+    # host buffers
+    hx = x.cpu().pin_memory()
+    ho = torch.empty(s.B, s.C_out, s.H, s.W, dtype=dt).pin_memory()
+    binding.msla_forward_host(desc, hx, weights, ho)
+    torch.cuda.synchronize()
+    assert np.array_equal(util.host(ho), ref)
+    # events between the steps
+    out = torch.empty(s.B, s.C_out, s.H, s.W, dtype=dt, device="cuda")
+    st = torch.cuda.current_stream()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+    for e in evs:
+        e.record(st)
+    launches = binding.msla_kernel_launches()
+    binding.msla_forward_profiled(desc, x, weights, out, st, evs)
+    torch.cuda.synchronize()
+    assert binding.msla_kernel_launches() - launches == 6
+    assert np.array_equal(util.host(out), ref)
+    assert all(evs[i].elapsed_time(evs[i + 1]) >= 0.0 for i in range(5))
+    # too small a workspace for the host variant is refused before anything runs
+    small = binding.make_desc(s.B, s.C, s.H, s.W, s.heads, s.d, s.C_out, binding.MSLA_BF16, s.eps,
+                              workspace=ws[:binding.msla_forward_workspace_bytes(d0)])
+    with pytest.raises(binding.MslaError) as err:
+        binding.msla_forward_host(small, hx, weights, ho)
+    assert err.value.status == 4
+
+
+def test_module_argument_errors_on_device():
+    s = inputs.ModuleShape("err", "bf16", 1, 64, 8, 8, 2, 32, seed=1)
+    x = torch.zeros(1, 64, 8, 8, dtype=torch.bfloat16, device="cuda")
+    w = [torch.zeros(n, dtype=torch.bfloat16, device="cuda") for n in (192 * 64, 192 * 25, 192 * 32, 64 * 128)]
+    weights = binding.make_weights(*w)
+    d0 = binding.make_desc(1, 64, 8, 8, 2, 32, 64, binding.MSLA_BF16)
+    ws = torch.empty(binding.msla_forward_workspace_bytes(d0), dtype=torch.uint8, device="cuda")
+    desc = binding.make_desc(1, 64, 8, 8, 2, 32, 64, binding.MSLA_BF16, workspace=ws)
+    with pytest.raises(binding.MslaError) as e:      # out aliases x
+        binding.msla_forward(desc, x, weights, x)
+    assert e.value.status == 1
+    out = torch.empty_like(x)
+    bad = binding.make_desc(1, 64, 8, 8, 2, 32, 64, binding.MSLA_BF16, workspace=ws[16:])
+    bad.workspace_bytes = 8
+    with pytest.raises(binding.MslaError) as e:
+        binding.msla_forward(bad, x, weights, out)
+    assert e.value.status == 4
+    binding.msla_forward(desc, x, weights, out)       # the context is still usable; zeros in, zeros out
+    torch.cuda.synchronize()
+    assert float(out.float().abs().max()) == 0.0
+
+
+def test_no_kernel_wait_timed_out():
+    """Every device-side wait in the library is bounded; none of the runs above may have hit its limit."""
+    assert binding.msla_debug_wait_timeouts() == 0
