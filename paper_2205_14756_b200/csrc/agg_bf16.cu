@@ -2,13 +2,16 @@
 // depthwise convolution and the grouped 1x1 convolution of one group of 32
 // channels in one kernel, on planar activations [planes][H*W][32].
 //
-// One CTA = one TW x TH pixel tile of one group.  A single TMA copy stages the
-// (TW+4) x (TH+4) halo tile in shared memory; coordinates outside the image are
-// zero-filled by the TMA unit, which is exactly the convolution's zero padding.
-// Each warp owns an 8x8 pixel block: lane (g = lane/4, t = lane%4) computes the
-// depthwise result of the 8 pixels of column g for channels 8t..8t+7 in fp32
-// registers (packed two-wide FMAs, sliding the 5-tap window down the column),
-// rounds it once to bf16 and uses it, in place, as the A operand of
+// One CTA = a run of TW x TH pixel tiles of one group.  TMA copies stage the
+// (TW+4) x (TH+4) halo tiles in a two-deep ring in shared memory; coordinates
+// outside the image are zero-filled by the TMA unit, which is exactly the
+// convolution's zero padding.  Each warp owns an 8x8 pixel block: lane
+// (g = lane/4, t = lane%4) accumulates, in fp32 registers, the depthwise result
+// of the 8 pixels of column g for channels 8t..8t+7.  Four of the five tap
+// columns are evaluated on tensor cores (a tap is a multiplication by a
+// diagonal matrix, and the lane's 16-byte loads are already the A fragments),
+// the fifth with packed fp32 FMAs sliding down the column.  The result is
+// rounded once to bf16 and used, in place, as the A operand of
 // mma.sync.m16n8k16 against the group's 32x32 pointwise weights: the grouped
 // 1x1 is fed from registers, with no shared-memory round trip in between.
 #include <cuda.h>
@@ -43,9 +46,6 @@ __device__ int g_agg_timeout_flag = 0;
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void fma2(float2& acc, const float2& a, const float2& b) {
-#ifdef MSLA_AGG_SCALAR_FMA
-  acc.x = fmaf(a.x, b.x, acc.x); acc.y = fmaf(a.y, b.y, acc.y); return;
-#endif
   unsigned long long& c = reinterpret_cast<unsigned long long&>(acc);
   asm("fma.rn.f32x2 %0, %1, %2, %0;"
       : "+l"(c)

@@ -3,10 +3,12 @@
 //
 // Both steps are HBM-bound only if their small contractions (d x (d+1) per
 // token) stay off the plain fp32 pipes, so each warp feeds mma.sync.m16n8k16
-// directly from registers filled by vectorised global loads.  The freedom that
-// makes this work without any shared-memory transpose: the contraction index
-// of an MMA may be assigned to tokens (reduction) or channels (apply) in any
-// order, as long as both operands use the same assignment.
+// from data that cp.async streams through per-warp shared-memory rings (bytes
+// in flight independent of registers and occupancy).  The freedom used to
+// avoid data shuffling: the contraction index of an MMA may be assigned to
+// tokens (reduction) or channels (apply) in any order, as long as both
+// operands use the same assignment; where a transpose is unavoidable (tokens
+// along the contraction, rows of channels in memory) ldmatrix.trans does it.
 #include "msla_common.cuh"
 #include "msla_host.h"
 

@@ -12,13 +12,18 @@
 //                    NCHW (the token index is contiguous: an "MN-major" operand),
 //                    B = w_qkv (K-major).
 // Output projection: m = output channel, n = token; A = w_proj (K-major),
-//                    B = attention output, token-major (K-major); D rows are
-//                    NCHW planes, so each thread stores runs of tokens.
+//                    B = attention output (K-major): either token-major
+//                    [N][2C'] or one [N][32] plane per head; D rows are NCHW
+//                    planes, so a row of the tile is a run of tokens.
 //
 // One persistent CTA per SM, warp-specialised: warp 0 issues TMA, warp 1
 // issues MMAs (and owns the tensor-memory allocation), warps 2-9 drain the
 // accumulators.  Two 128x256 fp32 accumulators (all 512 TMEM columns) let the
-// epilogue of one tile overlap the MMAs of the next.  Every mbarrier wait is
+// epilogue of one tile overlap the MMAs of the next.  The epilogue converts to
+// bf16, stages 32x32 blocks in shared memory and writes them with TMA stores
+// (whole lines; a lane-per-row store of 16-byte pieces was twice as slow).
+// A second kernel keeps the CTA's weight block resident in shared memory and
+// streams only activations (used for the input projection).  Every mbarrier wait is
 // bounded: on time-out the CTA raises a flag, all roles leave their loops, the
 // tensor memory is released and the kernel returns.
 #include <cuda.h>
