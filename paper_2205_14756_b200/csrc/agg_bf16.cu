@@ -76,12 +76,20 @@ struct AggParams {
   int tiles_per_cta;           // consecutive tiles of one plane handled by one CTA
 };
 
-template <int WX, int WY>
+// D16 = false: one group of 32 channels, planes [H*W][32].
+// D16 = true : d = 16.  Two neighbouring groups of 16 channels are handled as one block of 32 channels
+// (the depthwise part does not care about groups; the 1x1 becomes block-diagonal).  Their two planes
+// [H*W][16] are staged as two tiles; the second one is fetched two pixels further left, so that it sits
+// 64 bytes further on in shared memory and the two planes' 16-byte chunks fall into different banks.
+template <int WX, int WY, bool D16>
 __global__ void __launch_bounds__(WX * WY * 32, MSLA_AGG_MIN_BLOCKS)
 aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
-  constexpr int TW = 8 * WX, TH = 8 * WY, HW_ = TW + 4, HH = TH + 4;
-  constexpr int TILE_BYTES = HW_ * HH * D * 2;
-  constexpr int TILE_PITCH = (TILE_BYTES + 127) / 128 * 128;
+  constexpr int TW = 8 * WX, TH = 8 * WY, HH = TH + 4;
+  constexpr int HW_ = D16 ? TW + 6 : TW + 4;          // pixels per staged row (d = 16: two spare columns)
+  constexpr int PIXB = D16 ? 32 : 64;                  // bytes per staged pixel
+  constexpr int PLANE_BYTES = HW_ * HH * PIXB;         // one TMA box
+  constexpr int TILE_BYTES = D16 ? 2 * PLANE_BYTES : PLANE_BYTES;
+  constexpr int TILE_PITCH = (TILE_BYTES + 64 + 127) / 128 * 128;
   constexpr int TC_COLS = MSLA_AGG_TC_COLS;
   extern __shared__ __align__(128) unsigned char tiles[];  // two halo tiles (double buffer), dynamic
   __shared__ __align__(16) float wdw_s[5][5][D];           // [dx][dy][channel]
@@ -111,8 +119,13 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(TILE_BYTES) : "memory");
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(tiles0 + (k & 1) * TILE_PITCH), "l"(&tm_src), "r"(bar), "r"(0), "r"(tx0 - 2), "r"(ty0 - 2), "r"(plane_idx)
-        : "memory");
+        ::"r"(tiles0 + (k & 1) * TILE_PITCH), "l"(&tm_src), "r"(bar), "r"(0), "r"(tx0 - 2), "r"(ty0 - 2),
+          "r"(D16 ? 2 * plane_idx - b * p.src_planes_per_batch : plane_idx) : "memory");
+    if (D16)  // second plane of the pair, two pixels further left (see above)
+      asm volatile(
+          "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+          ::"r"(tiles0 + (k & 1) * TILE_PITCH + PLANE_BYTES), "l"(&tm_src), "r"(bar), "r"(0), "r"(tx0 - 4), "r"(ty0 - 2),
+            "r"(2 * plane_idx - b * p.src_planes_per_batch + 1) : "memory");
   };
 
   if (threadIdx.x == 0) {
@@ -149,11 +162,18 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
 #pragma unroll
       for (int r = 0; r < 2; ++r) {
         const int oc = 8 * (g >> 1) + 2 * jn + (g & 1);
-        bw[ks][jn][r] = *reinterpret_cast<const uint32_t*>(p.w_pw + (long long)(ch0 + oc) * D + 8 * t + 4 * ks + 2 * r);
+        const int ic = 8 * t + 4 * ks + 2 * r;  // first in-channel of the pair, inside the block of 32
+        if (D16)  // block-diagonal: two 16x16 groups
+          bw[ks][jn][r] = (oc >> 4) == (ic >> 4)
+                              ? *reinterpret_cast<const uint32_t*>(p.w_pw + (long long)(ch0 + oc) * 16 + (ic & 15)) : 0u;
+        else
+          bw[ks][jn][r] = *reinterpret_cast<const uint32_t*>(p.w_pw + (long long)(ch0 + oc) * D + ic);
       }
   __syncthreads();  // barriers initialised and taps staged before anyone proceeds
 
-  bf16* plane = p.dst + (long long)b * p.dst_batch_stride + (long long)group * p.H * p.W * D;
+  // output: plane `group` of 32 channels, or for d = 16 the plane (2*group + t/2) of 16 channels
+  bf16* plane = D16 ? p.dst + (long long)b * p.dst_batch_stride + (long long)(2 * group + (t >> 1)) * p.H * p.W * 16
+                    : p.dst + (long long)b * p.dst_batch_stride + (long long)group * p.H * p.W * D;
 #pragma unroll 1
   for (int k = 0; k < tile_count; ++k) {
     // prefetch the next tile into the buffer everyone left at the end of iteration k-1
@@ -186,7 +206,10 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
     for (int r = 0; r < 8; ++r)
 #pragma unroll
       for (int q = 0; q < 4; ++q) acc[r][q] = make_float2(0.f, 0.f);
-    const uint32_t col_base = tiles0 + (k & 1) * TILE_PITCH + (uint32_t)(((wy * 8) * HW_ + wx * 8 + g) * (D * 2) + t * 16);
+    // this lane's 16 bytes of the pixel at (row 0, column 0) of its column's window
+    const uint32_t col_base = tiles0 + (k & 1) * TILE_PITCH +
+                              (D16 ? (uint32_t)((t >> 1) * (PLANE_BYTES + 64) + ((wy * 8) * HW_ + wx * 8 + g) * PIXB + (t & 1) * 16)
+                                   : (uint32_t)(((wy * 8) * HW_ + wx * 8 + g) * PIXB + t * 16));
     // Tap columns 0 .. TC_COLS-1 on tensor cores, two columns per MMA.  For one tap (dy, dx) and one
     // block jn of 8 channels, out[pixel][ch] += in[pixel + (dy, dx)][ch] * w[ch] is the product of a
     // 16x8 pixel-by-channel matrix with the 8x8 matrix diag(w); m16n8k16 takes the taps (dy, dx) and
@@ -206,9 +229,9 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
       {
         uint32_t r0[4], r1[4];
         asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r0[0]), "=r"(r0[1]), "=r"(r0[2]), "=r"(r0[3])
-                     : "r"(col_base + (uint32_t)(dx * (D * 2))));
+                     : "r"(col_base + (uint32_t)(dx * PIXB)));
         asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r1[0]), "=r"(r1[1]), "=r"(r1[2]), "=r"(r1[3])
-                     : "r"(col_base + (uint32_t)((dx + 1) * (D * 2))));
+                     : "r"(col_base + (uint32_t)((dx + 1) * PIXB)));
 #pragma unroll
         for (int jn = 0; jn < 4; ++jn) { A[jn][1] = r0[jn]; A[jn][3] = r1[jn]; }
       }
@@ -216,9 +239,9 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
       for (int i = 0; i < 11; ++i) {  // input rows i and i+1 feed output rows (i-dy, i-dy+1)
         uint32_t r0[4], r1[4];
         asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r0[0]), "=r"(r0[1]), "=r"(r0[2]), "=r"(r0[3])
-                     : "r"(col_base + (uint32_t)(((i + 1) * HW_ + dx) * (D * 2))));
+                     : "r"(col_base + (uint32_t)(((i + 1) * HW_ + dx) * PIXB)));
         asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r1[0]), "=r"(r1[1]), "=r"(r1[2]), "=r"(r1[3])
-                     : "r"(col_base + (uint32_t)(((i + 1) * HW_ + dx + 1) * (D * 2))));
+                     : "r"(col_base + (uint32_t)(((i + 1) * HW_ + dx + 1) * PIXB)));
 #pragma unroll
         for (int jn = 0; jn < 4; ++jn) { A[jn][0] = A[jn][1]; A[jn][2] = A[jn][3]; A[jn][1] = r0[jn]; A[jn][3] = r1[jn]; }
 #pragma unroll
@@ -250,7 +273,7 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
         uint32_t raw[4];
         asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
                      : "=r"(raw[0]), "=r"(raw[1]), "=r"(raw[2]), "=r"(raw[3])
-                     : "r"(col_base + (uint32_t)((i * HW_ + dx) * (D * 2))));
+                     : "r"(col_base + (uint32_t)((i * HW_ + dx) * PIXB)));
         float2 in[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) in[q] = unpack_bf16x2(raw[q]);
@@ -287,7 +310,7 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
       for (int half = 0; half < 2; ++half) {
         const int y = y0 + wy * 8 + 2 * j + half;
         if (x < p.W && y < p.H) {
-          bf16* dst = plane + ((long long)y * p.W + x) * D + 8 * t;
+          bf16* dst = D16 ? plane + ((long long)y * p.W + x) * 16 + 8 * (t & 1) : plane + ((long long)y * p.W + x) * D + 8 * t;
           asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(dst),
                        "r"(pack_bf16(c[0][2 * half], c[0][2 * half + 1])), "r"(pack_bf16(c[1][2 * half], c[1][2 * half + 1])),
                        "r"(pack_bf16(c[2][2 * half], c[2][2 * half + 1])), "r"(pack_bf16(c[3][2 * half], c[3][2 * half + 1]))
@@ -302,19 +325,21 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
 }  // namespace
 
 bool aggregate_bf16_supported(int H, int W, int Ch, int d) {
-  return d == 32 && Ch % 32 == 0 && H >= 1 && W >= 1;
+  return (d == 32 || d == 16) && Ch % 32 == 0 && H >= 1 && W >= 1;
 }
 
-// src, dst: planar bf16 [.., planes, H*W, 32]; group g of image b is plane b*src_ppb + g of src
-// (src_planes_total planes in all) and lives at dst + b*dst_sb + g*H*W*32.
-msla_status_t run_aggregate_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
-                                 const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch,
-                                 cudaStream_t st) {
+namespace {
+template <bool D16>
+msla_status_t launch_aggregate(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
+                               const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch,
+                               cudaStream_t st) {
   constexpr int WX = MSLA_AGG_WX, WY = MSLA_AGG_WY, TW = 8 * WX, TH = 8 * WY;
+  constexpr int DP = D16 ? 16 : 32;           // channels per plane
+  constexpr int BOXW = D16 ? TW + 6 : TW + 4;  // staged pixels per row
   CUtensorMap tm;
-  const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)src_planes_total};
-  const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)W * D * 2, (cuuint64_t)H * W * D * 2};
-  const cuuint32_t box[4] = {(cuuint32_t)D, (cuuint32_t)(TW + 4), (cuuint32_t)(TH + 4), 1};
+  const cuuint64_t dims[4] = {(cuuint64_t)DP, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)src_planes_total};
+  const cuuint64_t strides[3] = {(cuuint64_t)DP * 2, (cuuint64_t)W * DP * 2, (cuuint64_t)H * W * DP * 2};
+  const cuuint32_t box[4] = {(cuuint32_t)DP, (cuuint32_t)BOXW, (cuuint32_t)(TH + 4), 1};
   if (!tma_make_map_bf16(&tm, src, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
     return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the aggregation input");
   AggParams p;
@@ -328,15 +353,26 @@ msla_status_t run_aggregate_bf16(const void* src, long long src_planes_total, in
   const long long units = tiles * (Ch / D) * B;
   p.tiles_per_cta = units >= 8 * 2400 ? 8 : units >= 4 * 2400 ? 4 : units >= 2 * 2400 ? 2 : 1;
   dim3 grid((unsigned)((tiles + p.tiles_per_cta - 1) / p.tiles_per_cta), (unsigned)(Ch / D), (unsigned)B);
-  constexpr int tile_bytes = 2 * (((TW + 4) * (TH + 4) * D * 2 + 127) / 128 * 128);
+  constexpr int one_tile = (D16 ? 2 : 1) * BOXW * (TH + 4) * DP * 2;
+  constexpr int tile_bytes = 2 * ((one_tile + 64 + 127) / 128 * 128);  // must match TILE_PITCH in the kernel
   static bool attr_done = false;
   if (!attr_done) {
-    cudaFuncSetAttribute(aggregate_bf16_kernel<WX, WY>, cudaFuncAttributeMaxDynamicSharedMemorySize, tile_bytes);
+    cudaFuncSetAttribute(aggregate_bf16_kernel<WX, WY, D16>, cudaFuncAttributeMaxDynamicSharedMemorySize, tile_bytes);
     attr_done = true;
   }
-  aggregate_bf16_kernel<WX, WY><<<grid, WX * WY * 32, tile_bytes, st>>>(tm, p);
+  aggregate_bf16_kernel<WX, WY, D16><<<grid, WX * WY * 32, tile_bytes, st>>>(tm, p);
   count_launches(1);
   return check_launch("token aggregation (bf16)");
+}
+}  // namespace
+
+// src, dst: planar bf16 [.., planes, H*W, d], d in {16, 32}; group g of image b is plane b*src_ppb + g of
+// src (src_planes_total planes in all) and lives at dst + b*dst_sb + g*H*W*d.  Ch must be a multiple of 32.
+msla_status_t run_aggregate_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
+                                 const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch, int d,
+                                 cudaStream_t st) {
+  return d == 16 ? launch_aggregate<true>(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_sb, B, H, W, Ch, st)
+                 : launch_aggregate<false>(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_sb, B, H, W, Ch, st);
 }
 
 int agg_timeout_flag() {

@@ -281,7 +281,7 @@ static msla_status_t run_aggregate(msla_dtype_t dt, const void* src, const void*
                                    long long dst_sb, cudaStream_t st) {
   const long long plane = (long long)H * W * d;
   if (dt == MSLA_BF16 && aggregate_bf16_supported(H, W, Ch, d) && src_sb % plane == 0)
-    return run_aggregate_bf16(src, (long long)B * (src_sb / plane), (int)(src_sb / plane), w_dw, w_pw, dst, dst_sb, B, H, W, Ch, st);
+    return run_aggregate_bf16(src, (long long)B * (src_sb / plane), (int)(src_sb / plane), w_dw, w_pw, dst, dst_sb, B, H, W, Ch, d, st);
   dim3 grid((unsigned)(ceil_div_ll(W, 8) * ceil_div_ll(H, 8)), (unsigned)(Ch / d), (unsigned)B);
   if (dt == MSLA_F32)
     generic::aggregate_kernel<float><<<grid, 256, 0, st>>>((const float*)src, (const float*)w_dw, (const float*)w_pw,

@@ -45,10 +45,10 @@ msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const vo
                                           int Cout, int N, cudaStream_t st);
 int gemm_timeout_flag();
 
-// bf16, d = 32 aggregation with TMA halo tiles (agg_bf16.cu).
+// bf16 aggregation (d = 16 or 32, Ch a multiple of 32) with TMA halo tiles (agg_bf16.cu).
 bool aggregate_bf16_supported(int H, int W, int Ch, int d);
 msla_status_t run_aggregate_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
-                                 const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch,
+                                 const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch, int d,
                                  cudaStream_t st);
 int agg_timeout_flag();
 

@@ -31,6 +31,8 @@ SMALL = [
     ("r5", "bf16", 1, 96, 24, 20, 3, 32),
     ("r6", "bf16", 3, 64, 17, 16, 4, 16),
     ("r7", "f32", 1, 16, 1, 1, 1, 16),
+    ("r8", "bf16", 1, 128, 40, 24, 8, 16),
+    ("r9", "bf16", 2, 48, 11, 13, 3, 16),
 ]
 
 
@@ -128,7 +130,9 @@ def test_stage_project_out(dtype, B, Cin, Cout, N):
 
 @pytest.mark.parametrize("dtype,B,H,W,Ch,d", [("f32", 1, 6, 9, 48, 16), ("bf16", 2, 13, 21, 96, 32), ("bf16", 1, 1, 5, 32, 32),
                                               ("bf16", 1, 64, 64, 192, 32), ("bf16", 1, 3, 70, 64, 16), ("bf16", 2, 16, 16, 32, 32),
-                                              ("bf16", 1, 17, 35, 64, 32), ("bf16", 1, 5, 3, 32, 32), ("bf16", 1, 40, 7, 32, 32)])
+                                              ("bf16", 1, 17, 35, 64, 32), ("bf16", 1, 5, 3, 32, 32), ("bf16", 1, 40, 7, 32, 32),
+                                              ("bf16", 2, 19, 37, 96, 16), ("bf16", 1, 64, 64, 192, 16), ("bf16", 1, 2, 2, 32, 16),
+                                              ("bf16", 1, 9, 9, 48, 16)])
 def test_stage_aggregate(dtype, B, H, W, Ch, d):
     t = inputs.quantise(inputs.normal(3, 0, B * Ch * H * W).reshape(B, Ch, H, W), dtype)
     w_dw = inputs.quantise(inputs.normal(3, 1, Ch * 25, 0.2).reshape(Ch, 5, 5), dtype)
