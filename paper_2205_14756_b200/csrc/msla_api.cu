@@ -280,8 +280,23 @@ static msla_status_t run_aggregate(msla_dtype_t dt, const void* src, const void*
                                    void* dst, int B, int H, int W, int Ch, int d, long long src_sb,
                                    long long dst_sb, cudaStream_t st) {
   const long long plane = (long long)H * W * d;
-  if (dt == MSLA_BF16 && aggregate_bf16_supported(H, W, Ch, d) && src_sb % plane == 0)
-    return run_aggregate_bf16(src, (long long)B * (src_sb / plane), (int)(src_sb / plane), w_dw, w_pw, dst, dst_sb, B, H, W, Ch, d, st);
+  if (dt == MSLA_BF16 && src_sb % plane == 0) {
+    if (aggregate_bf16_supported(H, W, Ch, d))
+      return run_aggregate_bf16(src, (long long)B * (src_sb / plane), (int)(src_sb / plane), w_dw, w_pw, dst, dst_sb, B, H, W, Ch, d, st);
+    if (d == 16 && Ch > 16 && aggregate_bf16_supported(H, W, Ch - 16, d)) {
+      // odd number of 16-channel groups: the tuned kernel takes them in pairs, the plain one the last group
+      msla_status_t s = run_aggregate_bf16(src, (long long)B * (src_sb / plane), (int)(src_sb / plane), w_dw, w_pw, dst, dst_sb, B, H, W, Ch - 16, d, st);
+      if (s != MSLA_OK) return s;
+      const __nv_bfloat16* s16 = (const __nv_bfloat16*)src + (long long)(Ch / 16 - 1) * plane;
+      __nv_bfloat16* d16 = (__nv_bfloat16*)dst + (long long)(Ch / 16 - 1) * plane;
+      dim3 grid1((unsigned)(ceil_div_ll(W, 8) * ceil_div_ll(H, 8)), 1u, (unsigned)B);
+      generic::aggregate_kernel<__nv_bfloat16><<<grid1, 256, 0, st>>>(s16, (const __nv_bfloat16*)w_dw + (long long)(Ch - 16) * 25,
+                                                                      (const __nv_bfloat16*)w_pw + (long long)(Ch - 16) * 16, d16, H, W, d,
+                                                                      src_sb, dst_sb);
+      count_launches(1);
+      return check_launch("token aggregation (last group)");
+    }
+  }
   dim3 grid((unsigned)(ceil_div_ll(W, 8) * ceil_div_ll(H, 8)), (unsigned)(Ch / d), (unsigned)B);
   if (dt == MSLA_F32)
     generic::aggregate_kernel<float><<<grid, 256, 0, st>>>((const float*)src, (const float*)w_dw, (const float*)w_pw,
