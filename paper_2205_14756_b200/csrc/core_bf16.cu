@@ -247,7 +247,10 @@ kv_combine_bf16path_kernel(const float* __restrict__ partial, float* __restrict_
 // The fp32 state is fed as bf16 hi + bf16 lo (two MMAs) to keep ~16 mantissa
 // bits; one extra tile whose columns all hold ks gives the denominator.
 // ---------------------------------------------------------------------------
-template <int D, int NWARPS, int STAGES, int U>
+// PAIR: one CTA serves heads 2p (even warps) and 2p+1 (odd warps) of a paired
+// output view, so that the two 64-byte halves of each 128-byte output row are
+// written at nearly the same time.
+template <int D, int NWARPS, int STAGES, int U, bool PAIR>
 __global__ void __launch_bounds__(NWARPS * 32)
 apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf16* __restrict__ out,
                  HeadView qv, HeadView ov, int heads, int N, float eps, int tok_per_cta) {
@@ -263,20 +266,23 @@ apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf
   __shared__ __align__(16) unsigned char fifo[NWARPS * STAGES * STAGEB];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int bh = blockIdx.y;
+  constexpr int NW = PAIR ? NWARPS / 2 : NWARPS;  // warps sharing one head's tokens
+  const int wslot = PAIR ? warp >> 1 : warp;
+  const int bh = PAIR ? 2 * blockIdx.y + (warp & 1) : blockIdx.y;
   const int b = bh / heads, h = bh % heads;
   const long long qbase = (long long)b * qv.batch + (long long)h * qv.head + t * CPT;
-  const long long obase = (long long)b * ov.batch + (long long)h * ov.head + t * CPT;
+  const long long obase = PAIR ? (long long)b * ov.batch + (long long)(h >> 1) * ov.head + (h & 1) * D + t * CPT
+                               : (long long)b * ov.batch + (long long)h * ov.head + t * CPT;
   const int n_begin = blockIdx.x * tok_per_cta;
   const int n_end = min(N, n_begin + tok_per_cta);
   constexpr int TS = 16 * U;
   const int groups = (n_end - n_begin + TS - 1) / TS;
-  const int my_groups = groups > warp ? (groups - warp + NWARPS - 1) / NWARPS : 0;
+  const int my_groups = groups > wslot ? (groups - wslot + NW - 1) / NW : 0;
   const uint32_t ring = smem_u32(fifo) + warp * (STAGES * STAGEB) + lane * LB;
 
   auto issue = [&](int it) {
     const uint32_t dst = ring + (it % STAGES) * STAGEB;
-    const int n0 = n_begin + (warp + it * NWARPS) * TS + g;
+    const int n0 = n_begin + (wslot + it * NW) * TS + g;
 #pragma unroll
     for (int u = 0; u < 2 * U; ++u) {  // u even: token g of tile u/2, odd: token g+8
       const int n = n0 + u * 8;
@@ -318,7 +324,7 @@ apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf
     cp_async_commit();
     cp_async_wait<STAGES - 1>();
     const uint32_t src = ring + (it % STAGES) * STAGEB;
-    const int n0 = n_begin + (warp + it * NWARPS) * TS;
+    const int n0 = n_begin + (wslot + it * NW) * TS;
     uint32_t qa[U][WQ], qb[U][WQ];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -388,9 +394,15 @@ msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out
   const long long total = BH * p.ne;
   kv_combine_bf16path_kernel<<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>(partial, state, p.S, p.ne, total);
   if (mid) cudaEventRecord(mid, st);
-  const int tok_per_cta = p.apply_tokens;
-  apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U><<<dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)BH), AP_WARPS * 32, 0, st>>>(
-      q, state, out, in, ov, heads, N, eps, tok_per_cta);
+  if (ov.pair) {  // heads is even here, so a pair never straddles two images
+    const int tok_per_cta = p.apply_tokens / 2;
+    apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, true><<<dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)(BH / 2)), AP_WARPS * 32, 0, st>>>(
+        q, state, out, in, ov, heads, N, eps, tok_per_cta);
+  } else {
+    const int tok_per_cta = p.apply_tokens;
+    apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, false><<<dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)BH), AP_WARPS * 32, 0, st>>>(
+        q, state, out, in, ov, heads, N, eps, tok_per_cta);
+  }
   count_launches(3);
   return check_launch("attention core kernels (bf16)");
 }

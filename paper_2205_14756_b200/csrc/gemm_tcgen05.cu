@@ -13,7 +13,7 @@
 //                    B = w_qkv (K-major).
 // Output projection: m = output channel, n = token; A = w_proj (K-major),
 //                    B = attention output (K-major): either token-major
-//                    [N][2C'] or one [N][32] plane per head; D rows are NCHW
+//                    [N][2C'] or one [N][64] plane per pair of heads; D rows are NCHW
 //                    planes, so a row of the tile is a run of tokens.
 //
 // One persistent CTA per SM, warp-specialised: warp 0 issues TMA, warp 1
@@ -118,12 +118,6 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
 __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo16, uint32_t sbo16) {
   return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)lbo16 << 16) | ((uint64_t)sbo16 << 32) |
          (1ull << 46) /* descriptor version */ | (2ull << 61) /* SWIZZLE_128B */;
-}
-
-// K-major operand with 64-byte rows and 64-byte swizzle: groups of 8 rows are 512 B apart.
-__device__ __forceinline__ uint64_t make_desc64(uint32_t addr) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(512 >> 4) << 32) | (1ull << 46) |
-         (4ull << 61) /* SWIZZLE_64B */;
 }
 
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -236,9 +230,8 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUt
   }
 }
 
-// B_PLANAR (output projection with the attention output kept as one [N][32]
-// plane per head): a 64-wide k-slice is two planes, each loaded as its own
-// 64-byte-swizzled sub-tile; the matching halves of the weight tile likewise.
+// B_PLANAR (output projection with the attention output kept as one [N][64]
+// plane per pair of heads): the 64-wide k-slice kb of B is plane kb of the image.
 template <bool A_MN_MAJOR, bool B_PLANAR>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -294,11 +287,9 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
           if (!ok) break;
           const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
           mbar_expect_tx(full_bar + 8 * s, STAGE_BYTES);
-          if (B_PLANAR) {    // per half: 32 k x 128 weight rows, and one head plane: 32 channels x 256 tokens
+          if (B_PLANAR) {    // 64 k x 128 weight rows, and one plane: 64 channels x 256 tokens
             tma_load_3d(sa, &tmA, full_bar + 8 * s, kb * BK, mt * BM, 0);
-            tma_load_3d(sa + A_STAGE_BYTES / 2, &tmA, full_bar + 8 * s, kb * BK + 32, mt * BM, 0);
-            tma_load_3d(sb, &tmB, full_bar + 8 * s, 0, nt * BN, b * p.planes_per_batch + 2 * kb);
-            tma_load_3d(sb + B_STAGE_BYTES / 2, &tmB, full_bar + 8 * s, 0, nt * BN, b * p.planes_per_batch + 2 * kb + 1);
+            tma_load_3d(sb, &tmB, full_bar + 8 * s, 0, nt * BN, b * p.planes_per_batch + kb);
           } else {
             if (A_MN_MAJOR) {  // two boxes of 64 tokens x 64 k
               tma_load_3d(sa, &tmA, full_bar + 8 * s, mt * BM, kb * BK, b);
@@ -335,14 +326,9 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
           for (int kk = 0; kk < BK / 16; ++kk) {
             // MN-major A: 16 k-slices of 128 B further on; K-major: 32 B along the swizzled row
             uint64_t ad, bd;
-            if (B_PLANAR) {  // half kk/2 of the stage, 32 B further along its 64-byte rows for odd kk
-              ad = make_desc64(sa + (kk >> 1) * (A_STAGE_BYTES / 2) + (kk & 1) * 32);
-              bd = make_desc64(sb + (kk >> 1) * (B_STAGE_BYTES / 2) + (kk & 1) * 32);
-            } else {
-              ad = A_MN_MAJOR ? make_desc(sa + kk * 2048, (A_STAGE_BYTES / 2) >> 4, 1024 >> 4)
-                              : make_desc(sa + kk * 32, 1, 1024 >> 4);
-              bd = make_desc(sb + kk * 32, 1, 1024 >> 4);
-            }
+            ad = A_MN_MAJOR ? make_desc(sa + kk * 2048, (A_STAGE_BYTES / 2) >> 4, 1024 >> 4)
+                            : make_desc(sa + kk * 32, 1, 1024 >> 4);
+            bd = make_desc(sb + kk * 32, 1, 1024 >> 4);
             umma_bf16(d_tmem, ad, bd, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
           }
           umma_commit(empty_bar + 8 * s);  // stage reusable once these MMAs have read it
@@ -678,23 +664,17 @@ msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bia
 
 bool project_out_planar_bf16_supported(int Cin, int Cout, int N) { return Cin % 64 == 0 && N % 8 == 0 && Cout >= 1; }
 
-// Same product with the attention output kept planar: a[b][j / 32][n][j % 32] (one [N][32] plane per head).
+// Same product with the attention output kept planar: a[b][j / 64][n][j % 64] (one [N][64] plane per pair of heads).
 msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin,
                                           int Cout, int N, cudaStream_t st) {
   CUtensorMap tmA, tmB, tmO;
-  const int planes = Cin / 32;
+  const int planes = Cin / 64;
   {
-    const cuuint64_t dA[3] = {(cuuint64_t)Cin, (cuuint64_t)Cout, 1};
-    const cuuint64_t sA[2] = {(cuuint64_t)Cin * 2, (cuuint64_t)Cin * Cout * 2};
-    const cuuint32_t bA[3] = {32, (cuuint32_t)BM, 1};
-    const cuuint64_t dB[3] = {32, (cuuint64_t)N, (cuuint64_t)B * planes};
-    const cuuint64_t sB[2] = {64, (cuuint64_t)N * 64};
-    const cuuint32_t bB[3] = {32, (cuuint32_t)BN, 1};
     const cuuint64_t dO[3] = {(cuuint64_t)N, (cuuint64_t)Cout, (cuuint64_t)B};
     const cuuint64_t sO[2] = {(cuuint64_t)N * 2, (cuuint64_t)Cout * N * 2};
     const cuuint32_t bO[3] = {32, 32, 1};
-    if (!tma_make_map_bf16(&tmA, w, 3, dA, sA, bA, CU_TENSOR_MAP_SWIZZLE_64B) ||
-        !tma_make_map_bf16(&tmB, a, 3, dB, sB, bB, CU_TENSOR_MAP_SWIZZLE_64B) ||
+    if (!make_map(&tmA, w, (uint64_t)Cin, (uint64_t)Cout, 1, (uint64_t)Cin * 2, (uint64_t)Cin * Cout * 2, BK, BM) ||
+        !make_map(&tmB, a, 64, (uint64_t)N, (uint64_t)B * planes, 128, (uint64_t)N * 128, BK, BN) ||
         !tma_make_map_bf16(&tmO, y, 3, dO, sO, bO, CU_TENSOR_MAP_SWIZZLE_64B))
       return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the output projection");
   }

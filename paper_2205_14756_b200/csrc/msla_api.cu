@@ -114,12 +114,15 @@ static msla_status_t run_core(msla_dtype_t dtype, const void* q, const void* k, 
                               void* out, HeadView in, HeadView ov, int B, int heads, int N, int d,
                               float eps, const CorePlan& p, void* ws, cudaStream_t st,
                               cudaEvent_t mid = nullptr) {
+  if (ov.pair && (dtype != MSLA_BF16 || (heads & 1)))  // only the bf16 tensor-core kernels write paired planes
+    return fail(MSLA_ERR_UNSUPPORTED, "paired output planes need bf16 and an even number of heads");
   if (dtype == MSLA_F32)
     return run_core_generic<float>((const float*)q, (const float*)k, (const float*)v, (float*)out,
                                    in, ov, B, heads, N, d, eps, p, (char*)ws, st, mid);
   const bool strides_ok = in.batch % 8 == 0 && in.head % 8 == 0 && in.ld % 8 == 0 && ov.batch % 8 == 0 &&
                           ov.head % 8 == 0 && ov.ld % 8 == 0;
   if (strides_ok) return run_core_bf16(q, k, v, out, in, ov, B, heads, N, d, eps, p, ws, st, mid);
+  if (ov.pair) return fail(MSLA_ERR_UNSUPPORTED, "paired output planes need strides that are multiples of 8 elements");
   return run_core_generic<__nv_bfloat16>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
                                          (const __nv_bfloat16*)v, (__nv_bfloat16*)out, in, ov, B,
                                          heads, N, d, eps, p, (char*)ws, st, mid);
@@ -371,11 +374,12 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   if ((s = record(events, 2, st)) != MSLA_OK) return s;
   // 3+4. attention over 2*heads heads of [q|k|v]; outputs land at channel head*d (concat)
   const HeadView in{ms_sb, 3LL * N * d, d};
-  // Attention output: one [N][d] plane per head when the tcgen05 output projection can take it
-  // (dense 64-byte rows for the apply kernel's stores), otherwise token-major [N][2C'].
+  // Attention output: one [N][2d] plane per pair of heads when the tcgen05 output projection can
+  // take it (dense 128-byte rows for the apply kernel's stores and the GEMM's tile loads),
+  // otherwise token-major [N][2C'].
   const bool att_planar = desc->dtype == MSLA_BF16 && d == 32 && project_out_planar_bf16_supported(2 * Cp, desc->C_out, N);
-  const HeadView ov = att_planar ? HeadView{(long long)N * ld_att, (long long)N * d, d}
-                                 : HeadView{(long long)N * ld_att, d, ld_att};
+  const HeadView ov = att_planar ? HeadView{(long long)N * ld_att, (long long)N * 2 * d, 2 * d, 1}
+                                 : HeadView{(long long)N * ld_att, d, ld_att, 0};
   s = run_core(desc->dtype, ms, ms + (size_t)N * d * e, ms + (size_t)2 * N * d * e, att, in, ov, desc->B, 2 * heads, N, d, desc->eps, p.core,
                ws + p.core_off, st, events ? (cudaEvent_t)events[3] : nullptr);
   if (s != MSLA_OK) return s;

@@ -12,10 +12,14 @@ namespace msla {
 // Dense [B, heads, N, d] input:        batch = heads*N*d, head = N*d, ld = d.
 // Token-major multi-scale buffer
 // [B, N, 6C'] with [q|k|v] per head:   batch = N*6C',  head = 3d,  ld = 6C'.
+// Paired heads (pair = 1, outputs only): heads 2p and 2p+1 share one [N][2d]
+// plane, head 2p+1 in its upper d columns:
+//   t[b * batch + (h / 2) * head + (h % 2) * d + n * ld + i],  ld = 2d.
 struct HeadView {
   long long batch;
   long long head;
   long long ld;
+  int pair;
 };
 
 __device__ __forceinline__ float to_f32(float v) { return v; }
