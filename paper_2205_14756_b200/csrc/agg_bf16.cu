@@ -128,11 +128,13 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
             "r"(2 * plane_idx - b * p.src_planes_per_batch + 1) : "memory");
   };
 
+  pdl_launch_dependents();
   if (threadIdx.x == 0) {
     timed_out = 0;
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0) : "memory");
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    pdl_wait();  // the planes read here come from the previous kernel; the tables below only need the weights
     issue(0);
   }
   // depthwise taps -> fp32 [dx][dy][c] while the first copy is in flight
@@ -170,6 +172,7 @@ aggregate_bf16_kernel(const __grid_constant__ CUtensorMap tm_src, AggParams p) {
           bw[ks][jn][r] = *reinterpret_cast<const uint32_t*>(p.w_pw + (long long)(ch0 + oc) * D + ic);
       }
   __syncthreads();  // barriers initialised and taps staged before anyone proceeds
+  pdl_wait();
 
   // output: plane `group` of 32 channels, or for d = 16 the plane (2*group + t/2) of 16 channels
   bf16* plane = D16 ? p.dst + (long long)b * p.dst_batch_stride + (long long)(2 * group + (t >> 1)) * p.H * p.W * 16
@@ -360,7 +363,7 @@ msla_status_t launch_aggregate(const void* src, long long src_planes_total, int 
     cudaFuncSetAttribute(aggregate_bf16_kernel<WX, WY, D16>, cudaFuncAttributeMaxDynamicSharedMemorySize, tile_bytes);
     attr_done = true;
   }
-  aggregate_bf16_kernel<WX, WY, D16><<<grid, WX * WY * 32, tile_bytes, st>>>(tm, p);
+  launch_pdl(aggregate_bf16_kernel<WX, WY, D16>, grid, dim3(WX * WY * 32), tile_bytes, st, tm, p);
   count_launches(1);
   return check_launch("token aggregation (bf16)");
 }

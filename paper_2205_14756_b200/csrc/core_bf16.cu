@@ -113,6 +113,8 @@ kv_state_mma_kernel(const bf16* __restrict__ k, const bf16* __restrict__ v, floa
   extern __shared__ __align__(128) unsigned char smem[];
   static_assert(NWARPS * STAGES * 2 * TILEB >= NWARPS * NE * 4, "reduction buffer must fit in the stage ring");
 
+  pdl_launch_dependents();
+  pdl_wait();  // k and v come from the previous kernel
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int bh = blockIdx.x, s = blockIdx.y;
@@ -224,6 +226,8 @@ kv_state_mma_kernel(const bf16* __restrict__ k, const bf16* __restrict__ v, floa
 // Level two: state[bh][e] = partial[bh][0][e] + partial[bh][1][e] + ... in index order.
 __global__ void __launch_bounds__(256)
 kv_combine_bf16path_kernel(const float* __restrict__ partial, float* __restrict__ state, int S, int ne, long long total) {
+  pdl_launch_dependents();
+  pdl_wait();
   const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
   if (idx >= total) return;
   const long long bh = idx / ne;
@@ -264,6 +268,8 @@ apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf
   // memory (cp.async in, plain load out), so loads run STAGES groups ahead of
   // the MMAs without holding registers and without any cross-lane hand-off.
   __shared__ __align__(16) unsigned char fifo[NWARPS * STAGES * STAGEB];
+  pdl_launch_dependents();
+  pdl_wait();  // the state comes from the previous kernel
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   constexpr int NW = PAIR ? NWARPS / 2 : NWARPS;  // warps sharing one head's tokens
@@ -390,18 +396,18 @@ msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out
     cudaFuncSetAttribute(kv_state_mma_kernel<D, KV_WARPS, KV_STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, kv_smem);
     attr_done = true;
   }
-  kv_state_mma_kernel<D, KV_WARPS, KV_STAGES><<<dim3((unsigned)BH, p.S), KV_WARPS * 32, kv_smem, st>>>(k, v, partial, in, heads, N, p.S, p.chunk);
+  launch_pdl(kv_state_mma_kernel<D, KV_WARPS, KV_STAGES>, dim3((unsigned)BH, p.S), dim3(KV_WARPS * 32), kv_smem, st, k, v, partial, in, heads, N, p.S, p.chunk);
   const long long total = BH * p.ne;
-  kv_combine_bf16path_kernel<<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>(partial, state, p.S, p.ne, total);
+  launch_pdl(kv_combine_bf16path_kernel, dim3((unsigned)ceil_div_ll(total, 256)), dim3(256), 0, st, partial, state, p.S, p.ne, total);
   if (mid) cudaEventRecord(mid, st);
   if (ov.pair) {  // heads is even here, so a pair never straddles two images
     const int tok_per_cta = p.apply_tokens / 2;
-    apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, true><<<dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)(BH / 2)), AP_WARPS * 32, 0, st>>>(
-        q, state, out, in, ov, heads, N, eps, tok_per_cta);
+    launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, true>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)(BH / 2)),
+               dim3(AP_WARPS * 32), 0, st, q, state, out, in, ov, heads, N, eps, tok_per_cta);
   } else {
     const int tok_per_cta = p.apply_tokens;
-    apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, false><<<dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)BH), AP_WARPS * 32, 0, st>>>(
-        q, state, out, in, ov, heads, N, eps, tok_per_cta);
+    launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, false>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)BH),
+               dim3(AP_WARPS * 32), 0, st, q, state, out, in, ov, heads, N, eps, tok_per_cta);
   }
   count_launches(3);
   return check_launch("attention core kernels (bf16)");

@@ -246,6 +246,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_sh;
 
+  pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_tiles = p.batches * p.m_tiles * p.n_tiles;
   const int k_iters = (p.K + BK - 1) / BK;
@@ -270,6 +271,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
   }
   __syncthreads();
   const uint32_t tmem_base = tmem_base_sh;
+  pdl_wait();  // barriers and tensor memory are set up; the activations come from the previous kernel
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -412,6 +414,7 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_sh;
 
+  pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int k_iters = (p.K + BK - 1) / BK;
   const int blk = blockIdx.x % blocks, worker = blockIdx.x / blocks;
@@ -451,6 +454,7 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
         if (RES_IS_B) tma_load_3d(res_base + kb * RES_SLICE, &tmB, res_bar, kb * BK, blk * BN, 0);
         else          tma_load_3d(res_base + kb * RES_SLICE, &tmA, res_bar, kb * BK, blk * BM, 0);
       }
+      pdl_wait();  // the streamed operand may come from the previous kernel; the weights above do not
       uint32_t it = 0;
       bool ok = true;
       for (int si = worker; ok && si < stream_total; si += workers) {
@@ -512,6 +516,7 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
     const int col_half = (warp - 2) >> 2;
     uint32_t local = 0;
     bool ok = true;
+    pdl_wait();  // no global write before the previous kernel is done with the output buffer
     for (int si = worker; ok && si < stream_total; si += workers, ++local) {
       const int b = si / stream_per_batch, st = si % stream_per_batch;
       const int mt = RES_IS_B ? st : blk, nt = RES_IS_B ? blk : st;
@@ -576,7 +581,7 @@ msla_status_t launch_stationary(const CUtensorMap& tmA, const CUtensorMap& tmB, 
   const long long stream_total = (long long)p.batches * (A_MN ? p.m_tiles : p.n_tiles);
   long long workers = sm_count() / blocks;
   if (workers > stream_total) workers = stream_total;
-  gemm_bf16_stationary_kernel<A_MN><<<(unsigned)(workers * blocks), NUM_THREADS, WS_SMEM_BYTES, st>>>(tmA, tmB, tmO, p, blocks, (int)workers);
+  launch_pdl(gemm_bf16_stationary_kernel<A_MN>, dim3((unsigned)(workers * blocks)), dim3(NUM_THREADS), WS_SMEM_BYTES, st, tmA, tmB, tmO, p, blocks, (int)workers);
   count_launches(1);
   return check_launch("projection GEMM (tcgen05, stationary weights)");
 }
@@ -598,7 +603,7 @@ msla_status_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUten
   }
   const long long tiles = (long long)p.batches * p.m_tiles * p.n_tiles;
   const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-  gemm_bf16_tcgen05_kernel<A_MN, B_PLANAR><<<grid, NUM_THREADS, SMEM_BYTES, st>>>(tmA, tmB, tmO, p);
+  launch_pdl(gemm_bf16_tcgen05_kernel<A_MN, B_PLANAR>, dim3(grid), dim3(NUM_THREADS), SMEM_BYTES, st, tmA, tmB, tmO, p);
   count_launches(1);
   return check_launch("projection GEMM (tcgen05)");
 }

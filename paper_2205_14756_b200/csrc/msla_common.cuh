@@ -31,6 +31,17 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(flo
   return __float2bfloat16_rn(v);
 }
 
+// Programmatic dependent launch.  The tuned kernels are launched so that a
+// kernel may become resident while its predecessor in the stream is still
+// running: it sets up what depends on no earlier kernel (barriers, tensor
+// memory, tables built from the weights) and then waits here, which returns
+// once the predecessor has finished and its writes are visible.  Every global
+// read of an earlier kernel's output, and every global write, comes after it.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream be scheduled as soon as every CTA of this
+// one has started (it still waits in pdl_wait for this kernel's completion).
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __host__ __device__ __forceinline__ long long ceil_div_ll(long long a, long long b) {
   return (a + b - 1) / b;
 }

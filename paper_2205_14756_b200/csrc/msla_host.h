@@ -27,6 +27,23 @@ msla_status_t check_launch(const char* what);
 
 void count_launches(int n);
 
+// Launches `kernel` with programmatic stream serialization allowed: it may become resident before the
+// previous kernel of the stream has finished, and orders itself with pdl_wait() (msla_common.cuh).
+template <typename... KArgs, typename... Args>
+inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);  // errors surface in check_launch()
+}
+
 struct HeadView;
 // Tuned bf16 attention core (d in {16, 32}); all view strides must be multiples of 8 elements.
 msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* out, HeadView in, HeadView ov, int B,
