@@ -385,7 +385,7 @@ apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf
 
 template <int D>
 msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out, HeadView in, HeadView ov, int B,
-                          int heads, int N, float eps, const CorePlan& p, char* ws, cudaStream_t st, cudaEvent_t mid) {
+                          int heads, int N, float eps, const CorePlan& p, char* ws, cudaStream_t st, cudaEvent_t mid, bool with_apply) {
   constexpr int KV_WARPS = MSLA_KV_WARPS, KV_STAGES = MSLA_KV_STAGES, AP_WARPS = MSLA_AP_WARPS, AP_STAGES = MSLA_AP_STAGES, AP_U = MSLA_AP_U;
   const long long BH = (long long)B * heads;
   float* partial = reinterpret_cast<float*>(ws + p.partial_off);
@@ -400,6 +400,10 @@ msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out
   const long long total = BH * p.ne;
   launch_pdl(kv_combine_bf16path_kernel, dim3((unsigned)ceil_div_ll(total, 256)), dim3(256), 0, st, partial, state, p.S, p.ne, total);
   if (mid) cudaEventRecord(mid, st);
+  if (!with_apply) {
+    count_launches(2);
+    return check_launch("attention state kernels (bf16)");
+  }
   if (ov.pair) {  // heads is even here, so a pair never straddles two images
     const int tok_per_cta = p.apply_tokens / 2;
     launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, true>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)(BH / 2)),
@@ -417,10 +421,10 @@ msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out
 
 msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* out, HeadView in, HeadView ov, int B,
                             int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st,
-                            cudaEvent_t mid) {
+                            cudaEvent_t mid, bool with_apply) {
   if (d == 32)
-    return launch_core<32>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid);
-  return launch_core<16>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid);
+    return launch_core<32>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid, with_apply);
+  return launch_core<16>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid, with_apply);
 }
 
 }  // namespace msla

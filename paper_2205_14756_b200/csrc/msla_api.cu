@@ -3,6 +3,7 @@
 
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -113,7 +114,8 @@ static msla_status_t run_core_generic(const T* q, const T* k, const T* v, T* out
 static msla_status_t run_core(msla_dtype_t dtype, const void* q, const void* k, const void* v,
                               void* out, HeadView in, HeadView ov, int B, int heads, int N, int d,
                               float eps, const CorePlan& p, void* ws, cudaStream_t st,
-                              cudaEvent_t mid = nullptr) {
+                              cudaEvent_t mid = nullptr, bool with_apply = true) {
+  if (!with_apply && dtype != MSLA_BF16) return fail(MSLA_ERR_UNSUPPORTED, "the state-only core exists for bf16 only");
   if (ov.pair && (dtype != MSLA_BF16 || (heads & 1)))  // only the bf16 tensor-core kernels write paired planes
     return fail(MSLA_ERR_UNSUPPORTED, "paired output planes need bf16 and an even number of heads");
   if (dtype == MSLA_F32)
@@ -121,7 +123,8 @@ static msla_status_t run_core(msla_dtype_t dtype, const void* q, const void* k, 
                                    in, ov, B, heads, N, d, eps, p, (char*)ws, st, mid);
   const bool strides_ok = in.batch % 8 == 0 && in.head % 8 == 0 && in.ld % 8 == 0 && ov.batch % 8 == 0 &&
                           ov.head % 8 == 0 && ov.ld % 8 == 0;
-  if (strides_ok) return run_core_bf16(q, k, v, out, in, ov, B, heads, N, d, eps, p, ws, st, mid);
+  if (strides_ok) return run_core_bf16(q, k, v, out, in, ov, B, heads, N, d, eps, p, ws, st, mid, with_apply);
+  if (!with_apply) return fail(MSLA_ERR_UNSUPPORTED, "the state-only core needs strides that are multiples of 8 elements");
   if (ov.pair) return fail(MSLA_ERR_UNSUPPORTED, "paired output planes need strides that are multiples of 8 elements");
   return run_core_generic<__nv_bfloat16>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
                                          (const __nv_bfloat16*)v, (__nv_bfloat16*)out, in, ov, B,
@@ -380,13 +383,20 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   const bool att_planar = desc->dtype == MSLA_BF16 && d == 32 && project_out_planar_bf16_supported(2 * Cp, desc->C_out, N);
   const HeadView ov = att_planar ? HeadView{(long long)N * ld_att, (long long)N * 2 * d, 2 * d, 1}
                                  : HeadView{(long long)N * ld_att, d, ld_att, 0};
+  // Steps 4 and 5 run as one kernel when it takes the shape: the head concat then stays in shared memory.
+  static const bool no_fused = getenv("MSLA_NO_FUSED_APPLY") != nullptr;
+  const bool fused = !no_fused && desc->dtype == MSLA_BF16 && apply_project_bf16_supported(2 * heads, d, desc->C_out, N, in);
   s = run_core(desc->dtype, ms, ms + (size_t)N * d * e, ms + (size_t)2 * N * d * e, att, in, ov, desc->B, 2 * heads, N, d, desc->eps, p.core,
-               ws + p.core_off, st, events ? (cudaEvent_t)events[3] : nullptr);
+               ws + p.core_off, st, events ? (cudaEvent_t)events[3] : nullptr, !fused);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 4, st)) != MSLA_OK) return s;
   // 5. output projection back to NCHW
-  s = att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st)
-                 : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st);
+  if (fused)
+    s = run_apply_project_bf16(ms, reinterpret_cast<const float*>(ws + p.core_off + p.core.state_off), w->w_proj, w->b_proj, out_dev, in,
+                               desc->B, 2 * heads, N, desc->C_out, desc->eps, st);
+  else
+    s = att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st)
+                   : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 5, st)) != MSLA_OK) return s;
   if (host_io) {
@@ -463,8 +473,8 @@ msla_status_t msla_forward_host(const msla_desc* desc, const void* x_host, const
 unsigned long long msla_kernel_launches(void) { return g_launches; }
 
 int msla_debug_wait_timeouts(void) {
-  const int a = gemm_timeout_flag(), b = agg_timeout_flag();
-  return (a < 0 || b < 0) ? -1 : (a | b);
+  const int a = gemm_timeout_flag(), b = agg_timeout_flag(), c = fused_timeout_flag();
+  return (a < 0 || b < 0 || c < 0) ? -1 : (a | b | c);
 }
 
 msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d, void* stream) {

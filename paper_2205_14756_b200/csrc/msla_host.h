@@ -46,9 +46,17 @@ inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 
 struct HeadView;
 // Tuned bf16 attention core (d in {16, 32}); all view strides must be multiples of 8 elements.
+// with_apply = false stops after the combined states (at ws + p.state_off); `out` and `ov` are then unused.
 msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* out, HeadView in, HeadView ov, int B,
                             int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st,
-                            cudaEvent_t mid);
+                            cudaEvent_t mid, bool with_apply);
+
+// Apply step and output projection in one kernel (fused_apply_project.cu): bf16, d = 32, an even
+// number of heads, Cout <= 256, query strides multiples of 8 elements.
+bool apply_project_bf16_supported(int heads, int d, int Cout, int N, HeadView qv);
+msla_status_t run_apply_project_bf16(const void* q, const float* state, const void* w, const void* bias, void* y,
+                                     HeadView qv, int B, int heads, int N, int Cout, float eps, cudaStream_t st);
+int fused_timeout_flag();
 
 // bf16 projections on tcgen05 tensor cores (gemm_tcgen05.cu).
 bool project_in_bf16_supported(int C, int Cout, int N, int d);
