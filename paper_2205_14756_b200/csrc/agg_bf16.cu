@@ -374,6 +374,8 @@ msla_status_t launch_aggregate(const void* src, long long src_planes_total, int 
 msla_status_t run_aggregate_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
                                  const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch, int d,
                                  cudaStream_t st) {
+  if (aggregate_toeplitz_bf16_supported(H, W, Ch, d))
+    return run_aggregate_toeplitz_bf16(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_sb, B, H, W, Ch, st);
   return d == 16 ? launch_aggregate<true>(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_sb, B, H, W, Ch, st)
                  : launch_aggregate<false>(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_sb, B, H, W, Ch, st);
 }
