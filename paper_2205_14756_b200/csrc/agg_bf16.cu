@@ -1,6 +1,7 @@
-// Fused multi-scale token aggregation for bf16, d = 32 (Section 3.1): the 5x5
-// depthwise convolution and the grouped 1x1 convolution of one group of 32
-// channels in one kernel, on planar activations [planes][H*W][32].
+// Fused multi-scale token aggregation for bf16 (Section 3.1): the 5x5 depthwise
+// convolution and the grouped 1x1 convolution of one block of 32 channels in
+// one kernel, on planar activations.  The library uses it for d = 16 (two
+// groups per block, D16 = true); d = 32 runs the kernel of agg_toeplitz.cu.
 //
 // One CTA = a run of TW x TH pixel tiles of one group.  TMA copies stage the
 // (TW+4) x (TH+4) halo tiles in a two-deep ring in shared memory; coordinates
@@ -371,13 +372,17 @@ msla_status_t launch_aggregate(const void* src, long long src_planes_total, int 
 
 // src, dst: planar bf16 [.., planes, H*W, d], d in {16, 32}; group g of image b is plane b*src_ppb + g of
 // src (src_planes_total planes in all) and lives at dst + b*dst_sb + g*H*W*d.  Ch must be a multiple of 32.
+// d = 32 goes to the Toeplitz kernel (agg_toeplitz.cu), d = 16 to the kernel above.
 msla_status_t run_aggregate_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
                                  const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch, int d,
                                  cudaStream_t st) {
-  if (aggregate_toeplitz_bf16_supported(H, W, Ch, d))
-    return run_aggregate_toeplitz_bf16(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_sb, B, H, W, Ch, st);
-  return d == 16 ? launch_aggregate<true>(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_sb, B, H, W, Ch, st)
-                 : launch_aggregate<false>(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_sb, B, H, W, Ch, st);
+  if (d == 16) return launch_aggregate<true>(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_sb, B, H, W, Ch, st);
+  const long long plane = (long long)H * W * d;
+  if (!aggregate_toeplitz_bf16_supported(H, W, Ch, d) || dst_sb % plane != 0)
+    return fail(MSLA_ERR_UNSUPPORTED, "aggregation: d = %d with an output batch stride of %lld elements", d, dst_sb);
+  const long long dst_ppb = dst_sb / plane;
+  return run_aggregate_toeplitz_bf16(src, src_planes_total, src_ppb, w_dw, w_pw, dst, (B - 1) * dst_ppb + Ch / d, (int)dst_ppb,
+                                     B, H, W, Ch, st);
 }
 
 int agg_timeout_flag() {

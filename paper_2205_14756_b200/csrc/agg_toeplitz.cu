@@ -23,8 +23,14 @@
 //       18 ldmatrix matrices feed 10 MMAs per channel.  fp32 accumulators, rounded
 //       once to bf16 into a [channel][pixel] tile.
 //   P3  grouped 1x1: A = that tile through ldmatrix.trans (pixels x channels),
-//       B = the group's 32x32 weights from registers; 16-byte stores to the plane.
+//       B = the group's 32x32 weights from registers; each warp stages its 8 x 4
+//       pixels and writes them with one TMA store, which also clips at the image
+//       border (stores issued by the lanes themselves cost the load/store pipe
+//       four times the cycles of the staging writes).
 // The single TMA buffer is refilled for the next tile as soon as P1 is over.
+// The grid is persistent: two CTAs per SM, each with a contiguous run of
+// (image, group, tile) units; the weight fragments are reloaded when the group
+// changes.
 #include <cuda.h>
 
 #include "msla_common.cuh"
@@ -49,9 +55,12 @@ constexpr int DWO_CH = TW * TH * 2 + 16;     // 528 = 16 * 33: depthwise output,
 constexpr int DWO_BYTES = TD * DWO_CH;
 constexpr int T_WARPS = 8;
 constexpr int T_THREADS = 32 * T_WARPS;
-constexpr int T_SMEM_BYTES = 1024 + BOX_BYTES + PL_BYTES + DWO_BYTES;
+constexpr int OUT_WARP_BYTES = 4 * 8 * 64;   // output staging per warp: 4 rows x 8 pixels x 32 channels
+constexpr int OUT_BYTES = T_WARPS * OUT_WARP_BYTES;
+constexpr int T_SMEM_BYTES = 1024 + BOX_BYTES + PL_BYTES + DWO_BYTES + OUT_BYTES;
 constexpr long long T_WAIT_LIMIT_CYCLES = 4000000000LL;
 static_assert(BOXH % 2 == 0 && (PL_CH / 16) % 2 == 1 && (DWO_CH / 16) % 2 == 1 && (PL_ROW / 16) % 2 == 1, "bank-conflict-free pitches");
+static_assert(PL_BYTES % 128 == 0 && DWO_BYTES % 128 == 0, "the output staging must stay 128-byte aligned");
 static_assert(BOX_ROW % 512 == 0, "the 64B swizzle pattern must restart with every staged row");
 
 __device__ int g_aggt_timeout_flag = 0;
@@ -81,40 +90,56 @@ __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) { asm volatile(
 struct ToeplitzParams {
   const bf16* w_dw;  // [Ch][5][5]
   const bf16* w_pw;  // [Ch][32]
-  bf16* dst;         // planar output
-  long long dst_batch_stride;  // elements
-  int src_planes_per_batch;    // plane index of (b, group) in the tensor map = b * this + group
-  int H, W;
+  int src_planes_per_batch;    // plane index of (b, group) in a tensor map = b * planes_per_batch + group
+  int dst_planes_per_batch;
+  int groups;
   int tiles_x, tiles_total;    // tiles per plane
-  int tiles_per_cta;           // consecutive tiles of one plane handled by one CTA
+  long long units;             // B * groups * tiles_total, tile fastest
+  long long units_per_cta;
 };
 
 __global__ void __launch_bounds__(T_THREADS, 2)
-aggregate_toeplitz_kernel(const __grid_constant__ CUtensorMap tm_src, ToeplitzParams p) {
+aggregate_toeplitz_kernel(const __grid_constant__ CUtensorMap tm_src, const __grid_constant__ CUtensorMap tm_dst, ToeplitzParams p) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t box = (smem_addr(smem_raw) + 1023u) & ~1023u;  // the swizzle pattern is a function of the address
-  const uint32_t pl = box + BOX_BYTES, dwo = pl + PL_BYTES;
+  const uint32_t pl = box + BOX_BYTES, dwo = pl + PL_BYTES, outs = dwo + DWO_BYTES;
   __shared__ __align__(8) unsigned long long bar_storage;
   __shared__ int timed_out;
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int group = blockIdx.y, b = blockIdx.z;
-  const int ch0 = group * TD;
-  const int tile_first = blockIdx.x * p.tiles_per_cta;
-  const int tile_count = min(p.tiles_per_cta, p.tiles_total - tile_first);
-  const int plane_idx = b * p.src_planes_per_batch + group;
+  const long long unit_first = (long long)blockIdx.x * p.units_per_cta;
+  const int unit_count = (int)max(0LL, min(p.units_per_cta, p.units - unit_first));
   const uint32_t bar = smem_addr(&bar_storage);
 
+  // Cursor over (image, group, tile) units, tile fastest, advanced without divisions.
+  struct Unit { int tile, tx, ty, group, b; };
+  auto locate = [&](long long u) {
+    const long long bg = u / p.tiles_total;
+    Unit r;
+    r.tile = (int)(u - bg * p.tiles_total);
+    r.ty = r.tile / p.tiles_x;
+    r.tx = r.tile - r.ty * p.tiles_x;
+    r.b = (int)(bg / p.groups);
+    r.group = (int)(bg - (long long)r.b * p.groups);
+    return r;
+  };
+  auto advance = [&](Unit& u) {
+    ++u.tile;
+    if (++u.tx == p.tiles_x) { u.tx = 0; ++u.ty; }
+    if (u.tile == p.tiles_total) {
+      u.tile = 0; u.ty = 0;
+      if (++u.group == p.groups) { u.group = 0; ++u.b; }
+    }
+  };
   // x and y may start below 0 and run past W, H: the TMA unit returns zeros there.
-  auto issue = [&](int k) {
-    const int tile = tile_first + k;
-    const int tx0 = (tile % p.tiles_x) * TW, ty0 = (tile / p.tiles_x) * TH;
+  auto issue = [&](const Unit& u) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(BOX_BYTES) : "memory");
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(box), "l"(&tm_src), "r"(bar), "r"(0), "r"(tx0 - 4), "r"(ty0 - 2), "r"(plane_idx) : "memory");
+        ::"r"(box), "l"(&tm_src), "r"(bar), "r"(0), "r"(u.tx * TW - 4), "r"(u.ty * TH - 2), "r"(u.b * p.src_planes_per_batch + u.group) : "memory");
   };
+  Unit un = locate(unit_first), nxt = un;  // nxt: the unit whose copy is issued next (thread 0 only)
 
   pdl_launch_dependents();
   if (threadIdx.x == 0) {
@@ -122,34 +147,38 @@ aggregate_toeplitz_kernel(const __grid_constant__ CUtensorMap tm_src, ToeplitzPa
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     pdl_wait();  // the planes read here come from the previous kernel; the fragments below only need the weights
-    issue(0);
+    if (unit_count > 0) issue(nxt);
   }
 
-  // Toeplitz B fragments of this warp's four channels: lane (g, t) holds rows k = 2t, 2t+1 (b0) and
-  // 2t+8, 2t+9 (b1) of column n = g, i.e. taps dx = k - g - 2 of filter row dy.
-  uint32_t bt[4][5][2];
+  uint32_t bt[4][5][2];  // Toeplitz B fragments of this warp's four channels
+  uint32_t bw[2][4][2];  // pointwise weights as B fragments
+  auto load_weights = [&](int group) {
+    const int ch0 = group * TD;
+    // lane (g, t) holds rows k = 2t, 2t+1 (b0) and 2t+8, 2t+9 (b1) of column n = g, i.e. taps dx = k - g - 2 of filter row dy
 #pragma unroll
-  for (int cc = 0; cc < 4; ++cc)
+    for (int cc = 0; cc < 4; ++cc)
 #pragma unroll
-    for (int dy = 0; dy < 5; ++dy) {
-      const bf16* wrow = p.w_dw + (long long)(ch0 + 4 * warp + cc) * 25 + dy * 5;
-      const int i0 = 2 * t - g - 2;
-      auto tap = [&](int i) -> uint32_t { return (i >= 0 && i < 5) ? (uint32_t)__bfloat16_as_ushort(wrow[i]) : 0u; };
-      bt[cc][dy][0] = tap(i0) | (tap(i0 + 1) << 16);
-      bt[cc][dy][1] = tap(i0 + 8) | (tap(i0 + 9) << 16);
-    }
-  // Pointwise weights as B fragments.  Contraction slots are the input channels in order; column n = g
-  // of block jn is output channel 8(g/2) + 2jn + (g&1), so that a lane ends up with channels 8t .. 8t+7.
-  uint32_t bw[2][4][2];
+      for (int dy = 0; dy < 5; ++dy) {
+        const bf16* wrow = p.w_dw + (long long)(ch0 + 4 * warp + cc) * 25 + dy * 5;
+        const int i0 = 2 * t - g - 2;
+        auto tap = [&](int i) -> uint32_t { return (i >= 0 && i < 5) ? (uint32_t)__bfloat16_as_ushort(wrow[i]) : 0u; };
+        bt[cc][dy][0] = tap(i0) | (tap(i0 + 1) << 16);
+        bt[cc][dy][1] = tap(i0 + 8) | (tap(i0 + 9) << 16);
+      }
+    // Contraction slots are the input channels in order; column n = g of block jn is output channel
+    // 8(g/2) + 2jn + (g&1), so that a lane ends up with channels 8t .. 8t+7.
 #pragma unroll
-  for (int ks = 0; ks < 2; ++ks)
+    for (int ks = 0; ks < 2; ++ks)
 #pragma unroll
-    for (int jn = 0; jn < 4; ++jn) {
-      const int oc = 8 * (g >> 1) + 2 * jn + (g & 1);
-      const bf16* wr = p.w_pw + (long long)(ch0 + oc) * TD + 16 * ks + 2 * t;
-      bw[ks][jn][0] = *reinterpret_cast<const uint32_t*>(wr);
-      bw[ks][jn][1] = *reinterpret_cast<const uint32_t*>(wr + 8);
-    }
+      for (int jn = 0; jn < 4; ++jn) {
+        const int oc = 8 * (g >> 1) + 2 * jn + (g & 1);
+        const bf16* wr = p.w_pw + (long long)(ch0 + oc) * TD + 16 * ks + 2 * t;
+        bw[ks][jn][0] = *reinterpret_cast<const uint32_t*>(wr);
+        bw[ks][jn][1] = *reinterpret_cast<const uint32_t*>(wr + 8);
+      }
+  };
+  int cur_group = un.group;
+  load_weights(cur_group);
 
   // Per-lane address offsets of the six ldmatrix loads of a channel.  Matrix (r, h) = staged rows
   // 2g'+r (g' = 0..7), 16-byte piece h of the row; lane l supplies row l&7 of matrix l>>3.
@@ -170,9 +199,10 @@ aggregate_toeplitz_kernel(const __grid_constant__ CUtensorMap tm_src, ToeplitzPa
   __syncthreads();  // barrier initialised before anyone waits on it
   pdl_wait();
 
-  bf16* plane = p.dst + (long long)b * p.dst_batch_stride + (long long)group * p.H * p.W * TD;
+  // this warp's 8 x 4 pixels of a tile: columns 8(w/4) .. +7, rows 4(w%4) .. +3
+  const uint32_t my_out = outs + (uint32_t)(warp * OUT_WARP_BYTES);
 #pragma unroll 1
-  for (int k = 0; k < tile_count; ++k) {
+  for (int k = 0; k < unit_count; ++k, advance(un)) {
     {  // bounded wait for this tile
       const uint32_t parity = k & 1;
       uint32_t ok = 0;
@@ -185,8 +215,11 @@ aggregate_toeplitz_kernel(const __grid_constant__ CUtensorMap tm_src, ToeplitzPa
         if (timed_out || clock64() - t_start > T_WAIT_LIMIT_CYCLES) { timed_out = 1; break; }
       }
     }
-    const int tile = tile_first + k;
-    const int x0 = (tile % p.tiles_x) * TW, y0 = (tile / p.tiles_x) * TH;
+    const int x0 = un.tx * TW, y0 = un.ty * TH;
+    if (un.group != cur_group) {  // uniform over the CTA
+      cur_group = un.group;
+      load_weights(cur_group);
+    }
 
     // ---- P1: [row][pixel][channel] -> [channel][row parity][row/2][pixel].  One unit = one staged row
     // and 8 pixels: four 8x8 matrices (8 pixels x 8 channels each), transposed by ldmatrix, so that lane
@@ -206,9 +239,10 @@ aggregate_toeplitz_kernel(const __grid_constant__ CUtensorMap tm_src, ToeplitzPa
       if (threadIdx.x == 0) atomicExch(&g_aggt_timeout_flag, 1);
       return;
     }
-    if (threadIdx.x == 0 && k + 1 < tile_count) {
+    if (threadIdx.x == 0 && k + 1 < unit_count) {
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // order the generic reads above before the async write
-      issue(k + 1);
+      advance(nxt);
+      issue(nxt);
     }
 
     // ---- P2: depthwise 5x5 of channels 4w .. 4w+3
@@ -244,10 +278,13 @@ aggregate_toeplitz_kernel(const __grid_constant__ CUtensorMap tm_src, ToeplitzPa
     __syncthreads();
 
     // ---- P3: grouped 1x1 on 32 pixels per warp.  8-pixel block q of the depthwise tile is image row
-    // 2(q&7) + ((q>>3)&1), columns 8(q>>4) .. +7.
+    // 2(q&7) + ((q>>3)&1), columns 8(q>>4) .. +7; rows 4a .. 4a+3 of column block xb are q = 16xb + 2a,
+    // 16xb + 8 + 2a, 16xb + 2a + 1, 16xb + 8 + 2a + 1.
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // the previous tile's store has read the staging
+    __syncwarp();
 #pragma unroll
     for (int mb = 0; mb < 2; ++mb) {
-      const int qa = 4 * warp + 2 * mb;
+      const int qa = 16 * (warp >> 2) + 2 * (warp & 3) + mb;  // MMA rows g: block qa (row 4a + 2mb), rows g+8: block qa + 8 (row 4a + 2mb + 1)
       float c[4][4];
 #pragma unroll
       for (int jn = 0; jn < 4; ++jn)
@@ -256,25 +293,30 @@ aggregate_toeplitz_kernel(const __grid_constant__ CUtensorMap tm_src, ToeplitzPa
 #pragma unroll
       for (int ks = 0; ks < 2; ++ks) {
         const int mi = lane >> 3;
-        uint32_t a0, a1, a2, a3;  // rows = pixels of block qa / qa+1, contraction = channels 16ks .. 16ks+15
-        ldsm_x4_trans(a0, a1, a2, a3, dwo + (uint32_t)((16 * ks + 8 * (mi >> 1) + (lane & 7)) * DWO_CH + (qa + (mi & 1)) * 16));
+        uint32_t a0, a1, a2, a3;  // rows = pixels of block qa / qa+8, contraction = channels 16ks .. 16ks+15
+        ldsm_x4_trans(a0, a1, a2, a3, dwo + (uint32_t)((16 * ks + 8 * (mi >> 1) + (lane & 7)) * DWO_CH + (qa + 8 * (mi & 1)) * 16));
 #pragma unroll
         for (int jn = 0; jn < 4; ++jn) mma_bf16(c[jn], a0, a1, a2, a3, bw[ks][jn][0], bw[ks][jn][1]);
       }
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const int q = qa + half;
-        const int y = y0 + 2 * (q & 7) + ((q >> 3) & 1), x = x0 + 8 * (q >> 4) + g;
-        if (x < p.W && y < p.H)
-          asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(plane + ((long long)y * p.W + x) * TD + 8 * t),
-                       "r"(pack_bf16x2(c[0][2 * half], c[0][2 * half + 1])), "r"(pack_bf16x2(c[1][2 * half], c[1][2 * half + 1])),
-                       "r"(pack_bf16x2(c[2][2 * half], c[2][2 * half + 1])), "r"(pack_bf16x2(c[3][2 * half], c[3][2 * half + 1]))
-                       : "memory");
-      }
+      for (int half = 0; half < 2; ++half)  // staging: [row 2mb + half][pixel g][channels 8t .. 8t+7]
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(my_out + (uint32_t)(((2 * mb + half) * 8 + g) * 64 + t * 16)),
+                     "r"(pack_bf16x2(c[0][2 * half], c[0][2 * half + 1])), "r"(pack_bf16x2(c[1][2 * half], c[1][2 * half + 1])),
+                     "r"(pack_bf16x2(c[2][2 * half], c[2][2 * half + 1])), "r"(pack_bf16x2(c[3][2 * half], c[3][2 * half + 1]))
+                     : "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) {  // pixels outside the image are clipped by the TMA unit
+      asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                   ::"l"(&tm_dst), "r"(my_out), "r"(0), "r"(x0 + 8 * (warp >> 2)), "r"(y0 + 4 * (warp & 3)),
+                     "r"(un.b * p.dst_planes_per_batch + un.group) : "memory");
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
     }
     // No barrier here: the next tile's P1 only writes the planar tile (last read before the barrier
     // above), and its trailing barrier comes before anything overwrites the depthwise tile.
   }
+  if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // stores done before the CTA retires
 }
 
 }  // namespace
@@ -282,27 +324,37 @@ aggregate_toeplitz_kernel(const __grid_constant__ CUtensorMap tm_src, ToeplitzPa
 bool aggregate_toeplitz_bf16_supported(int H, int W, int Ch, int d) { return d == TD && Ch % TD == 0 && H >= 1 && W >= 1; }
 
 // src, dst: planar bf16 [.., planes, H*W, 32]; group g of image b is plane b*src_ppb + g of src
-// (src_planes_total planes in all) and lives at dst + b*dst_sb + g*H*W*32.
+// (src_planes_total planes in all) and plane b*dst_ppb + g of dst (dst_planes_total in all).
 msla_status_t run_aggregate_toeplitz_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
-                                          const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch,
-                                          cudaStream_t st) {
-  CUtensorMap tm;
-  const cuuint64_t dims[4] = {(cuuint64_t)TD, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)src_planes_total};
-  const cuuint64_t strides[3] = {(cuuint64_t)TD * 2, (cuuint64_t)W * TD * 2, (cuuint64_t)H * W * TD * 2};
-  const cuuint32_t bx[4] = {(cuuint32_t)TD, (cuuint32_t)BOXW, (cuuint32_t)BOXH, 1};
-  if (!tma_make_map_bf16(&tm, src, 4, dims, strides, bx, CU_TENSOR_MAP_SWIZZLE_64B))
-    return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the aggregation input");
+                                          const void* w_pw, void* dst, long long dst_planes_total, int dst_ppb, int B,
+                                          int H, int W, int Ch, cudaStream_t st) {
+  CUtensorMap tm_src, tm_dst;
+  {
+    const cuuint64_t dims[4] = {(cuuint64_t)TD, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)src_planes_total};
+    const cuuint64_t ddims[4] = {(cuuint64_t)TD, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)dst_planes_total};
+    const cuuint64_t strides[3] = {(cuuint64_t)TD * 2, (cuuint64_t)W * TD * 2, (cuuint64_t)H * W * TD * 2};
+    const cuuint32_t bx[4] = {(cuuint32_t)TD, (cuuint32_t)BOXW, (cuuint32_t)BOXH, 1};
+    const cuuint32_t ob[4] = {(cuuint32_t)TD, 8, 4, 1};
+    if (!tma_make_map_bf16(&tm_src, src, 4, dims, strides, bx, CU_TENSOR_MAP_SWIZZLE_64B) ||
+        !tma_make_map_bf16(&tm_dst, dst, 4, ddims, strides, ob, CU_TENSOR_MAP_SWIZZLE_NONE))
+      return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the aggregation");
+  }
   ToeplitzParams p;
-  p.w_dw = (const bf16*)w_dw; p.w_pw = (const bf16*)w_pw; p.dst = (bf16*)dst;
-  p.dst_batch_stride = dst_sb; p.src_planes_per_batch = src_ppb; p.H = H; p.W = W;
+  p.w_dw = (const bf16*)w_dw; p.w_pw = (const bf16*)w_pw;
+  p.src_planes_per_batch = src_ppb; p.dst_planes_per_batch = dst_ppb; p.groups = Ch / TD;
   p.tiles_x = (W + TW - 1) / TW;
   const long long tiles = (long long)p.tiles_x * ((H + TH - 1) / TH);
   if (tiles > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many aggregation tiles");
   p.tiles_total = (int)tiles;
-  // enough CTAs for a few waves over the GPU, otherwise as many tiles per CTA as possible (up to 8)
-  const long long units = tiles * (Ch / TD) * B;
-  p.tiles_per_cta = units >= 8 * 2400 ? 8 : units >= 4 * 2400 ? 4 : units >= 2 * 2400 ? 2 : 1;
-  dim3 grid((unsigned)((tiles + p.tiles_per_cta - 1) / p.tiles_per_cta), (unsigned)(Ch / TD), (unsigned)B);
+  p.units = tiles * p.groups * B;
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+  // two CTAs per SM; small problems get one unit per CTA
+  const long long ctas = p.units < 2LL * sms ? p.units : 2LL * sms;
+  p.units_per_cta = (p.units + ctas - 1) / ctas;
+  if (p.units_per_cta > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many aggregation tiles");
+  const unsigned grid = (unsigned)((p.units + p.units_per_cta - 1) / p.units_per_cta);
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(aggregate_toeplitz_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_BYTES) != cudaSuccess) {
@@ -311,7 +363,7 @@ msla_status_t run_aggregate_toeplitz_bf16(const void* src, long long src_planes_
     }
     attr_done = true;
   }
-  launch_pdl(aggregate_toeplitz_kernel, grid, dim3(T_THREADS), T_SMEM_BYTES, st, tm, p);
+  launch_pdl(aggregate_toeplitz_kernel, dim3(grid), dim3(T_THREADS), T_SMEM_BYTES, st, tm_src, tm_dst, p);
   count_launches(1);
   return check_launch("token aggregation (bf16, Toeplitz)");
 }

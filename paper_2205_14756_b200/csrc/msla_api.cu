@@ -286,7 +286,7 @@ static msla_status_t run_aggregate(msla_dtype_t dt, const void* src, const void*
                                    void* dst, int B, int H, int W, int Ch, int d, long long src_sb,
                                    long long dst_sb, cudaStream_t st) {
   const long long plane = (long long)H * W * d;
-  if (dt == MSLA_BF16 && src_sb % plane == 0) {
+  if (dt == MSLA_BF16 && src_sb % plane == 0 && dst_sb % plane == 0) {
     if (aggregate_bf16_supported(H, W, Ch, d))
       return run_aggregate_bf16(src, (long long)B * (src_sb / plane), (int)(src_sb / plane), w_dw, w_pw, dst, dst_sb, B, H, W, Ch, d, st);
     if (d == 16 && Ch > 16 && aggregate_bf16_supported(H, W, Ch - 16, d)) {

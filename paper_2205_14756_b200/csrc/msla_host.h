@@ -80,8 +80,8 @@ int agg_timeout_flag();
 // bf16 aggregation for d = 32 with the depthwise filter as banded matrices on tensor cores (agg_toeplitz.cu).
 bool aggregate_toeplitz_bf16_supported(int H, int W, int Ch, int d);
 msla_status_t run_aggregate_toeplitz_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
-                                          const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch,
-                                          cudaStream_t st);
+                                          const void* w_pw, void* dst, long long dst_planes_total, int dst_ppb, int B,
+                                          int H, int W, int Ch, cudaStream_t st);
 int aggt_timeout_flag();
 
 }  // namespace msla
