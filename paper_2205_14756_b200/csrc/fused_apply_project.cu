@@ -52,9 +52,11 @@ constexpr int F_SMEM_BYTES = F_SLICES * F_SLICE_BYTES + F_ASTAGES * F_A_BYTES + 
 
 __device__ int g_fused_timeout_flag = 0;
 
+constexpr int F_FRAG_WORDS = 2 * (FD / 16) * (FD / 8 + 1) * 2;  // 40 words per lane and head: hi, then lo
+
 struct FusedParams {
   const bf16* q;        // query planes, strides in qv
-  const float* state;   // [B * heads][32 * 33] fp32: KV | key sum
+  const uint4* frags;   // [B * heads][10][32 lanes]: the states as mma.sync B fragments (state_fragments_kernel)
   const bf16* bias;     // [Cout] or nullptr
   HeadView qv;
   int heads;            // heads per image over all scales (even); K = 32 * heads
@@ -81,6 +83,35 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
   asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ void mma_bf16_first(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {  // C = 0
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
+}
+
+// The fp32 states [heads][32][33] (KV | key sum) as the per-lane B fragments the apply warps feed to
+// mma.sync: word (ks*5 + j)*2 + e of lane (g, t) packs rows a0, a0+1 (a0 = 8t + 4ks + 2e) of column
+// c = 8(g/2) + 2j + (g&1), or of the key-sum column for j = 4; words 0-19 hold the bf16 roundings,
+// words 20-39 the bf16 roundings of the remainders.  Laid out so that a lane fetches its 40 words
+// with ten 16-byte loads, consecutive lanes 16 bytes apart.
+__global__ void __launch_bounds__(256) state_fragments_kernel(const float* __restrict__ state, uint32_t* __restrict__ table) {
+  pdl_launch_dependents();
+  pdl_wait();  // the states come from the previous kernel
+  const float* sp = state + (long long)blockIdx.x * (FD * (FD + 1));
+  uint32_t* tp = table + (long long)blockIdx.x * (F_FRAG_WORDS * 32);
+  for (int i = threadIdx.x; i < F_FRAG_WORDS * 32; i += blockDim.x) {
+    const int lane = i & 31, w = i >> 5;
+    const int lo = w >= F_FRAG_WORDS / 2, ww = lo ? w - F_FRAG_WORDS / 2 : w;
+    const int e = ww & 1, j = (ww >> 1) % (FD / 8 + 1), ks = (ww >> 1) / (FD / 8 + 1);
+    const int g = lane >> 2, t = lane & 3;
+    const int a0 = 8 * t + 4 * ks + 2 * e;
+    const int c = j < FD / 8 ? (g >> 1) * 8 + 2 * j + (g & 1) : FD;
+    const float v0 = sp[a0 * (FD + 1) + c], v1 = sp[(a0 + 1) * (FD + 1) + c];
+    const float r0 = v0 - __bfloat162float(__float2bfloat16_rn(v0)), r1 = v1 - __bfloat162float(__float2bfloat16_rn(v1));
+    tp[((w >> 2) * 32 + lane) * 4 + (w & 3)] = lo ? pack2(r0, r1) : pack2(v0, v1);
+  }
 }
 
 __global__ void __launch_bounds__(F_THREADS, 1)
@@ -236,7 +267,7 @@ apply_project_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
       cp_async_commit();
     }
 
-    uint32_t bhi[KS][NT + 1][2], blo[KS][NT + 1][2];
+    uint32_t bf[F_FRAG_WORDS];  // word (ks*(NT+1) + j)*2 + e: bf16 rounding of the state; + F_FRAG_WORDS/2: of the remainder
     bool ok = true, head_ok = false;
     for (int stp = 0; stp < total_steps; ++stp, advance(cc)) {
       const int ti = cc.ti, r = cc.r, st = cc.st;
@@ -246,20 +277,12 @@ apply_project_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
         const int h = r * F_APPLY_WARPS + aw;
         head_ok = h < p.heads;
         if (head_ok) {
-          const float* sp = p.state + ((long long)cc.b * p.heads + h) * (FD * (FD + 1));
+          const uint4* fp = p.frags + ((long long)cc.b * p.heads + h) * (F_FRAG_WORDS / 4 * 32) + lane;
 #pragma unroll
-          for (int ks = 0; ks < KS; ++ks)
-#pragma unroll
-            for (int j = 0; j <= NT; ++j)
-#pragma unroll
-              for (int e = 0; e < 2; ++e) {
-                const int a0 = 8 * t + 4 * ks + 2 * e;
-                const int c = j < NT ? (g >> 1) * 8 + 2 * j + (g & 1) : FD;
-                const float v0 = sp[a0 * (FD + 1) + c], v1 = sp[(a0 + 1) * (FD + 1) + c];
-                const bf16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
-                bhi[ks][j][e] = pack2(v0, v1);
-                blo[ks][j][e] = pack2(v0 - __bfloat162float(h0), v1 - __bfloat162float(h1));
-              }
+          for (int v = 0; v < F_FRAG_WORDS / 4; ++v) {
+            const uint4 x = fp[v * 32];
+            bf[4 * v] = x.x; bf[4 * v + 1] = x.y; bf[4 * v + 2] = x.z; bf[4 * v + 3] = x.w;
+          }
           // the MMAs that read this slice in its previous use must be done
           const uint32_t use = (uint32_t)(ti * uses_per_tile + r);
           ok = mbar_wait(bempty + 8 * s, (use & 1) ^ 1, &abort_flag);
@@ -278,12 +301,6 @@ apply_project_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
       }
       float acc[F_U][NT + 1][4];
 #pragma unroll
-      for (int u = 0; u < F_U; ++u)
-#pragma unroll
-        for (int j = 0; j <= NT; ++j)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) acc[u][j][e] = 0.f;
-#pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
         uint32_t A[F_U][4];
 #pragma unroll
@@ -294,11 +311,18 @@ apply_project_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
 #pragma unroll
         for (int j = 0; j <= NT; ++j)
 #pragma unroll
-          for (int u = 0; u < F_U; ++u) mma_bf16(acc[u][j], A[u], bhi[ks][j][0], bhi[ks][j][1]);
+          for (int u = 0; u < F_U; ++u) {
+            const int w = (ks * (NT + 1) + j) * 2;
+            if (ks == 0) mma_bf16_first(acc[u][j], A[u], bf[w], bf[w + 1]);
+            else mma_bf16(acc[u][j], A[u], bf[w], bf[w + 1]);
+          }
 #pragma unroll
         for (int j = 0; j <= NT; ++j)
 #pragma unroll
-          for (int u = 0; u < F_U; ++u) mma_bf16(acc[u][j], A[u], blo[ks][j][0], blo[ks][j][1]);
+          for (int u = 0; u < F_U; ++u) {
+            const int w = F_FRAG_WORDS / 2 + (ks * (NT + 1) + j) * 2;
+            mma_bf16(acc[u][j], A[u], bf[w], bf[w + 1]);
+          }
       }
       // normalise and store into the slice: row = token of the tile (128 bytes = 64 channels of the pair),
       // this head's half = 16-byte chunks 4*(aw&1) + t, XOR-swizzled with the row as the 128B mode expects
@@ -406,7 +430,10 @@ bool apply_project_bf16_supported(int heads, int d, int Cout, int N, HeadView qv
 
 // y[b][m][n] = sum_h sum_c w[m][32 h + c] * att[b][h][n][c] + bias[m], att = Eq. 3 applied to query head h with
 // state[b * heads + h] ([32][33] fp32: KV, then the key sum in column 32); y is NCHW [B, Cout, N].
-msla_status_t run_apply_project_bf16(const void* q, const float* state, const void* w, const void* bias, void* y,
+// scratch: apply_project_scratch_bytes(B, heads) bytes of device memory, 16-byte aligned (the states as fragments).
+size_t apply_project_scratch_bytes(int B, int heads) { return (size_t)B * heads * F_FRAG_WORDS * 32 * sizeof(uint32_t); }
+
+msla_status_t run_apply_project_bf16(const void* q, const float* state, void* scratch, const void* w, const void* bias, void* y,
                                      HeadView qv, int B, int heads, int N, int Cout, float eps, cudaStream_t st) {
   const int K = heads * FD;
   CUtensorMap tmA, tmO;
@@ -422,7 +449,7 @@ msla_status_t run_apply_project_bf16(const void* q, const float* state, const vo
       return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the fused apply + output projection");
   }
   FusedParams p{};
-  p.q = (const bf16*)q; p.state = state; p.bias = (const bf16*)bias; p.qv = qv;
+  p.q = (const bf16*)q; p.frags = (const uint4*)scratch; p.bias = (const bf16*)bias; p.qv = qv;
   p.heads = heads; p.B = B; p.N = N; p.Cout = Cout; p.eps = eps;
   p.m_tiles = (Cout + FBM - 1) / FBM;
   p.tiles_per_batch = (N + FT - 1) / FT;
@@ -441,8 +468,9 @@ msla_status_t run_apply_project_bf16(const void* q, const float* state, const vo
   cudaGetDevice(&dev);
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
   const int grid = (int)(tiles < sms ? tiles : sms);
+  launch_pdl(state_fragments_kernel, dim3((unsigned)(B * heads)), dim3(256), 0, st, state, (uint32_t*)scratch);
   launch_pdl(apply_project_fused_kernel, dim3(grid), dim3(F_THREADS), F_SMEM_BYTES, st, tmA, tmO, p);
-  count_launches(1);
+  count_launches(2);
   return check_launch("fused apply + output projection (tcgen05)");
 }
 

@@ -250,7 +250,11 @@ static msla_status_t validate_desc(const msla_desc* d, ForwardPlan* plan) {
   plan->core = make_core_plan((long long)d->B * 2 * d->heads, plan->N, d->d);
   plan->ms_off = 0;
   plan->att_off = align_up(tokens * 6 * plan->Cp * e, 256);
-  plan->core_off = plan->att_off + align_up(tokens * 2 * plan->Cp * e, 256);
+  // the attention output's region doubles as scratch of the fused apply + projection kernel, which writes no attention output
+  size_t att_bytes = tokens * 2 * plan->Cp * e;
+  const size_t fused_scratch = apply_project_scratch_bytes(d->B, 2 * d->heads);
+  if (att_bytes < fused_scratch) att_bytes = fused_scratch;
+  plan->core_off = plan->att_off + align_up(att_bytes, 256);
   plan->bytes = plan->core_off + plan->core.bytes;
   return MSLA_OK;
 }
@@ -392,7 +396,7 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   if ((s = record(events, 4, st)) != MSLA_OK) return s;
   // 5. output projection back to NCHW
   if (fused)
-    s = run_apply_project_bf16(ms, reinterpret_cast<const float*>(ws + p.core_off + p.core.state_off), w->w_proj, w->b_proj, out_dev, in,
+    s = run_apply_project_bf16(ms, reinterpret_cast<const float*>(ws + p.core_off + p.core.state_off), att, w->w_proj, w->b_proj, out_dev, in,
                                desc->B, 2 * heads, N, desc->C_out, desc->eps, st);
   else
     s = att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st)

@@ -54,7 +54,8 @@ msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* o
 // Apply step and output projection in one kernel (fused_apply_project.cu): bf16, d = 32, an even
 // number of heads, Cout <= 256, query strides multiples of 8 elements.
 bool apply_project_bf16_supported(int heads, int d, int Cout, int N, HeadView qv);
-msla_status_t run_apply_project_bf16(const void* q, const float* state, const void* w, const void* bias, void* y,
+size_t apply_project_scratch_bytes(int B, int heads);
+msla_status_t run_apply_project_bf16(const void* q, const float* state, void* scratch, const void* w, const void* bias, void* y,
                                      HeadView qv, int B, int heads, int N, int Cout, float eps, cudaStream_t st);
 int fused_timeout_flag();
 
