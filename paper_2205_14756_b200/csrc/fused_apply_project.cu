@@ -9,8 +9,8 @@
 //   warp 1      issues tcgen05.mma 128x128x16; owns the tensor-memory allocation
 //   warps 2-9   "apply" warps.  In round r warp a serves head 8r + a: it streams that
 //               head's query rows through a per-lane cp.async FIFO, multiplies them
-//               with the head's fp32 state (fed as bf16 hi + lo, one extra column
-//               block for the denominator) on mma.sync, normalises, and writes the
+//               with the head's state (rounded to bf16, one extra column block for
+//               the denominator) on mma.sync, normalises, and writes the
 //               128 x 32 result into its half of B slice a/2 (128 tokens x 64
 //               channels, the layout a 128B-swizzled TMA load would have produced)
 //   warps 10-13 drain the accumulators: TMEM -> bf16 (+ bias) -> swizzled staging ->
@@ -52,7 +52,7 @@ constexpr int F_SMEM_BYTES = F_SLICES * F_SLICE_BYTES + F_ASTAGES * F_A_BYTES + 
 
 __device__ int g_fused_timeout_flag = 0;
 
-constexpr int F_FRAG_WORDS = 2 * (FD / 16) * (FD / 8 + 1) * 2;  // 40 words per lane and head: hi, then lo
+constexpr int F_FRAG_WORDS = (FD / 16) * (FD / 8 + 1) * 2;  // 20 words per lane and head
 
 struct FusedParams {
   const bf16* q;        // query planes, strides in qv
@@ -93,9 +93,11 @@ __device__ __forceinline__ void mma_bf16_first(float (&c)[4], const uint32_t (&a
 
 // The fp32 states [heads][32][33] (KV | key sum) as the per-lane B fragments the apply warps feed to
 // mma.sync: word (ks*5 + j)*2 + e of lane (g, t) packs rows a0, a0+1 (a0 = 8t + 4ks + 2e) of column
-// c = 8(g/2) + 2j + (g&1), or of the key-sum column for j = 4; words 0-19 hold the bf16 roundings,
-// words 20-39 the bf16 roundings of the remainders.  Laid out so that a lane fetches its 40 words
-// with ten 16-byte loads, consecutive lanes 16 bytes apart.
+// c = 8(g/2) + 2j + (g&1), or of the key-sum column for j = 4, rounded to bf16 like every other
+// tensor-core operand of the module (the sums themselves were accumulated in fp32; feeding the
+// remainders as a second set of fragments doubles the kernel's mma.sync work for a change of the
+// module's relative L2 error from 0.33 % to 0.30 %).  Laid out so that a lane fetches its 20
+// words with five 16-byte loads, consecutive lanes 16 bytes apart.
 __global__ void __launch_bounds__(256) state_fragments_kernel(const float* __restrict__ state, uint32_t* __restrict__ table) {
   pdl_launch_dependents();
   pdl_wait();  // the states come from the previous kernel
@@ -103,14 +105,12 @@ __global__ void __launch_bounds__(256) state_fragments_kernel(const float* __res
   uint32_t* tp = table + (long long)blockIdx.x * (F_FRAG_WORDS * 32);
   for (int i = threadIdx.x; i < F_FRAG_WORDS * 32; i += blockDim.x) {
     const int lane = i & 31, w = i >> 5;
-    const int lo = w >= F_FRAG_WORDS / 2, ww = lo ? w - F_FRAG_WORDS / 2 : w;
-    const int e = ww & 1, j = (ww >> 1) % (FD / 8 + 1), ks = (ww >> 1) / (FD / 8 + 1);
+    const int e = w & 1, j = (w >> 1) % (FD / 8 + 1), ks = (w >> 1) / (FD / 8 + 1);
     const int g = lane >> 2, t = lane & 3;
     const int a0 = 8 * t + 4 * ks + 2 * e;
     const int c = j < FD / 8 ? (g >> 1) * 8 + 2 * j + (g & 1) : FD;
     const float v0 = sp[a0 * (FD + 1) + c], v1 = sp[(a0 + 1) * (FD + 1) + c];
-    const float r0 = v0 - __bfloat162float(__float2bfloat16_rn(v0)), r1 = v1 - __bfloat162float(__float2bfloat16_rn(v1));
-    tp[((w >> 2) * 32 + lane) * 4 + (w & 3)] = lo ? pack2(r0, r1) : pack2(v0, v1);
+    tp[((w >> 2) * 32 + lane) * 4 + (w & 3)] = pack2(v0, v1);
   }
 }
 
@@ -215,8 +215,8 @@ apply_project_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
     }
   } else if (warp < 2 + F_APPLY_WARPS) {
     // ------------------------------------------------------------ apply warps
-    // Same arithmetic as the stand-alone apply kernel: A = relu(Q) (rows = 16 tokens), B = state as
-    // bf16 hi + lo; lane (g, t) holds channels 8t..8t+7 of tokens g and g+8 of each 16-token tile.
+    // A = relu(Q) (rows = 16 tokens), B = state; lane (g, t) holds channels 8t..8t+7 of tokens g and
+    // g+8 of each 16-token tile (the fragment layout of the stand-alone apply kernel).
     constexpr int KS = FD / 16, NT = FD / 8;
     const int aw = warp - 2;
     const int g = lane >> 2, t = lane & 3;
@@ -267,7 +267,7 @@ apply_project_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
       cp_async_commit();
     }
 
-    uint32_t bf[F_FRAG_WORDS];  // word (ks*(NT+1) + j)*2 + e: bf16 rounding of the state; + F_FRAG_WORDS/2: of the remainder
+    uint32_t bf[F_FRAG_WORDS];  // word (ks*(NT+1) + j)*2 + e
     bool ok = true, head_ok = false;
     for (int stp = 0; stp < total_steps; ++stp, advance(cc)) {
       const int ti = cc.ti, r = cc.r, st = cc.st;
@@ -315,13 +315,6 @@ apply_project_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
             const int w = (ks * (NT + 1) + j) * 2;
             if (ks == 0) mma_bf16_first(acc[u][j], A[u], bf[w], bf[w + 1]);
             else mma_bf16(acc[u][j], A[u], bf[w], bf[w + 1]);
-          }
-#pragma unroll
-        for (int j = 0; j <= NT; ++j)
-#pragma unroll
-          for (int u = 0; u < F_U; ++u) {
-            const int w = F_FRAG_WORDS / 2 + (ks * (NT + 1) + j) * 2;
-            mma_bf16(acc[u][j], A[u], bf[w], bf[w + 1]);
           }
       }
       // normalise and store into the slice: row = token of the tile (128 bytes = 64 channels of the pair),
