@@ -2,7 +2,8 @@
 """Benchmark of the multi-scale linear attention module forward on B200.
 
 A step is one whole-module forward (QKV projection, 5x5 aggregation, KV-state
-reduction, apply, output projection) on one seeded synthetic feature map.
+reduction, apply, output projection; the last two as one kernel where the
+library fuses them) on one seeded synthetic feature map.
 Prints one JSON line (rank 0).  See the design doc for the meaning of every field.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
@@ -29,6 +30,8 @@ from paper_2205_14756_b200 import inputs  # noqa: E402
 METRIC = "msla_fwd_tokens_per_s"
 UNIT = "tokens/s"
 STAGES = ("project_in", "aggregate", "kv_state", "apply", "project_out")
+# when the library runs steps 4 and 5 as one kernel (msla_forward_fuses_apply), they are one stage
+STAGES_FUSED = ("project_in", "aggregate", "kv_state", "apply_project")
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -47,6 +50,7 @@ def stage_bytes_per_token(s: inputs.ModuleShape) -> dict:
         "kv_state": 2 * 2 * Cp * e,              # K and V of both scales
         "apply": (2 * Cp + 2 * Cp) * e,          # Q of both scales in, attention out
         "project_out": (2 * Cp + Co) * e,
+        "apply_project": (2 * Cp + Co) * e,      # fused: Q of both scales in, y out; the head concat stays on chip
     }
 
 
@@ -58,6 +62,7 @@ def stage_flops_per_token(s: inputs.ModuleShape) -> dict:
         "kv_state": 2 * 2 * Cp * (d + 1),
         "apply": 2 * 2 * Cp * (d + 1),
         "project_out": 2 * 2 * Cp * Co,
+        "apply_project": 2 * 2 * Cp * (d + 1) + 2 * 2 * Cp * Co,
     }
 
 
@@ -333,38 +338,67 @@ def main() -> None:
     barrier()
     ms_e2e = e_a.elapsed_time(e_b)
     clocks = sampler.stop() if rank == 0 else None
+    del lanes
+
+    # The attention core (steps 3 + 4) on its own entry point, at this workload's head and token counts:
+    # in the fused module the apply step has no kernel of its own to time.
+    core = None
+    if s.dtype == "bf16" and rank == 0:
+        cB, cH, cN, cd = s.B, 2 * s.heads, s.N, s.d
+        q, k, v = (torch.randn(cB, cH, cN, cd, device="cuda").to(tdt) for _ in range(3))
+        o = torch.empty_like(q)
+        nb = binding.msla_linattn_relu_workspace_bytes(cB, cH, cN, cd)
+        cws = torch.empty(nb, dtype=torch.uint8, device="cuda")
+        for _ in range(3):
+            binding.msla_linattn_relu_ws(code, q, k, v, o, cB, cH, cN, cd, s.eps, cws, nb)
+        c_a, c_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c_a.record(stream)
+        for _ in range(K):
+            binding.msla_linattn_relu_ws(code, q, k, v, o, cB, cH, cN, cd, s.eps, cws, nb)
+        c_b.record(stream)
+        torch.cuda.synchronize()
+        core = (c_a.elapsed_time(c_b) / K, 4 * cB * cH * cN * cd * 2)
+        del q, k, v, o, cws
 
     ms_total, ms_e2e, ms_e2e_serial, ms_plain = max_over_ranks([ms_total, ms_e2e, ms_e2e_serial, ms_plain], device="cuda")
 
     if rank == 0:
-        tokens_step = s.B * s.N * world
+        fused = binding.msla_forward_fuses_apply(desc) == 1
+        stage_names = STAGES_FUSED if fused else STAGES
         stage_ms = {}
         for j, name in enumerate(STAGES):
             stage_ms[name] = statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(K))
+        if fused:  # the event between steps 4 and 5 falls directly after the one that ends step 3
+            stage_ms["apply_project"] = stage_ms.pop("apply") + stage_ms.pop("project_out")
         bpt, fpt = stage_bytes_per_token(s), stage_flops_per_token(s)
         peak, peak_kind = measured_peaks()
         stages = {}
-        for name in STAGES:
+        for name in stage_names:
             sec = stage_ms[name] * 1e-3
             stages[name] = {"ms": round(stage_ms[name], 5),
                             "GBps": round(bpt[name] * s.B * s.N / sec / 1e9, 1),
                             "frac_of_%s_hbm" % peak_kind: round(bpt[name] * s.B * s.N / sec / 1e9 / peak, 4),
                             "frac_of_8TBps": round(bpt[name] * s.B * s.N / sec / 8e12, 4),
                             "TFLOPps": round(fpt[name] * s.B * s.N / sec / 1e12, 2)}
-        dom = max(STAGES, key=lambda n: stage_ms[n])
+        dom = max(stage_names, key=lambda n: stage_ms[n])
         achieved = bpt[dom] * s.B * s.N / (stage_ms[dom] * 1e-3) / 1e9
-        core_ms = stage_ms["kv_state"] + stage_ms["apply"]
-        core_gbps = (bpt["kv_state"] + bpt["apply"]) * s.B * s.N / (core_ms * 1e-3) / 1e9
+        if core is not None:
+            core_ms, core_how = core[0], "stand-alone core entry (msla_linattn_relu_ws) on [B, 2*heads, N, d] of this workload"
+            core_gbps = core[1] / (core_ms * 1e-3) / 1e9
+        else:
+            core_ms, core_how = stage_ms["kv_state"] + stage_ms["apply"], "steps 3 + 4 inside the module"
+            core_gbps = (bpt["kv_state"] + bpt["apply"]) * s.B * s.N / (core_ms * 1e-3) / 1e9
+        module_bytes = sum(bpt[n] for n in stage_names) * s.B * s.N
         e = 4 if s.dtype == "f32" else 2
         roofline = {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                     "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}",
                     "traffic": recorded_traffic(dom, s.name),
                     "algorithmic_bytes_per_launch": bpt[dom] * s.B * s.N}
         if dom == "aggregate":
-            # HBM is the roof this step is judged against.  What limits the kernel as built is the issue rate of
-            # mma.sync: four of the five tap columns of the depthwise filter and the grouped 1x1 run as
-            # 192 warp-level MMAs per 8x8 pixel block (about 2.8 SM cycles each, measured).
-            roofline["limiter"] = "mma.sync issue rate (depthwise taps as diagonal-matrix MMAs) + fp32 pipes (fifth tap column)"
+            # HBM is the roof this step is judged against.  What limits the kernel as built is the shared-memory
+            # pipe (the staged tile is turned to channel-planar there, then read as MMA operands: about 65 % busy)
+            # together with the issue rate of mma.sync (112 warp-level MMAs per 8x8 pixel block).
+            roofline["limiter"] = "shared-memory pipe (tile transposition + ldmatrix operand loads) and mma.sync issue rate"
         result = {
             "metric": METRIC, "value": whole_job_value(s.B * s.N, world, ms_total, K), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": W, "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -372,7 +406,8 @@ def main() -> None:
             "config": {"workload": s.name, "B": s.B, "C": s.C, "H": s.H, "W": s.W, "heads_per_scale": s.heads, "d": s.d,
                        "tokens_per_step_per_gpu": s.B * s.N, "accumulate": "f32",
                        "l2": "inputs and intermediates of one step exceed the 126 MB L2" if
-                       sum(bpt.values()) * s.B * s.N > 4 * 126e6 else "working set fits L2: numbers are L2-resident",
+                       module_bytes > 4 * 126e6 else "working set fits L2: numbers are L2-resident",
+                       "steps_4_5_fused": fused,
                        "parallelism": f"replicas x{world}, one image per GPU, no collective"},
             "e2e": {"value": whole_job_value(s.B * s.N, world, ms_e2e, K), "unit": UNIT,
                     "h2d_bytes_per_step": s.B * s.C * s.N * e, "d2h_bytes_per_step": s.B * s.C_out * s.N * e,
@@ -380,12 +415,12 @@ def main() -> None:
                     "single_stream_ms_per_step": ms_e2e_serial / K},
             "gpu_launches": int(launches),
             "roofline": roofline,
-            "attention_core": {"ms": round(core_ms, 5), "GBps": round(core_gbps, 1),
+            "attention_core": {"how": core_how, "ms": round(core_ms, 5), "GBps": round(core_gbps, 1),
                                "frac_of_%s_hbm" % peak_kind: round(core_gbps / peak, 4),
                                "frac_of_8TBps": round(core_gbps / 8000.0, 4)},
             "stages": stages,
             "ms_per_step_without_stage_events": round(ms_plain / K, 5),
-            "module_GBps": round(sum(bpt.values()) * s.B * s.N / (ms_total * 1e-3 / K) / 1e9, 1),
+            "module_GBps": round(module_bytes / (ms_total * 1e-3 / K) / 1e9, 1),
             "clocks": clocks,
         }
         if world == 1 and not args.no_cpu_baseline:

@@ -178,6 +178,13 @@ size_t msla_forward_host_workspace_bytes(const msla_desc* desc);
 msla_status_t msla_forward_host(const msla_desc* desc, const void* x_host, const msla_weights* weights,
                                 void* out_host, void* stream);
 
+/* 1 if msla_forward runs steps 4 and 5 of Section 3.1 (apply and output
+ * projection) as one kernel for this descriptor, so that the head concat never
+ * goes to device memory; 0 if they run as two kernels; -1 on an invalid
+ * descriptor.  A pure function of the descriptor (workspace fields ignored);
+ * host only, launches nothing.  Benchmarks use it to attribute time and bytes. */
+int msla_forward_fuses_apply(const msla_desc* desc);
+
 /* Number of kernels this library has launched from the calling thread since it
  * was loaded (a bookkeeping counter for benchmarks; no paper counterpart). */
 unsigned long long msla_kernel_launches(void);

@@ -52,6 +52,7 @@ EXPORTS = {
                                       ctypes.POINTER(c_void_p), c_int]),
     "msla_forward_host_workspace_bytes": (c_size_t, [ctypes.POINTER(msla_desc)]),
     "msla_forward_host": (c_int, [ctypes.POINTER(msla_desc), c_void_p, ctypes.POINTER(msla_weights), c_void_p, c_void_p]),
+    "msla_forward_fuses_apply": (c_int, [ctypes.POINTER(msla_desc)]),
     "msla_kernel_launches": (ctypes.c_ulonglong, []),
     "msla_debug_wait_timeouts": (c_int, []),
     "msla_project_in": (c_int, [c_int] + [c_void_p] * 3 + [c_int] * 5 + [c_void_p]),
@@ -179,6 +180,10 @@ def msla_forward_host(desc: msla_desc, x_host, weights: msla_weights, out_host, 
 
 def msla_debug_wait_timeouts() -> int:
     return lib().msla_debug_wait_timeouts()
+
+
+def msla_forward_fuses_apply(desc: msla_desc) -> int:
+    return lib().msla_forward_fuses_apply(ctypes.byref(desc))
 
 
 def msla_kernel_launches() -> int:

@@ -3,7 +3,6 @@
 
 #include <cstdarg>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -388,8 +387,7 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   const HeadView ov = att_planar ? HeadView{(long long)N * ld_att, (long long)N * 2 * d, 2 * d, 1}
                                  : HeadView{(long long)N * ld_att, d, ld_att, 0};
   // Steps 4 and 5 run as one kernel when it takes the shape: the head concat then stays in shared memory.
-  static const bool no_fused = getenv("MSLA_NO_FUSED_APPLY") != nullptr;
-  const bool fused = !no_fused && desc->dtype == MSLA_BF16 && apply_project_bf16_supported(2 * heads, d, desc->C_out, N, in);
+  const bool fused = desc->dtype == MSLA_BF16 && apply_project_bf16_supported(2 * heads, d, desc->C_out, N, in);
   s = run_core(desc->dtype, ms, ms + (size_t)N * d * e, ms + (size_t)2 * N * d * e, att, in, ov, desc->B, 2 * heads, N, d, desc->eps, p.core,
                ws + p.core_off, st, events ? (cudaEvent_t)events[3] : nullptr, !fused);
   if (s != MSLA_OK) return s;
@@ -472,6 +470,13 @@ size_t msla_forward_host_workspace_bytes(const msla_desc* desc) {
 
 msla_status_t msla_forward_host(const msla_desc* desc, const void* x_host, const msla_weights* w, void* out_host, void* stream) {
   return forward_impl(desc, x_host, w, out_host, (cudaStream_t)stream, nullptr, true);
+}
+
+int msla_forward_fuses_apply(const msla_desc* desc) {
+  ForwardPlan p;
+  if (validate_desc(desc, &p) != MSLA_OK) return -1;
+  const HeadView in{6LL * p.Cp * p.N, 3LL * p.N * desc->d, desc->d};
+  return desc->dtype == MSLA_BF16 && apply_project_bf16_supported(2 * desc->heads, desc->d, desc->C_out, p.N, in) ? 1 : 0;
 }
 
 unsigned long long msla_kernel_launches(void) { return g_launches; }
