@@ -53,6 +53,7 @@ constexpr int PL_CH = 2 * PL_HALF + 16;      // 976 = 16 * 61: channel pitch, od
 constexpr int PL_BYTES = TD * PL_CH;
 constexpr int DWO_CH = TW * TH * 2 + 16;     // 528 = 16 * 33: depthwise output, bytes per channel
 constexpr int DWO_BYTES = TD * DWO_CH;
+constexpr int T_BAND = 4;                    // tile rows per band of the traversal
 constexpr int T_WARPS = 8;
 constexpr int T_THREADS = 32 * T_WARPS;
 constexpr int OUT_WARP_BYTES = 4 * 8 * 64;   // output staging per warp: 4 rows x 8 pixels x 32 channels
@@ -93,7 +94,7 @@ struct ToeplitzParams {
   int src_planes_per_batch;    // plane index of (b, group) in a tensor map = b * planes_per_batch + group
   int dst_planes_per_batch;
   int groups;
-  int tiles_x, tiles_total;    // tiles per plane
+  int tiles_x, tiles_y, tiles_total;  // tiles per plane
   long long units;             // B * groups * tiles_total, tile fastest
   long long units_per_cta;
 };
@@ -112,23 +113,32 @@ aggregate_toeplitz_kernel(const __grid_constant__ CUtensorMap tm_src, const __gr
   const int unit_count = (int)max(0LL, min(p.units_per_cta, p.units - unit_first));
   const uint32_t bar = smem_addr(&bar_storage);
 
-  // Cursor over (image, group, tile) units, tile fastest, advanced without divisions.
-  struct Unit { int tile, tx, ty, group, b; };
+  // Cursor over (image, group, tile) units, tile fastest, advanced without divisions.  Inside a plane the
+  // tiles run down bands of T_BAND tile rows, column by column, so that a tile's lower and right
+  // neighbours follow within a few iterations and find the shared halo rows and columns in L2.
+  struct Unit { int tile, tx, ty, band_end, group, b; };  // band_end: first tile row below the current band
   auto locate = [&](long long u) {
     const long long bg = u / p.tiles_total;
     Unit r;
     r.tile = (int)(u - bg * p.tiles_total);
-    r.ty = r.tile / p.tiles_x;
-    r.tx = r.tile - r.ty * p.tiles_x;
+    const int band = r.tile / (T_BAND * p.tiles_x), rem = r.tile - band * (T_BAND * p.tiles_x);
+    r.band_end = min(band * T_BAND + T_BAND, p.tiles_y);
+    const int bh = r.band_end - band * T_BAND;
+    r.tx = rem / bh;
+    r.ty = band * T_BAND + rem - r.tx * bh;
     r.b = (int)(bg / p.groups);
     r.group = (int)(bg - (long long)r.b * p.groups);
     return r;
   };
   auto advance = [&](Unit& u) {
     ++u.tile;
-    if (++u.tx == p.tiles_x) { u.tx = 0; ++u.ty; }
+    if (++u.ty == u.band_end) {
+      const int band_start = (u.band_end - 1) / T_BAND * T_BAND;
+      if (++u.tx == p.tiles_x) { u.tx = 0; u.ty = u.band_end; u.band_end = min(u.band_end + T_BAND, p.tiles_y); }
+      else u.ty = band_start;
+    }
     if (u.tile == p.tiles_total) {
-      u.tile = 0; u.ty = 0;
+      u.tile = 0; u.ty = 0; u.band_end = min(T_BAND, p.tiles_y);
       if (++u.group == p.groups) { u.group = 0; ++u.b; }
     }
   };
@@ -343,7 +353,8 @@ msla_status_t run_aggregate_toeplitz_bf16(const void* src, long long src_planes_
   p.w_dw = (const bf16*)w_dw; p.w_pw = (const bf16*)w_pw;
   p.src_planes_per_batch = src_ppb; p.dst_planes_per_batch = dst_ppb; p.groups = Ch / TD;
   p.tiles_x = (W + TW - 1) / TW;
-  const long long tiles = (long long)p.tiles_x * ((H + TH - 1) / TH);
+  p.tiles_y = (H + TH - 1) / TH;
+  const long long tiles = (long long)p.tiles_x * p.tiles_y;
   if (tiles > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many aggregation tiles");
   p.tiles_total = (int)tiles;
   p.units = tiles * p.groups * B;
