@@ -33,6 +33,9 @@ SMALL = [
     ("r7", "f32", 1, 16, 1, 1, 1, 16),
     ("r8", "bf16", 1, 128, 40, 24, 8, 16),
     ("r9", "bf16", 2, 48, 11, 13, 3, 16),
+    # 10 heads over both scales: the fused apply + projection kernel runs a second round with two heads only;
+    # 240 tokens per image: a ragged last token tile in each of two images
+    ("r10", "bf16", 2, 160, 12, 20, 5, 32),
 ]
 
 
@@ -132,7 +135,10 @@ def test_stage_project_out(dtype, B, Cin, Cout, N):
                                               ("bf16", 1, 64, 64, 192, 32), ("bf16", 1, 3, 70, 64, 16), ("bf16", 2, 16, 16, 32, 32),
                                               ("bf16", 1, 17, 35, 64, 32), ("bf16", 1, 5, 3, 32, 32), ("bf16", 1, 40, 7, 32, 32),
                                               ("bf16", 2, 19, 37, 96, 16), ("bf16", 1, 64, 64, 192, 16), ("bf16", 1, 2, 2, 32, 16),
-                                              ("bf16", 1, 9, 9, 48, 16)])
+                                              ("bf16", 1, 9, 9, 48, 16),
+                                              # 432 (image, group, tile) units of 9 tiles per plane: the persistent CTAs' runs cross
+                                              # tile-band, group and image boundaries
+                                              ("bf16", 4, 48, 48, 384, 32)])
 def test_stage_aggregate(dtype, B, H, W, Ch, d):
     t = inputs.quantise(inputs.normal(3, 0, B * Ch * H * W).reshape(B, Ch, H, W), dtype)
     w_dw = inputs.quantise(inputs.normal(3, 1, Ch * 25, 0.2).reshape(Ch, 5, 5), dtype)
