@@ -220,6 +220,9 @@ apply_project_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
     constexpr int KS = FD / 16, NT = FD / 8;
     const int aw = warp - 2;
     const int g = lane >> 2, t = lane & 3;
+    // MMA rows g and g+8 of a 16-token tile are tokens gp and gp+8: the eight lanes of a quarter-warp
+    // (g = 2i, 2i+1) then write slice rows i and i+4, whose 16-byte pieces fall into different banks
+    const int gp = (g >> 1) | ((g & 1) << 2);
     const int s = aw >> 1;                                 // B slice of this warp's pair
     const int uses_per_tile = P > s ? (P - s + F_SLICES - 1) / F_SLICES : 0;
     const uint32_t ring = fifo + aw * (F_QSTAGES * F_QSTAGE_BYTES) + lane * 16;
@@ -250,7 +253,7 @@ apply_project_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
       if (h < p.heads) {                                   // else idle in the last round
         const bf16* qh = p.q + (long long)ic.b * p.qv.batch + (long long)h * p.qv.head + t * 8;
         const uint32_t dst = ring + (issued % F_QSTAGES) * F_QSTAGE_BYTES;
-        const int n0 = ic.nt * FT + ic.st * F_STEP_TOKENS + g;
+        const int n0 = ic.nt * FT + ic.st * F_STEP_TOKENS + gp;
 #pragma unroll
         for (int u = 0; u < 2 * F_U; ++u) {                // u even: token g of tile u/2, odd: token g+8
           const int n = n0 + u * 8;
@@ -328,7 +331,7 @@ apply_project_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
           oa[j] = pack2(acc[u][j][0] * inv_a, acc[u][j][1] * inv_a);
           ob[j] = pack2(acc[u][j][2] * inv_b, acc[u][j][3] * inv_b);
         }
-        const uint32_t ra = (uint32_t)(st * F_STEP_TOKENS + u * 16 + g), rb = ra + 8;
+        const uint32_t ra = (uint32_t)(st * F_STEP_TOKENS + u * 16 + gp), rb = ra + 8;
         const uint32_t chunk = (uint32_t)(4 * (aw & 1) + t);
         asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(slice + ra * 128 + ((chunk ^ (ra & 7)) << 4)),
                      "r"(oa[0]), "r"(oa[1]), "r"(oa[2]), "r"(oa[3]) : "memory");
