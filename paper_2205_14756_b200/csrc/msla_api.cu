@@ -482,8 +482,8 @@ int msla_forward_fuses_apply(const msla_desc* desc) {
 unsigned long long msla_kernel_launches(void) { return g_launches; }
 
 int msla_debug_wait_timeouts(void) {
-  const int a = gemm_timeout_flag(), b = agg_timeout_flag(), c = fused_timeout_flag(), d = aggt_timeout_flag();
-  return (a < 0 || b < 0 || c < 0 || d < 0) ? -1 : (a | b | c | d);
+  const int a = gemm_timeout_flag(), b = agg_timeout_flag(), c = fused_timeout_flag();
+  return (a < 0 || b < 0 || c < 0) ? -1 : (a | b | c);
 }
 
 msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d, void* stream) {

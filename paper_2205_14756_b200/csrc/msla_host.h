@@ -71,18 +71,12 @@ msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const vo
                                           int Cout, int N, cudaStream_t st);
 int gemm_timeout_flag();
 
-// bf16 aggregation (d = 16 or 32, Ch a multiple of 32) with TMA halo tiles (agg_bf16.cu).
+// bf16 aggregation (d = 16 or 32, Ch a multiple of 32): TMA halo tiles, depthwise filter as banded matrices on
+// tensor cores (agg_bf16.cu).  dst_sb must be a multiple of the plane size H*W*d.
 bool aggregate_bf16_supported(int H, int W, int Ch, int d);
 msla_status_t run_aggregate_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
                                  const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch, int d,
                                  cudaStream_t st);
 int agg_timeout_flag();
-
-// bf16 aggregation for d = 32 with the depthwise filter as banded matrices on tensor cores (agg_toeplitz.cu).
-bool aggregate_toeplitz_bf16_supported(int H, int W, int Ch, int d);
-msla_status_t run_aggregate_toeplitz_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
-                                          const void* w_pw, void* dst, long long dst_planes_total, int dst_ppb, int B,
-                                          int H, int W, int Ch, cudaStream_t st);
-int aggt_timeout_flag();
 
 }  // namespace msla
