@@ -397,13 +397,14 @@ msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out
     attr_done = true;
   }
   launch_pdl(kv_state_mma_kernel<D, KV_WARPS, KV_STAGES>, dim3((unsigned)BH, p.S), dim3(KV_WARPS * 32), kv_smem, st, k, v, partial, in, heads, N, p.S, p.chunk);
+  if (!with_apply) {  // the caller combines the partial states itself
+    if (mid) cudaEventRecord(mid, st);
+    count_launches(1);
+    return check_launch("attention state kernel (bf16)");
+  }
   const long long total = BH * p.ne;
   launch_pdl(kv_combine_bf16path_kernel, dim3((unsigned)ceil_div_ll(total, 256)), dim3(256), 0, st, partial, state, p.S, p.ne, total);
   if (mid) cudaEventRecord(mid, st);
-  if (!with_apply) {
-    count_launches(2);
-    return check_launch("attention state kernels (bf16)");
-  }
   if (ov.pair) {  // heads is even here, so a pair never straddles two images
     const int tok_per_cta = p.apply_tokens / 2;
     launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, true>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)(BH / 2)),

@@ -91,26 +91,35 @@ __device__ __forceinline__ void mma_bf16_first(float (&c)[4], const uint32_t (&a
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
 }
 
-// The fp32 states [heads][32][33] (KV | key sum) as the per-lane B fragments the apply warps feed to
-// mma.sync: word (ks*5 + j)*2 + e of lane (g, t) packs rows a0, a0+1 (a0 = 8t + 4ks + 2e) of column
-// c = 8(g/2) + 2j + (g&1), or of the key-sum column for j = 4, rounded to bf16 like every other
-// tensor-core operand of the module (the sums themselves were accumulated in fp32; feeding the
-// remainders as a second set of fragments doubles the kernel's mma.sync work for a change of the
-// module's relative L2 error from 0.33 % to 0.30 %).  Laid out so that a lane fetches its 20
-// words with five 16-byte loads, consecutive lanes 16 bytes apart.
-__global__ void __launch_bounds__(256) state_fragments_kernel(const float* __restrict__ state, uint32_t* __restrict__ table) {
+// Second level of the state reduction, straight into the form the apply warps consume.  One CTA per
+// head: every state entry [32][33] (KV | key sum) is the sum of its S partial states in index order (a
+// fixed order, so results are reproducible bit for bit), accumulated in fp32 and kept in shared
+// memory; the CTA then writes the state as per-lane B fragments of mma.sync.  Word (ks*5 + j)*2 + e
+// of lane (g, t) packs rows a0, a0+1 (a0 = 8t + 4ks + 2e) of column c = 8(g/2) + 2j + (g&1), or of the
+// key-sum column for j = 4, rounded to bf16 like every other tensor-core operand of the module
+// (feeding the remainders as a second set of fragments doubles the kernel's mma.sync work for a
+// change of the module's relative L2 error from 0.33 % to 0.30 %).  Laid out so that a lane fetches
+// its 20 words with five 16-byte loads, consecutive lanes 16 bytes apart.
+constexpr int F_NE = FD * (FD + 1);
+__global__ void __launch_bounds__(F_NE / 2) state_fragments_kernel(const float* __restrict__ partial, int S, uint32_t* __restrict__ table) {
+  __shared__ float st[F_NE];
   pdl_launch_dependents();
-  pdl_wait();  // the states come from the previous kernel
-  const float* sp = state + (long long)blockIdx.x * (FD * (FD + 1));
+  pdl_wait();  // the partial states come from the previous kernel
+  const float* sp = partial + (long long)blockIdx.x * S * F_NE + threadIdx.x;
+  float v0 = 0.f, v1 = 0.f;
+#pragma unroll 8
+  for (int s = 0; s < S; ++s) { v0 += sp[(long long)s * F_NE]; v1 += sp[(long long)s * F_NE + F_NE / 2]; }
+  st[threadIdx.x] = v0;
+  st[threadIdx.x + F_NE / 2] = v1;
+  __syncthreads();
   uint32_t* tp = table + (long long)blockIdx.x * (F_FRAG_WORDS * 32);
-  for (int i = threadIdx.x; i < F_FRAG_WORDS * 32; i += blockDim.x) {
+  for (int i = threadIdx.x; i < F_FRAG_WORDS * 32; i += F_NE / 2) {
     const int lane = i & 31, w = i >> 5;
     const int e = w & 1, j = (w >> 1) % (FD / 8 + 1), ks = (w >> 1) / (FD / 8 + 1);
     const int g = lane >> 2, t = lane & 3;
     const int a0 = 8 * t + 4 * ks + 2 * e;
     const int c = j < FD / 8 ? (g >> 1) * 8 + 2 * j + (g & 1) : FD;
-    const float v0 = sp[a0 * (FD + 1) + c], v1 = sp[(a0 + 1) * (FD + 1) + c];
-    tp[((w >> 2) * 32 + lane) * 4 + (w & 3)] = pack2(v0, v1);
+    tp[((w >> 2) * 32 + lane) * 4 + (w & 3)] = pack2(st[a0 * (FD + 1) + c], st[(a0 + 1) * (FD + 1) + c]);
   }
 }
 
@@ -425,11 +434,12 @@ bool apply_project_bf16_supported(int heads, int d, int Cout, int N, HeadView qv
 }
 
 // y[b][m][n] = sum_h sum_c w[m][32 h + c] * att[b][h][n][c] + bias[m], att = Eq. 3 applied to query head h with
-// state[b * heads + h] ([32][33] fp32: KV, then the key sum in column 32); y is NCHW [B, Cout, N].
+// the state of (b, h) = sum over s < S of partial[(b * heads + h) * S + s] ([32][33] fp32 each: KV, then the
+// key sum in column 32); y is NCHW [B, Cout, N].
 // scratch: apply_project_scratch_bytes(B, heads) bytes of device memory, 16-byte aligned (the states as fragments).
 size_t apply_project_scratch_bytes(int B, int heads) { return (size_t)B * heads * F_FRAG_WORDS * 32 * sizeof(uint32_t); }
 
-msla_status_t run_apply_project_bf16(const void* q, const float* state, void* scratch, const void* w, const void* bias, void* y,
+msla_status_t run_apply_project_bf16(const void* q, const float* partial, int S, void* scratch, const void* w, const void* bias, void* y,
                                      HeadView qv, int B, int heads, int N, int Cout, float eps, cudaStream_t st) {
   const int K = heads * FD;
   CUtensorMap tmA, tmO;
@@ -464,7 +474,7 @@ msla_status_t run_apply_project_bf16(const void* q, const float* state, void* sc
   cudaGetDevice(&dev);
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
   const int grid = (int)(tiles < sms ? tiles : sms);
-  launch_pdl(state_fragments_kernel, dim3((unsigned)(B * heads)), dim3(256), 0, st, state, (uint32_t*)scratch);
+  launch_pdl(state_fragments_kernel, dim3((unsigned)(B * heads)), dim3(F_NE / 2), 0, st, partial, S, (uint32_t*)scratch);
   launch_pdl(apply_project_fused_kernel, dim3(grid), dim3(F_THREADS), F_SMEM_BYTES, st, tmA, tmO, p);
   count_launches(2);
   return check_launch("fused apply + output projection (tcgen05)");

@@ -394,7 +394,7 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   if ((s = record(events, 4, st)) != MSLA_OK) return s;
   // 5. output projection back to NCHW
   if (fused)
-    s = run_apply_project_bf16(ms, reinterpret_cast<const float*>(ws + p.core_off + p.core.state_off), att, w->w_proj, w->b_proj, out_dev, in,
+    s = run_apply_project_bf16(ms, reinterpret_cast<const float*>(ws + p.core_off + p.core.partial_off), p.core.S, att, w->w_proj, w->b_proj, out_dev, in,
                                desc->B, 2 * heads, N, desc->C_out, desc->eps, st);
   else
     s = att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st)

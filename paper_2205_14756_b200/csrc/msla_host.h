@@ -46,7 +46,7 @@ inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 
 struct HeadView;
 // Tuned bf16 attention core (d in {16, 32}); all view strides must be multiples of 8 elements.
-// with_apply = false stops after the combined states (at ws + p.state_off); `out` and `ov` are then unused.
+// with_apply = false stops after the partial states (at ws + p.partial_off, p.S per head); `out` and `ov` are then unused.
 msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* out, HeadView in, HeadView ov, int B,
                             int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st,
                             cudaEvent_t mid, bool with_apply);
@@ -55,7 +55,7 @@ msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* o
 // number of heads, Cout <= 256, query strides multiples of 8 elements.
 bool apply_project_bf16_supported(int heads, int d, int Cout, int N, HeadView qv);
 size_t apply_project_scratch_bytes(int B, int heads);
-msla_status_t run_apply_project_bf16(const void* q, const float* state, void* scratch, const void* w, const void* bias, void* y,
+msla_status_t run_apply_project_bf16(const void* q, const float* partial, int S, void* scratch, const void* w, const void* bias, void* y,
                                      HeadView qv, int B, int heads, int N, int Cout, float eps, cudaStream_t st);
 int fused_timeout_flag();
 
