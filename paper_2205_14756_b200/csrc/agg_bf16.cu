@@ -388,13 +388,14 @@ msla_status_t launch_toeplitz(const void* src, long long src_planes_total, int s
   p.units_per_cta = (p.units + ctas - 1) / ctas;
   if (p.units_per_cta > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many aggregation tiles");
   const unsigned grid = (unsigned)((p.units + p.units_per_cta - 1) / p.units_per_cta);
-  static bool attr_done = false;  // one flag per instantiation
-  if (!attr_done) {
+  static unsigned long long attr_done = 0;  // devices on which the attribute is set (a race only repeats the call)
+  const unsigned long long dev_bit = current_device_bit();
+  if (!(attr_done & dev_bit)) {
     if (cudaFuncSetAttribute(aggregate_toeplitz_kernel<D16>, cudaFuncAttributeMaxDynamicSharedMemorySize, T_SMEM_BYTES) != cudaSuccess) {
       cudaGetLastError();
       return fail(MSLA_ERR_CUDA, "cannot reserve %d bytes of shared memory for the aggregation", T_SMEM_BYTES);
     }
-    attr_done = true;
+    attr_done |= dev_bit;
   }
   launch_pdl(aggregate_toeplitz_kernel<D16>, dim3(grid), dim3(T_THREADS), T_SMEM_BYTES, st, tm_src, tm_dst, p);
   count_launches(1);

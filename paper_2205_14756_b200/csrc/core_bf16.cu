@@ -391,10 +391,11 @@ msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out
   float* partial = reinterpret_cast<float*>(ws + p.partial_off);
   float* state = reinterpret_cast<float*>(ws + p.state_off);
   constexpr int kv_smem = KV_WARPS * KV_STAGES * 2 * 32 * D * 2;
-  static bool attr_done = false;  // idempotent; a race only repeats the call
-  if (!attr_done) {
+  static unsigned long long attr_done = 0;  // devices on which the attribute is set (a race only repeats the call)
+  const unsigned long long dev_bit = current_device_bit();
+  if (!(attr_done & dev_bit)) {
     cudaFuncSetAttribute(kv_state_mma_kernel<D, KV_WARPS, KV_STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, kv_smem);
-    attr_done = true;
+    attr_done |= dev_bit;
   }
   launch_pdl(kv_state_mma_kernel<D, KV_WARPS, KV_STAGES>, dim3((unsigned)BH, p.S), dim3(KV_WARPS * 32), kv_smem, st, k, v, partial, in, heads, N, p.S, p.chunk);
   if (!with_apply) {  // the caller combines the partial states itself

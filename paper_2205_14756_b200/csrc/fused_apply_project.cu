@@ -462,13 +462,14 @@ msla_status_t run_apply_project_bf16(const void* q, const float* partial, int S,
   const long long tiles = (long long)B * p.tiles_per_batch;
   if (tiles > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many token tiles");
   p.num_tiles = (int)tiles;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static unsigned long long attr_done = 0;  // devices on which the attribute is set (a race only repeats the call)
+  const unsigned long long dev_bit = current_device_bit();
+  if (!(attr_done & dev_bit)) {
     if (cudaFuncSetAttribute(apply_project_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, F_SMEM_BYTES) != cudaSuccess) {
       cudaGetLastError();
       return fail(MSLA_ERR_CUDA, "cannot reserve %d bytes of shared memory for the fused apply + output projection", F_SMEM_BYTES);
     }
-    attr_done = true;
+    attr_done |= dev_bit;
   }
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);

@@ -485,13 +485,14 @@ int sm_count() {
 template <bool A_MN>
 msla_status_t launch_stationary(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO, const GemmParams& p,
                                 int blocks, cudaStream_t st) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static unsigned long long attr_done = 0;  // devices on which the attribute is set (a race only repeats the call)
+  const unsigned long long dev_bit = current_device_bit();
+  if (!(attr_done & dev_bit)) {
     if (cudaFuncSetAttribute(gemm_bf16_stationary_kernel<A_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, WS_SMEM_BYTES) != cudaSuccess) {
       cudaGetLastError();
       return fail(MSLA_ERR_CUDA, "cannot reserve %d bytes of shared memory for the projection GEMM", WS_SMEM_BYTES);
     }
-    attr_done = true;
+    attr_done |= dev_bit;
   }
   const long long stream_total = (long long)p.batches * (A_MN ? p.m_tiles : p.n_tiles);
   long long workers = sm_count() / blocks;
@@ -508,13 +509,14 @@ msla_status_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUten
   const int k_iters = (p.K + BK - 1) / BK;
   if (A_MN && k_iters * B_STAGE_BYTES <= RES_BYTES && blocks <= 16 && blocks <= sm_count())
     return launch_stationary<A_MN>(tmA, tmB, tmO, p, blocks, st);
-  static bool attr_done = false;
-  if (!attr_done) {
+  static unsigned long long attr_done = 0;  // devices on which the attribute is set (a race only repeats the call)
+  const unsigned long long dev_bit = current_device_bit();
+  if (!(attr_done & dev_bit)) {
     if (cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel<A_MN, B_PLANAR>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
       cudaGetLastError();
       return fail(MSLA_ERR_CUDA, "cannot reserve %d bytes of shared memory for the projection GEMM", SMEM_BYTES);
     }
-    attr_done = true;
+    attr_done |= dev_bit;
   }
   const long long tiles = (long long)p.batches * p.m_tiles * p.n_tiles;
   const int grid = (int)(tiles < sm_count() ? tiles : sm_count());

@@ -27,6 +27,15 @@ msla_status_t check_launch(const char* what);
 
 void count_launches(int n);
 
+// Function attributes (the dynamic shared-memory limit) belong to one device: a launch site keeps a
+// mask of the devices on which it has set them.  Bit of the current device; 0 for device numbers past
+// 63, which makes the site set the attribute on every call there.
+inline unsigned long long current_device_bit() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 0; }
+  return (dev >= 0 && dev < 64) ? 1ull << dev : 0ull;
+}
+
 // Launches `kernel` with programmatic stream serialization allowed: it may become resident before the
 // previous kernel of the stream has finished, and orders itself with pdl_wait() (msla_common.cuh).
 template <typename... KArgs, typename... Args>
