@@ -91,8 +91,8 @@ __device__ __forceinline__ void mma_bf16_first(float (&c)[4], const uint32_t (&a
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
 }
 
-// Second level of the state reduction, straight into the form the apply warps consume.  One CTA per
-// head: every state entry [32][33] (KV | key sum) is the sum of its S partial states in index order (a
+// Second level of the state reduction, straight into the form the apply warps consume.  Four CTAs per
+// head, eight state rows each: every state entry [32][33] (KV | key sum) is the sum of its S partial states in index order (a
 // fixed order, so results are reproducible bit for bit), accumulated in fp32 and kept in shared
 // memory; the CTA then writes the state as per-lane B fragments of mma.sync.  Word (ks*5 + j)*2 + e
 // of lane (g, t) packs rows a0, a0+1 (a0 = 8t + 4ks + 2e) of column c = 8(g/2) + 2j + (g&1), or of the
@@ -101,23 +101,24 @@ __device__ __forceinline__ void mma_bf16_first(float (&c)[4], const uint32_t (&a
 // change of the module's relative L2 error from 0.33 % to 0.30 %).  Laid out so that a lane fetches
 // its 20 words with five 16-byte loads, consecutive lanes 16 bytes apart.
 constexpr int F_NE = FD * (FD + 1);
-__global__ void __launch_bounds__(F_NE / 2) state_fragments_kernel(const float* __restrict__ partial, int S, uint32_t* __restrict__ table) {
-  __shared__ float st[F_NE];
+constexpr int F_FRAG_ROWS = 8;                       // state rows per CTA: rows 8q .. 8q+7 feed exactly the lanes with t = q
+constexpr int F_FRAG_THREADS = F_FRAG_ROWS * (FD + 1);  // one state entry per thread
+__global__ void __launch_bounds__(F_FRAG_THREADS) state_fragments_kernel(const float* __restrict__ partial, int S, uint32_t* __restrict__ table) {
+  __shared__ float st[F_FRAG_ROWS * (FD + 1)];
   pdl_launch_dependents();
   pdl_wait();  // the partial states come from the previous kernel
-  const float* sp = partial + (long long)blockIdx.x * S * F_NE + threadIdx.x;
-  float v0 = 0.f, v1 = 0.f;
+  const int head = blockIdx.x, q = blockIdx.y;
+  const float* sp = partial + (long long)head * S * F_NE + q * F_FRAG_ROWS * (FD + 1) + threadIdx.x;
+  float v = 0.f;
 #pragma unroll 8
-  for (int s = 0; s < S; ++s) { v0 += sp[(long long)s * F_NE]; v1 += sp[(long long)s * F_NE + F_NE / 2]; }
-  st[threadIdx.x] = v0;
-  st[threadIdx.x + F_NE / 2] = v1;
+  for (int s = 0; s < S; ++s) v += sp[(long long)s * F_NE];
+  st[threadIdx.x] = v;
   __syncthreads();
-  uint32_t* tp = table + (long long)blockIdx.x * (F_FRAG_WORDS * 32);
-  for (int i = threadIdx.x; i < F_FRAG_WORDS * 32; i += F_NE / 2) {
-    const int lane = i & 31, w = i >> 5;
+  uint32_t* tp = table + (long long)head * (F_FRAG_WORDS * 32);
+  for (int i = threadIdx.x; i < F_FRAG_WORDS * 8; i += F_FRAG_THREADS) {  // the 20 words of the 8 lanes (g, t = q)
+    const int g = i & 7, w = i >> 3, lane = 4 * g + q;
     const int e = w & 1, j = (w >> 1) % (FD / 8 + 1), ks = (w >> 1) / (FD / 8 + 1);
-    const int g = lane >> 2, t = lane & 3;
-    const int a0 = 8 * t + 4 * ks + 2 * e;
+    const int a0 = 4 * ks + 2 * e;                     // row 8q + a0 of the state, local row a0
     const int c = j < FD / 8 ? (g >> 1) * 8 + 2 * j + (g & 1) : FD;
     tp[((w >> 2) * 32 + lane) * 4 + (w & 3)] = pack2(st[a0 * (FD + 1) + c], st[(a0 + 1) * (FD + 1) + c]);
   }
@@ -475,7 +476,7 @@ msla_status_t run_apply_project_bf16(const void* q, const float* partial, int S,
   cudaGetDevice(&dev);
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
   const int grid = (int)(tiles < sms ? tiles : sms);
-  launch_pdl(state_fragments_kernel, dim3((unsigned)(B * heads)), dim3(F_NE / 2), 0, st, partial, S, (uint32_t*)scratch);
+  launch_pdl(state_fragments_kernel, dim3((unsigned)(B * heads), FD / F_FRAG_ROWS), dim3(F_FRAG_THREADS), 0, st, partial, S, (uint32_t*)scratch);
   launch_pdl(apply_project_fused_kernel, dim3(grid), dim3(F_THREADS), F_SMEM_BYTES, st, tmA, tmO, p);
   count_launches(2);
   return check_launch("fused apply + output projection (tcgen05)");
