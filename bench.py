@@ -4,7 +4,13 @@
 A step is one whole-module forward (QKV projection, 5x5 aggregation, KV-state
 reduction, apply, output projection; the last two as one kernel where the
 library fuses them) on one seeded synthetic feature map.
-Prints one JSON line (rank 0).  See the design doc for the meaning of every field.
+Prints one JSON line (rank 0): `value` is tokens/s of the whole job from CUDA
+events around the timed steps, `stages` the per-step times and algorithmic
+HBM rates from events recorded between the steps, `roofline` the slowest
+step against the measured HBM copy rate, `attention_core` the stand-alone
+core entry point at the workload's head and token counts, `e2e` the same
+metric with pinned host buffers and the copies inside the timed region,
+`cpu_baseline` the fp64 oracle on the host cores.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 """
