@@ -1,0 +1,499 @@
+// Steps 4 and 5 of the module (Section 3.1: apply step of Eq. 3, head concat,
+// final linear projection) as one tensor-core GEMM per image.
+//
+// Eq. 3 gives, for head h and token n,  O_h[n][c] = sum_a relu(q_h[n][a]) S_h[a][c] / den_h[n]
+// with den_h[n] = sum_a relu(q_h[n][a]) ks_h[a] + eps, and the projection is
+// y[m][n] = sum_h sum_c w[m][h*d + c] O_h[n][c] + bias[m].  Re-associating the two sums,
+//
+//   y[m][n] = sum_h sum_a  M[m][h*d + a] * qt[h*d + a][n]  + bias[m],
+//   M[m][h*d + a] = sum_c w[m][h*d + c] S_h[a][c]          (per image, C_out x 2C', tiny)
+//   qt[h*d + a][n] = relu(q_h[n][a]) / den_h[n]            (the queries, scaled per head and token)
+//
+// which is exact in real arithmetic: the d x d contraction of the apply step moves
+// from every token into the small matrix M, and what is left per token and head is
+// one d-term dot product (the normaliser) and a scaling.  M and qt are rounded to
+// bf16 where the unfused path rounds S and O.
+//
+// state_fold_kernel : sums the partial states in index order (fixed order, so the result
+//                     is reproducible bit for bit), writes ks and M (fp32 accumulate, bf16 out).
+// fused_out_kernel  : clusters of two CTAs, paired tensor-core MMAs (cta_group::2, M = 256).
+//   Each CTA keeps its 128 rows of M (<= 128 KB) in shared memory while the image lasts and
+//   owns 128 of the pair's 256 tokens per tile.  Per 64-channel slice of the queries:
+//     warp 0       TMA: two boxes of 64 channels x 64 tokens (token index contiguous, 128B swizzle)
+//     warps 2-9    turn q into qt in place (normaliser on the fp32 pipes, one token pair per lane)
+//     warp 1       (leader CTA only) issues tcgen05.mma 256 x 256 x 16: A = M (K-major), B = qt
+//                  (MN-major), fp32 accumulators in both CTAs' tensor memory
+//     warps 10-13  drain the accumulators: TMEM -> bf16 (+ bias) -> swizzled staging -> TMA
+//                  stores of 32-channel x 64-token blocks into the NCHW output
+//   Two accumulator sets (2 x 256 TMEM columns) let the drain of a tile overlap the next.
+// No TMA load is multicast: each CTA loads its own operands; only tcgen05.commit signals
+// both CTAs' barriers.  Every mbarrier wait is bounded as in the GEMM.
+#include <cuda.h>
+
+#include "msla_common.cuh"
+#include "msla_host.h"
+#include "tma_host.h"
+#include "tcgen05_util.cuh"
+
+namespace msla {
+namespace {
+
+using bf16 = __nv_bfloat16;
+
+constexpr int OT = 128;                  // tokens per CTA and tile (256 per pair)
+constexpr int OM = 128;                  // output channels per CTA (256 per pair)
+constexpr int OKS = 64;                  // channels per k-slice
+constexpr int O_BOX = 64 * OKS * 2;      // 8 KB: 64 channels x 64 tokens
+constexpr int O_SLICE = (OT / 64) * O_BOX;  // 16 KB
+constexpr int O_A_SLICE = OM * OKS * 2;  // 16 KB: 128 rows of M x 64 k
+constexpr int O_MAX_KS = 8;              // K = 2C' <= 512
+constexpr int O_STAGES = 4;
+constexpr int O_XWARPS = 8;              // transform warps: two groups of four, alternating slices
+constexpr int O_THREADS = 32 * (2 + O_XWARPS + 4);
+constexpr int O_STAGING_WARP = 32 * 128;
+constexpr int O_STAGING = 4 * O_STAGING_WARP;
+constexpr int O_BAR_BYTES = 256;
+
+__device__ int g_fused_timeout_flag = 0;
+
+struct OutParams {
+  const float* ks;   // [B][Ht][d] key sums
+  const bf16* bias;  // [Cout] or nullptr
+  int B, N, Cout, Ht, d;
+  int kslices;       // ceil(Ht * d / 64)
+  int tiles_per_image, num_tiles;  // tiles of 256 tokens
+  float eps;
+};
+
+// ---- cluster helpers
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {  // shared::cta address -> shared::cluster address in CTA `rank`
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred P1;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P1, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, P1;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait on a barrier that other CTAs of the cluster (or tcgen05.commit) arrive on.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait_cluster(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait_cluster(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void umma2_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives (once the MMAs issued so far have completed) on the barrier at this shared-memory offset in both CTAs of the pair.
+__device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+
+// ---------------------------------------------------------------------------
+// Second level of the state reduction (Eq. 3) and the fold of the state into the projection weights.
+// Grid (B * Ht, ceil(Cout / 64)).  partial: [B*Ht][S][d*(d+1)] fp32, entry [a][c], column d = key sum.
+//   ks[bh][a]            = sum_s partial[bh][s][a][d]
+//   M[b][m][hh*d + a]    = sum_c w[m][hh*d + c] * (sum_s partial[bh][s][a][c])        (bf16, row stride Kp)
+// ---------------------------------------------------------------------------
+constexpr int FOLD_ROWS = 64;
+__global__ void __launch_bounds__(256)
+state_fold_kernel(const float* __restrict__ partial, int S, const bf16* __restrict__ w, bf16* __restrict__ M, float* __restrict__ ks,
+                  int Ht, int d, int Cout, int K) {
+  __shared__ float st[32 * 33];
+  pdl_launch_dependents();
+  pdl_wait();  // the partial states come from the previous kernel
+  const int bh = blockIdx.x, b = bh / Ht, hh = bh % Ht;
+  const int d1 = d + 1, ne = d * d1;
+  const float* sp = partial + (long long)bh * S * ne;
+  for (int e = threadIdx.x; e < ne; e += 256) {
+    float v = 0.f;
+    for (int s = 0; s < S; ++s) v += sp[(long long)s * ne + e];
+    st[e] = v;
+  }
+  __syncthreads();
+  if (blockIdx.y == 0)
+    for (int a = threadIdx.x; a < d; a += 256) ks[(long long)bh * d + a] = st[a * d1 + d];
+  const int m0 = blockIdx.y * FOLD_ROWS;
+  for (int idx = threadIdx.x; idx < FOLD_ROWS * d; idx += 256) {
+    const int m = m0 + idx / d, a = idx % d;
+    if (m >= Cout) break;
+    const bf16* wr = w + (long long)m * K + hh * d;
+    float acc = 0.f;
+    for (int c = 0; c < d; ++c) acc = fmaf(__bfloat162float(wr[c]), st[a * d1 + c], acc);
+    M[((long long)b * Cout + m) * K + hh * d + a] = __float2bfloat16_rn(acc);
+  }
+}
+
+__global__ void __launch_bounds__(O_THREADS, 1)
+fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmQ,
+                 const __grid_constant__ CUtensorMap tmO, OutParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
+  const uint32_t a_base = smem_base;                                  // resident rows of M: kslices x 16 KB
+  const uint32_t ring = a_base + (uint32_t)p.kslices * O_A_SLICE;
+  const uint32_t staging = ring + O_STAGES * O_SLICE;
+  const uint32_t bars = staging + O_STAGING;
+  const uint32_t full_bar = bars;                        // [stage] TMA landed (own CTA)
+  const uint32_t empty_bar = bars + 8 * O_STAGES;        // [stage] MMAs have read the slice (commit, both CTAs)
+  const uint32_t ready_bar = bars + 16 * O_STAGES;       // [stage] both CTAs' slices transformed (leader only)
+  const uint32_t tfull_bar = bars + 24 * O_STAGES;       // [acc] accumulator complete (commit, both CTAs)
+  const uint32_t tempty_bar = tfull_bar + 16;            // [acc] both CTAs' epilogues have drained it (leader only)
+  const uint32_t res_bar = tempty_bar + 16;              // rows of M landed (own CTA)
+  const uint32_t peer_res_bar = res_bar + 8;             // the peer's rows of M landed (leader only)
+  const uint32_t tmem_slot = peer_res_bar + 8;
+  __shared__ int abort_flag;
+  __shared__ uint32_t tmem_base_sh;
+
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();               // 0 = leader of the pair
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < O_STAGES; ++s) {
+      mbar_init(full_bar + 8 * s, 1);
+      mbar_init(empty_bar + 8 * s, 1);
+      mbar_init(ready_bar + 8 * s, 2 * (O_XWARPS / 2));
+    }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar + 8 * a, 1); mbar_init(tempty_bar + 8 * a, 2 * 4); }
+    mbar_init(res_bar, 1);
+    mbar_init(peer_res_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // one warp of each CTA of the pair: all 512 tensor-memory columns in both
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (threadIdx.x == 0) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(tmem_slot));
+    tmem_base_sh = v;
+  }
+  cluster_sync_all();  // both CTAs' barriers exist before anything arrives on them from the other CTA
+  const uint32_t tmem_base = tmem_base_sh;
+  pdl_wait();  // queries, states and M come from earlier kernels
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (each CTA for itself)
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmM) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmQ) : "memory");
+      uint32_t it = 0, local = 0;
+      int cur_b = -1;
+      bool ok = true;
+      const int heads_per_slice = OKS / p.d;
+      for (int tile = pair; ok && tile < p.num_tiles; tile += npairs, ++local) {
+        const int b = tile / p.tiles_per_image, nt = tile % p.tiles_per_image;
+        if (b != cur_b) {
+          if (cur_b >= 0) {  // every MMA that reads the previous image's rows of M must be complete
+            const uint32_t last = local - 1;
+            ok = mbar_wait_cluster(tfull_bar + 8 * (last & 1), (last >> 1) & 1, &abort_flag);
+            if (!ok) break;
+          }
+          cur_b = b;
+          mbar_expect_tx(res_bar, (uint32_t)(p.kslices * O_A_SLICE));
+          for (int ks = 0; ks < p.kslices; ++ks)
+            tma_load_3d(a_base + ks * O_A_SLICE, &tmM, res_bar, ks * OKS, (int)rank * OM, b);
+        }
+        const int n0 = nt * (2 * OT) + (int)rank * OT;
+        for (int ks = 0; ok && ks < p.kslices; ++ks, ++it) {
+          const uint32_t s = it % O_STAGES, ph = (it / O_STAGES) & 1;
+          ok = mbar_wait_cluster(empty_bar + 8 * s, ph ^ 1, &abort_flag);
+          if (!ok) break;
+          const uint32_t dst = ring + s * O_SLICE;
+          mbar_expect_tx(full_bar + 8 * s, O_SLICE);
+          tma_load_4d(dst, &tmQ, full_bar + 8 * s, n0, 0, ks * heads_per_slice, b);
+          tma_load_4d(dst + O_BOX, &tmQ, full_bar + 8 * s, n0 + 64, 0, ks * heads_per_slice, b);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (leader) / M hand-shake (peer)
+    if (lane == 0) {
+      // instruction descriptor: D = f32, A = B = bf16, A K-major, B MN-major, N = 256, M = 256 (pair)
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+      const uint32_t peer_res_remote = map_to_cta(peer_res_bar, 0);
+      uint32_t it = 0, local = 0, res_ph = 0;
+      int cur_b = -1;
+      bool ok = true;
+      for (int tile = pair; ok && tile < p.num_tiles; tile += npairs, ++local) {
+        const int b = tile / p.tiles_per_image;
+        if (b != cur_b) {
+          cur_b = b;
+          ok = mbar_wait(res_bar, res_ph, &abort_flag);  // own rows of M
+          if (!ok) break;
+          if (rank == 0) {
+            ok = mbar_wait_cluster(peer_res_bar, res_ph, &abort_flag);  // the peer's rows of M
+            if (!ok) break;
+          } else {
+            mbar_arrive_cluster(peer_res_remote);
+          }
+          res_ph ^= 1;
+        }
+        if (rank != 0) continue;
+        const uint32_t acc = local & 1, acc_ph = (local >> 1) & 1;
+        ok = mbar_wait_cluster(tempty_bar + 8 * acc, acc_ph ^ 1, &abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * 256;
+        for (int ks = 0; ok && ks < p.kslices; ++ks, ++it) {
+          const uint32_t s = it % O_STAGES, ph = (it / O_STAGES) & 1;
+          ok = mbar_wait_cluster(ready_bar + 8 * s, ph, &abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sa = a_base + ks * O_A_SLICE, sb = ring + s * O_SLICE;
+#pragma unroll
+          for (int kk = 0; kk < OKS / 16; ++kk)
+            umma2_bf16(d_tmem, make_desc(sa + kk * 32, 1, 1024 >> 4), make_desc(sb + kk * 2048, O_BOX >> 4, 1024 >> 4), idesc,
+                       (ks > 0 || kk > 0) ? 1u : 0u);
+          umma2_commit_both(empty_bar + 8 * s);  // both CTAs may refill the slice once these MMAs have read it
+        }
+        if (ok) umma2_commit_both(tfull_bar + 8 * acc);
+      }
+    }
+  } else if (warp < 2 + O_XWARPS) {
+    // ------------------------------------------------------------ transform warps: q -> relu(q) / den, in place
+    // Group xg of four warps takes the slices with (slice counter & 1) == xg.  A lane owns one pair of
+    // neighbouring tokens of one head: word `lane` of every 128-byte channel row of its 64-token box
+    // (16-byte pieces XOR-swizzled with the row, as the TMA unit's 128B mode wrote them), so a warp
+    // reads and writes whole rows without bank conflicts.
+    const int xw = warp - 2, xg = xw >> 2, wig = xw & 3;
+    const int d = p.d;
+    const int heads_per_slice = OKS / d;
+    const uint32_t ready_remote = map_to_cta(ready_bar, 0);
+    const uint32_t box_off = (uint32_t)(wig & 1) * O_BOX;   // warps 0, 2: tokens 0-63; warps 1, 3: tokens 64-127
+    const uint32_t piece = (uint32_t)(lane >> 2), word = (uint32_t)(lane & 3);
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = pair; ok && tile < p.num_tiles; tile += npairs) {
+      const int b = tile / p.tiles_per_image;
+      for (int ks = 0; ok && ks < p.kslices; ++ks, ++it) {
+        if ((int)(it & 1) != xg) continue;
+        const uint32_t s = it % O_STAGES, ph = (it / O_STAGES) & 1;
+        ok = mbar_wait(full_bar + 8 * s, ph, &abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const uint32_t base = ring + s * O_SLICE + box_off + word * 4;
+        // d = 32: warps 0, 1 take the first head of the slice, warps 2, 3 the second;
+        // d = 16: warps 0, 1 take heads 0 and 2, warps 2, 3 heads 1 and 3
+        for (int hs = wig >> 1; hs < heads_per_slice; hs += 2) {
+          const int h = ks * heads_per_slice + hs;
+          if (h >= p.Ht) break;  // rows past the last head were filled with zeros and multiply zero columns of M
+          const float4* ksp = reinterpret_cast<const float4*>(p.ks + ((long long)b * p.Ht + h) * d);
+          const uint32_t row0 = (uint32_t)(hs * d);
+          uint32_t q[32];
+          float den0 = 0.f, den1 = 0.f;
+#pragma unroll
+          for (int a4 = 0; a4 < 8; ++a4) {
+            if (a4 * 4 >= d) break;
+            const float4 kv = __ldg(ksp + a4);
+            const float kk[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const uint32_t r = row0 + (uint32_t)(a4 * 4 + e);
+              uint32_t v;
+              asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(base + r * 128 + ((piece ^ (r & 7)) << 4)));
+              asm("max.bf16x2 %0, %1, %2;" : "=r"(v) : "r"(v), "r"(0u));
+              q[a4 * 4 + e] = v;
+              den0 = fmaf(__uint_as_float(v << 16), kk[e], den0);
+              den1 = fmaf(__uint_as_float(v & 0xffff0000u), kk[e], den1);
+            }
+          }
+          const float inv0 = 1.f / (den0 + p.eps), inv1 = 1.f / (den1 + p.eps);
+#pragma unroll
+          for (int a = 0; a < 32; ++a) {
+            if (a >= d) break;
+            const uint32_t r = row0 + (uint32_t)a;
+            const uint32_t o = pack2(__uint_as_float(q[a] << 16) * inv0, __uint_as_float(q[a] & 0xffff0000u) * inv1);
+            asm volatile("st.shared.u32 [%0], %1;" ::"r"(base + r * 128 + ((piece ^ (r & 7)) << 4)), "r"(o) : "memory");
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the tensor cores read what was just written
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(ready_remote + 8 * s);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue
+    // Four warps; warp % 4 selects the TMEM lane quarter (a hardware rule).  A lane owns one output
+    // channel of this CTA's 128; the accumulator's 256 columns are the pair's 256 tokens.
+    const int quarter = warp & 3;
+    const uint32_t stage = staging + (uint32_t)(warp - 2 - O_XWARPS) * O_STAGING_WARP;
+    const uint32_t my_row = stage + lane * 128, sw = (uint32_t)(lane & 7);
+    const int row0 = (int)rank * OM + quarter * 32;
+    const float bias = (p.bias && row0 + lane < p.Cout) ? __bfloat162float(p.bias[row0 + lane]) : 0.f;
+    const uint32_t tempty_remote = map_to_cta(tempty_bar, 0);
+    uint32_t local = 0;
+    bool ok = true;
+    for (int tile = pair; ok && tile < p.num_tiles; tile += npairs, ++local) {
+      const int b = tile / p.tiles_per_image, nt = tile % p.tiles_per_image;
+      const uint32_t acc = local & 1, acc_ph = (local >> 1) & 1;
+      ok = mbar_wait_cluster(tfull_bar + 8 * acc, acc_ph, &abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + acc * 256 + ((uint32_t)(quarter * 32) << 16);
+      uint32_t r[2][32];
+      tmem_ld32(taddr, r[0]);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        tmem_ld_wait();
+        if (c + 1 < 8) tmem_ld32(taddr + (c + 1) * 32, r[(c + 1) & 1]);  // next chunk streams in meanwhile
+        const uint32_t(&rc)[32] = r[c & 1];
+        const int n0 = nt * (2 * OT) + (c >> 1) * 64;  // first token of the 64-token block
+        if (n0 >= p.N || row0 >= p.Cout) continue;    // warp-uniform
+        if ((c & 1) == 0) {  // the previous block must have been read out of the staging buffer
+          if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          __syncwarp();
+        }
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          uint32_t w[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            w[e] = pack2(__uint_as_float(rc[v * 8 + 2 * e]) + bias, __uint_as_float(rc[v * 8 + 2 * e + 1]) + bias);
+          const uint32_t pc = (uint32_t)((c & 1) * 4 + v);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(my_row + ((pc ^ sw) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                       "r"(w[3]) : "memory");
+        }
+        if (c & 1) {
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_3d(&tmO, stage, n0, row0, b);
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(tempty_remote + 8 * acc);  // this warp's quarter of the accumulator is drained
+    }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // stores done before the CTA retires
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
+    // give copies and MMAs still in flight time to land before memory is released
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    if (threadIdx.x == 0) atomicExch(&g_fused_timeout_flag, 1);
+    __syncthreads();
+  }
+  cluster_sync_all();  // neither CTA leaves (or frees tensor memory) while the other may still touch its barriers or shared memory
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
+}  // namespace
+
+bool fused_out_bf16_supported(int Ht, int d, int Cout, int N) {
+  return (d == 16 || d == 32) && Ht >= 1 && Ht * d <= O_MAX_KS * OKS && Cout >= 1 && Cout <= 2 * OM && Cout % 8 == 0 && N >= 8 && N % 8 == 0;
+}
+
+// Scratch: M [B][Cout][Ht*d] bf16, then ks [B][Ht][d] fp32 (256-byte aligned).
+static size_t fused_out_m_bytes(int B, int Ht, int d, int Cout) { return ((size_t)B * Cout * Ht * d * 2 + 255) / 256 * 256; }
+size_t fused_out_scratch_bytes(int B, int Ht, int d, int Cout) { return fused_out_m_bytes(B, Ht, d, Cout) + (size_t)B * Ht * d * sizeof(float); }
+
+// y[b][m][n] = sum_h sum_c w[m][h*d + c] * att[b][h][n][c] + bias[m], att = Eq. 3 applied to query head h with the
+// state of (b, h) = sum over s < S of partial[(b * Ht + h) * S + s] ([d][d+1] fp32 each: KV, then the key sum in
+// column d).  q: channel-major, head h of image b at q + b*q_sb + h*q_sh, channel stride N (elements); y: NCHW
+// [B, Cout, N].
+msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, const float* partial, int S, void* scratch,
+                                 const void* w, const void* bias, void* y, int B, int Ht, int d, int N, int Cout, float eps,
+                                 cudaStream_t st) {
+  if (!fused_out_bf16_supported(Ht, d, Cout, N) || q_sb % 8 != 0 || q_sh % 8 != 0)
+    return fail(MSLA_ERR_UNSUPPORTED, "fused apply + projection: %d heads of %d channels, %d output channels, %d tokens", Ht, d, Cout, N);
+  const int K = Ht * d;
+  bf16* M = (bf16*)scratch;
+  float* ks = (float*)((char*)scratch + fused_out_m_bytes(B, Ht, d, Cout));
+  CUtensorMap tmM, tmQ, tmO;
+  {
+    const cuuint64_t dM[3] = {(cuuint64_t)K, (cuuint64_t)Cout, (cuuint64_t)B};
+    const cuuint64_t sM[2] = {(cuuint64_t)K * 2, (cuuint64_t)K * Cout * 2};
+    const cuuint32_t bM[3] = {OKS, OM, 1};
+    const cuuint64_t dQ[4] = {(cuuint64_t)N, (cuuint64_t)d, (cuuint64_t)Ht, (cuuint64_t)B};
+    const cuuint64_t sQ[3] = {(cuuint64_t)N * 2, (cuuint64_t)q_sh * 2, (cuuint64_t)q_sb * 2};
+    const cuuint32_t bQ[4] = {64, (cuuint32_t)d, (cuuint32_t)(OKS / d), 1};
+    const cuuint64_t dO[3] = {(cuuint64_t)N, (cuuint64_t)Cout, (cuuint64_t)B};
+    const cuuint64_t sO[2] = {(cuuint64_t)N * 2, (cuuint64_t)Cout * N * 2};
+    const cuuint32_t bO[3] = {64, 32, 1};
+    if (!tma_make_map_bf16(&tmM, M, 3, dM, sM, bM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !tma_make_map_bf16(&tmQ, q, 4, dQ, sQ, bQ, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !tma_make_map_bf16(&tmO, y, 3, dO, sO, bO, CU_TENSOR_MAP_SWIZZLE_128B))
+      return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the fused apply + output projection");
+  }
+  OutParams p{};
+  p.ks = ks; p.bias = (const bf16*)bias;
+  p.B = B; p.N = N; p.Cout = Cout; p.Ht = Ht; p.d = d; p.eps = eps;
+  p.kslices = (K + OKS - 1) / OKS;
+  p.tiles_per_image = (N + 2 * OT - 1) / (2 * OT);
+  const long long tiles = (long long)B * p.tiles_per_image;
+  if (tiles > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many token tiles");
+  p.num_tiles = (int)tiles;
+  const int smem = p.kslices * O_A_SLICE + O_STAGES * O_SLICE + O_STAGING + O_BAR_BYTES + 1024;
+  static std::atomic<unsigned long long> attr_done{0};
+  msla_status_t s = ensure_smem_attr(attr_done, fused_out_kernel, O_MAX_KS * O_A_SLICE + O_STAGES * O_SLICE + O_STAGING + O_BAR_BYTES + 1024);
+  if (s != MSLA_OK) return s;
+  const int sms = device_sm_count();
+  long long pairs = sms / 2;
+  if (pairs > tiles) pairs = tiles;
+  if (pairs < 1) pairs = 1;
+  launch_pdl(state_fold_kernel, dim3((unsigned)(B * Ht), (unsigned)((Cout + FOLD_ROWS - 1) / FOLD_ROWS)), dim3(256), 0, st, partial, S,
+             (const bf16*)w, M, ks, Ht, d, Cout, K);
+  launch_pdl_cluster2(fused_out_kernel, dim3((unsigned)(2 * pairs)), dim3(O_THREADS), (size_t)smem, st, tmM, tmQ, tmO, p);
+  count_launches(2);
+  return check_launch("fused apply + output projection (tcgen05, paired CTAs)");
+}
+
+int fused_timeout_flag() {
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, g_fused_timeout_flag, sizeof(int)) != cudaSuccess) {
+    cudaGetLastError();
+    return -1;
+  }
+  return v;
+}
+
+}  // namespace msla

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stddef.h>
 
+#include <atomic>
+
 #include "../../include/msla.h"
 
 namespace msla {
@@ -27,14 +29,31 @@ msla_status_t check_launch(const char* what);
 
 void count_launches(int n);
 
-// Function attributes (the dynamic shared-memory limit) belong to one device: a launch site keeps a
-// mask of the devices on which it has set them.  Bit of the current device; 0 for device numbers past
-// 63, which makes the site set the attribute on every call there.
+// Function attributes (the dynamic shared-memory limit) belong to one device: a launch site keeps an
+// atomic mask of the devices on which it has set them.  Bit of the current device; 0 for device numbers
+// past 63, which makes the site set the attribute on every call there.
 inline unsigned long long current_device_bit() {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 0; }
   return (dev >= 0 && dev < 64) ? 1ull << dev : 0ull;
 }
+
+// Raises the dynamic shared-memory limit of `kernel` to `bytes` on the current device, once per device
+// (two threads racing on the first call both set it, which is harmless).
+template <typename Kernel>
+inline msla_status_t ensure_smem_attr(std::atomic<unsigned long long>& done, Kernel kernel, int bytes) {
+  const unsigned long long bit = current_device_bit();
+  if (bit && (done.load(std::memory_order_acquire) & bit)) return MSLA_OK;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) {
+    cudaGetLastError();
+    return fail(MSLA_ERR_CUDA, "cannot reserve %d bytes of shared memory for a kernel", bytes);
+  }
+  done.fetch_or(bit, std::memory_order_release);
+  return MSLA_OK;
+}
+
+// Number of SMs of the current device (looked up once per device).
+int device_sm_count();
 
 // Launches `kernel` with programmatic stream serialization allowed: it may become resident before the
 // previous kernel of the stream has finished, and orders itself with pdl_wait() (msla_common.cuh).
@@ -53,39 +72,54 @@ inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);  // errors surface in check_launch()
 }
 
+// The same for a kernel that runs as clusters of two CTAs (grid.x must be even).
+template <typename... KArgs, typename... Args>
+inline void launch_pdl_cluster2(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = 2;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);  // errors surface in check_launch()
+}
+
 struct HeadView;
-// Tuned bf16 attention core (d in {16, 32}); all view strides must be multiples of 8 elements.
-// with_apply = false stops after the partial states (at ws + p.partial_off, p.S per head); `out` and `ov` are then unused.
+// Tuned bf16 attention core on dense [B, heads, N, d] tensors (d in {16, 32}, channel stride 1); all view strides
+// must be multiples of 8 elements.
 msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* out, HeadView in, HeadView ov, int B,
-                            int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st,
-                            cudaEvent_t mid, bool with_apply);
+                            int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st);
 
-// Apply step and output projection in one kernel (fused_apply_project.cu): bf16, d = 32, an even
-// number of heads, Cout <= 256, query strides multiples of 8 elements.
-bool apply_project_bf16_supported(int heads, int d, int Cout, int N, HeadView qv);
-size_t apply_project_scratch_bytes(int B, int heads);
-msla_status_t run_apply_project_bf16(const void* q, const float* partial, int S, void* scratch, const void* w, const void* bias, void* y,
-                                     HeadView qv, int B, int heads, int N, int Cout, float eps, cudaStream_t st);
-int fused_timeout_flag();
-
-// bf16 projections on tcgen05 tensor cores (gemm_tcgen05.cu).
-bool project_in_bf16_supported(int C, int Cout, int N, int d);
-msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d,
-                                  long long y_batch_stride, cudaStream_t st);
-bool project_out_bf16_supported(int Cin, int Cout, int N);
-msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin, int Cout,
-                                   int N, cudaStream_t st);
-bool project_out_planar_bf16_supported(int Cin, int Cout, int N);
-msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin,
-                                          int Cout, int N, cudaStream_t st);
+// bf16 1x1 projection on channel-major activations, tcgen05 tensor cores (gemm_tcgen05.cu):
+// y[b][m][n] = sum_k w[m][k] x[b][k][n] + bias[m]; batch strides in elements.
+bool gemm_bf16_supported(int M, int N, int K);
+msla_status_t run_gemm_bf16(const void* x, const void* w, const void* bias, void* y, int B, int K, int M, int N,
+                            long long x_sb, long long y_sb, cudaStream_t st);
 int gemm_timeout_flag();
 
-// bf16 aggregation (d = 16 or 32, Ch a multiple of 32): TMA halo tiles, depthwise filter as banded matrices on
-// tensor cores (agg_bf16.cu).  dst_sb must be a multiple of the plane size H*W*d.
+// bf16 aggregation on channel-major activations (agg_nchw.cu): TMA halo tiles, depthwise filter as banded matrices
+// on tensor cores, grouped 1x1 on tensor cores.  Batch strides in elements.
 bool aggregate_bf16_supported(int H, int W, int Ch, int d);
-msla_status_t run_aggregate_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
-                                 const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch, int d,
-                                 cudaStream_t st);
+msla_status_t run_aggregate_bf16(const void* src, long long src_sb, const void* w_dw, const void* w_pw, void* dst,
+                                 long long dst_sb, int B, int H, int W, int Ch, int d, cudaStream_t st);
 int agg_timeout_flag();
+
+// Apply step and output projection as one GEMM per image (fused_out.cu): bf16, d in {16, 32}, at most 512 attention
+// channels and 256 output channels.  q: channel-major query planes (channel stride N), head h of image b at
+// q + b*q_sb + h*q_sh.
+bool fused_out_bf16_supported(int Ht, int d, int Cout, int N);
+size_t fused_out_scratch_bytes(int B, int Ht, int d, int Cout);
+msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, const float* partial, int S, void* scratch,
+                                 const void* w, const void* bias, void* y, int B, int Ht, int d, int N, int Cout, float eps,
+                                 cudaStream_t st);
+int fused_timeout_flag();
 
 }  // namespace msla
