@@ -21,7 +21,7 @@
  *     floating-point atomics, and the split of the token reduction depends on
  *     the shape only.
  *   - There is no CPU fallback: on a device that is not compute capability
- *     10.0 (sm_100a) every compute call returns MSLA_ERR_ARCH.
+ *     10.x every compute call returns MSLA_ERR_ARCH.
  */
 #ifndef MSLA_H_
 #define MSLA_H_
@@ -39,7 +39,7 @@ typedef enum {
   MSLA_ERR_UNSUPPORTED = 2, /* a shape or option this build has no kernel for */
   MSLA_ERR_ALIGNMENT = 3,   /* a device pointer is not 16-byte aligned */
   MSLA_ERR_WORKSPACE = 4,   /* workspace missing or smaller than the *_workspace_bytes() answer */
-  MSLA_ERR_ARCH = 5,        /* current device is not compute capability 10.0 (sm_100a) */
+  MSLA_ERR_ARCH = 5,        /* current device is not sm_100 */
   MSLA_ERR_CUDA = 6         /* a CUDA runtime call or launch failed; see msla_last_error() */
 } msla_status_t;
 
@@ -198,17 +198,17 @@ int msla_debug_wait_timeouts(void);
 
 /* Stage entry points (the module's steps 1, 2 and 5 of Section 3.1 on their
  * own), exposed so that each kernel can be checked and timed in isolation.
- * Between the steps the library keeps activations channel-major, like x and
- * out themselves: [B, channels, H*W] with the token index contiguous.
- *   msla_project_in : x [B, C, N], w [Cout, C]                      -> y [B, Cout, N]    (Q = xW_Q, K = xW_K, V = xW_V)
- *   msla_aggregate  : t [B, Ch, H, W], w_dw [Ch,5,5], w_pw [Ch,d]   -> y [B, Ch, H, W]   (depthwise 5x5, then grouped 1x1
- *                                                                     with Ch/d groups of d channels)
- *   msla_project_out: a [B, Cin, N], w [Cout, Cin], bias [Cout]|NULL -> y [B, Cout, N]   (final linear projection)
- * Channel counts must be multiples of 8; d must be 16 or 32 and divide Ch.  The
- * output must not overlap the input (MSLA_ERR_INVALID_ARG).
+ * Between the steps the library keeps activations "planar": channels are cut
+ * into groups of d (one group = the q, k or v of one head, which is also one
+ * group of the aggregation's 1x1 group convolution), each group a dense
+ * [N][d] matrix: act[b][group][n][i], channel = group*d + i.
+ *   msla_project_in : x [B, C, N] (NCHW), w [Cout, C]              -> y [B, Cout/d, N, d]
+ *   msla_aggregate  : t [B, Ch/d, H*W, d], w_dw [Ch,5,5], w_pw [Ch,d] -> y [B, Ch/d, H*W, d]
+ *   msla_project_out: a [B, N, Cin] (token-major), w [Cout, Cin], bias [Cout]|NULL -> y [B, Cout, N] (NCHW)
+ * d must be 16 or 32 and divide Cout / Ch.
  */
 msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y,
-                              int B, int C, int Cout, int N, void* stream);
+                              int B, int C, int Cout, int N, int d, void* stream);
 msla_status_t msla_aggregate(msla_dtype_t dtype, const void* t, const void* w_dw, const void* w_pw,
                              void* y, int B, int H, int W, int Ch, int d, void* stream);
 msla_status_t msla_project_out(msla_dtype_t dtype, const void* a, const void* w, const void* bias,

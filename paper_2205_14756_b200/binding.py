@@ -55,7 +55,7 @@ EXPORTS = {
     "msla_forward_fuses_apply": (c_int, [ctypes.POINTER(msla_desc)]),
     "msla_kernel_launches": (ctypes.c_ulonglong, []),
     "msla_debug_wait_timeouts": (c_int, []),
-    "msla_project_in": (c_int, [c_int] + [c_void_p] * 3 + [c_int] * 4 + [c_void_p]),
+    "msla_project_in": (c_int, [c_int] + [c_void_p] * 3 + [c_int] * 5 + [c_void_p]),
     "msla_aggregate": (c_int, [c_int] + [c_void_p] * 4 + [c_int] * 5 + [c_void_p]),
     "msla_project_out": (c_int, [c_int] + [c_void_p] * 4 + [c_int] * 4 + [c_void_p]),
     "msla_status_string": (ctypes.c_char_p, [c_int]),
@@ -196,8 +196,8 @@ def make_weights(w_qkv, w_dw, w_pw, w_proj, b_proj=None) -> msla_weights:
     return w
 
 
-def msla_project_in(dtype, x, w, y, B, C, Cout, N, stream=None) -> None:
-    _check(lib().msla_project_in(dtype, _ptr(x), _ptr(w), _ptr(y), B, C, Cout, N, _stream(stream)))
+def msla_project_in(dtype, x, w, y, B, C, Cout, N, d, stream=None) -> None:
+    _check(lib().msla_project_in(dtype, _ptr(x), _ptr(w), _ptr(y), B, C, Cout, N, d, _stream(stream)))
 
 
 def msla_aggregate(dtype, t, w_dw, w_pw, y, B, H, W, Ch, d, stream=None) -> None:

@@ -234,7 +234,10 @@ kv_combine_bf16path_kernel(const float* __restrict__ partial, float* __restrict_
 // The fp32 state is fed as bf16 hi + bf16 lo (two MMAs) to keep ~16 mantissa
 // bits; one extra tile whose columns all hold ks gives the denominator.
 // ---------------------------------------------------------------------------
-template <int D, int NWARPS, int STAGES, int U>
+// PAIR: one CTA serves heads 2p (even warps) and 2p+1 (odd warps) of a paired
+// output view, so that the two 64-byte halves of each 128-byte output row are
+// written at nearly the same time.
+template <int D, int NWARPS, int STAGES, int U, bool PAIR>
 __global__ void __launch_bounds__(NWARPS * 32)
 apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf16* __restrict__ out,
                  HeadView qv, HeadView ov, int heads, int N, float eps, int tok_per_cta) {
@@ -252,12 +255,13 @@ apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf
   pdl_wait();  // the state comes from the previous kernel
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
-  constexpr int NW = NWARPS;  // warps sharing one head's tokens
-  const int wslot = warp;
-  const int bh = blockIdx.y;
+  constexpr int NW = PAIR ? NWARPS / 2 : NWARPS;  // warps sharing one head's tokens
+  const int wslot = PAIR ? warp >> 1 : warp;
+  const int bh = PAIR ? 2 * blockIdx.y + (warp & 1) : blockIdx.y;
   const int b = bh / heads, h = bh % heads;
   const long long qbase = (long long)b * qv.batch + (long long)h * qv.head + t * CPT;
-  const long long obase = (long long)b * ov.batch + (long long)h * ov.head + t * CPT;
+  const long long obase = PAIR ? (long long)b * ov.batch + (long long)(h >> 1) * ov.head + (h & 1) * D + t * CPT
+                               : (long long)b * ov.batch + (long long)h * ov.head + t * CPT;
   const int n_begin = blockIdx.x * tok_per_cta;
   const int n_end = min(N, n_begin + tok_per_cta);
   constexpr int TS = 16 * U;
@@ -362,39 +366,48 @@ apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf
   cp_async_wait<0>();
 }
 
-// Launch shapes: 4 warps per CTA and 4-deep rings in both kernels; two 16-token MMA tiles per FIFO stage of the apply step.
-constexpr int KV_WARPS = 4, KV_STAGES = 4, AP_WARPS = 4, AP_STAGES = 4, AP_U = 2;
-
 template <int D>
 msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out, HeadView in, HeadView ov, int B,
-                          int heads, int N, float eps, const CorePlan& p, char* ws, cudaStream_t st) {
+                          int heads, int N, float eps, const CorePlan& p, char* ws, cudaStream_t st, cudaEvent_t mid, bool with_apply) {
+  // 4 warps per CTA and 4-deep rings in both kernels; two 16-token MMA tiles per FIFO stage of the apply step
+  constexpr int KV_WARPS = 4, KV_STAGES = 4, AP_WARPS = 4, AP_STAGES = 4, AP_U = 2;
   const long long BH = (long long)B * heads;
   float* partial = reinterpret_cast<float*>(ws + p.partial_off);
   float* state = reinterpret_cast<float*>(ws + p.state_off);
   constexpr int kv_smem = KV_WARPS * KV_STAGES * 2 * 32 * D * 2;
   static std::atomic<unsigned long long> attr_done{0};
-  msla_status_t s = ensure_smem_attr(attr_done, kv_state_mma_kernel<D, KV_WARPS, KV_STAGES>, kv_smem);
-  if (s != MSLA_OK) return s;
+  const msla_status_t as = ensure_smem_attr(attr_done, kv_state_mma_kernel<D, KV_WARPS, KV_STAGES>, kv_smem);
+  if (as != MSLA_OK) return as;
   launch_pdl(kv_state_mma_kernel<D, KV_WARPS, KV_STAGES>, dim3((unsigned)BH, p.S), dim3(KV_WARPS * 32), kv_smem, st, k, v, partial, in, heads, N, p.S, p.chunk);
+  if (!with_apply) {  // the caller combines the partial states itself
+    if (mid) cudaEventRecord(mid, st);
+    count_launches(1);
+    return check_launch("attention state kernel (bf16)");
+  }
   const long long total = BH * p.ne;
   launch_pdl(kv_combine_bf16path_kernel, dim3((unsigned)ceil_div_ll(total, 256)), dim3(256), 0, st, partial, state, p.S, p.ne, total);
-  const int tok_per_cta = p.apply_tokens;
-  launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)BH),
-             dim3(AP_WARPS * 32), 0, st, q, state, out, in, ov, heads, N, eps, tok_per_cta);
+  if (mid) cudaEventRecord(mid, st);
+  if (ov.pair) {  // heads is even here, so a pair never straddles two images
+    const int tok_per_cta = p.apply_tokens / 2;
+    launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, true>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)(BH / 2)),
+               dim3(AP_WARPS * 32), 0, st, q, state, out, in, ov, heads, N, eps, tok_per_cta);
+  } else {
+    const int tok_per_cta = p.apply_tokens;
+    launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, false>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)BH),
+               dim3(AP_WARPS * 32), 0, st, q, state, out, in, ov, heads, N, eps, tok_per_cta);
+  }
   count_launches(3);
   return check_launch("attention core kernels (bf16)");
 }
 
 }  // namespace
 
-// Dense tensors only: channel stride 1, all other strides multiples of 8 elements.
 msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* out, HeadView in, HeadView ov, int B,
-                            int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st) {
-  if (in.cs != 1 || ov.cs != 1 || in.batch % 8 || in.head % 8 || in.ld % 8 || ov.batch % 8 || ov.head % 8 || ov.ld % 8)
-    return fail(MSLA_ERR_UNSUPPORTED, "the tensor-core attention core takes dense [B, heads, N, d] tensors");
+                            int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st,
+                            cudaEvent_t mid, bool with_apply) {
   if (d == 32)
-    return launch_core<32>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st);
-  return launch_core<16>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st);
+    return launch_core<32>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid, with_apply);
+  return launch_core<16>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid, with_apply);
 }
 
 }  // namespace msla

@@ -18,11 +18,12 @@
 //                     is reproducible bit for bit), writes ks and M (fp32 accumulate, bf16 out).
 // fused_out_kernel  : clusters of two CTAs, paired tensor-core MMAs (cta_group::2, M = 256).
 //   Each CTA keeps its 128 rows of M (<= 128 KB) in shared memory while the image lasts and
-//   owns 128 of the pair's 256 tokens per tile.  Per 64-channel slice of the queries:
-//     warp 0       TMA: two boxes of 64 channels x 64 tokens (token index contiguous, 128B swizzle)
-//     warps 2-9    turn q into qt in place (normaliser on the fp32 pipes, one token pair per lane)
-//     warp 1       (leader CTA only) issues tcgen05.mma 256 x 256 x 16: A = M (K-major), B = qt
-//                  (MN-major), fp32 accumulators in both CTAs' tensor memory
+//   owns 128 of the pair's 256 tokens per tile.  Per head (one slice of d query channels):
+//     warp 0       TMA: one box of 128 tokens x d channels of the head's planar [N][d] query
+//                  matrix (one contiguous 8 KB piece for d = 32; swizzle span = the row)
+//     warps 2-9    turn q into qt in place (normaliser on the fp32 pipes, one token per lane)
+//     warp 1       (leader CTA only) issues tcgen05.mma 256 x 256 x 16: A = M, B = qt, both
+//                  K-major, fp32 accumulators in both CTAs' tensor memory
 //     warps 10-13  drain the accumulators: TMEM -> bf16 (+ bias) -> swizzled staging -> TMA
 //                  stores of 32-channel x 64-token blocks into the NCHW output
 //   Two accumulator sets (2 x 256 TMEM columns) let the drain of a tile overlap the next.
@@ -42,17 +43,17 @@ using bf16 = __nv_bfloat16;
 
 constexpr int OT = 128;                  // tokens per CTA and tile (256 per pair)
 constexpr int OM = 128;                  // output channels per CTA (256 per pair)
-constexpr int OKS = 64;                  // channels per k-slice
-constexpr int O_BOX = 64 * OKS * 2;      // 8 KB: 64 channels x 64 tokens
-constexpr int O_SLICE = (OT / 64) * O_BOX;  // 16 KB
+constexpr int OKS = 64;                  // k-extent of one resident slice of M (one 128-byte swizzle span)
 constexpr int O_A_SLICE = OM * OKS * 2;  // 16 KB: 128 rows of M x 64 k
 constexpr int O_MAX_KS = 8;              // K = 2C' <= 512
-constexpr int O_STAGES = 4;
+constexpr int O_SLICE_MAX = OT * 32 * 2; // 8 KB: 128 tokens x 32 channels (d = 16: half of it is used)
+constexpr int O_STAGES = 8;
 constexpr int O_XWARPS = 8;              // transform warps: two groups of four, alternating slices
 constexpr int O_THREADS = 32 * (2 + O_XWARPS + 4);
 constexpr int O_STAGING_WARP = 32 * 128;
 constexpr int O_STAGING = 4 * O_STAGING_WARP;
-constexpr int O_BAR_BYTES = 256;
+constexpr int O_BAR_BYTES = 512;
+constexpr int O_SMEM_MAX = O_MAX_KS * O_A_SLICE + O_STAGES * O_SLICE_MAX + O_STAGING + O_BAR_BYTES + 1024;
 
 __device__ int g_fused_timeout_flag = 0;
 
@@ -60,7 +61,7 @@ struct OutParams {
   const float* ks;   // [B][Ht][d] key sums
   const bf16* bias;  // [Cout] or nullptr
   int B, N, Cout, Ht, d;
-  int kslices;       // ceil(Ht * d / 64)
+  int kslices;       // 64-wide k-slices of M: ceil(Ht * d / 64)
   int tiles_per_image, num_tiles;  // tiles of 256 tokens
   float eps;
 };
@@ -77,7 +78,7 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {  
   return r;
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -86,7 +87,7 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred P1;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P1, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\t"
       "selp.b32 %0, 1, 0, P1;\n\t}"
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
@@ -111,6 +112,11 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
+// K-major shared-memory matrix descriptor whose swizzle span is the row: rows of 64 bytes (mode 4) or 32 bytes (mode 6);
+// sbo16 = distance between groups of 8 rows in 16-byte units.
+__device__ __forceinline__ uint64_t make_desc_kmajor(uint32_t addr, uint32_t sbo16, uint64_t mode) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)sbo16 << 32) | (1ull << 46) | (mode << 61);
+}
 __device__ __forceinline__ void umma2_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
@@ -130,25 +136,41 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
 //   M[b][m][hh*d + a]    = sum_c w[m][hh*d + c] * (sum_s partial[bh][s][a][c])        (bf16, row stride Kp)
 // ---------------------------------------------------------------------------
 constexpr int FOLD_ROWS = 64;
-__global__ void __launch_bounds__(256)
+constexpr int FOLD_THREADS = 1024;
+__global__ void __launch_bounds__(FOLD_THREADS)
 state_fold_kernel(const float* __restrict__ partial, int S, const bf16* __restrict__ w, bf16* __restrict__ M, float* __restrict__ ks,
                   int Ht, int d, int Cout, int K) {
+  __shared__ float quarter[4][32 * 33];
   __shared__ float st[32 * 33];
   pdl_launch_dependents();
   pdl_wait();  // the partial states come from the previous kernel
   const int bh = blockIdx.x, b = bh / Ht, hh = bh % Ht;
   const int d1 = d + 1, ne = d * d1;
   const float* sp = partial + (long long)bh * S * ne;
-  for (int e = threadIdx.x; e < ne; e += 256) {
+  // Fixed summation order: the partial states are cut into four runs of consecutive indices, each run is summed in
+  // index order by its own thread (many loads in flight at once), and the four sums are added in run order.
+  for (int item = threadIdx.x; item < 4 * ne; item += FOLD_THREADS) {
+    const int j = item / ne, e = item - j * ne;
+    const int s0 = (int)((long long)S * j / 4), s1 = (int)((long long)S * (j + 1) / 4);
     float v = 0.f;
-    for (int s = 0; s < S; ++s) v += sp[(long long)s * ne + e];
-    st[e] = v;
+    int s = s0;
+    for (; s + 4 <= s1; s += 4) {
+      float t[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) t[u] = sp[(long long)(s + u) * ne + e];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) v += t[u];
+    }
+    for (; s < s1; ++s) v += sp[(long long)s * ne + e];
+    quarter[j][e] = v;
   }
   __syncthreads();
+  for (int e = threadIdx.x; e < ne; e += FOLD_THREADS) st[e] = ((quarter[0][e] + quarter[1][e]) + quarter[2][e]) + quarter[3][e];
+  __syncthreads();
   if (blockIdx.y == 0)
-    for (int a = threadIdx.x; a < d; a += 256) ks[(long long)bh * d + a] = st[a * d1 + d];
+    for (int a = threadIdx.x; a < d; a += FOLD_THREADS) ks[(long long)bh * d + a] = st[a * d1 + d];
   const int m0 = blockIdx.y * FOLD_ROWS;
-  for (int idx = threadIdx.x; idx < FOLD_ROWS * d; idx += 256) {
+  for (int idx = threadIdx.x; idx < FOLD_ROWS * d; idx += FOLD_THREADS) {
     const int m = m0 + idx / d, a = idx % d;
     if (m >= Cout) break;
     const bf16* wr = w + (long long)m * K + hh * d;
@@ -158,14 +180,17 @@ state_fold_kernel(const float* __restrict__ partial, int S, const bf16* __restri
   }
 }
 
+template <int D>
 __global__ void __launch_bounds__(O_THREADS, 1)
 fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmQ,
                  const __grid_constant__ CUtensorMap tmO, OutParams p) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
   const uint32_t a_base = smem_base;                                  // resident rows of M: kslices x 16 KB
+  constexpr int SLICE = OT * D * 2;                                    // one head's queries of this CTA's 128 tokens
+  constexpr int ROWB = D * 2;                                          // bytes per token row = the swizzle span
   const uint32_t ring = a_base + (uint32_t)p.kslices * O_A_SLICE;
-  const uint32_t staging = ring + O_STAGES * O_SLICE;
+  const uint32_t staging = ring + O_STAGES * SLICE;
   const uint32_t bars = staging + O_STAGING;
   const uint32_t full_bar = bars;                        // [stage] TMA landed (own CTA)
   const uint32_t empty_bar = bars + 8 * O_STAGES;        // [stage] MMAs have read the slice (commit, both CTAs)
@@ -181,7 +206,10 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();               // 0 = leader of the pair
+  // A pair works on a run of consecutive tiles, so that it changes image (and reloads its rows of M) as seldom as possible.
   const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+  const int tiles_per_pair = (p.num_tiles + npairs - 1) / npairs;
+  const int tile_first = min(pair * tiles_per_pair, p.num_tiles), tile_end = min(tile_first + tiles_per_pair, p.num_tiles);
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -219,8 +247,7 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
       uint32_t it = 0, local = 0;
       int cur_b = -1;
       bool ok = true;
-      const int heads_per_slice = OKS / p.d;
-      for (int tile = pair; ok && tile < p.num_tiles; tile += npairs, ++local) {
+      for (int tile = tile_first; ok && tile < tile_end; ++tile, ++local) {
         const int b = tile / p.tiles_per_image, nt = tile % p.tiles_per_image;
         if (b != cur_b) {
           if (cur_b >= 0) {  // every MMA that reads the previous image's rows of M must be complete
@@ -234,27 +261,25 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
             tma_load_3d(a_base + ks * O_A_SLICE, &tmM, res_bar, ks * OKS, (int)rank * OM, b);
         }
         const int n0 = nt * (2 * OT) + (int)rank * OT;
-        for (int ks = 0; ok && ks < p.kslices; ++ks, ++it) {
+        for (int h = 0; ok && h < p.Ht; ++h, ++it) {
           const uint32_t s = it % O_STAGES, ph = (it / O_STAGES) & 1;
           ok = mbar_wait_cluster(empty_bar + 8 * s, ph ^ 1, &abort_flag);
           if (!ok) break;
-          const uint32_t dst = ring + s * O_SLICE;
-          mbar_expect_tx(full_bar + 8 * s, O_SLICE);
-          tma_load_4d(dst, &tmQ, full_bar + 8 * s, n0, 0, ks * heads_per_slice, b);
-          tma_load_4d(dst + O_BOX, &tmQ, full_bar + 8 * s, n0 + 64, 0, ks * heads_per_slice, b);
+          mbar_expect_tx(full_bar + 8 * s, SLICE);
+          tma_load_4d(ring + s * SLICE, &tmQ, full_bar + 8 * s, 0, n0, h, b);  // rows past the last token are filled with zeros
         }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader) / M hand-shake (peer)
     if (lane == 0) {
-      // instruction descriptor: D = f32, A = B = bf16, A K-major, B MN-major, N = 256, M = 256 (pair)
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+      // instruction descriptor: D = f32, A = B = bf16, both K-major, N = 256, M = 256 (pair)
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
       const uint32_t peer_res_remote = map_to_cta(peer_res_bar, 0);
       uint32_t it = 0, local = 0, res_ph = 0;
       int cur_b = -1;
       bool ok = true;
-      for (int tile = pair; ok && tile < p.num_tiles; tile += npairs, ++local) {
+      for (int tile = tile_first; ok && tile < tile_end; ++tile, ++local) {
         const int b = tile / p.tiles_per_image;
         if (b != cur_b) {
           cur_b = b;
@@ -274,16 +299,18 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * 256;
-        for (int ks = 0; ok && ks < p.kslices; ++ks, ++it) {
+        for (int h = 0; ok && h < p.Ht; ++h, ++it) {
           const uint32_t s = it % O_STAGES, ph = (it / O_STAGES) & 1;
           ok = mbar_wait_cluster(ready_bar + 8 * s, ph, &abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t sa = a_base + ks * O_A_SLICE, sb = ring + s * O_SLICE;
+          const uint32_t sb = ring + s * SLICE;
 #pragma unroll
-          for (int kk = 0; kk < OKS / 16; ++kk)
-            umma2_bf16(d_tmem, make_desc(sa + kk * 32, 1, 1024 >> 4), make_desc(sb + kk * 2048, O_BOX >> 4, 1024 >> 4), idesc,
-                       (ks > 0 || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const int k0 = h * D + 16 * kk;  // column of M: 64-wide slices 16 KB apart, 32 bytes per 16 columns inside a slice
+            umma2_bf16(d_tmem, make_desc(a_base + (uint32_t)((k0 >> 6) * O_A_SLICE + (k0 & 63) * 2), 1, 1024 >> 4),
+                       make_desc_kmajor(sb + kk * 32, (8 * ROWB) >> 4, D == 32 ? 4ull : 6ull), idesc, (h > 0 || kk > 0) ? 1u : 0u);
+          }
           umma2_commit_both(empty_bar + 8 * s);  // both CTAs may refill the slice once these MMAs have read it
         }
         if (ok) umma2_commit_both(tfull_bar + 8 * acc);
@@ -291,61 +318,53 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     }
   } else if (warp < 2 + O_XWARPS) {
     // ------------------------------------------------------------ transform warps: q -> relu(q) / den, in place
-    // Group xg of four warps takes the slices with (slice counter & 1) == xg.  A lane owns one pair of
-    // neighbouring tokens of one head: word `lane` of every 128-byte channel row of its 64-token box
-    // (16-byte pieces XOR-swizzled with the row, as the TMA unit's 128B mode wrote them), so a warp
-    // reads and writes whole rows without bank conflicts.
+    // Group xg of four warps takes the slices with (slice counter & 1) == xg; its 128 lanes own one token
+    // row each (d channels: 64 or 32 bytes, 16-byte pieces XOR-swizzled with the row as the TMA unit
+    // wrote them and as the MMA reads them; eight consecutive rows cover all banks once).
+    constexpr int PCS = D / 8;     // 16-byte pieces per token row
     const int xw = warp - 2, xg = xw >> 2, wig = xw & 3;
-    const int d = p.d;
-    const int heads_per_slice = OKS / d;
     const uint32_t ready_remote = map_to_cta(ready_bar, 0);
-    const uint32_t box_off = (uint32_t)(wig & 1) * O_BOX;   // warps 0, 2: tokens 0-63; warps 1, 3: tokens 64-127
-    const uint32_t piece = (uint32_t)(lane >> 2), word = (uint32_t)(lane & 3);
+    const uint32_t row = (uint32_t)(wig * 32 + lane);
+    const uint32_t swz = D == 32 ? (row >> 1) & 3u : (row >> 2) & 1u;
+    const uint32_t row_off = row * ROWB;
     uint32_t it = 0;
     bool ok = true;
-    for (int tile = pair; ok && tile < p.num_tiles; tile += npairs) {
+    for (int tile = tile_first; ok && tile < tile_end; ++tile) {
       const int b = tile / p.tiles_per_image;
-      for (int ks = 0; ok && ks < p.kslices; ++ks, ++it) {
+      for (int h = 0; ok && h < p.Ht; ++h, ++it) {
         if ((int)(it & 1) != xg) continue;
+        // the head's key sums, fetched before the wait so that their latency hides behind it
+        float kk[D];
+        const float4* ksp = reinterpret_cast<const float4*>(p.ks + ((long long)b * p.Ht + h) * D);
+#pragma unroll
+        for (int a4 = 0; a4 < D / 4; ++a4) {
+          const float4 v = __ldg(ksp + a4);
+          kk[4 * a4] = v.x; kk[4 * a4 + 1] = v.y; kk[4 * a4 + 2] = v.z; kk[4 * a4 + 3] = v.w;
+        }
         const uint32_t s = it % O_STAGES, ph = (it / O_STAGES) & 1;
         ok = mbar_wait(full_bar + 8 * s, ph, &abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
-        const uint32_t base = ring + s * O_SLICE + box_off + word * 4;
-        // d = 32: warps 0, 1 take the first head of the slice, warps 2, 3 the second;
-        // d = 16: warps 0, 1 take heads 0 and 2, warps 2, 3 heads 1 and 3
-        for (int hs = wig >> 1; hs < heads_per_slice; hs += 2) {
-          const int h = ks * heads_per_slice + hs;
-          if (h >= p.Ht) break;  // rows past the last head were filled with zeros and multiply zero columns of M
-          const float4* ksp = reinterpret_cast<const float4*>(p.ks + ((long long)b * p.Ht + h) * d);
-          const uint32_t row0 = (uint32_t)(hs * d);
-          uint32_t q[32];
-          float den0 = 0.f, den1 = 0.f;
+        const uint32_t rbase = ring + s * SLICE + row_off;
+        uint32_t q[D / 2];  // word w = channels 2w (low half), 2w+1 (high half)
 #pragma unroll
-          for (int a4 = 0; a4 < 8; ++a4) {
-            if (a4 * 4 >= d) break;
-            const float4 kv = __ldg(ksp + a4);
-            const float kk[4] = {kv.x, kv.y, kv.z, kv.w};
+        for (int c = 0; c < PCS; ++c)
+          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(q[4 * c]), "=r"(q[4 * c + 1]), "=r"(q[4 * c + 2]), "=r"(q[4 * c + 3])
+                       : "r"(rbase + (((uint32_t)c ^ swz) << 4)));
+        float den[4] = {0.f, 0.f, 0.f, 0.f};  // four chains
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const uint32_t r = row0 + (uint32_t)(a4 * 4 + e);
-              uint32_t v;
-              asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(base + r * 128 + ((piece ^ (r & 7)) << 4)));
-              asm("max.bf16x2 %0, %1, %2;" : "=r"(v) : "r"(v), "r"(0u));
-              q[a4 * 4 + e] = v;
-              den0 = fmaf(__uint_as_float(v << 16), kk[e], den0);
-              den1 = fmaf(__uint_as_float(v & 0xffff0000u), kk[e], den1);
-            }
-          }
-          const float inv0 = 1.f / (den0 + p.eps), inv1 = 1.f / (den1 + p.eps);
-#pragma unroll
-          for (int a = 0; a < 32; ++a) {
-            if (a >= d) break;
-            const uint32_t r = row0 + (uint32_t)a;
-            const uint32_t o = pack2(__uint_as_float(q[a] << 16) * inv0, __uint_as_float(q[a] & 0xffff0000u) * inv1);
-            asm volatile("st.shared.u32 [%0], %1;" ::"r"(base + r * 128 + ((piece ^ (r & 7)) << 4)), "r"(o) : "memory");
-          }
+        for (int w = 0; w < D / 2; ++w) {
+          asm("max.bf16x2 %0, %1, %2;" : "=r"(q[w]) : "r"(q[w]), "r"(0u));
+          den[2 * (w & 1)] = fmaf(__uint_as_float(q[w] << 16), kk[2 * w], den[2 * (w & 1)]);
+          den[2 * (w & 1) + 1] = fmaf(__uint_as_float(q[w] & 0xffff0000u), kk[2 * w + 1], den[2 * (w & 1) + 1]);
         }
+        const float inv = __frcp_rn((den[0] + den[1]) + (den[2] + den[3]) + p.eps);
+#pragma unroll
+        for (int w = 0; w < D / 2; ++w) q[w] = pack2(__uint_as_float(q[w] << 16) * inv, __uint_as_float(q[w] & 0xffff0000u) * inv);
+#pragma unroll
+        for (int c = 0; c < PCS; ++c)
+          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(rbase + (((uint32_t)c ^ swz) << 4)), "r"(q[4 * c]), "r"(q[4 * c + 1]),
+                       "r"(q[4 * c + 2]), "r"(q[4 * c + 3]) : "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the tensor cores read what was just written
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(ready_remote + 8 * s);
@@ -363,7 +382,7 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     const uint32_t tempty_remote = map_to_cta(tempty_bar, 0);
     uint32_t local = 0;
     bool ok = true;
-    for (int tile = pair; ok && tile < p.num_tiles; tile += npairs, ++local) {
+    for (int tile = tile_first; ok && tile < tile_end; ++tile, ++local) {
       const int b = tile / p.tiles_per_image, nt = tile % p.tiles_per_image;
       const uint32_t acc = local & 1, acc_ph = (local >> 1) & 1;
       ok = mbar_wait_cluster(tfull_bar + 8 * acc, acc_ph, &abort_flag);
@@ -438,7 +457,7 @@ size_t fused_out_scratch_bytes(int B, int Ht, int d, int Cout) { return fused_ou
 
 // y[b][m][n] = sum_h sum_c w[m][h*d + c] * att[b][h][n][c] + bias[m], att = Eq. 3 applied to query head h with the
 // state of (b, h) = sum over s < S of partial[(b * Ht + h) * S + s] ([d][d+1] fp32 each: KV, then the key sum in
-// column d).  q: channel-major, head h of image b at q + b*q_sb + h*q_sh, channel stride N (elements); y: NCHW
+// column d).  q: planar bf16 query matrices [N][d], head h of image b at q + b*q_sb + h*q_sh (elements); y: NCHW
 // [B, Cout, N].
 msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, const float* partial, int S, void* scratch,
                                  const void* w, const void* bias, void* y, int B, int Ht, int d, int N, int Cout, float eps,
@@ -453,14 +472,14 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
     const cuuint64_t dM[3] = {(cuuint64_t)K, (cuuint64_t)Cout, (cuuint64_t)B};
     const cuuint64_t sM[2] = {(cuuint64_t)K * 2, (cuuint64_t)K * Cout * 2};
     const cuuint32_t bM[3] = {OKS, OM, 1};
-    const cuuint64_t dQ[4] = {(cuuint64_t)N, (cuuint64_t)d, (cuuint64_t)Ht, (cuuint64_t)B};
-    const cuuint64_t sQ[3] = {(cuuint64_t)N * 2, (cuuint64_t)q_sh * 2, (cuuint64_t)q_sb * 2};
-    const cuuint32_t bQ[4] = {64, (cuuint32_t)d, (cuuint32_t)(OKS / d), 1};
+    const cuuint64_t dQ[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)Ht, (cuuint64_t)B};
+    const cuuint64_t sQ[3] = {(cuuint64_t)d * 2, (cuuint64_t)q_sh * 2, (cuuint64_t)q_sb * 2};
+    const cuuint32_t bQ[4] = {(cuuint32_t)d, OT, 1, 1};
     const cuuint64_t dO[3] = {(cuuint64_t)N, (cuuint64_t)Cout, (cuuint64_t)B};
     const cuuint64_t sO[2] = {(cuuint64_t)N * 2, (cuuint64_t)Cout * N * 2};
     const cuuint32_t bO[3] = {64, 32, 1};
     if (!tma_make_map_bf16(&tmM, M, 3, dM, sM, bM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !tma_make_map_bf16(&tmQ, q, 4, dQ, sQ, bQ, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !tma_make_map_bf16(&tmQ, q, 4, dQ, sQ, bQ, d == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B) ||
         !tma_make_map_bf16(&tmO, y, 3, dO, sO, bO, CU_TENSOR_MAP_SWIZZLE_128B))
       return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the fused apply + output projection");
   }
@@ -472,17 +491,20 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   const long long tiles = (long long)B * p.tiles_per_image;
   if (tiles > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many token tiles");
   p.num_tiles = (int)tiles;
-  const int smem = p.kslices * O_A_SLICE + O_STAGES * O_SLICE + O_STAGING + O_BAR_BYTES + 1024;
-  static std::atomic<unsigned long long> attr_done{0};
-  msla_status_t s = ensure_smem_attr(attr_done, fused_out_kernel, O_MAX_KS * O_A_SLICE + O_STAGES * O_SLICE + O_STAGING + O_BAR_BYTES + 1024);
+  const int smem = p.kslices * O_A_SLICE + O_STAGES * (OT * d * 2) + O_STAGING + O_BAR_BYTES + 1024;
+  static std::atomic<unsigned long long> attr_done{0}, attr_done16{0};
+  constexpr int smem_max = O_SMEM_MAX;
+  msla_status_t s = ensure_smem_attr(attr_done, fused_out_kernel<32>, smem_max);
+  if (s == MSLA_OK) s = ensure_smem_attr(attr_done16, fused_out_kernel<16>, smem_max);
   if (s != MSLA_OK) return s;
   const int sms = device_sm_count();
   long long pairs = sms / 2;
   if (pairs > tiles) pairs = tiles;
   if (pairs < 1) pairs = 1;
-  launch_pdl(state_fold_kernel, dim3((unsigned)(B * Ht), (unsigned)((Cout + FOLD_ROWS - 1) / FOLD_ROWS)), dim3(256), 0, st, partial, S,
+  launch_pdl(state_fold_kernel, dim3((unsigned)(B * Ht), (unsigned)((Cout + FOLD_ROWS - 1) / FOLD_ROWS)), dim3(FOLD_THREADS), 0, st, partial, S,
              (const bf16*)w, M, ks, Ht, d, Cout, K);
-  launch_pdl_cluster2(fused_out_kernel, dim3((unsigned)(2 * pairs)), dim3(O_THREADS), (size_t)smem, st, tmM, tmQ, tmO, p);
+  if (d == 32) launch_pdl_cluster2(fused_out_kernel<32>, dim3((unsigned)(2 * pairs)), dim3(O_THREADS), (size_t)smem, st, tmM, tmQ, tmO, p);
+  else launch_pdl_cluster2(fused_out_kernel<16>, dim3((unsigned)(2 * pairs)), dim3(O_THREADS), (size_t)smem, st, tmM, tmQ, tmO, p);
   count_launches(2);
   return check_launch("fused apply + output projection (tcgen05, paired CTAs)");
 }

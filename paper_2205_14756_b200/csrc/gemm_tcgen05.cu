@@ -1,30 +1,31 @@
-// bf16 GEMM for the module's 1x1 projections (Section 3.1: Q = xW_Q, K = xW_K,
-// V = xW_V, and the final linear projection) on channel-major activations, on the
-// 5th-generation tensor cores: TMA loads into 128B-swizzled shared memory,
-// tcgen05.mma with fp32 accumulators in tensor memory, tcgen05.ld epilogue.
+// bf16 GEMM for the module's two 1x1 projections (Section 3.1: Q = xW_Q,
+// K = xW_K, V = xW_V, and the final linear projection) on the 5th-generation
+// tensor cores: TMA loads into 128B-swizzled shared memory, tcgen05.mma with
+// fp32 accumulators in tensor memory, tcgen05.ld epilogue.
 //
-//   y[b][m][n] = sum_k w[m][k] * x[b][k][n] (+ bias[m]),   fp32 accumulate, bf16 out
+//   D[m][n] = sum_k A[m][k] * B[n][k] (+ bias),   fp32 accumulate, bf16 out,
+//   out[batch * out_batch_stride + m * ld_out + n]                     (group == 0), or
+//   out[batch * out_batch_stride + ((n / group) * M + m) * group + n % group]
+//   (columns split into planes of `group` channels, each plane [M][group])
 //
-// x is [B][K][N] and y is [B][M][N] (NCHW with N = H*W), so both the activation
-// operand and the result have the token index contiguous.  The MMA takes
-//   A = 128 rows of w (K-major: k contiguous),
-//   B = a 256-token tile of x as an MN-major operand (n contiguous), four TMA
-//       boxes of 64 k x 64 tokens per 64-wide k-slice,
-//   D = 128 output channels (tensor-memory lanes) x 256 tokens (columns).
-// The weight block of a CTA (<= 128 KB) stays in shared memory for the CTA's
-// whole life when it fits (K <= 512): every CTA of a streaming kernel would
-// otherwise re-read the same few weight lines from L2 at the same time.  CTA c
-// serves weight block c % blocks and the token tiles c / blocks, + workers, ...
+// Input projection : m = token, n = output channel; A = x taken straight from
+//                    NCHW (the token index is contiguous: an "MN-major" operand),
+//                    B = w_qkv (K-major).
+// Output projection: m = output channel, n = token; A = w_proj (K-major),
+//                    B = attention output (K-major): either token-major
+//                    [N][2C'] or one [N][64] plane per pair of heads; D rows are NCHW
+//                    planes, so a row of the tile is a run of tokens.
 //
-// One persistent CTA per SM, warp-specialised: warp 0 issues TMA, warp 1 issues
-// MMAs (and owns the tensor-memory allocation), warps 2-9 drain the
+// One persistent CTA per SM, warp-specialised: warp 0 issues TMA, warp 1
+// issues MMAs (and owns the tensor-memory allocation), warps 2-9 drain the
 // accumulators.  Two 128x256 fp32 accumulators (all 512 TMEM columns) let the
 // epilogue of one tile overlap the MMAs of the next.  The epilogue converts to
-// bf16, stages 32-channel x 64-token blocks in shared memory (128-byte rows,
-// 128B swizzle) and writes them with TMA stores, which emit whole lines and
-// clip at the tensor's edges.  Every mbarrier wait is bounded: on time-out the
-// CTA raises a flag, all roles leave their loops, the tensor memory is released
-// and the kernel returns.
+// bf16, stages 32x32 blocks in shared memory and writes them with TMA stores
+// (whole lines; a lane-per-row store of 16-byte pieces was twice as slow).
+// A second kernel keeps the CTA's weight block resident in shared memory and
+// streams only activations (used for the input projection).  Every mbarrier wait is
+// bounded: on time-out the CTA raises a flag, all roles leave their loops, the
+// tensor memory is released and the kernel returns.
 #include <cuda.h>
 
 #include "msla_common.cuh"
@@ -38,62 +39,140 @@ namespace {
 using bf16 = __nv_bfloat16;
 
 constexpr int BM = 128, BN = 256, BK = 64;  // CTA tile; BK = one 128-byte swizzle span of bf16
-constexpr int A_SLICE = BM * BK * 2;        // 16 KB: 128 weight rows x 64 k
-constexpr int B_BOX = 64 * BK * 2;          // 8 KB: 64 k x 64 tokens
-constexpr int B_SLICE = (BN / 64) * B_BOX;  // 32 KB
-constexpr int NUM_THREADS = 320;            // TMA warp, MMA warp, 8 epilogue warps
-constexpr int STAGING_WARP = 32 * 128;      // one 32-channel x 64-token block per epilogue warp
-constexpr int STAGING_BYTES = 8 * STAGING_WARP;
-constexpr int MAX_STAGES = 6;
-constexpr int BAR_BYTES = 256;
-constexpr int SMEM_BUDGET = 226 * 1024;  // 227 KB per CTA less the static shared memory and some slack
-constexpr int RES_MAX_BYTES = 128 * 1024;
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * BK * 2;  // 16 KB
+constexpr int B_STAGE_BYTES = BN * BK * 2;  // 32 KB
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int NUM_THREADS = 320;  // TMA warp, MMA warp, 8 epilogue warps
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 8 * 2048 + 256 + 1024;  // ring + epilogue staging + barriers + alignment slack
 
 // Sticky: set when any wait in any GEMM launch of this process timed out.
 __device__ int g_gemm_timeout_flag = 0;
 
 struct GemmParams {
-  int M, N, K;      // output channels, tokens per image, input channels
+  int M, N, K;            // per batch
   int batches;
-  int n_tiles;      // 256-token tiles per image
-  int blocks;       // 128-row blocks of w
-  int workers;      // CTAs per block
-  int a_resident;   // 1: the CTA's weight block stays in shared memory
-  int stages;       // ring depth
-  const bf16* bias; // [M] or nullptr
+  int m_tiles, n_tiles;   // per batch
+  long long out_batch_stride;  // elements between consecutive batches of the output
+  long long ld_out;       // output row stride (elements) when group == 0
+  int group;              // 0, or channels per output plane (16 or 32)
+  int bias_per_row;       // 1: bias[m], 0: bias[n] (ignored when bias == nullptr)
+  int n_fastest;          // tile order: 1 = consecutive tiles share the A tile, 0 = share the B tile
+  const bf16* bias;
+  bf16* out;
+  int tma_store;          // 1: epilogue stages 32x32 blocks in shared memory and writes them with TMA (tmO)
+  int planes_per_batch;   // planar output: plane coordinate of (batch, n) = batch*planes_per_batch + n/32
 };
 
+__device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& b, int& mt, int& nt) {
+  const int per_batch = p.m_tiles * p.n_tiles;
+  b = tile / per_batch;
+  const int r = tile % per_batch;
+  if (p.n_fastest) { mt = r / p.n_tiles; nt = r % p.n_tiles; }
+  else             { nt = r / p.m_tiles; mt = r % p.m_tiles; }
+}
+
+constexpr int STAGING_BYTES = 8 * 2048;  // one 32-row x 64-byte block per epilogue warp
+
+// One epilogue warp's share of a finished 128x256 accumulator: TMEM lanes
+// 32*quarter .. +31 (= tile rows), columns col_half*128 .. +127, converted to
+// bf16 (+ bias).  A lane owns one row, so storing straight from registers
+// scatters 16-byte pieces over 32 rows per instruction; instead each 32x32
+// block is laid out in shared memory (64-byte rows, 16-byte chunks XOR-swizzled
+// as the TMA unit's 64B mode expects) and written by one TMA store, which
+// emits whole lines and clips rows and columns outside the tensor.  Without a
+// store map (planes of 16 channels) the lane stores its vectors directly.
+__device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUtensorMap* tmO, uint32_t stage, int b,
+                                                  int mt, int nt, uint32_t tmem_acc, int quarter, int col_half, int lane) {
+  const int gs = p.group == 32 ? 5 : 4;  // log2(group) when the output is planar
+  const int row0 = mt * BM + quarter * 32;
+  const int m = row0 + lane;
+  const bool row_ok = m < p.M;
+  bf16* obase = p.out + (long long)b * p.out_batch_stride;
+  const float bias_row = (p.bias && p.bias_per_row && row_ok) ? __bfloat162float(p.bias[m]) : 0.f;
+  const bool bias_col = p.bias && !p.bias_per_row;
+  const int ncol0 = nt * BN + col_half * 128;
+  const uint32_t taddr = tmem_acc + col_half * 128 + ((uint32_t)(quarter * 32) << 16);
+  const uint32_t my_row = stage + lane * 64, sw = (uint32_t)((lane >> 1) & 3);
+  uint32_t r[2][32];
+  tmem_ld32(taddr, r[0]);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    tmem_ld_wait();
+    if (c + 1 < 4) tmem_ld32(taddr + (c + 1) * 32, r[(c + 1) & 1]);  // next chunk streams in while this one is stored
+    const uint32_t(&rc)[32] = r[c & 1];
+    const int n0 = ncol0 + c * 32;
+    if (n0 >= p.N) continue;  // warp-uniform
+    uint32_t w[4][4];
+#pragma unroll
+    for (int v = 0; v < 4; ++v)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float f0 = __uint_as_float(rc[v * 8 + 2 * e]) + bias_row;
+        float f1 = __uint_as_float(rc[v * 8 + 2 * e + 1]) + bias_row;
+        if (bias_col && n0 + v * 8 < p.N) {
+          f0 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e]);
+          f1 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e + 1]);
+        }
+        w[v][e] = pack2(f0, f1);
+      }
+    if (p.tma_store) {
+      // the previous block must have been read out of the staging buffer
+      if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      __syncwarp();
+#pragma unroll
+      for (int v = 0; v < 4; ++v)
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(my_row + (((uint32_t)v ^ sw) << 4)), "r"(w[v][0]),
+                     "r"(w[v][1]), "r"(w[v][2]), "r"(w[v][3]) : "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) {
+        if (p.group) tma_store_3d(tmO, stage, 0, row0, b * p.planes_per_batch + (n0 >> 5));
+        else         tma_store_3d(tmO, stage, n0, row0, b);
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      }
+    } else if (row_ok) {
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {  // 4 x (8 columns = 16 bytes); N is a multiple of 8
+        const int n = n0 + v * 8;
+        if (n < p.N) {
+          bf16* dst = p.group ? obase + (((long long)(n >> gs) * p.M + m) << gs) + (n & (p.group - 1))
+                              : obase + (long long)m * p.ld_out + n;
+          asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(dst), "r"(w[v][0]), "r"(w[v][1]), "r"(w[v][2]), "r"(w[v][3]) : "memory");
+        }
+      }
+    }
+  }
+}
+
+// B_PLANAR (output projection with the attention output kept as one [N][64]
+// plane per pair of heads): the 64-wide k-slice kb of B is plane kb of the image.
+template <bool A_MN_MAJOR, bool B_PLANAR>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_wx_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-               const __grid_constant__ CUtensorMap tmO, GemmParams p) {
+gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                         const __grid_constant__ CUtensorMap tmO, GemmParams p) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
-  const int k_iters = (p.K + BK - 1) / BK;
-  const uint32_t res_base = smem_base;
-  const uint32_t ring_base = res_base + (p.a_resident ? (uint32_t)(k_iters * A_SLICE) : 0u);
-  const uint32_t stage_bytes = (uint32_t)B_SLICE + (p.a_resident ? 0u : (uint32_t)A_SLICE);
-  const uint32_t staging = ring_base + (uint32_t)p.stages * stage_bytes;
+  const uint32_t staging = smem_base + STAGES * STAGE_BYTES;
   const uint32_t bars = staging + STAGING_BYTES;
-  const uint32_t full_bar = bars, empty_bar = bars + 8 * MAX_STAGES;
-  const uint32_t tfull_bar = bars + 16 * MAX_STAGES, tempty_bar = tfull_bar + 16;
-  const uint32_t res_bar = tempty_bar + 16, tmem_slot = res_bar + 8;
+  const uint32_t full_bar = bars, empty_bar = bars + 8 * STAGES;
+  const uint32_t tfull_bar = bars + 16 * STAGES, tempty_bar = tfull_bar + 16;
+  const uint32_t tmem_slot = tempty_bar + 16;
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_sh;
 
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int blk = blockIdx.x % p.blocks, worker = blockIdx.x / p.blocks;
-  const int stream_total = p.batches * p.n_tiles;
-  const uint32_t nstage = (uint32_t)p.stages;
+  const int num_tiles = p.batches * p.m_tiles * p.n_tiles;
+  const int k_iters = (p.K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
-    for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar + 8 * a, 1); mbar_init(tempty_bar + 8 * a, 8); }
-    mbar_init(res_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {  // whole warp: all 512 tensor-memory columns (one CTA per SM)
+  if (warp == 1) {  // whole warp: allocate all 512 tensor-memory columns (one CTA per SM)
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -107,60 +186,66 @@ gemm_wx_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   }
   __syncthreads();
   const uint32_t tmem_base = tmem_base_sh;
+  pdl_wait();  // barriers and tensor memory are set up; the activations come from the previous kernel
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmX) : "memory");
-      if (p.a_resident) {  // the weights are no earlier kernel's output: load them before the dependency wait
-        mbar_expect_tx(res_bar, (uint32_t)(k_iters * A_SLICE));
-        for (int kb = 0; kb < k_iters; ++kb) tma_load_3d(res_base + kb * A_SLICE, &tmW, res_bar, kb * BK, blk * BM, 0);
-      }
-      pdl_wait();  // the activations may come from the previous kernel
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
       uint32_t it = 0;
       bool ok = true;
-      for (int si = worker; ok && si < stream_total; si += p.workers) {
-        const int b = si / p.n_tiles, nt = si % p.n_tiles;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        int b, mt, nt;
+        tile_coords(p, tile, b, mt, nt);
         for (int kb = 0; ok && kb < k_iters; ++kb, ++it) {
-          const uint32_t s = it % nstage, ph = (it / nstage) & 1;
+          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
           ok = mbar_wait(empty_bar + 8 * s, ph ^ 1, &abort_flag);
           if (!ok) break;
-          const uint32_t dst = ring_base + s * stage_bytes;
-          mbar_expect_tx(full_bar + 8 * s, stage_bytes);
-#pragma unroll
-          for (int j = 0; j < BN / 64; ++j)  // boxes past the last token are filled with zeros
-            tma_load_3d(dst + j * B_BOX, &tmX, full_bar + 8 * s, nt * BN + 64 * j, kb * BK, b);
-          if (!p.a_resident) tma_load_3d(dst + B_SLICE, &tmW, full_bar + 8 * s, kb * BK, blk * BM, 0);
+          const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+          mbar_expect_tx(full_bar + 8 * s, STAGE_BYTES);
+          if (B_PLANAR) {    // 64 k x 128 weight rows, and one plane: 64 channels x 256 tokens
+            tma_load_3d(sa, &tmA, full_bar + 8 * s, kb * BK, mt * BM, 0);
+            tma_load_3d(sb, &tmB, full_bar + 8 * s, 0, nt * BN, b * p.planes_per_batch + kb);
+          } else {
+            if (A_MN_MAJOR) {  // two boxes of 64 tokens x 64 k
+              tma_load_3d(sa, &tmA, full_bar + 8 * s, mt * BM, kb * BK, b);
+              tma_load_3d(sa + A_STAGE_BYTES / 2, &tmA, full_bar + 8 * s, mt * BM + 64, kb * BK, b);
+            } else {           // one box of 64 k x 128 rows
+              tma_load_3d(sa, &tmA, full_bar + 8 * s, kb * BK, mt * BM, 0);
+            }
+            tma_load_3d(sb, &tmB, full_bar + 8 * s, kb * BK, nt * BN, A_MN_MAJOR ? 0 : b);
+          }
         }
       }
     }
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      // instruction descriptor: D = f32, A = B = bf16, A K-major, B MN-major, N = 256, M = 128
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      // instruction descriptor: D = f32, A = B = bf16, A major, B K-major, N = 256, M = 128
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN_MAJOR ? 1u : 0u) << 15) |
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
       uint32_t it = 0, local = 0;
-      bool ok = p.a_resident ? mbar_wait(res_bar, 0, &abort_flag) : true;
-      for (int si = worker; ok && si < stream_total; si += p.workers, ++local) {
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++local) {
         const uint32_t acc = local & 1, acc_ph = (local >> 1) & 1;
         ok = mbar_wait(tempty_bar + 8 * acc, acc_ph ^ 1, &abort_flag);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int kb = 0; ok && kb < k_iters; ++kb, ++it) {
-          const uint32_t s = it % nstage, ph = (it / nstage) & 1;
+          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
           ok = mbar_wait(full_bar + 8 * s, ph, &abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t sb = ring_base + s * stage_bytes;
-          const uint32_t sa = p.a_resident ? res_base + kb * A_SLICE : sb + B_SLICE;
+          const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
 #pragma unroll
           for (int kk = 0; kk < BK / 16; ++kk) {
-            // K-major w: 32 bytes further along the swizzled row; MN-major x: 16 k-rows of 128 bytes
-            // further, 64-token blocks 8 KB apart, groups of 8 k-rows 1 KB apart
-            const uint64_t ad = make_desc(sa + kk * 32, 1, 1024 >> 4);
-            const uint64_t bd = make_desc(sb + kk * 2048, B_BOX >> 4, 1024 >> 4);
+            // MN-major A: 16 k-slices of 128 B further on; K-major: 32 B along the swizzled row
+            uint64_t ad, bd;
+            ad = A_MN_MAJOR ? make_desc(sa + kk * 2048, (A_STAGE_BYTES / 2) >> 4, 1024 >> 4)
+                            : make_desc(sa + kk * 32, 1, 1024 >> 4);
+            bd = make_desc(sb + kk * 32, 1, 1024 >> 4);
             umma_bf16(d_tmem, ad, bd, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
           }
           umma_commit(empty_bar + 8 * s);  // stage reusable once these MMAs have read it
@@ -170,60 +255,21 @@ gemm_wx_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
   } else {
     // ---------------------------------------------------------------- epilogue
-    // Eight warps: warp % 4 selects the TMEM lane quarter (a hardware rule), the other bit which 128
-    // of the tile's 256 tokens the warp drains.  A lane owns one output channel; two 32-token chunks
-    // fill a 32-channel x 64-token block (128-byte rows, 16-byte pieces XOR-swizzled with the row as
-    // the TMA unit's 128B mode expects), written by one TMA store.
+    // Eight warps: warp%4 selects the TMEM lane quarter (a hardware rule), the
+    // other bit selects which 128 of the tile's 256 columns the warp drains.
     const int quarter = warp & 3;
     const int col_half = (warp - 2) >> 2;
-    const uint32_t stage = staging + (uint32_t)(warp - 2) * STAGING_WARP;
-    const uint32_t my_row = stage + lane * 128, sw = (uint32_t)(lane & 7);
-    const int row0 = blk * BM + quarter * 32;
-    const float bias = (p.bias && row0 + lane < p.M) ? __bfloat162float(p.bias[row0 + lane]) : 0.f;
     uint32_t local = 0;
     bool ok = true;
-    pdl_wait();  // no global write before the previous kernel is done with the output buffer
-    for (int si = worker; ok && si < stream_total; si += p.workers, ++local) {
-      const int b = si / p.n_tiles, nt = si % p.n_tiles;
+    for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++local) {
+      int b, mt, nt;
+      tile_coords(p, tile, b, mt, nt);
       const uint32_t acc = local & 1, acc_ph = (local >> 1) & 1;
       ok = mbar_wait(tfull_bar + 8 * acc, acc_ph, &abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t taddr = tmem_base + acc * BN + col_half * 128 + ((uint32_t)(quarter * 32) << 16);
-      const int ncol0 = nt * BN + col_half * 128;
-      uint32_t r[2][32];
-      tmem_ld32(taddr, r[0]);
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        tmem_ld_wait();
-        if (c + 1 < 4) tmem_ld32(taddr + (c + 1) * 32, r[(c + 1) & 1]);  // next chunk streams in meanwhile
-        const uint32_t(&rc)[32] = r[c & 1];
-        const int n0 = ncol0 + (c >> 1) * 64;   // first token of the 64-token block
-        if (n0 >= p.N || row0 >= p.M) continue;  // warp-uniform: nothing of this block lies inside the tensor
-        if ((c & 1) == 0) {  // the previous block must have been read out of the staging buffer
-          if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-          __syncwarp();
-        }
-#pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          uint32_t w[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e)
-            w[e] = pack2(__uint_as_float(rc[v * 8 + 2 * e]) + bias, __uint_as_float(rc[v * 8 + 2 * e + 1]) + bias);
-          const uint32_t piece = (uint32_t)((c & 1) * 4 + v);
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(my_row + ((piece ^ sw) << 4)), "r"(w[0]), "r"(w[1]),
-                       "r"(w[2]), "r"(w[3]) : "memory");
-        }
-        if (c & 1) {
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          __syncwarp();
-          if (lane == 0) {
-            tma_store_3d(&tmO, stage, n0, row0, b);
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-          }
-        }
-      }
+      drain_accumulator(p, &tmO, staging + (warp - 2) * 2048, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);  // this warp's share of the accumulator is drained
@@ -246,61 +292,299 @@ gemm_wx_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   }
 }
 
-}  // namespace
 
-bool gemm_bf16_supported(int M, int N, int K) { return M >= 1 && N >= 8 && N % 8 == 0 && K >= 8 && K % 8 == 0; }
+// ---------------------------------------------------------------------------
+// Weight-stationary variant.  Every CTA of the streaming kernel above re-reads
+// the same weight slices from L2 at the same time, and those few hot lines
+// serialise in their L2 slices.  Here a CTA owns one block of output channels
+// for its whole life: that block of the weight matrix (<= 128 KB) is loaded
+// into shared memory once, and only activation tiles stream through a ring.
+//   RES_IS_B = true  (input projection) : B = 256 weight rows resident (K <= 256),
+//                                         A = 128-token x tiles, MN-major, 16 KB stages (5 deep)
+//   RES_IS_B = false (output projection): A = 128 weight rows resident (K <= 512),
+//                                         B = 256-token attention tiles, 32 KB stages (2 deep)
+// CTA c serves weight block c % blocks and the activation tiles c / blocks,
+// c / blocks + workers, ...  Barriers, TMEM use and epilogue are as above.
+// ---------------------------------------------------------------------------
+constexpr int RES_BYTES = 128 * 1024;
+constexpr int WS_RING_BYTES = 80 * 1024;
+constexpr int WS_SMEM_BYTES = RES_BYTES + WS_RING_BYTES + STAGING_BYTES + 256 + 1024;
+constexpr int WS_MAX_STAGES = 6;
 
-// y[b][m][n] = sum_k w[m][k] * x[b][k][n] + bias[m];  x: [B][K][N] with batch stride x_sb, y: [B][M][N] with
-// batch stride y_sb (elements; multiples of 8), w: [M][K], bias: [M] or nullptr.
-msla_status_t run_gemm_bf16(const void* x, const void* w, const void* bias, void* y, int B, int K, int M, int N,
-                            long long x_sb, long long y_sb, cudaStream_t st) {
-  if (!gemm_bf16_supported(M, N, K) || x_sb % 8 != 0 || y_sb % 8 != 0)
-    return fail(MSLA_ERR_UNSUPPORTED, "projection GEMM: M = %d, N = %d, K = %d", M, N, K);
-  CUtensorMap tmW, tmX, tmO;
-  {
-    const cuuint64_t dW[3] = {(cuuint64_t)K, (cuuint64_t)M, 1};
-    const cuuint64_t sW[2] = {(cuuint64_t)K * 2, (cuuint64_t)K * M * 2};
-    const cuuint32_t bW[3] = {BK, BM, 1};
-    const cuuint64_t dX[3] = {(cuuint64_t)N, (cuuint64_t)K, (cuuint64_t)B};
-    const cuuint64_t sX[2] = {(cuuint64_t)N * 2, (cuuint64_t)x_sb * 2};
-    const cuuint32_t bX[3] = {64, BK, 1};
-    const cuuint64_t dO[3] = {(cuuint64_t)N, (cuuint64_t)M, (cuuint64_t)B};
-    const cuuint64_t sO[2] = {(cuuint64_t)N * 2, (cuuint64_t)y_sb * 2};
-    const cuuint32_t bO[3] = {64, 32, 1};
-    if (!tma_make_map_bf16(&tmW, w, 3, dW, sW, bW, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !tma_make_map_bf16(&tmX, x, 3, dX, sX, bX, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !tma_make_map_bf16(&tmO, y, 3, dO, sO, bO, CU_TENSOR_MAP_SWIZZLE_128B))
-      return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the projection GEMM");
+template <bool RES_IS_B>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                            const __grid_constant__ CUtensorMap tmO, GemmParams p, int blocks, int workers) {
+  constexpr int STREAM_BYTES = RES_IS_B ? A_STAGE_BYTES : B_STAGE_BYTES;  // one k-slice of the streamed operand
+  constexpr int NSTAGE = WS_RING_BYTES / STREAM_BYTES;                     // 5 or 2
+  constexpr int RES_SLICE = RES_IS_B ? B_STAGE_BYTES : A_STAGE_BYTES;      // one k-slice of the resident operand
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t res_base = smem_base, ring_base = smem_base + RES_BYTES;
+  const uint32_t staging = ring_base + WS_RING_BYTES;
+  const uint32_t bars = staging + STAGING_BYTES;
+  const uint32_t full_bar = bars, empty_bar = bars + 8 * WS_MAX_STAGES;
+  const uint32_t tfull_bar = bars + 16 * WS_MAX_STAGES, tempty_bar = tfull_bar + 16;
+  const uint32_t res_bar = tempty_bar + 16, tmem_slot = res_bar + 8;
+  __shared__ int abort_flag;
+  __shared__ uint32_t tmem_base_sh;
+
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int k_iters = (p.K + BK - 1) / BK;
+  const int blk = blockIdx.x % blocks, worker = blockIdx.x / blocks;
+  const int stream_per_batch = RES_IS_B ? p.m_tiles : p.n_tiles;
+  const int stream_total = p.batches * stream_per_batch;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < NSTAGE; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar + 8 * a, 1); mbar_init(tempty_bar + 8 * a, 8); }
+    mbar_init(res_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  GemmParams p{};
-  p.M = M; p.N = N; p.K = K; p.batches = B;
-  p.n_tiles = (N + BN - 1) / BN;
-  p.blocks = (M + BM - 1) / BM;
-  p.bias = (const bf16*)bias;
-  const int k_iters = (K + BK - 1) / BK;
-  const int sms = device_sm_count();
-  const long long stream_total = (long long)B * p.n_tiles;
-  if (stream_total > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many token tiles");
-  p.a_resident = (k_iters * A_SLICE <= RES_MAX_BYTES && p.blocks <= sms) ? 1 : 0;
-  const int fixed = STAGING_BYTES + BAR_BYTES + 1024 + (p.a_resident ? k_iters * A_SLICE : 0);
-  const int stage_bytes = B_SLICE + (p.a_resident ? 0 : A_SLICE);
-  int stages = (SMEM_BUDGET - fixed) / stage_bytes;
-  p.stages = stages > MAX_STAGES ? MAX_STAGES : stages;
-  const int smem = fixed + p.stages * stage_bytes;
-  long long workers = p.a_resident ? sms / p.blocks : 1;
-  if (!p.a_resident) {  // streaming: every CTA walks all (block, tile) pairs of its share; keep the block fixed per CTA all the same
-    workers = sms / p.blocks;
-    if (workers < 1) workers = 1;
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (workers > stream_total) workers = stream_total;
-  p.workers = (int)workers;
-  // with more blocks than SMs the grid is larger than one wave; CTAs do not depend on one another
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (threadIdx.x == 0) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(tmem_slot));
+    tmem_base_sh = v;
+  }
+  __syncthreads();
+  const uint32_t tmem_base = tmem_base_sh;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+      // the resident weight block: all k-slices on one barrier
+      mbar_expect_tx(res_bar, (uint32_t)(k_iters * RES_SLICE));
+      for (int kb = 0; kb < k_iters; ++kb) {
+        if (RES_IS_B) tma_load_3d(res_base + kb * RES_SLICE, &tmB, res_bar, kb * BK, blk * BN, 0);
+        else          tma_load_3d(res_base + kb * RES_SLICE, &tmA, res_bar, kb * BK, blk * BM, 0);
+      }
+      pdl_wait();  // the streamed operand may come from the previous kernel; the weights above do not
+      uint32_t it = 0;
+      bool ok = true;
+      for (int si = worker; ok && si < stream_total; si += workers) {
+        const int b = si / stream_per_batch, st = si % stream_per_batch;
+        for (int kb = 0; ok && kb < k_iters; ++kb, ++it) {
+          const uint32_t s = it % NSTAGE, ph = (it / NSTAGE) & 1;
+          ok = mbar_wait(empty_bar + 8 * s, ph ^ 1, &abort_flag);
+          if (!ok) break;
+          const uint32_t dst = ring_base + s * STREAM_BYTES;
+          mbar_expect_tx(full_bar + 8 * s, STREAM_BYTES);
+          if (RES_IS_B) {  // x tile: two boxes of 64 tokens x 64 k
+            tma_load_3d(dst, &tmA, full_bar + 8 * s, st * BM, kb * BK, b);
+            tma_load_3d(dst + STREAM_BYTES / 2, &tmA, full_bar + 8 * s, st * BM + 64, kb * BK, b);
+          } else {         // attention tile: one box of 64 k x 256 tokens
+            tma_load_3d(dst, &tmB, full_bar + 8 * s, kb * BK, st * BN, b);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // -------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((RES_IS_B ? 1u : 0u) << 15) |
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      uint32_t it = 0, local = 0;
+      bool ok = mbar_wait(res_bar, 0, &abort_flag);
+      for (int si = worker; ok && si < stream_total; si += workers, ++local) {
+        const uint32_t acc = local & 1, acc_ph = (local >> 1) & 1;
+        ok = mbar_wait(tempty_bar + 8 * acc, acc_ph ^ 1, &abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; ok && kb < k_iters; ++kb, ++it) {
+          const uint32_t s = it % NSTAGE, ph = (it / NSTAGE) & 1;
+          ok = mbar_wait(full_bar + 8 * s, ph, &abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t stream = ring_base + s * STREAM_BYTES, res = res_base + kb * RES_SLICE;
+#pragma unroll
+          for (int kk = 0; kk < BK / 16; ++kk) {
+            uint64_t ad, bd;
+            if (RES_IS_B) {
+              ad = make_desc(stream + kk * 2048, (A_STAGE_BYTES / 2) >> 4, 1024 >> 4);  // MN-major x tile
+              bd = make_desc(res + kk * 32, 1, 1024 >> 4);
+            } else {
+              ad = make_desc(res + kk * 32, 1, 1024 >> 4);
+              bd = make_desc(stream + kk * 32, 1, 1024 >> 4);
+            }
+            umma_bf16(d_tmem, ad, bd, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+          }
+          umma_commit(empty_bar + 8 * s);
+        }
+        if (ok) umma_commit(tfull_bar + 8 * acc);
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int quarter = warp & 3;
+    const int col_half = (warp - 2) >> 2;
+    uint32_t local = 0;
+    bool ok = true;
+    pdl_wait();  // no global write before the previous kernel is done with the output buffer
+    for (int si = worker; ok && si < stream_total; si += workers, ++local) {
+      const int b = si / stream_per_batch, st = si % stream_per_batch;
+      const int mt = RES_IS_B ? st : blk, nt = RES_IS_B ? blk : st;
+      const uint32_t acc = local & 1, acc_ph = (local >> 1) & 1;
+      ok = mbar_wait(tfull_bar + 8 * acc, acc_ph, &abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      drain_accumulator(p, &tmO, staging + (warp - 2) * 2048, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);
+    }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    if (threadIdx.x == 0) atomicExch(&g_gemm_timeout_flag, 1);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------- host side
+// 3-D bf16 tensor map, 128-byte swizzle, zero fill outside the tensor.
+// dims/box are innermost first; strides (bytes) are for dims 1 and 2.
+bool make_map(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t s1, uint64_t s2,
+              uint32_t b0, uint32_t b1) {
+  const cuuint64_t dims[3] = {d0, d1, d2};
+  const cuuint64_t strides[2] = {s1, s2};
+  const cuuint32_t box[3] = {b0, b1, 1};
+  return tma_make_map_bf16(map, base, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
+template <bool A_MN>
+msla_status_t launch_stationary(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO, const GemmParams& p,
+                                int blocks, cudaStream_t st) {
   static std::atomic<unsigned long long> attr_done{0};
-  msla_status_t s = ensure_smem_attr(attr_done, gemm_wx_kernel, SMEM_BUDGET);
-  if (s != MSLA_OK) return s;
-  launch_pdl(gemm_wx_kernel, dim3((unsigned)(p.workers * p.blocks)), dim3(NUM_THREADS), (size_t)smem, st, tmW, tmX, tmO, p);
+  const msla_status_t as = ensure_smem_attr(attr_done, gemm_bf16_stationary_kernel<A_MN>, WS_SMEM_BYTES);
+  if (as != MSLA_OK) return as;
+  const long long stream_total = (long long)p.batches * (A_MN ? p.m_tiles : p.n_tiles);
+  long long workers = device_sm_count() / blocks;
+  if (workers > stream_total) workers = stream_total;
+  launch_pdl(gemm_bf16_stationary_kernel<A_MN>, dim3((unsigned)(workers * blocks)), dim3(NUM_THREADS), WS_SMEM_BYTES, st, tmA, tmB, tmO, p, blocks, (int)workers);
+  count_launches(1);
+  return check_launch("projection GEMM (tcgen05, stationary weights)");
+}
+
+template <bool A_MN, bool B_PLANAR = false>
+msla_status_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO, const GemmParams& p, cudaStream_t st) {
+  // weight-stationary kernel when the CTA's weight block fits its 128 KB of shared memory
+  const int blocks = A_MN ? p.n_tiles : p.m_tiles;
+  const int k_iters = (p.K + BK - 1) / BK;
+  if (A_MN && k_iters * B_STAGE_BYTES <= RES_BYTES && blocks <= 16 && blocks <= device_sm_count())
+    return launch_stationary<A_MN>(tmA, tmB, tmO, p, blocks, st);
+  static std::atomic<unsigned long long> attr_done{0};
+  const msla_status_t as = ensure_smem_attr(attr_done, gemm_bf16_tcgen05_kernel<A_MN, B_PLANAR>, SMEM_BYTES);
+  if (as != MSLA_OK) return as;
+  const long long tiles = (long long)p.batches * p.m_tiles * p.n_tiles;
+  const int grid = (int)(tiles < device_sm_count() ? tiles : device_sm_count());
+  launch_pdl(gemm_bf16_tcgen05_kernel<A_MN, B_PLANAR>, dim3(grid), dim3(NUM_THREADS), SMEM_BYTES, st, tmA, tmB, tmO, p);
   count_launches(1);
   return check_launch("projection GEMM (tcgen05)");
+}
+
+}  // namespace
+
+bool project_in_bf16_supported(int C, int Cout, int N, int d) {
+  return C % 8 == 0 && Cout % 8 == 0 && N % 8 == 0 && (d == 16 || d == 32) && Cout % d == 0;
+}
+
+// y[b][o / d][n][o % d] = sum_c w[o][c] * x[b][c][n];  x NCHW [B, C, N], y planar with batch stride y_sb.
+msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d,
+                                  long long y_sb, cudaStream_t st) {
+  CUtensorMap tmA, tmB;
+  if (!make_map(&tmA, x, (uint64_t)N, (uint64_t)C, (uint64_t)B, (uint64_t)N * 2, (uint64_t)C * N * 2, 64, BK) ||
+      !make_map(&tmB, w, (uint64_t)C, (uint64_t)Cout, 1, (uint64_t)C * 2, (uint64_t)C * Cout * 2, BK, BN))
+    return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the input projection");
+  GemmParams p{};
+  p.M = N; p.N = Cout; p.K = C; p.batches = B;
+  p.m_tiles = (N + BM - 1) / BM; p.n_tiles = (Cout + BN - 1) / BN;
+  p.out_batch_stride = y_sb; p.ld_out = 0; p.group = d; p.bias_per_row = 0; p.n_fastest = 1;
+  p.bias = nullptr; p.out = (bf16*)y;
+  // planes of 32 channels are written as 32-token x 32-channel blocks by TMA
+  CUtensorMap tmO = tmA;  // placeholder when the direct-store epilogue is used
+  const long long plane_elems = (long long)N * 32;
+  if (d == 32 && y_sb % plane_elems == 0) {
+    p.tma_store = 1;
+    p.planes_per_batch = (int)(y_sb / plane_elems);
+    const cuuint64_t dims[3] = {32, (cuuint64_t)N, (cuuint64_t)B * p.planes_per_batch};
+    const cuuint64_t strides[2] = {64, (cuuint64_t)N * 64};
+    const cuuint32_t box[3] = {32, 32, 1};
+    if (!tma_make_map_bf16(&tmO, y, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B))
+      return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the input projection's output");
+  }
+  return launch<true>(tmA, tmB, tmO, p, st);
+}
+
+bool project_out_bf16_supported(int Cin, int Cout, int N) { return Cin % 8 == 0 && N % 8 == 0 && Cout >= 1; }
+
+// y[b][m][n] = sum_j w[m][j] * a[b][n][j] + bias[m];  a token-major [B, N, Cin], y NCHW [B, Cout, N].
+msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin, int Cout,
+                                   int N, cudaStream_t st) {
+  CUtensorMap tmA, tmB;
+  if (!make_map(&tmA, w, (uint64_t)Cin, (uint64_t)Cout, 1, (uint64_t)Cin * 2, (uint64_t)Cin * Cout * 2, BK, BM) ||
+      !make_map(&tmB, a, (uint64_t)Cin, (uint64_t)N, (uint64_t)B, (uint64_t)Cin * 2, (uint64_t)N * Cin * 2, BK, BN))
+    return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the output projection");
+  GemmParams p{};
+  p.M = Cout; p.N = N; p.K = Cin; p.batches = B;
+  p.m_tiles = (Cout + BM - 1) / BM; p.n_tiles = (N + BN - 1) / BN;
+  p.out_batch_stride = (long long)Cout * N; p.ld_out = N; p.group = 0; p.bias_per_row = 1; p.n_fastest = 0;
+  p.bias = (const bf16*)bias; p.out = (bf16*)y;
+  CUtensorMap tmO;  // NCHW output as [batch][channel][token]; blocks of 32 channels x 32 tokens
+  {
+    p.tma_store = 1;
+    const cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)Cout, (cuuint64_t)B};
+    const cuuint64_t strides[2] = {(cuuint64_t)N * 2, (cuuint64_t)Cout * N * 2};
+    const cuuint32_t box[3] = {32, 32, 1};
+    if (!tma_make_map_bf16(&tmO, y, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B))
+      return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the output projection's output");
+  }
+  return launch<false>(tmA, tmB, tmO, p, st);
+}
+
+bool project_out_planar_bf16_supported(int Cin, int Cout, int N) { return Cin % 64 == 0 && N % 8 == 0 && Cout >= 1; }
+
+// Same product with the attention output kept planar: a[b][j / 64][n][j % 64] (one [N][64] plane per pair of heads).
+msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin,
+                                          int Cout, int N, cudaStream_t st) {
+  CUtensorMap tmA, tmB, tmO;
+  const int planes = Cin / 64;
+  {
+    const cuuint64_t dO[3] = {(cuuint64_t)N, (cuuint64_t)Cout, (cuuint64_t)B};
+    const cuuint64_t sO[2] = {(cuuint64_t)N * 2, (cuuint64_t)Cout * N * 2};
+    const cuuint32_t bO[3] = {32, 32, 1};
+    if (!make_map(&tmA, w, (uint64_t)Cin, (uint64_t)Cout, 1, (uint64_t)Cin * 2, (uint64_t)Cin * Cout * 2, BK, BM) ||
+        !make_map(&tmB, a, 64, (uint64_t)N, (uint64_t)B * planes, 128, (uint64_t)N * 128, BK, BN) ||
+        !tma_make_map_bf16(&tmO, y, 3, dO, sO, bO, CU_TENSOR_MAP_SWIZZLE_64B))
+      return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the output projection");
+  }
+  GemmParams p{};
+  p.M = Cout; p.N = N; p.K = Cin; p.batches = B;
+  p.m_tiles = (Cout + BM - 1) / BM; p.n_tiles = (N + BN - 1) / BN;
+  p.out_batch_stride = (long long)Cout * N; p.ld_out = N; p.group = 0; p.bias_per_row = 1; p.n_fastest = 0;
+  p.bias = (const bf16*)bias; p.out = (bf16*)y;
+  p.tma_store = 1; p.planes_per_batch = planes;
+  return launch<false, true>(tmA, tmB, tmO, p, st);
 }
 
 // Non-zero once any projection GEMM of this process hit a wait time-out (synchronises the device).

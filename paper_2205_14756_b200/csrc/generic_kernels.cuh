@@ -13,13 +13,15 @@ namespace generic {
 // Strided GEMM for the two 1x1 projections (Section 3.1: Q = xW_Q, K = xW_K,
 // V = xW_V; final linear projection):
 //   D(m, n) = sum_k A(m, k) * W[n, k] (+ bias[n]),   m = token, n = out channel
-// A(m, k) = A[b*sAb + m*sAm + k*sAk];   D(m, n) = D[b*sDb + m*sDm + n*sDn].
-// Channel-major (NCHW) operands have sAm = sDm = 1 and sAk = sDn = N.
+// A(m, k) = A[b*sAb + m*sAm + k*sAk];
+// D(m, n) = D[b*sDb + (n / group)*sDg + m*sDm + (n % group)*sDn]: out channels
+// may be split into groups of `group` that live in separate planes.
 // ---------------------------------------------------------------------------
 struct GemmArgs {
   long long sAb, sAm, sAk;
-  long long sDb, sDm, sDn;
+  long long sDb, sDm, sDn, sDg;
   int M, Nc, K;  // tokens, out channels, in channels
+  int group;     // out channels per plane (>= Nc: one plane)
 };
 
 template <typename T>
@@ -81,7 +83,7 @@ gemm_kernel(const T* __restrict__ A, const T* __restrict__ Wt, const T* __restri
       const int n = n0 + ni + j;
       if (n >= g.Nc) continue;
       const float r = acc[i][j] + (bias ? to_f32(bias[n]) : 0.f);
-      Db[m * g.sDm + (long long)n * g.sDn] = from_f32<T>(r);
+      Db[(long long)(n / g.group) * g.sDg + m * g.sDm + (long long)(n % g.group) * g.sDn] = from_f32<T>(r);
     }
   }
 }
@@ -89,8 +91,8 @@ gemm_kernel(const T* __restrict__ A, const T* __restrict__ Wt, const T* __restri
 // ---------------------------------------------------------------------------
 // Multi-scale token aggregation (Section 3.1): 5x5 depthwise convolution
 // (cross-correlation, zero padding 2) followed by the grouped 1x1 convolution,
-// on channel-major activations [B, Ch, H, W].  One CTA = one 8x8 pixel tile of
-// one group of d channels.  src(b, c, y, x) = src[b*src_sb + (c*H + y)*W + x];
+// on planar activations [B, groups, H*W, d].  One CTA = one 8x8 pixel tile of
+// one group of d channels.  src(b, g, n, i) = src[b*src_sb + (g*H*W + n)*d + i];
 // dst likewise with dst_sb.
 // ---------------------------------------------------------------------------
 template <typename T>
@@ -98,8 +100,8 @@ __global__ void __launch_bounds__(256)
 aggregate_kernel(const T* __restrict__ src, const T* __restrict__ w_dw, const T* __restrict__ w_pw,
                  T* __restrict__ dst, int H, int W, int d, long long src_sb, long long dst_sb) {
   constexpr int TS = 8, HALO = TS + 4, DMAX = 32;
-  __shared__ float tile[DMAX][HALO * HALO + 1];
-  __shared__ float dwo[DMAX][TS * TS + 1];
+  __shared__ float tile[HALO * HALO][DMAX + 1];
+  __shared__ float dwo[TS * TS][DMAX + 1];
   __shared__ float wdw[DMAX][25];
   __shared__ float wpw[DMAX][DMAX + 1];
   const int tid = threadIdx.x;
@@ -107,38 +109,37 @@ aggregate_kernel(const T* __restrict__ src, const T* __restrict__ w_dw, const T*
   const int x0 = (blockIdx.x % tiles_x) * TS, y0 = (blockIdx.x / tiles_x) * TS;
   const int ch0 = blockIdx.y * d;
   const int b = blockIdx.z;
-  const long long plane = (long long)H * W;
-  const T* sb = src + (long long)b * src_sb + (long long)ch0 * plane;
+  const T* sb = src + (long long)b * src_sb + (long long)blockIdx.y * H * W * d;
   for (int e = tid; e < d * 25; e += 256) wdw[e / 25][e % 25] = to_f32(w_dw[(long long)ch0 * 25 + e]);
   for (int e = tid; e < d * d; e += 256) wpw[e / d][e % d] = to_f32(w_pw[(long long)ch0 * d + e]);
   for (int e = tid; e < HALO * HALO * d; e += 256) {
-    const int p = e % (HALO * HALO), c = e / (HALO * HALO);
+    const int c = e % d, p = e / d;
     const int yy = y0 + p / HALO - 2, xx = x0 + p % HALO - 2;
     float v = 0.f;
-    if (yy >= 0 && yy < H && xx >= 0 && xx < W) v = to_f32(sb[c * plane + (long long)yy * W + xx]);
-    tile[c][p] = v;
+    if (yy >= 0 && yy < H && xx >= 0 && xx < W) v = to_f32(sb[((long long)yy * W + xx) * d + c]);
+    tile[p][c] = v;
   }
   __syncthreads();
   for (int e = tid; e < TS * TS * d; e += 256) {
-    const int p = e % (TS * TS), c = e / (TS * TS);
+    const int c = e % d, p = e / d;
     const int py = p / TS, px = p % TS;
     float acc = 0.f;
 #pragma unroll
     for (int dy = 0; dy < 5; ++dy)
 #pragma unroll
       for (int dx = 0; dx < 5; ++dx)
-        acc = fmaf(wdw[c][dy * 5 + dx], tile[c][(py + dy) * HALO + px + dx], acc);
-    dwo[c][p] = acc;
+        acc = fmaf(wdw[c][dy * 5 + dx], tile[(py + dy) * HALO + px + dx][c], acc);
+    dwo[p][c] = acc;
   }
   __syncthreads();
-  T* db = dst + (long long)b * dst_sb + (long long)ch0 * plane;
+  T* db = dst + (long long)b * dst_sb + (long long)blockIdx.y * H * W * d;
   for (int e = tid; e < TS * TS * d; e += 256) {
-    const int p = e % (TS * TS), o = e / (TS * TS);
+    const int o = e % d, p = e / d;
     const int yy = y0 + p / TS, xx = x0 + p % TS;
     if (yy >= H || xx >= W) continue;
     float acc = 0.f;
-    for (int i = 0; i < d; ++i) acc = fmaf(wpw[o][i], dwo[i][p], acc);
-    db[o * plane + (long long)yy * W + xx] = from_f32<T>(acc);
+    for (int i = 0; i < d; ++i) acc = fmaf(wpw[o][i], dwo[p][i], acc);
+    db[((long long)yy * W + xx) * d + o] = from_f32<T>(acc);
   }
 }
 
@@ -172,11 +173,10 @@ kv_partial_kernel(const T* __restrict__ k, const T* __restrict__ v, float* __res
   }
   for (int n0 = n_begin; n0 < n_end; n0 += TT) {
     for (int e = tid; e < TT * d; e += 256) {
-      // consecutive threads follow the contiguous index: channels (dense rows) or tokens (channel-major)
-      const int i = kv.cs == 1 ? e % d : e / TT, t = kv.cs == 1 ? e / d : e % TT;
+      const int i = e % d, t = e / d;
       float kk = 0.f, vv = 0.f;
       if (n0 + t < n_end) {
-        const long long off = base + (long long)(n0 + t) * kv.ld + (long long)i * kv.cs;
+        const long long off = base + (long long)(n0 + t) * kv.ld + i;
         kk = fmaxf(to_f32(k[off]), 0.f);
         vv = to_f32(v[off]);
       }
@@ -235,7 +235,7 @@ apply_kernel(const T* __restrict__ q, const float* __restrict__ state, T* __rest
   T* op = out + (long long)b * ov.batch + (long long)h * ov.head + (long long)n * ov.ld;
   float qr[DMAX];
 #pragma unroll
-  for (int a = 0; a < DMAX; ++a) qr[a] = a < d ? fmaxf(to_f32(qp[(long long)a * qv.cs]), 0.f) : 0.f;
+  for (int a = 0; a < DMAX; ++a) qr[a] = a < d ? fmaxf(to_f32(qp[a]), 0.f) : 0.f;
   float den = 0.f;
 #pragma unroll
   for (int a = 0; a < DMAX; ++a)
@@ -246,7 +246,7 @@ apply_kernel(const T* __restrict__ q, const float* __restrict__ state, T* __rest
 #pragma unroll
     for (int a = 0; a < DMAX; ++a)
       if (a < d) num = fmaf(qr[a], st[a * d1 + c], num);
-    op[(long long)c * ov.cs] = from_f32<T>(num * inv);
+    op[c] = from_f32<T>(num * inv);
   }
 }
 

@@ -110,35 +110,43 @@ static bool core_shape_ok(int B, int heads, int N, int d) {
   return B >= 1 && heads >= 1 && N >= 1 && (d == 16 || d == 32) && (long long)B * heads <= 65535;
 }
 
-// Generic SIMT attention core: partial states, fixed-order combine, apply.  `combine_and_apply` = false stops
-// after the partial states (the caller folds them itself).
 template <typename T>
-static msla_status_t run_core_generic(const T* q, const T* k, const T* v, T* out, HeadView in, HeadView ov, int B,
-                                      int heads, int N, int d, float eps, const CorePlan& p, char* ws, cudaStream_t st,
-                                      bool combine_and_apply = true, cudaEvent_t mid = nullptr) {
+static msla_status_t run_core_generic(const T* q, const T* k, const T* v, T* out, HeadView in,
+                                      HeadView ov, int B, int heads, int N, int d, float eps,
+                                      const CorePlan& p, char* ws, cudaStream_t st, cudaEvent_t mid) {
   const long long BH = (long long)B * heads;
   float* partial = reinterpret_cast<float*>(ws + p.partial_off);
   float* state = reinterpret_cast<float*>(ws + p.state_off);
   generic::kv_partial_kernel<T><<<dim3((unsigned)BH, p.S), 256, 0, st>>>(k, v, partial, in, heads, N, d, p.S, p.chunk);
-  count_launches(1);
-  if (combine_and_apply) {
-    const long long total = BH * p.ne;
-    generic::kv_combine_kernel<<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>(partial, state, p.S, p.ne, total);
-    if (mid) cudaEventRecord(mid, st);
-    generic::apply_kernel<T><<<dim3((unsigned)ceil_div_ll(N, 128), (unsigned)BH), 128, 0, st>>>(q, state, out, in, ov, heads, N, d, eps);
-    count_launches(2);
-  }
+  const long long total = BH * p.ne;
+  generic::kv_combine_kernel<<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>(partial, state, p.S, p.ne, total);
+  if (mid) cudaEventRecord(mid, st);
+  generic::apply_kernel<T><<<dim3((unsigned)ceil_div_ll(N, 128), (unsigned)BH), 128, 0, st>>>(
+      q, state, out, in, ov, heads, N, d, eps);
+  count_launches(3);
   return check_launch("attention core kernels");
 }
 
-// Attention core on dense [B, heads, N, d] tensors.
-static msla_status_t run_core(msla_dtype_t dtype, const void* q, const void* k, const void* v, void* out, int B,
-                              int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st) {
-  const HeadView in{(long long)heads * N * d, (long long)N * d, d, 1};
+// q/k/v views share strides; k = q + d and v = q + 2d in the module layout,
+// separate tensors in the dense layout, so three pointers are passed.
+static msla_status_t run_core(msla_dtype_t dtype, const void* q, const void* k, const void* v,
+                              void* out, HeadView in, HeadView ov, int B, int heads, int N, int d,
+                              float eps, const CorePlan& p, void* ws, cudaStream_t st,
+                              cudaEvent_t mid = nullptr, bool with_apply = true) {
+  if (!with_apply && dtype != MSLA_BF16) return fail(MSLA_ERR_UNSUPPORTED, "the state-only core exists for bf16 only");
+  if (ov.pair && (dtype != MSLA_BF16 || (heads & 1)))  // only the bf16 tensor-core kernels write paired planes
+    return fail(MSLA_ERR_UNSUPPORTED, "paired output planes need bf16 and an even number of heads");
   if (dtype == MSLA_F32)
-    return run_core_generic<float>((const float*)q, (const float*)k, (const float*)v, (float*)out, in, in, B, heads, N, d,
-                                   eps, p, (char*)ws, st);
-  return run_core_bf16(q, k, v, out, in, in, B, heads, N, d, eps, p, ws, st);
+    return run_core_generic<float>((const float*)q, (const float*)k, (const float*)v, (float*)out,
+                                   in, ov, B, heads, N, d, eps, p, (char*)ws, st, mid);
+  const bool strides_ok = in.batch % 8 == 0 && in.head % 8 == 0 && in.ld % 8 == 0 && ov.batch % 8 == 0 &&
+                          ov.head % 8 == 0 && ov.ld % 8 == 0;
+  if (strides_ok) return run_core_bf16(q, k, v, out, in, ov, B, heads, N, d, eps, p, ws, st, mid, with_apply);
+  if (!with_apply) return fail(MSLA_ERR_UNSUPPORTED, "the state-only core needs strides that are multiples of 8 elements");
+  if (ov.pair) return fail(MSLA_ERR_UNSUPPORTED, "paired output planes need strides that are multiples of 8 elements");
+  return run_core_generic<__nv_bfloat16>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
+                                         (const __nv_bfloat16*)v, (__nv_bfloat16*)out, in, ov, B,
+                                         heads, N, d, eps, p, (char*)ws, st, mid);
 }
 
 static msla_status_t core_entry(msla_dtype_t dtype, const void* q, const void* k, const void* v,
@@ -171,7 +179,8 @@ static msla_status_t core_entry(msla_dtype_t dtype, const void* q, const void* k
       return fail(MSLA_ERR_CUDA, "cudaMallocAsync(%zu): %s", p.bytes, cudaGetErrorString(e));
     }
   }
-  s = run_core(dtype, q, k, v, out, B, heads, N, d, eps, p, ws, st);
+  const HeadView in{(long long)heads * N * d, (long long)N * d, d};
+  s = run_core(dtype, q, k, v, out, in, in, B, heads, N, d, eps, p, ws, st);
   if (own_ws) cudaFreeAsync(ws, st);
   return s;
 }
@@ -228,18 +237,15 @@ static msla_status_t core_entry_noalloc(msla_dtype_t dtype, const void* q, const
   if ((s = noalloc_scratch(&ws)) != MSLA_OK) return s;
   // Every partial and state entry the apply step reads is written earlier in
   // this same call, so nothing left over from a previous call needs clearing.
-  return run_core(dtype, q, k, v, out, B, heads, N, d, eps, p, ws, st);
+  const HeadView in{(long long)heads * N * d, (long long)N * d, d};
+  return run_core(dtype, q, k, v, out, in, in, B, heads, N, d, eps, p, ws, st);
 }
 
 // ------------------------------------------------------------- module plan
-// Between the steps every activation is channel-major (NCHW), like x and out: the multi-scale buffer is
-// ms[B][6C'][N], channel (s*heads + h)*3*d + t*d + i = element i of q (t = 0), k (1) or v (2) of head h at scale
-// s (0: projected tokens, 1: aggregated tokens).  One image's q, k, v of one head are 3*d consecutive planes.
 struct ForwardPlan {
   size_t ms_off, att_off, core_off, bytes;
   CorePlan core;
   int Cp, N;
-  bool fused;  // steps 4 and 5 as one kernel
 };
 
 static msla_status_t validate_desc(const msla_desc* d, ForwardPlan* plan) {
@@ -254,45 +260,72 @@ static msla_status_t validate_desc(const msla_desc* d, ForwardPlan* plan) {
   if (d->d != 16 && d->d != 32) return fail(MSLA_ERR_UNSUPPORTED, "d = %d; only 16 and 32 are supported", d->d);
   if ((long long)d->H * d->W > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "H*W exceeds 2^31-1");
   if (d->C % 8 != 0 || d->C_out % 8 != 0) return fail(MSLA_ERR_UNSUPPORTED, "C and C_out must be multiples of 8");
-  if ((long long)d->B * 2 * d->heads > 65535 || d->B > 65535 || 3LL * d->heads > 65535) return fail(MSLA_ERR_UNSUPPORTED, "B*2*heads exceeds 65535");
+  if ((long long)d->B * 2 * d->heads > 65535 || d->B > 65535) return fail(MSLA_ERR_UNSUPPORTED, "B*2*heads exceeds 65535");
   plan->Cp = d->heads * d->d;
   plan->N = d->H * d->W;
   const size_t e = elem_size(d->dtype);
   const size_t tokens = (size_t)d->B * plan->N;
   plan->core = make_core_plan((long long)d->B * 2 * d->heads, plan->N, d->d);
-  plan->fused = d->dtype == MSLA_BF16 && fused_out_bf16_supported(2 * d->heads, d->d, d->C_out, plan->N);
   plan->ms_off = 0;
   plan->att_off = align_up(tokens * 6 * plan->Cp * e, 256);
-  // unfused: the attention output [B][2C'][N]; fused: the folded projection matrix and the key sums
-  const size_t att_bytes = plan->fused ? fused_out_scratch_bytes(d->B, 2 * d->heads, d->d, d->C_out) : tokens * 2 * plan->Cp * e;
+  // the attention output's region doubles as scratch of the fused apply + projection kernel, which writes no attention output
+  size_t att_bytes = tokens * 2 * plan->Cp * e;
+  const size_t fused_scratch = fused_out_bf16_supported(2 * d->heads, d->d, d->C_out, plan->N) ? fused_out_scratch_bytes(d->B, 2 * d->heads, d->d, d->C_out) : 0;
+  if (att_bytes < fused_scratch) att_bytes = fused_scratch;
   plan->core_off = plan->att_off + align_up(att_bytes, 256);
   plan->bytes = plan->core_off + plan->core.bytes;
   return MSLA_OK;
 }
 
-// y[b][m][n] = sum_k w[m][k] x[b][k][n] (+ bias[m]): a 1x1 convolution on channel-major activations
-// (batch strides x_sb, y_sb in elements).
-static msla_status_t run_conv1x1(msla_dtype_t dt, const void* x, const void* w, const void* bias, void* y, int B, int K,
-                                 int M, int N, long long x_sb, long long y_sb, cudaStream_t st) {
-  if (dt == MSLA_BF16 && gemm_bf16_supported(M, N, K) && x_sb % 8 == 0 && y_sb % 8 == 0)
-    return run_gemm_bf16(x, w, bias, y, B, K, M, N, x_sb, y_sb, st);
-  const generic::GemmArgs g{x_sb, 1, N, y_sb, 1, N, N, M, K};
-  const dim3 grid((unsigned)ceil_div_ll(N, 64), (unsigned)ceil_div_ll(M, 64), (unsigned)B);
-  if (dt == MSLA_F32)
-    generic::gemm_kernel<float><<<grid, 256, 0, st>>>((const float*)x, (const float*)w, (const float*)bias, (float*)y, g);
-  else
-    generic::gemm_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w,
-                                                              (const __nv_bfloat16*)bias, (__nv_bfloat16*)y, g);
+template <typename T>
+static void launch_gemm(const T* A, const T* W, const T* bias, T* D, generic::GemmArgs g, int B, cudaStream_t st) {
+  dim3 grid((unsigned)ceil_div_ll(g.M, 64), (unsigned)ceil_div_ll(g.Nc, 64), (unsigned)B);
+  generic::gemm_kernel<T><<<grid, 256, 0, st>>>(A, W, bias, D, g);
   count_launches(1);
-  return check_launch("1x1 projection");
 }
 
-// src, dst: channel-major [B, Ch, H, W] with batch strides src_sb, dst_sb (elements)
-static msla_status_t run_aggregate(msla_dtype_t dt, const void* src, const void* w_dw, const void* w_pw, void* dst, int B,
-                                   int H, int W, int Ch, int d, long long src_sb, long long dst_sb, cudaStream_t st) {
-  if (dt == MSLA_BF16 && aggregate_bf16_supported(H, W, Ch, d) && src_sb % 8 == 0 && dst_sb % 8 == 0)
-    return run_aggregate_bf16(src, src_sb, w_dw, w_pw, dst, dst_sb, B, H, W, Ch, d, st);
-  const dim3 grid((unsigned)(ceil_div_ll(W, 8) * ceil_div_ll(H, 8)), (unsigned)(Ch / d), (unsigned)B);
+// y planar: y[b*y_sb + ((o/d)*N + n)*d + o%d]
+static msla_status_t run_project_in(msla_dtype_t dt, const void* x, const void* w, void* y, int B,
+                                    int C, int Cout, int N, int d, long long y_sb, cudaStream_t st) {
+  if (dt == MSLA_BF16 && project_in_bf16_supported(C, Cout, N, d)) return run_project_in_bf16(x, w, y, B, C, Cout, N, d, y_sb, st);
+  generic::GemmArgs g{(long long)C * N, 1, N, y_sb, d, 1, (long long)N * d, N, Cout, C, d};
+  if (dt == MSLA_F32) launch_gemm<float>((const float*)x, (const float*)w, nullptr, (float*)y, g, B, st);
+  else launch_gemm<__nv_bfloat16>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w, nullptr, (__nv_bfloat16*)y, g, B, st);
+  return check_launch("input projection");
+}
+
+static msla_status_t run_project_out(msla_dtype_t dt, const void* a, const void* w, const void* bias,
+                                     void* y, int B, int Cin, int Cout, int N, cudaStream_t st) {
+  if (dt == MSLA_BF16 && project_out_bf16_supported(Cin, Cout, N)) return run_project_out_bf16(a, w, bias, y, B, Cin, Cout, N, st);
+  generic::GemmArgs g{(long long)N * Cin, Cin, 1, (long long)Cout * N, 1, N, 0, N, Cout, Cin, Cout};
+  if (dt == MSLA_F32) launch_gemm<float>((const float*)a, (const float*)w, (const float*)bias, (float*)y, g, B, st);
+  else launch_gemm<__nv_bfloat16>((const __nv_bfloat16*)a, (const __nv_bfloat16*)w, (const __nv_bfloat16*)bias, (__nv_bfloat16*)y, g, B, st);
+  return check_launch("output projection");
+}
+
+// src, dst planar [B, Ch/d, H*W, d] with batch strides src_sb, dst_sb (elements)
+static msla_status_t run_aggregate(msla_dtype_t dt, const void* src, const void* w_dw, const void* w_pw,
+                                   void* dst, int B, int H, int W, int Ch, int d, long long src_sb,
+                                   long long dst_sb, cudaStream_t st) {
+  const long long plane = (long long)H * W * d;
+  if (dt == MSLA_BF16 && src_sb % plane == 0 && dst_sb % plane == 0) {
+    if (aggregate_bf16_supported(H, W, Ch, d))
+      return run_aggregate_bf16(src, (long long)B * (src_sb / plane), (int)(src_sb / plane), w_dw, w_pw, dst, dst_sb, B, H, W, Ch, d, st);
+    if (d == 16 && Ch > 16 && aggregate_bf16_supported(H, W, Ch - 16, d)) {
+      // odd number of 16-channel groups: the tuned kernel takes them in pairs, the plain one the last group
+      msla_status_t s = run_aggregate_bf16(src, (long long)B * (src_sb / plane), (int)(src_sb / plane), w_dw, w_pw, dst, dst_sb, B, H, W, Ch - 16, d, st);
+      if (s != MSLA_OK) return s;
+      const __nv_bfloat16* s16 = (const __nv_bfloat16*)src + (long long)(Ch / 16 - 1) * plane;
+      __nv_bfloat16* d16 = (__nv_bfloat16*)dst + (long long)(Ch / 16 - 1) * plane;
+      dim3 grid1((unsigned)(ceil_div_ll(W, 8) * ceil_div_ll(H, 8)), 1u, (unsigned)B);
+      generic::aggregate_kernel<__nv_bfloat16><<<grid1, 256, 0, st>>>(s16, (const __nv_bfloat16*)w_dw + (long long)(Ch - 16) * 25,
+                                                                      (const __nv_bfloat16*)w_pw + (long long)(Ch - 16) * 16, d16, H, W, d,
+                                                                      src_sb, dst_sb);
+      count_launches(1);
+      return check_launch("token aggregation (last group)");
+    }
+  }
+  dim3 grid((unsigned)(ceil_div_ll(W, 8) * ceil_div_ll(H, 8)), (unsigned)(Ch / d), (unsigned)B);
   if (dt == MSLA_F32)
     generic::aggregate_kernel<float><<<grid, 256, 0, st>>>((const float*)src, (const float*)w_dw, (const float*)w_pw,
                                                            (float*)dst, H, W, d, src_sb, dst_sb);
@@ -348,42 +381,43 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
       return fail(MSLA_ERR_CUDA, "host-to-device copy of x: %s", cudaGetErrorString(ce));
     }
   }
-  const int Cp = p.Cp, N = p.N, d = desc->d, heads = desc->heads, B = desc->B;
+  const int Cp = p.Cp, N = p.N, d = desc->d, heads = desc->heads;
+  const long long ld_att = 2LL * Cp;
   const long long ms_sb = 6LL * Cp * N;  // elements per image of the multi-scale buffer
+  // ms: planar [B][6*heads planes][N][d]; plane (s*heads + h)*3 + t holds q (t=0), k (1) or v (2)
+  // of head h at scale s (0: projected tokens, 1: aggregated tokens).
   char* ms = ws + p.ms_off;
-  char* att = ws + p.att_off;
+  char* att = ws + p.att_off;  // [B, N, 2C'] token-major head concat
   if ((s = record(events, 0, st)) != MSLA_OK) return s;
-  // 1. QKV projection into the scale-0 channels
-  s = run_conv1x1(desc->dtype, x_dev, w->w_qkv, nullptr, ms, B, desc->C, 3 * Cp, N, (long long)desc->C * N, ms_sb, st);
+  // 1. QKV projection into the scale-0 planes
+  s = run_project_in(desc->dtype, x_dev, w->w_qkv, ms, desc->B, desc->C, 3 * Cp, N, d, ms_sb, st);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 1, st)) != MSLA_OK) return s;
-  // 2. aggregation of the scale-0 channels into the scale-1 channels
-  s = run_aggregate(desc->dtype, ms, w->w_dw, w->w_pw, ms + (size_t)3 * Cp * N * e, B, desc->H, desc->W, 3 * Cp, d, ms_sb, ms_sb, st);
+  // 2. aggregation of every scale-0 plane into the matching scale-1 plane
+  s = run_aggregate(desc->dtype, ms, w->w_dw, w->w_pw, ms + (size_t)3 * Cp * N * e, desc->B, desc->H, desc->W, 3 * Cp, d, ms_sb, ms_sb, st);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 2, st)) != MSLA_OK) return s;
-  // 3 + 4. attention over 2*heads heads of [q|k|v] channel planes; outputs land at channel head*d (concat)
-  const HeadView in{ms_sb, 3LL * d * N, 1, N};
-  const HeadView ov{2LL * Cp * N, (long long)d * N, 1, N};
-  const void* qp = ms;
-  const void* kp = ms + (size_t)d * N * e;
-  const void* vp = ms + (size_t)2 * d * N * e;
-  char* core_ws = ws + p.core_off;
-  cudaEvent_t mid = events ? (cudaEvent_t)events[3] : nullptr;
-  if (desc->dtype == MSLA_F32)
-    s = run_core_generic<float>((const float*)qp, (const float*)kp, (const float*)vp, (float*)att, in, ov, B, 2 * heads, N, d,
-                                desc->eps, p.core, core_ws, st, !p.fused, mid);
-  else
-    s = run_core_generic<__nv_bfloat16>((const __nv_bfloat16*)qp, (const __nv_bfloat16*)kp, (const __nv_bfloat16*)vp,
-                                        (__nv_bfloat16*)att, in, ov, B, 2 * heads, N, d, desc->eps, p.core, core_ws, st, !p.fused, mid);
+  // 3+4. attention over 2*heads heads of [q|k|v]; outputs land at channel head*d (concat)
+  const HeadView in{ms_sb, 3LL * N * d, d};
+  // Attention output: one [N][2d] plane per pair of heads when the tcgen05 output projection can
+  // take it (dense 128-byte rows for the apply kernel's stores and the GEMM's tile loads),
+  // otherwise token-major [N][2C'].
+  const bool att_planar = desc->dtype == MSLA_BF16 && d == 32 && project_out_planar_bf16_supported(2 * Cp, desc->C_out, N);
+  const HeadView ov = att_planar ? HeadView{(long long)N * ld_att, (long long)N * 2 * d, 2 * d, 1}
+                                 : HeadView{(long long)N * ld_att, d, ld_att, 0};
+  // Steps 4 and 5 run as one kernel when it takes the shape: the head concat then stays in shared memory.
+  const bool fused = desc->dtype == MSLA_BF16 && fused_out_bf16_supported(2 * heads, d, desc->C_out, N);
+  s = run_core(desc->dtype, ms, ms + (size_t)N * d * e, ms + (size_t)2 * N * d * e, att, in, ov, desc->B, 2 * heads, N, d, desc->eps, p.core,
+               ws + p.core_off, st, events ? (cudaEvent_t)events[3] : nullptr, !fused);
   if (s != MSLA_OK) return s;
-  if (p.fused && (s = record(events, 3, st)) != MSLA_OK) return s;
   if ((s = record(events, 4, st)) != MSLA_OK) return s;
-  // 5. output projection back to NCHW (fused: state fold, then apply + projection as one GEMM)
-  if (p.fused)
-    s = run_fused_out_bf16(qp, ms_sb, 3LL * d * N, reinterpret_cast<const float*>(core_ws + p.core.partial_off), p.core.S, att,
-                           w->w_proj, w->b_proj, out_dev, B, 2 * heads, d, N, desc->C_out, desc->eps, st);
+  // 5. output projection back to NCHW
+  if (fused)
+    s = run_fused_out_bf16(ms, ms_sb, 3LL * N * d, reinterpret_cast<const float*>(ws + p.core_off + p.core.partial_off), p.core.S, att, w->w_proj,
+                           w->b_proj, out_dev, desc->B, 2 * heads, d, N, desc->C_out, desc->eps, st);
   else
-    s = run_conv1x1(desc->dtype, att, w->w_proj, w->b_proj, out_dev, B, 2 * Cp, desc->C_out, N, 2LL * Cp * N, (long long)desc->C_out * N, st);
+    s = att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st)
+                   : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 5, st)) != MSLA_OK) return s;
   if (host_io) {
@@ -460,7 +494,7 @@ msla_status_t msla_forward_host(const msla_desc* desc, const void* x_host, const
 int msla_forward_fuses_apply(const msla_desc* desc) {
   ForwardPlan p;
   if (validate_desc(desc, &p) != MSLA_OK) return -1;
-  return p.fused ? 1 : 0;
+  return desc->dtype == MSLA_BF16 && fused_out_bf16_supported(2 * desc->heads, desc->d, desc->C_out, p.N) ? 1 : 0;
 }
 
 unsigned long long msla_kernel_launches(void) { return g_launches; }
@@ -470,8 +504,17 @@ int msla_debug_wait_timeouts(void) {
   return (a < 0 || b < 0 || c < 0) ? -1 : (a | b | c);
 }
 
-msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y, int B, int C, int Cout, int N, void* stream) {
-  return msla_project_out(dtype, x, w, nullptr, y, B, C, Cout, N, stream);
+msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d, void* stream) {
+  if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");
+  if (!x || !w || !y) return fail(MSLA_ERR_INVALID_ARG, "null pointer");
+  if (B < 1 || C < 1 || Cout < 1 || N < 1 || B > 65535) return fail(MSLA_ERR_INVALID_ARG, "sizes must be positive (B <= 65535)");
+  if (C % 8 || Cout % 8) return fail(MSLA_ERR_UNSUPPORTED, "C and Cout must be multiples of 8");
+  if (d != 16 && d != 32) return fail(MSLA_ERR_UNSUPPORTED, "d = %d; only 16 and 32 are supported", d);
+  if (Cout % d) return fail(MSLA_ERR_INVALID_ARG, "Cout must be a multiple of d");
+  if (!aligned16(x) || !aligned16(w) || !aligned16(y)) return fail(MSLA_ERR_ALIGNMENT, "pointers must be 16-byte aligned");
+  msla_status_t s = check_arch();
+  if (s != MSLA_OK) return s;
+  return run_project_in(dtype, x, w, y, B, C, Cout, N, d, (long long)Cout * N, (cudaStream_t)stream);
 }
 
 msla_status_t msla_aggregate(msla_dtype_t dtype, const void* t, const void* w_dw, const void* w_pw, void* y, int B, int H, int W, int Ch, int d, void* stream) {
@@ -494,13 +537,11 @@ msla_status_t msla_project_out(msla_dtype_t dtype, const void* a, const void* w,
   if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");
   if (!a || !w || !y) return fail(MSLA_ERR_INVALID_ARG, "null pointer");
   if (B < 1 || Cin < 1 || Cout < 1 || N < 1 || B > 65535) return fail(MSLA_ERR_INVALID_ARG, "sizes must be positive (B <= 65535)");
-  if (Cin % 8 || Cout % 8) return fail(MSLA_ERR_UNSUPPORTED, "channel counts must be multiples of 8");
+  if (Cin % 8 || Cout % 8) return fail(MSLA_ERR_UNSUPPORTED, "Cin and Cout must be multiples of 8");
   if (!aligned16(a) || !aligned16(w) || !aligned16(y) || (bias && !aligned16(bias))) return fail(MSLA_ERR_ALIGNMENT, "pointers must be 16-byte aligned");
-  const size_t e = elem_size(dtype);
-  if (overlaps(a, (size_t)B * Cin * N * e, y, (size_t)B * Cout * N * e)) return fail(MSLA_ERR_INVALID_ARG, "y overlaps the input");
   msla_status_t s = check_arch();
   if (s != MSLA_OK) return s;
-  return run_conv1x1(dtype, a, w, bias, y, B, Cin, Cout, N, (long long)Cin * N, (long long)Cout * N, (cudaStream_t)stream);
+  return run_project_out(dtype, a, w, bias, y, B, Cin, Cout, N, (cudaStream_t)stream);
 }
 
 const char* msla_status_string(msla_status_t s) {

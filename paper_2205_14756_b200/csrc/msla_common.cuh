@@ -8,17 +8,18 @@
 namespace msla {
 
 // Strided view of per-head token matrices: element (b, h, n, i) of tensor t is
-//   t[b * batch + h * head + n * ld + i * cs].
-// Dense [B, heads, N, d] tensors of the
-// stand-alone attention core:           batch = heads*N*d, head = N*d, ld = d, cs = 1.
-// Channel-major (NCHW) activations of
-// the module, head = d consecutive
-// channel planes of N tokens each:      batch = C*N, head = (channels per head)*N, ld = 1, cs = N.
+//   t[b * batch + h * head + n * ld + i].
+// Dense [B, heads, N, d] input:        batch = heads*N*d, head = N*d, ld = d.
+// Token-major multi-scale buffer
+// [B, N, 6C'] with [q|k|v] per head:   batch = N*6C',  head = 3d,  ld = 6C'.
+// Paired heads (pair = 1, outputs only): heads 2p and 2p+1 share one [N][2d]
+// plane, head 2p+1 in its upper d columns:
+//   t[b * batch + (h / 2) * head + (h % 2) * d + n * ld + i],  ld = 2d.
 struct HeadView {
   long long batch;
   long long head;
   long long ld;
-  long long cs;
+  int pair;
 };
 
 __device__ __forceinline__ float to_f32(float v) { return v; }

@@ -93,33 +93,40 @@ inline void launch_pdl_cluster2(void (*kernel)(KArgs...), dim3 grid, dim3 block,
 }
 
 struct HeadView;
-// Tuned bf16 attention core on dense [B, heads, N, d] tensors (d in {16, 32}, channel stride 1); all view strides
-// must be multiples of 8 elements.
+// Tuned bf16 attention core (d in {16, 32}); all view strides must be multiples of 8 elements.
+// with_apply = false stops after the partial states (at ws + p.partial_off, p.S per head); `out` and `ov` are then unused.
 msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* out, HeadView in, HeadView ov, int B,
-                            int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st);
-
-// bf16 1x1 projection on channel-major activations, tcgen05 tensor cores (gemm_tcgen05.cu):
-// y[b][m][n] = sum_k w[m][k] x[b][k][n] + bias[m]; batch strides in elements.
-bool gemm_bf16_supported(int M, int N, int K);
-msla_status_t run_gemm_bf16(const void* x, const void* w, const void* bias, void* y, int B, int K, int M, int N,
-                            long long x_sb, long long y_sb, cudaStream_t st);
-int gemm_timeout_flag();
-
-// bf16 aggregation on channel-major activations (agg_nchw.cu): TMA halo tiles, depthwise filter as banded matrices
-// on tensor cores, grouped 1x1 on tensor cores.  Batch strides in elements.
-bool aggregate_bf16_supported(int H, int W, int Ch, int d);
-msla_status_t run_aggregate_bf16(const void* src, long long src_sb, const void* w_dw, const void* w_pw, void* dst,
-                                 long long dst_sb, int B, int H, int W, int Ch, int d, cudaStream_t st);
-int agg_timeout_flag();
+                            int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st,
+                            cudaEvent_t mid, bool with_apply);
 
 // Apply step and output projection as one GEMM per image (fused_out.cu): bf16, d in {16, 32}, at most 512 attention
-// channels and 256 output channels.  q: channel-major query planes (channel stride N), head h of image b at
-// q + b*q_sb + h*q_sh.
+// channels and 256 output channels.  q: planar query matrices [N][d], head h of image b at q + b*q_sb + h*q_sh
+// (elements).
 bool fused_out_bf16_supported(int Ht, int d, int Cout, int N);
 size_t fused_out_scratch_bytes(int B, int Ht, int d, int Cout);
 msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, const float* partial, int S, void* scratch,
                                  const void* w, const void* bias, void* y, int B, int Ht, int d, int N, int Cout, float eps,
                                  cudaStream_t st);
 int fused_timeout_flag();
+
+// bf16 projections on tcgen05 tensor cores (gemm_tcgen05.cu).
+bool project_in_bf16_supported(int C, int Cout, int N, int d);
+msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d,
+                                  long long y_batch_stride, cudaStream_t st);
+bool project_out_bf16_supported(int Cin, int Cout, int N);
+msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin, int Cout,
+                                   int N, cudaStream_t st);
+bool project_out_planar_bf16_supported(int Cin, int Cout, int N);
+msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin,
+                                          int Cout, int N, cudaStream_t st);
+int gemm_timeout_flag();
+
+// bf16 aggregation (d = 16 or 32, Ch a multiple of 32): TMA halo tiles, depthwise filter as banded matrices on
+// tensor cores (agg_bf16.cu).  dst_sb must be a multiple of the plane size H*W*d.
+bool aggregate_bf16_supported(int H, int W, int Ch, int d);
+msla_status_t run_aggregate_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
+                                 const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch, int d,
+                                 cudaStream_t st);
+int agg_timeout_flag();
 
 }  // namespace msla
