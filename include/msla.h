@@ -98,8 +98,12 @@ msla_status_t msla_linattn_relu_ws(msla_dtype_t dtype, const void* q, const void
  * is launched.  The call never allocates or frees memory, on host or device.
  *
  * The first call on each device looks up the array's device address (a
- * symbol query, not an allocation); make that first call outside any stream
- * capture.  All calls on a device share the one array, and its contents
+ * symbol query, not an allocation), and the first call for each (device,
+ * dtype, d) loads and configures that variant's kernels, which the driver may
+ * back with device memory of its own: make one warm-up call per (device,
+ * dtype, d) at start-up, outside any stream capture; from then on a call does
+ * no set-up and no allocation.  The looked-up address does not survive
+ * cudaDeviceReset.  All calls on a device share the one array, and its contents
  * persist from call to call, so two calls whose kernels may overlap on the GPU
  * (different streams, no ordering between them) race; order them on one stream
  * or with events. */
@@ -162,7 +166,13 @@ msla_status_t msla_forward(const msla_desc* desc, const void* x, const msla_weig
  * array of n_events = 6 cudaEvent_t handles (as void*): events[0] is recorded
  * on `stream` before step 1 and events[i] after step i (1 projection, 2
  * aggregation, 3 KV-state reduction, 4 apply, 5 output projection; Section
- * 3.1).  Everything else is as for msla_forward. */
+ * 3.1).  When msla_forward_fuses_apply(desc) == 1 steps 4 and 5 are one
+ * kernel: events[3] is then recorded after the first level of the state
+ * reduction (the per-chunk partial states), events[4] directly after it, so
+ * the interval of step 4 is empty and events[4]..events[5] covers the second
+ * level of the state reduction (fixed-order sum of the partial states, folded
+ * into the projection weights) together with apply + projection.  Everything
+ * else is as for msla_forward. */
 msla_status_t msla_forward_profiled(const msla_desc* desc, const void* x, const msla_weights* weights,
                                     void* out, void* stream, void* const* events, int n_events);
 
@@ -195,6 +205,15 @@ unsigned long long msla_kernel_launches(void);
  * SYNCHRONISES the device and returns 1 if that ever happened in this process,
  * 0 if not, -1 if the flag could not be read. */
 int msla_debug_wait_timeouts(void);
+
+/* Diagnostic (no paper counterpart): runs the bounded wait itself on a barrier
+ * that nothing ever arrives at, with a limit of `limit_cycles` SM cycles
+ * (1 .. 2e9, i.e. at most about a second), in a one-warp kernel of its own on
+ * `stream`, and SYNCHRONISES the stream.  `scratch` is device memory for two
+ * ints.  Returns 1 if the wait gave up at the limit and raised the kernel's
+ * abort flag (what every kernel of the library relies on), 0 if not, -1 on a
+ * bad argument or CUDA error.  The context stays usable either way. */
+int msla_debug_wait_selftest(long long limit_cycles, void* scratch, void* stream);
 
 /* Stage entry points (the module's steps 1, 2 and 5 of Section 3.1 on their
  * own), exposed so that each kernel can be checked and timed in isolation.

@@ -55,6 +55,7 @@ EXPORTS = {
     "msla_forward_fuses_apply": (c_int, [ctypes.POINTER(msla_desc)]),
     "msla_kernel_launches": (ctypes.c_ulonglong, []),
     "msla_debug_wait_timeouts": (c_int, []),
+    "msla_debug_wait_selftest": (c_int, [ctypes.c_longlong, c_void_p, c_void_p]),
     "msla_project_in": (c_int, [c_int] + [c_void_p] * 3 + [c_int] * 5 + [c_void_p]),
     "msla_aggregate": (c_int, [c_int] + [c_void_p] * 4 + [c_int] * 5 + [c_void_p]),
     "msla_project_out": (c_int, [c_int] + [c_void_p] * 4 + [c_int] * 4 + [c_void_p]),
@@ -180,6 +181,11 @@ def msla_forward_host(desc: msla_desc, x_host, weights: msla_weights, out_host, 
 
 def msla_debug_wait_timeouts() -> int:
     return lib().msla_debug_wait_timeouts()
+
+
+def msla_debug_wait_selftest(limit_cycles: int, scratch, stream=None) -> int:
+    """Runs the library's bounded wait on a barrier nobody arrives at; 1 = it gave up at the limit."""
+    return lib().msla_debug_wait_selftest(limit_cycles, _ptr(scratch), _stream(stream))
 
 
 def msla_forward_fuses_apply(desc: msla_desc) -> int:

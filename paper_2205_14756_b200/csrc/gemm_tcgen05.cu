@@ -587,6 +587,35 @@ msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const vo
   return launch<false, true>(tmA, tmB, tmO, p, st);
 }
 
+// Self-test of the bounded wait every kernel of the library relies on: one thread waits, with the given cycle
+// limit, on a barrier nothing ever arrives at, and reports how the wait ended.  No product kernel is involved.
+namespace {
+__global__ void wait_selftest_kernel(long long limit_cycles, int* result) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const bool ok = mbar_wait_limit(smem_u32(&bar), 0, &abort_flag, limit_cycles);
+    result[0] = ok ? 0 : 1;     // 1: the wait gave up
+    result[1] = abort_flag;     // and raised the flag the other roles of a kernel poll
+  }
+}
+}  // namespace
+
+// 1 if a wait on a barrier nobody arrives at gave up after `limit_cycles` and raised the abort flag (the expected
+// outcome), 0 if it claimed success, -1 on a CUDA error.  `scratch` is device memory for two ints.
+int run_wait_selftest(long long limit_cycles, int* scratch, cudaStream_t st) {
+  wait_selftest_kernel<<<1, 32, 0, st>>>(limit_cycles, scratch);
+  int host[2] = {-1, -1};
+  if (cudaMemcpyAsync(host, scratch, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaGetLastError();
+    return -1;
+  }
+  return (host[0] == 1 && host[1] == 1) ? 1 : 0;
+}
+
 // Non-zero once any projection GEMM of this process hit a wait time-out (synchronises the device).
 int gemm_timeout_flag() {
   int v = 0;

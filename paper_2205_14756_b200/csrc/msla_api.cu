@@ -504,6 +504,12 @@ int msla_debug_wait_timeouts(void) {
   return (a < 0 || b < 0 || c < 0) ? -1 : (a | b | c);
 }
 
+int msla_debug_wait_selftest(long long limit_cycles, void* scratch, void* stream) {
+  if (limit_cycles < 1 || limit_cycles > 2000000000LL || !scratch) return -1;  // at most about a second
+  if (check_arch() != MSLA_OK) return -1;
+  return run_wait_selftest(limit_cycles, (int*)scratch, (cudaStream_t)stream);
+}
+
 msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d, void* stream) {
   if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");
   if (!x || !w || !y) return fail(MSLA_ERR_INVALID_ARG, "null pointer");

@@ -120,6 +120,7 @@ bool project_out_planar_bf16_supported(int Cin, int Cout, int N);
 msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin,
                                           int Cout, int N, cudaStream_t st);
 int gemm_timeout_flag();
+int run_wait_selftest(long long limit_cycles, int* scratch, cudaStream_t st);
 
 // bf16 aggregation (d = 16 or 32, Ch a multiple of 32): TMA halo tiles, depthwise filter as banded matrices on
 // tensor cores (agg_bf16.cu).  dst_sb must be a multiple of the plane size H*W*d.

@@ -43,35 +43,40 @@ SMALL = [
 def test_small_modules(name, dtype, B, C, H, W, heads, d):
     s = inputs.ModuleShape(name, dtype, B, C, H, W, heads, d, seed=40 + H)
     t = inputs.module_inputs(s)
-    util.assert_close(util.run_module(s, t), _ref(s, t), dtype, name)
+    util.assert_close(util.run_module(s, t), _ref(s, t), dtype, name, block=util.MODULE_BLOCK)
 
 
-def test_module_with_bias_and_different_c_out():
-    s = inputs.ModuleShape("bias", "bf16", 1, 64, 8, 8, 2, 32, seed=77)
+# Output widths and biases that differ from the input's: C_out = 40 (one ragged block of output channels in the fused
+# apply + projection), and two shapes with d = 32 and C_out > 256, which the fused kernel does not take: they run the
+# tensor-core apply step on paired head planes followed by the planar output-projection GEMM (one with a bias, one
+# with a ragged token tile and an odd number of head pairs).
+@pytest.mark.parametrize("B,C,H,W,heads,d,c_out,with_bias,fused", [(1, 64, 8, 8, 2, 32, 40, True, 1),
+                                                                    (2, 64, 8, 16, 2, 32, 264, True, 0),
+                                                                    (1, 64, 12, 20, 3, 32, 320, False, 0),
+                                                                    (1, 64, 16, 16, 4, 16, 72, True, 1)])
+def test_module_with_bias_and_different_c_out(B, C, H, W, heads, d, c_out, with_bias, fused):
+    s = inputs.ModuleShape("cout", "bf16", B, C, H, W, heads, d, seed=77)
     t = inputs.module_inputs(s)
-    t["w_proj"] = inputs.quantise(inputs.normal(77, 9, 40 * 128, 128 ** -0.5).reshape(40, 128), "bf16")
-    bias = inputs.quantise(inputs.normal(77, 10, 40), "bf16")
-    dt = s.dtype
-    x, w_qkv, w_dw, w_pw, w_proj, b = (util.dev(a, dt) for a in (t["x"], t["w_qkv"], t["w_dw"], t["w_pw"], t["w_proj"], bias))
-    desc = binding.make_desc(1, 64, 8, 8, 2, 32, 40, binding.MSLA_BF16)
-    ws = torch.empty(binding.msla_forward_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
-    desc = binding.make_desc(1, 64, 8, 8, 2, 32, 40, binding.MSLA_BF16, workspace=ws)
-    out = torch.empty(1, 40, 8, 8, dtype=torch.bfloat16, device="cuda")
-    binding.msla_forward(desc, x, binding.make_weights(w_qkv, w_dw, w_pw, w_proj, b), out)
-    torch.cuda.synchronize()
-    util.assert_close(util.host(out), _ref(s, t, bias), "bf16", "bias + C_out=40")
+    k = 2 * heads * d
+    t["w_proj"] = inputs.quantise(inputs.normal(77, 9, c_out * k, k ** -0.5).reshape(c_out, k), "bf16")
+    bias = inputs.quantise(inputs.normal(77, 10, c_out), "bf16") if with_bias else None
+    desc = binding.make_desc(B, C, H, W, heads, d, c_out, binding.MSLA_BF16)
+    assert binding.msla_forward_fuses_apply(desc) == fused
+    got = util.run_module(s, t, bias)
+    util.assert_close(got, _ref(s, t, bias), "bf16", f"C_out = {c_out}", block=util.MODULE_BLOCK)
+    assert binding.msla_debug_wait_timeouts() == 0
 
 
 def test_config3_bf16():
     s = inputs.CONFIG3
     t = inputs.module_inputs(s)
-    util.assert_close(util.run_module(s, t), _ref(s, t), "bf16", "config 3")
+    util.assert_close(util.run_module(s, t), _ref(s, t), "bf16", "config 3", block=util.MODULE_BLOCK)
 
 
 def test_config4_bf16():
     s = inputs.CONFIG4
     t = inputs.module_inputs(s)
-    util.assert_close(util.run_module(s, t), _ref(s, t), "bf16", "config 4")
+    util.assert_close(util.run_module(s, t), _ref(s, t), "bf16", "config 4", block=util.MODULE_BLOCK)
 
 
 @pytest.mark.parametrize("idx", [0, 1, 2, 3, 4])
@@ -80,7 +85,7 @@ def test_config5_sweep_bf16(idx):
     262144 tokens) is the shape and launch configuration the benchmark times."""
     s = inputs.CONFIG5[idx]
     t = inputs.module_inputs(s)
-    util.assert_close(util.run_module(s, t), _ref(s, t), "bf16", s.name)
+    util.assert_close(util.run_module(s, t), _ref(s, t), "bf16", s.name, block=util.MODULE_BLOCK)
 
 
 def test_module_is_bitwise_reproducible():
@@ -213,6 +218,19 @@ def test_module_argument_errors_on_device():
     binding.msla_forward(desc, x, weights, out)       # the context is still usable; zeros in, zeros out
     torch.cuda.synchronize()
     assert float(out.float().abs().max()) == 0.0
+
+
+def test_bounded_wait_gives_up_and_leaves_the_context_usable():
+    """The wait every kernel relies on, run on a barrier nobody arrives at with a limit of about a millisecond: it
+    must give up and say so (no product kernel is made to time out), and the library must work afterwards."""
+    scratch = torch.zeros(2, dtype=torch.int32, device="cuda")
+    assert binding.msla_debug_wait_selftest(2_000_000, scratch) == 1
+    assert scratch.tolist() == [1, 1]
+    assert binding.msla_debug_wait_selftest(0, scratch) == -1          # refused: no limit given
+    s = inputs.ModuleShape("after", "bf16", 1, 64, 8, 8, 2, 32, seed=3)
+    t = inputs.module_inputs(s)
+    util.assert_close(util.run_module(s, t), _ref(s, t), "bf16", "forward after the wait self-test")
+    assert binding.msla_debug_wait_timeouts() == 0                     # the self-test does not touch the product kernels' flag
 
 
 def test_no_kernel_wait_timed_out():

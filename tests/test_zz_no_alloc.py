@@ -6,7 +6,9 @@ allocation may block or fail), a plug-in inside a runtime that owns all device
 memory.  msla_linattn_relu_noalloc serves them from a fixed scratch array built
 into the library.  Here it must reproduce the workspace-taking entry point on
 two calls in a row (the second reuses the array with the first call's leftovers
-in it), and must refuse shapes whose scratch does not fit.
+in it), must agree with the CPU oracle like every other entry point, must leave
+the device's free memory untouched once its kernels are warm, and must refuse
+shapes whose scratch does not fit.
 
 Collected last on purpose: a failure here cannot hide the other tests from a
 run that stops at the first failure."""
@@ -15,6 +17,7 @@ import pytest
 import torch
 
 import __graft_entry__  # noqa: F401
+import oracle
 import util
 from paper_2205_14756_b200 import binding, inputs
 
@@ -39,6 +42,26 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row(dtype):
         assert np.all(np.isfinite(got))
         util.assert_close(got, ref, dtype, f"noalloc {dtype} {B}x{heads}x{N}x{d}")
         assert np.array_equal(got, ref), "same kernels and same split: results should be identical"
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_noalloc_matches_the_oracle_and_allocates_nothing(dtype):
+    B, heads, N, d = 2, 3, 3000, 32
+    t = inputs.core_inputs(inputs.CoreShape("noalloc_oracle", dtype, B, heads, N, d, seed=24))
+    q, k, v = (util.dev(t[n], dtype) for n in ("q", "k", "v"))
+    og = util.Guarded(q.numel() * q.element_size())
+    out = og.view(q.dtype, q.shape)
+    binding.msla_linattn_relu_noalloc(util.CODE[dtype], q, k, v, out, B, heads, N, d, 1e-15)   # warm-up: loads the kernels
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    out.fill_(float("nan"))
+    binding.msla_linattn_relu_noalloc(util.CODE[dtype], q, k, v, out, B, heads, N, d, 1e-15)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "a warmed call changed the device's free memory"
+    og.check("noalloc output")
+    util.assert_close(util.host(out), oracle.linattn_relu(t["q"], t["k"], t["v"], 1e-15), dtype, f"noalloc vs oracle {dtype}",
+                      block=util.CORE_BLOCK)
 
 
 def test_noalloc_full_config2_fits():
