@@ -4,13 +4,17 @@
 A step is one whole-module forward (QKV projection, 5x5 aggregation, KV-state
 reduction, apply, output projection; the last two as one kernel where the
 library fuses them) on one seeded synthetic feature map.
-Prints one JSON line (rank 0): `value` is tokens/s of the whole job from CUDA
-events around the timed steps, `stages` the per-step times and algorithmic
-HBM rates from events recorded between the steps, `roofline` the slowest
-step against the measured HBM copy rate, `attention_core` the stand-alone
-core entry point at the workload's head and token counts, `e2e` the same
-metric with pinned host buffers and the copies inside the timed region,
-`cpu_baseline` the fp64 oracle on the host cores.
+Prints one JSON line (rank 0).  The timed region is BLOCKS blocks of `--steps`
+forwards, each block bracketed by CUDA events: `ms_per_step` is the median
+block (`ms_per_step_min/max` the fastest and slowest), `value` tokens/s of the
+whole job from it; `stages` the per-step times and algorithmic HBM rates from
+events recorded between the steps, `roofline` the slowest step against the
+measured HBM copy rate, `attention_core` the stand-alone core entry point at
+the workload's head and token counts, `e2e` the same metric with pinned host
+buffers and the copies inside the timed region, `configs` the other
+configurations (attention core alone, the two feature-map shapes, the
+resolution sweep with its linear fit), `cpu_baseline` the oracle's source
+instantiated in fp32 at -O3 on the host cores.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 """
@@ -39,6 +43,7 @@ STAGES = ("project_in", "aggregate", "kv_state", "apply", "project_out")
 # when the library runs steps 4 and 5 as one kernel (msla_forward_fuses_apply), they are one stage
 STAGES_FUSED = ("project_in", "aggregate", "kv_state", "apply_project")
 FALLBACK_HBM_GBS = 6650.0
+BLOCKS = 7           # timed blocks of --steps forwards; the median block is reported
 
 
 def workload_by_name(name: str) -> inputs.ModuleShape:
@@ -186,6 +191,57 @@ def time_oracle(s: inputs.ModuleShape, side: int, repeats: int = 1) -> tuple:
     return ss.B * ss.N / best, best, ss, oracle.num_threads()
 
 
+def _oracle_f32_lib():
+    """The oracle's own source file, unchanged, compiled a second time with every `double` read as `float` at
+    -O3 -march=native: the fp32 instantiation the CPU baseline is quoted on.  A three-line wrapper includes the
+    system headers first (their `long double` declarations must not see the macro), defines it, and includes the
+    source."""
+    import ctypes
+    import tempfile
+    src = os.path.join(ROOT, "oracle", "msla_oracle.c")
+    tag = f"{os.getuid()}_{int(os.path.getmtime(src))}"
+    out = os.path.join(tempfile.gettempdir(), f"libmsla_oracle_f32_{tag}.so")
+    if not os.path.exists(out):
+        wrap = os.path.join(tempfile.gettempdir(), f"msla_oracle_f32_{tag}_{os.getpid()}.c")
+        with open(wrap, "w") as f:
+            f.write('#include <stddef.h>\n#include <stdlib.h>\n#include <string.h>\n#if defined(_OPENMP)\n#include <omp.h>\n#endif\n'
+                    f'#define double float\n#include "{src}"\n')
+        tmp = out + f".tmp{os.getpid()}"
+        subprocess.run(["gcc", "-O3", "-march=native", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-o", tmp, wrap, "-lm"], check=True)
+        os.replace(tmp, out)
+        os.remove(wrap)
+    lib = ctypes.CDLL(out)
+    fp = ctypes.POINTER(ctypes.c_float)
+    lib.oracle_msla_forward.argtypes = [fp] * 7 + [ctypes.c_int] * 8 + [ctypes.c_float]
+    lib.oracle_msla_forward.restype = ctypes.c_int
+    lib.oracle_num_threads.restype = ctypes.c_int
+    lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
+    return lib, fp
+
+
+def time_oracle_f32(s: inputs.ModuleShape, side: int, threads: int, repeats: int = 3) -> tuple:
+    """Best of `repeats` runs of the fp32 instantiation on a side x side crop of the token grid with `threads`
+    threads (0 = all).  Returns (tokens/s, seconds, threads used)."""
+    lib, fp = _oracle_f32_lib()
+    ss = oracle_sample_shape(s, side)
+    t = inputs.module_inputs(ss)
+    a = {k: np.ascontiguousarray(v, dtype=np.float32) for k, v in t.items()}
+    out = np.empty((ss.B, ss.C_out, ss.H, ss.W), dtype=np.float32)
+    all_threads = lib.oracle_num_threads()
+    lib.oracle_set_num_threads(threads if threads > 0 else all_threads)
+    used = lib.oracle_num_threads()
+    best = float("inf")
+    p = lambda v: v.ctypes.data_as(fp)
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        rc = lib.oracle_msla_forward(p(a["x"]), p(a["w_qkv"]), p(a["w_dw"]), p(a["w_pw"]), p(a["w_proj"]), None, p(out),
+                                     ss.B, ss.C, ss.H, ss.W, ss.heads, ss.d, 5, ss.C_out, ss.eps)
+        best = min(best, time.perf_counter() - t0)
+        assert rc == 0
+    lib.oracle_set_num_threads(all_threads)
+    return ss.B * ss.N / best, best, used
+
+
 def run_reference(args, s: inputs.ModuleShape, rank: int) -> None:
     if rank != 0:
         return
@@ -225,6 +281,7 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=inputs.CONFIG5[-1].name)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the other configurations (the `configs` key)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -281,26 +338,37 @@ def main() -> None:
     if rank == 0:
         sampler.start()
     barrier()
-    launches0 = binding.msla_kernel_launches()
-    ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev_a.record(stream)
-    for i in range(K):
-        binding.msla_forward_profiled(desc, x, weights, out, stream, evs[i])
-    ev_b.record(stream)
-    barrier()
-    launches = binding.msla_kernel_launches() - launches0
-    ms_total = ev_a.elapsed_time(ev_b)
 
-    # The same K steps through msla_forward, i.e. without the event records between the steps,
-    # which lets each kernel's set-up overlap its predecessor's tail.  Reported beside the
-    # headline, not as the headline: the per-step durations above come from the profiled loop.
-    p_a, p_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    p_a.record(stream)
-    for _ in range(K):
-        binding.msla_forward(desc, x, weights, out, stream)
-    p_b.record(stream)
-    barrier()
-    ms_plain = p_a.elapsed_time(p_b)
+    def timed_blocks(call, blocks=BLOCKS, steps=K):
+        """ms of each of `blocks` blocks of `steps` calls (CUDA events on the launching stream around each block)."""
+        res = []
+        for _ in range(blocks):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for i in range(steps):
+                call(i)
+            b.record(stream)
+            barrier()
+            res.append(a.elapsed_time(b))
+        return res
+
+    # Headline: BLOCKS blocks of K forwards with the events between the steps.
+    launches0 = binding.msla_kernel_launches()
+    stage_acc = {name: [] for name in STAGES}
+
+    def profiled(i):
+        binding.msla_forward_profiled(desc, x, weights, out, stream, evs[i])
+
+    ms_blocks = []
+    for _ in range(BLOCKS):
+        ms_blocks += timed_blocks(profiled, blocks=1)
+        for j, name in enumerate(STAGES):
+            stage_acc[name] += [evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(K)]
+    launches = (binding.msla_kernel_launches() - launches0) // BLOCKS   # per block of K steps
+
+    # The same through msla_forward, i.e. without the event records between the steps, which lets each
+    # kernel's set-up overlap its predecessor's tail.  Reported beside the headline, not as the headline.
+    ms_plain_blocks = timed_blocks(lambda i: binding.msla_forward(desc, x, weights, out, stream))
 
     # end to end: pinned host input -> device -> five steps -> host result, every step.
     # (a) one stream: the latency of a single call; (b) three calls in flight on three
@@ -309,13 +377,7 @@ def main() -> None:
     for _ in range(2):
         binding.msla_forward_host(desc, host_x, weights, host_out, stream)
     barrier()
-    e_a, e_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e_a.record(stream)
-    for _ in range(K):
-        binding.msla_forward_host(desc, host_x, weights, host_out, stream)
-    e_b.record(stream)
-    barrier()
-    ms_e2e_serial = e_a.elapsed_time(e_b)
+    ms_e2e_serial_blocks = timed_blocks(lambda i: binding.msla_forward_host(desc, host_x, weights, host_out, stream), blocks=3)
 
     PIPE = 3
     lanes = []
@@ -329,51 +391,99 @@ def main() -> None:
     for st_i, d_i, hx_i, ho_i, _ in lanes:          # warm-up of every lane
         binding.msla_forward_host(d_i, hx_i, weights, ho_i, st_i)
     barrier()
-    e_a, e_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e_a.record(stream)
-    for st_i, *_ in lanes:
-        st_i.wait_event(e_a)
-    for k in range(K):
-        st_i, d_i, hx_i, ho_i, _ = lanes[k % PIPE]
-        binding.msla_forward_host(d_i, hx_i, weights, ho_i, st_i)
-    for st_i, *_ in lanes:
-        done = torch.cuda.Event()
-        done.record(st_i)
-        stream.wait_event(done)
-    e_b.record(stream)
-    barrier()
-    ms_e2e = e_a.elapsed_time(e_b)
+    ms_e2e_blocks = []
+    for _ in range(3):
+        e_a, e_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e_a.record(stream)
+        for st_i, *_ in lanes:
+            st_i.wait_event(e_a)
+        for k in range(K):
+            st_i, d_i, hx_i, ho_i, _ = lanes[k % PIPE]
+            binding.msla_forward_host(d_i, hx_i, weights, ho_i, st_i)
+        for st_i, *_ in lanes:
+            done = torch.cuda.Event()
+            done.record(st_i)
+            stream.wait_event(done)
+        e_b.record(stream)
+        barrier()
+        ms_e2e_blocks.append(e_a.elapsed_time(e_b))
     clocks = sampler.stop() if rank == 0 else None
     del lanes
 
-    # The attention core (steps 3 + 4) on its own entry point, at this workload's head and token counts:
+    med = statistics.median
+
+    def time_core(cs: inputs.CoreShape, blocks=BLOCKS, steps=K):
+        """Stand-alone attention core (steps 3 + 4) on seeded q, k, v: (median ms per call, min, max, bytes)."""
+        ct = inputs.core_inputs(cs)
+        q, k, v = (torch.from_numpy(ct[n]).to("cuda").to(tdt).contiguous() for n in ("q", "k", "v"))
+        o = torch.empty_like(q)
+        nb = binding.msla_linattn_relu_workspace_bytes(cs.B, cs.heads, cs.N, cs.d)
+        cws = torch.empty(nb, dtype=torch.uint8, device="cuda")
+        call = lambda i: binding.msla_linattn_relu_ws(code, q, k, v, o, cs.B, cs.heads, cs.N, cs.d, cs.eps, cws, nb)
+        for i in range(3):
+            call(i)
+        ms = [m / steps for m in timed_blocks(call, blocks=blocks, steps=steps)]
+        return med(ms), min(ms), max(ms), 4 * q.numel() * q.element_size()
+
+    # The attention core on its own entry point, at this workload's head and token counts:
     # in the fused module the apply step has no kernel of its own to time.
     core = None
     if s.dtype == "bf16" and rank == 0:
-        cB, cH, cN, cd = s.B, 2 * s.heads, s.N, s.d
-        q, k, v = (torch.randn(cB, cH, cN, cd, device="cuda").to(tdt) for _ in range(3))
-        o = torch.empty_like(q)
-        nb = binding.msla_linattn_relu_workspace_bytes(cB, cH, cN, cd)
-        cws = torch.empty(nb, dtype=torch.uint8, device="cuda")
-        for _ in range(3):
-            binding.msla_linattn_relu_ws(code, q, k, v, o, cB, cH, cN, cd, s.eps, cws, nb)
-        c_a, c_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        c_a.record(stream)
-        for _ in range(K):
-            binding.msla_linattn_relu_ws(code, q, k, v, o, cB, cH, cN, cd, s.eps, cws, nb)
-        c_b.record(stream)
-        torch.cuda.synchronize()
-        core = (c_a.elapsed_time(c_b) / K, 4 * cB * cH * cN * cd * 2)
-        del q, k, v, o, cws
+        core = time_core(inputs.CoreShape("core_of_workload", "bf16", s.B, 2 * s.heads, s.N, s.d, seed=s.seed))
 
-    ms_total, ms_e2e, ms_e2e_serial, ms_plain = max_over_ranks([ms_total, ms_e2e, ms_e2e_serial, ms_plain], device="cuda")
+    def time_module(ms_shape: inputs.ModuleShape, blocks=5, steps=10):
+        """Plain msla_forward on another configuration: dict with ms per step, tokens/s and module GB/s."""
+        mt = inputs.module_inputs(ms_shape)
+        mdt = torch.float32 if ms_shape.dtype == "f32" else torch.bfloat16
+        mcode = binding.MSLA_F32 if ms_shape.dtype == "f32" else binding.MSLA_BF16
+        mx = torch.from_numpy(mt["x"]).to("cuda").to(mdt).contiguous()
+        mw = [torch.from_numpy(mt[n]).to("cuda").to(mdt).contiguous() for n in ("w_qkv", "w_dw", "w_pw", "w_proj")]
+        mweights = binding.make_weights(*mw)
+        mo = torch.empty(ms_shape.B, ms_shape.C_out, ms_shape.H, ms_shape.W, dtype=mdt, device="cuda")
+        md0 = binding.make_desc(ms_shape.B, ms_shape.C, ms_shape.H, ms_shape.W, ms_shape.heads, ms_shape.d, ms_shape.C_out, mcode, ms_shape.eps)
+        mws = torch.empty(binding.msla_forward_workspace_bytes(md0), dtype=torch.uint8, device="cuda")
+        mdesc = binding.make_desc(ms_shape.B, ms_shape.C, ms_shape.H, ms_shape.W, ms_shape.heads, ms_shape.d, ms_shape.C_out, mcode,
+                                  ms_shape.eps, workspace=mws)
+        call = lambda i: binding.msla_forward(mdesc, mx, mweights, mo, stream)
+        for i in range(3):
+            call(i)
+        ms = [m / steps for m in timed_blocks(call, blocks=blocks, steps=steps)]
+        fused_m = binding.msla_forward_fuses_apply(mdesc) == 1
+        bpt_m = stage_bytes_per_token(ms_shape)
+        names = STAGES_FUSED if fused_m else STAGES
+        mbytes = sum(bpt_m[n] for n in names) * ms_shape.B * ms_shape.N
+        return {"workload": ms_shape.name, "tokens": ms_shape.B * ms_shape.N, "ms": round(med(ms), 5), "ms_min": round(min(ms), 5),
+                "ms_max": round(max(ms), 5), "tokens_per_s": ms_shape.B * ms_shape.N / (med(ms) * 1e-3),
+                "module_GBps": round(mbytes / (med(ms) * 1e-3) / 1e9, 1),
+                "l2": "exceeds L2" if mbytes > 4 * 126e6 else "L2-resident", "steps_4_5_fused": fused_m}
+
+    other = None
+    if rank == 0 and world == 1 and not args.no_configs:
+        other = {}
+        c2 = inputs.CONFIG2
+        m2, lo2, hi2, b2 = time_core(c2, blocks=5, steps=10)
+        other["cfg2_core"] = {"workload": c2.name, "ms": round(m2, 5), "ms_min": round(lo2, 5), "ms_max": round(hi2, 5),
+                              "token_heads_per_s": c2.B * c2.heads * c2.N / (m2 * 1e-3), "GBps": round(b2 / (m2 * 1e-3) / 1e9, 1),
+                              "l2": "L2-resident (134 MB in and out)"}
+        other["cfg3"] = time_module(inputs.CONFIG3)
+        other["cfg4"] = time_module(inputs.CONFIG4)
+        # a bf16, d = 16 sibling of config 1's width at 256 x 256 tokens, 384 channels
+        other["d16_256x256_c384"] = time_module(inputs.ModuleShape("bf16_d16_256x256_c384", "bf16", 1, 384, 256, 256, 24, 16, seed=7))
+        sweep = [time_module(c) for c in inputs.CONFIG5]
+        ns = np.array([c["tokens"] for c in sweep], dtype=np.float64)
+        ts = np.array([c["ms"] for c in sweep], dtype=np.float64) * 1e3
+        slope, icpt = np.polyfit(ns, ts, 1)     # least squares: t [us] = a + b * N
+        other["cfg5_sweep"] = {"points": sweep, "fit_us": {"a_us": round(float(icpt), 2), "b_ns_per_token": round(float(slope) * 1e3, 4),
+                                                           "max_rel_residual": round(float(np.max(np.abs(icpt + slope * ns - ts) / ts)), 3)}}
+
+    ms_total, ms_lo, ms_hi = med(ms_blocks), min(ms_blocks), max(ms_blocks)
+    ms_total, ms_lo, ms_hi, ms_e2e, ms_e2e_serial, ms_plain = max_over_ranks(
+        [ms_total, ms_lo, ms_hi, med(ms_e2e_blocks), med(ms_e2e_serial_blocks), med(ms_plain_blocks)], device="cuda")
 
     if rank == 0:
         fused = binding.msla_forward_fuses_apply(desc) == 1
         stage_names = STAGES_FUSED if fused else STAGES
-        stage_ms = {}
-        for j, name in enumerate(STAGES):
-            stage_ms[name] = statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(K))
+        stage_ms = {name: statistics.mean(v) for name, v in stage_acc.items()}
         if fused:  # the event between steps 4 and 5 falls directly after the one that ends step 3
             stage_ms["apply_project"] = stage_ms.pop("apply") + stage_ms.pop("project_out")
         bpt, fpt = stage_bytes_per_token(s), stage_flops_per_token(s)
@@ -389,8 +499,8 @@ def main() -> None:
         dom = max(stage_names, key=lambda n: stage_ms[n])
         achieved = bpt[dom] * s.B * s.N / (stage_ms[dom] * 1e-3) / 1e9
         if core is not None:
-            core_ms, core_how = core[0], "stand-alone core entry (msla_linattn_relu_ws) on [B, 2*heads, N, d] of this workload"
-            core_gbps = core[1] / (core_ms * 1e-3) / 1e9
+            core_ms, core_how = core[0], "stand-alone core entry (msla_linattn_relu_ws) on seeded [B, 2*heads, N, d] tensors of this workload"
+            core_gbps = core[3] / (core_ms * 1e-3) / 1e9
         else:
             core_ms, core_how = stage_ms["kv_state"] + stage_ms["apply"], "steps 3 + 4 inside the module"
             core_gbps = (bpt["kv_state"] + bpt["apply"]) * s.B * s.N / (core_ms * 1e-3) / 1e9
@@ -407,13 +517,15 @@ def main() -> None:
             roofline["limiter"] = "shared-memory pipe (tile transposition + ldmatrix operand loads) and mma.sync issue rate"
         result = {
             "metric": METRIC, "value": whole_job_value(s.B * s.N, world, ms_total, K), "unit": UNIT, "n_gpus": world, "steps": K,
-            "warmup": W, "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "warmup": W, "ms_per_step": ms_total / K, "ms_per_step_min": ms_lo / K, "ms_per_step_max": ms_hi / K,
+            "timed_blocks": BLOCKS, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if s.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": s.name, "B": s.B, "C": s.C, "H": s.H, "W": s.W, "heads_per_scale": s.heads, "d": s.d,
                        "tokens_per_step_per_gpu": s.B * s.N, "accumulate": "f32",
                        "l2": "inputs and intermediates of one step exceed the 126 MB L2" if
                        module_bytes > 4 * 126e6 else "working set fits L2: numbers are L2-resident",
                        "steps_4_5_fused": fused,
+                       "timing": f"median of {BLOCKS} blocks of {K} steps, CUDA events around each block",
                        "parallelism": f"replicas x{world}, one image per GPU, no collective"},
             "e2e": {"value": whole_job_value(s.B * s.N, world, ms_e2e, K), "unit": UNIT,
                     "h2d_bytes_per_step": s.B * s.C * s.N * e, "d2h_bytes_per_step": s.B * s.C_out * s.N * e,
@@ -427,14 +539,22 @@ def main() -> None:
             "stages": stages,
             "ms_per_step_without_stage_events": round(ms_plain / K, 5),
             "module_GBps": round(module_bytes / (ms_total * 1e-3 / K) / 1e9, 1),
+            "module_GBps_of_the_unfused_21Ce_plan": round(sum(bpt[n] for n in STAGES) * s.B * s.N / (ms_total * 1e-3 / K) / 1e9, 1),
             "clocks": clocks,
         }
+        if core is not None:
+            result["attention_core"]["ms_min"], result["attention_core"]["ms_max"] = round(core[1], 5), round(core[2], 5)
+        if other is not None:
+            result["configs"] = other
         if world == 1 and not args.no_cpu_baseline:
             side = 512 if max(s.H, s.W) >= 512 else max(s.H, s.W)
-            v, sec, ss, cores = time_oracle(s, side)
-            result["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                      "sample": f"{ss.H}x{ss.W} crop of the token grid (same C, heads, d), one pass, "
-                                                f"{sec:.1f} s, fp64 oracle as it stands"}
+            v_all, sec_all, cores = time_oracle_f32(s, side, 0)
+            v_one, sec_one, _ = time_oracle_f32(s, min(side, 128), 1)
+            result["cpu_baseline"] = {"value": v_all, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                      "sample": f"the oracle's source instantiated in fp32 (-Ddouble=float, gcc -O3 -march=native), best of 3: "
+                                                f"{min(side, s.H)}x{min(side, s.W)} crop of the token grid on {cores} threads ({sec_all:.1f} s per pass); "
+                                                f"one thread on a {min(side, 128, s.H)}x{min(side, 128, s.W)} crop: {v_one:.0f} tokens/s ({sec_one:.1f} s per pass)",
+                                      "single_thread_value": v_one}
         print(json.dumps(result))
     if world > 1:
         dist.destroy_process_group()
