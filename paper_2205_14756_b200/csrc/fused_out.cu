@@ -131,15 +131,14 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
 
 // ---------------------------------------------------------------------------
 // Second level of the state reduction (Eq. 3) and the fold of the state into the projection weights.
-// Grid (B * Ht, ceil(Cout / 64)).  partial: [B*Ht][S][d*(d+1)] fp32, entry [a][c], column d = key sum.
+// Grid (B * Ht, ceil(Cout / rows)): a CTA folds `rows` rows of the projection weights with one head's state.  partial: [B*Ht][S][d*(d+1)] fp32, entry [a][c], column d = key sum.
 //   ks[bh][a]            = sum_s partial[bh][s][a][d]
 //   M[b][m][hh*d + a]    = sum_c w[m][hh*d + c] * (sum_s partial[bh][s][a][c])        (bf16, row stride Kp)
 // ---------------------------------------------------------------------------
-constexpr int FOLD_ROWS = 64;
 constexpr int FOLD_THREADS = 1024;
 __global__ void __launch_bounds__(FOLD_THREADS)
 state_fold_kernel(const float* __restrict__ partial, int S, const bf16* __restrict__ w, bf16* __restrict__ M, float* __restrict__ ks,
-                  int Ht, int d, int Cout, int K) {
+                  int Ht, int d, int Cout, int K, int rows) {
   __shared__ float quarter[4][32 * 33];
   __shared__ float st[32 * 33];
   pdl_launch_dependents();
@@ -169,8 +168,8 @@ state_fold_kernel(const float* __restrict__ partial, int S, const bf16* __restri
   __syncthreads();
   if (blockIdx.y == 0)
     for (int a = threadIdx.x; a < d; a += FOLD_THREADS) ks[(long long)bh * d + a] = st[a * d1 + d];
-  const int m0 = blockIdx.y * FOLD_ROWS;
-  for (int idx = threadIdx.x; idx < FOLD_ROWS * d; idx += FOLD_THREADS) {
+  const int m0 = blockIdx.y * rows;
+  for (int idx = threadIdx.x; idx < rows * d; idx += FOLD_THREADS) {
     const int m = m0 + idx / d, a = idx % d;
     if (m >= Cout) break;
     const bf16* wr = w + (long long)m * K + hh * d;
@@ -501,8 +500,12 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   long long pairs = sms / 2;
   if (pairs > tiles) pairs = tiles;
   if (pairs < 1) pairs = 1;
-  launch_pdl(state_fold_kernel, dim3((unsigned)(B * Ht), (unsigned)((Cout + FOLD_ROWS - 1) / FOLD_ROWS)), dim3(FOLD_THREADS), 0, st, partial, S,
-             (const bf16*)w, M, ks, Ht, d, Cout, K);
+  // about one CTA per SM: few heads -> several CTAs per head (each repeats the short sum over the partial states)
+  int fold_chunks = sms / (B * Ht);
+  fold_chunks = fold_chunks < 1 ? 1 : (fold_chunks > 4 ? 4 : fold_chunks);
+  const int fold_rows = (Cout + fold_chunks - 1) / fold_chunks;
+  launch_pdl(state_fold_kernel, dim3((unsigned)(B * Ht), (unsigned)((Cout + fold_rows - 1) / fold_rows)), dim3(FOLD_THREADS), 0, st, partial, S,
+             (const bf16*)w, M, ks, Ht, d, Cout, K, fold_rows);
   if (d == 32) launch_pdl_cluster2(fused_out_kernel<32>, dim3((unsigned)(2 * pairs)), dim3(O_THREADS), (size_t)smem, st, tmM, tmQ, tmO, p);
   else launch_pdl_cluster2(fused_out_kernel<16>, dim3((unsigned)(2 * pairs)), dim3(O_THREADS), (size_t)smem, st, tmM, tmQ, tmO, p);
   count_launches(2);

@@ -299,25 +299,21 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
 // serialise in their L2 slices.  Here a CTA owns one block of output channels
 // for its whole life: that block of the weight matrix (<= 128 KB) is loaded
 // into shared memory once, and only activation tiles stream through a ring.
-//   RES_IS_B = true  (input projection) : B = 256 weight rows resident (K <= 256),
-//                                         A = 128-token x tiles, MN-major, 16 KB stages (5 deep)
-//   RES_IS_B = false (output projection): A = 128 weight rows resident (K <= 512),
-//                                         B = 256-token attention tiles, 32 KB stages (2 deep)
-// CTA c serves weight block c % blocks and the activation tiles c / blocks,
-// c / blocks + workers, ...  Barriers, TMEM use and epilogue are as above.
+// Used for the input projection: B = 256 weight rows resident (K <= 256), A = 128-token x tiles,
+// MN-major, 16 KB stages (5 deep).  CTA c serves weight block c % blocks and the activation
+// tiles c / blocks, c / blocks + workers, ...  Barriers, TMEM use and epilogue are as above.
 // ---------------------------------------------------------------------------
 constexpr int RES_BYTES = 128 * 1024;
 constexpr int WS_RING_BYTES = 80 * 1024;
 constexpr int WS_SMEM_BYTES = RES_BYTES + WS_RING_BYTES + STAGING_BYTES + 256 + 1024;
 constexpr int WS_MAX_STAGES = 6;
 
-template <bool RES_IS_B>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                             const __grid_constant__ CUtensorMap tmO, GemmParams p, int blocks, int workers) {
-  constexpr int STREAM_BYTES = RES_IS_B ? A_STAGE_BYTES : B_STAGE_BYTES;  // one k-slice of the streamed operand
-  constexpr int NSTAGE = WS_RING_BYTES / STREAM_BYTES;                     // 5 or 2
-  constexpr int RES_SLICE = RES_IS_B ? B_STAGE_BYTES : A_STAGE_BYTES;      // one k-slice of the resident operand
+  constexpr int STREAM_BYTES = A_STAGE_BYTES;             // one k-slice of the streamed operand (the x tile)
+  constexpr int NSTAGE = WS_RING_BYTES / STREAM_BYTES;    // 5
+  constexpr int RES_SLICE = B_STAGE_BYTES;                // one k-slice of the resident operand (256 weight rows)
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t res_base = smem_base, ring_base = smem_base + RES_BYTES;
@@ -333,7 +329,7 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int k_iters = (p.K + BK - 1) / BK;
   const int blk = blockIdx.x % blocks, worker = blockIdx.x / blocks;
-  const int stream_per_batch = RES_IS_B ? p.m_tiles : p.n_tiles;
+  const int stream_per_batch = p.m_tiles;
   const int stream_total = p.batches * stream_per_batch;
 
   if (threadIdx.x == 0) {
@@ -365,10 +361,7 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
       // the resident weight block: all k-slices on one barrier
       mbar_expect_tx(res_bar, (uint32_t)(k_iters * RES_SLICE));
-      for (int kb = 0; kb < k_iters; ++kb) {
-        if (RES_IS_B) tma_load_3d(res_base + kb * RES_SLICE, &tmB, res_bar, kb * BK, blk * BN, 0);
-        else          tma_load_3d(res_base + kb * RES_SLICE, &tmA, res_bar, kb * BK, blk * BM, 0);
-      }
+      for (int kb = 0; kb < k_iters; ++kb) tma_load_3d(res_base + kb * RES_SLICE, &tmB, res_bar, kb * BK, blk * BN, 0);
       pdl_wait();  // the streamed operand may come from the previous kernel; the weights above do not
       uint32_t it = 0;
       bool ok = true;
@@ -380,19 +373,16 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
           if (!ok) break;
           const uint32_t dst = ring_base + s * STREAM_BYTES;
           mbar_expect_tx(full_bar + 8 * s, STREAM_BYTES);
-          if (RES_IS_B) {  // x tile: two boxes of 64 tokens x 64 k
-            tma_load_3d(dst, &tmA, full_bar + 8 * s, st * BM, kb * BK, b);
-            tma_load_3d(dst + STREAM_BYTES / 2, &tmA, full_bar + 8 * s, st * BM + 64, kb * BK, b);
-          } else {         // attention tile: one box of 64 k x 256 tokens
-            tma_load_3d(dst, &tmB, full_bar + 8 * s, kb * BK, st * BN, b);
-          }
+          // x tile: two boxes of 64 tokens x 64 k
+          tma_load_3d(dst, &tmA, full_bar + 8 * s, st * BM, kb * BK, b);
+          tma_load_3d(dst + STREAM_BYTES / 2, &tmA, full_bar + 8 * s, st * BM + 64, kb * BK, b);
         }
       }
     }
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((RES_IS_B ? 1u : 0u) << 15) |
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) |
                              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
       uint32_t it = 0, local = 0;
       bool ok = mbar_wait(res_bar, 0, &abort_flag);
@@ -410,14 +400,8 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
           const uint32_t stream = ring_base + s * STREAM_BYTES, res = res_base + kb * RES_SLICE;
 #pragma unroll
           for (int kk = 0; kk < BK / 16; ++kk) {
-            uint64_t ad, bd;
-            if (RES_IS_B) {
-              ad = make_desc(stream + kk * 2048, (A_STAGE_BYTES / 2) >> 4, 1024 >> 4);  // MN-major x tile
-              bd = make_desc(res + kk * 32, 1, 1024 >> 4);
-            } else {
-              ad = make_desc(res + kk * 32, 1, 1024 >> 4);
-              bd = make_desc(stream + kk * 32, 1, 1024 >> 4);
-            }
+            const uint64_t ad = make_desc(stream + kk * 2048, (A_STAGE_BYTES / 2) >> 4, 1024 >> 4);  // MN-major x tile
+            const uint64_t bd = make_desc(res + kk * 32, 1, 1024 >> 4);
             umma_bf16(d_tmem, ad, bd, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
           }
           umma_commit(empty_bar + 8 * s);
@@ -434,7 +418,7 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
     pdl_wait();  // no global write before the previous kernel is done with the output buffer
     for (int si = worker; ok && si < stream_total; si += workers, ++local) {
       const int b = si / stream_per_batch, st = si % stream_per_batch;
-      const int mt = RES_IS_B ? st : blk, nt = RES_IS_B ? blk : st;
+      const int mt = st, nt = blk;
       const uint32_t acc = local & 1, acc_ph = (local >> 1) & 1;
       ok = mbar_wait(tfull_bar + 8 * acc, acc_ph, &abort_flag);
       ok = __all_sync(0xffffffffu, ok);
@@ -472,16 +456,15 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint
   return tma_make_map_bf16(map, base, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
-template <bool A_MN>
 msla_status_t launch_stationary(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO, const GemmParams& p,
                                 int blocks, cudaStream_t st) {
   static std::atomic<unsigned long long> attr_done{0};
-  const msla_status_t as = ensure_smem_attr(attr_done, gemm_bf16_stationary_kernel<A_MN>, WS_SMEM_BYTES);
+  const msla_status_t as = ensure_smem_attr(attr_done, gemm_bf16_stationary_kernel, WS_SMEM_BYTES);
   if (as != MSLA_OK) return as;
-  const long long stream_total = (long long)p.batches * (A_MN ? p.m_tiles : p.n_tiles);
+  const long long stream_total = (long long)p.batches * p.m_tiles;
   long long workers = device_sm_count() / blocks;
   if (workers > stream_total) workers = stream_total;
-  launch_pdl(gemm_bf16_stationary_kernel<A_MN>, dim3((unsigned)(workers * blocks)), dim3(NUM_THREADS), WS_SMEM_BYTES, st, tmA, tmB, tmO, p, blocks, (int)workers);
+  launch_pdl(gemm_bf16_stationary_kernel, dim3((unsigned)(workers * blocks)), dim3(NUM_THREADS), WS_SMEM_BYTES, st, tmA, tmB, tmO, p, blocks, (int)workers);
   count_launches(1);
   return check_launch("projection GEMM (tcgen05, stationary weights)");
 }
@@ -492,7 +475,7 @@ msla_status_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUten
   const int blocks = A_MN ? p.n_tiles : p.m_tiles;
   const int k_iters = (p.K + BK - 1) / BK;
   if (A_MN && k_iters * B_STAGE_BYTES <= RES_BYTES && blocks <= 16 && blocks <= device_sm_count())
-    return launch_stationary<A_MN>(tmA, tmB, tmO, p, blocks, st);
+    return launch_stationary(tmA, tmB, tmO, p, blocks, st);
   static std::atomic<unsigned long long> attr_done{0};
   const msla_status_t as = ensure_smem_attr(attr_done, gemm_bf16_tcgen05_kernel<A_MN, B_PLANAR>, SMEM_BYTES);
   if (as != MSLA_OK) return as;
