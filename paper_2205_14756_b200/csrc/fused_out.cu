@@ -41,7 +41,7 @@ namespace {
 
 using bf16 = __nv_bfloat16;
 
-constexpr int OT = 128;                  // tokens per CTA and tile (256 per pair)
+constexpr int OT = 128;                  // tokens per CTA and tile (256 per pair); 64 where that spreads a small problem over more pairs
 constexpr int OM = 128;                  // output channels per CTA (256 per pair)
 constexpr int OKS = 64;                  // k-extent of one resident slice of M (one 128-byte swizzle span)
 constexpr int O_A_SLICE = OM * OKS * 2;  // 16 KB: 128 rows of M x 64 k
@@ -62,7 +62,8 @@ struct OutParams {
   const bf16* bias;  // [Cout] or nullptr
   int B, N, Cout, Ht, d;
   int kslices;       // 64-wide k-slices of M: ceil(Ht * d / 64)
-  int tiles_per_image, num_tiles;  // tiles of 256 tokens
+  int ot;            // tokens per CTA and tile: 128 or 64
+  int tiles_per_image, num_tiles;  // tiles of 2 * ot tokens
   float eps;
 };
 
@@ -186,7 +187,7 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
   const uint32_t a_base = smem_base;                                  // resident rows of M: kslices x 16 KB
-  constexpr int SLICE = OT * D * 2;                                    // one head's queries of this CTA's 128 tokens
+  constexpr int SLICE = OT * D * 2;                                    // ring slot: one head's queries of this CTA's (up to) 128 tokens
   constexpr int ROWB = D * 2;                                          // bytes per token row = the swizzle span
   const uint32_t ring = a_base + (uint32_t)p.kslices * O_A_SLICE;
   const uint32_t staging = ring + O_STAGES * SLICE;
@@ -259,12 +260,12 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
           for (int ks = 0; ks < p.kslices; ++ks)
             tma_load_3d(a_base + ks * O_A_SLICE, &tmM, res_bar, ks * OKS, (int)rank * OM, b);
         }
-        const int n0 = nt * (2 * OT) + (int)rank * OT;
+        const int n0 = nt * (2 * p.ot) + (int)rank * p.ot;
         for (int h = 0; ok && h < p.Ht; ++h, ++it) {
           const uint32_t s = it % O_STAGES, ph = (it / O_STAGES) & 1;
           ok = mbar_wait_cluster(empty_bar + 8 * s, ph ^ 1, &abort_flag);
           if (!ok) break;
-          mbar_expect_tx(full_bar + 8 * s, SLICE);
+          mbar_expect_tx(full_bar + 8 * s, (uint32_t)(p.ot * ROWB));
           tma_load_4d(ring + s * SLICE, &tmQ, full_bar + 8 * s, 0, n0, h, b);  // rows past the last token are filled with zeros
         }
       }
@@ -273,7 +274,7 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     // ------------------------------------------------------------ MMA issuer (leader) / M hand-shake (peer)
     if (lane == 0) {
       // instruction descriptor: D = f32, A = B = bf16, both K-major, N = 256, M = 256 (pair)
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * p.ot) >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
       const uint32_t peer_res_remote = map_to_cta(peer_res_bar, 0);
       uint32_t it = 0, local = 0, res_ph = 0;
       int cur_b = -1;
@@ -332,6 +333,7 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
       const int b = tile / p.tiles_per_image;
       for (int h = 0; ok && h < p.Ht; ++h, ++it) {
         if ((int)(it & 1) != xg) continue;
+        const bool has_row = (int)row < p.ot;  // with 64-token tiles only the first two warps of a group own rows
         // the head's key sums, fetched before the wait so that their latency hides behind it
         float kk[D];
         const float4* ksp = reinterpret_cast<const float4*>(p.ks + ((long long)b * p.Ht + h) * D);
@@ -345,6 +347,10 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         const uint32_t rbase = ring + s * SLICE + row_off;
+        if (!has_row) {  // warp-uniform
+          if (lane == 0) mbar_arrive_cluster(ready_remote + 8 * s);
+          continue;
+        }
         uint32_t q[D / 2];  // word w = channels 2w (low half), 2w+1 (high half)
 #pragma unroll
         for (int c = 0; c < PCS; ++c)
@@ -391,12 +397,14 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
       const uint32_t taddr = tmem_base + acc * 256 + ((uint32_t)(quarter * 32) << 16);
       uint32_t r[2][32];
       tmem_ld32(taddr, r[0]);
+      const int chunks = (2 * p.ot) / 32;  // the accumulator's columns are the pair's tokens
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
+        if (c >= chunks) break;
         tmem_ld_wait();
-        if (c + 1 < 8) tmem_ld32(taddr + (c + 1) * 32, r[(c + 1) & 1]);  // next chunk streams in meanwhile
+        if (c + 1 < chunks) tmem_ld32(taddr + (c + 1) * 32, r[(c + 1) & 1]);  // next chunk streams in meanwhile
         const uint32_t(&rc)[32] = r[c & 1];
-        const int n0 = nt * (2 * OT) + (c >> 1) * 64;  // first token of the 64-token block
+        const int n0 = nt * (2 * p.ot) + (c >> 1) * 64;  // first token of the 64-token block
         if (n0 >= p.N || row0 >= p.Cout) continue;    // warp-uniform
         if ((c & 1) == 0) {  // the previous block must have been read out of the staging buffer
           if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -464,6 +472,10 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   if (!fused_out_bf16_supported(Ht, d, Cout, N) || q_sb % 8 != 0 || q_sh % 8 != 0)
     return fail(MSLA_ERR_UNSUPPORTED, "fused apply + projection: %d heads of %d channels, %d output channels, %d tokens", Ht, d, Cout, N);
   const int K = Ht * d;
+  // 256-token tiles per pair of CTAs; 128-token tiles for problems so small that half the pairs would have nothing
+  // to do (the larger tile is the more efficient one as soon as every pair has work)
+  const int sms = device_sm_count();
+  const int ot = 2LL * B * ((N + 2 * OT - 1) / (2 * OT)) <= sms / 2 ? OT / 2 : OT;
   bf16* M = (bf16*)scratch;
   float* ks = (float*)((char*)scratch + fused_out_m_bytes(B, Ht, d, Cout));
   CUtensorMap tmM, tmQ, tmO;
@@ -473,7 +485,7 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
     const cuuint32_t bM[3] = {OKS, OM, 1};
     const cuuint64_t dQ[4] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)Ht, (cuuint64_t)B};
     const cuuint64_t sQ[3] = {(cuuint64_t)d * 2, (cuuint64_t)q_sh * 2, (cuuint64_t)q_sb * 2};
-    const cuuint32_t bQ[4] = {(cuuint32_t)d, OT, 1, 1};
+    const cuuint32_t bQ[4] = {(cuuint32_t)d, (cuuint32_t)ot, 1, 1};
     const cuuint64_t dO[3] = {(cuuint64_t)N, (cuuint64_t)Cout, (cuuint64_t)B};
     const cuuint64_t sO[2] = {(cuuint64_t)N * 2, (cuuint64_t)Cout * N * 2};
     const cuuint32_t bO[3] = {64, 32, 1};
@@ -486,7 +498,8 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   p.ks = ks; p.bias = (const bf16*)bias;
   p.B = B; p.N = N; p.Cout = Cout; p.Ht = Ht; p.d = d; p.eps = eps;
   p.kslices = (K + OKS - 1) / OKS;
-  p.tiles_per_image = (N + 2 * OT - 1) / (2 * OT);
+  p.ot = ot;
+  p.tiles_per_image = (N + 2 * ot - 1) / (2 * ot);
   const long long tiles = (long long)B * p.tiles_per_image;
   if (tiles > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many token tiles");
   p.num_tiles = (int)tiles;
@@ -496,7 +509,6 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   msla_status_t s = ensure_smem_attr(attr_done, fused_out_kernel<32>, smem_max);
   if (s == MSLA_OK) s = ensure_smem_attr(attr_done16, fused_out_kernel<16>, smem_max);
   if (s != MSLA_OK) return s;
-  const int sms = device_sm_count();
   long long pairs = sms / 2;
   if (pairs > tiles) pairs = tiles;
   if (pairs < 1) pairs = 1;
