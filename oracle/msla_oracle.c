@@ -66,8 +66,9 @@ void oracle_conv1x1(const double* x, const double* w, const double* bias, double
 }
 
 /*
- * Depthwise k x k convolution used for token aggregation (Section 3.1,
- * "small-kernel depthwise-separable convolutions"; Section 4.1 fixes 5x5).
+ * Depthwise k x k convolution used for token aggregation (last paragraph of
+ * Section 3.1: a depthwise convolution with a small kernel followed by a grouped
+ * 1x1 convolution; Section 4.1 fixes 5x5).
  * Cross-correlation, stride 1, zero padding k/2, output size = input size.
  * x [B, Ch, H, W], w [Ch, k, k] with taps indexed [dy][dx], y [B, Ch, H, W].
  *   y[b,o,r,s] = sum_{dy,dx} w[o,dy,dx] * x[b,o,r+dy-k/2,s+dx-k/2]   (0 outside)

@@ -173,9 +173,17 @@ state_fold_kernel(const float* __restrict__ partial, int S, const bf16* __restri
   for (int idx = threadIdx.x; idx < rows * d; idx += FOLD_THREADS) {
     const int m = m0 + idx / d, a = idx % d;
     if (m >= Cout) break;
-    const bf16* wr = w + (long long)m * K + hh * d;
+    const uint4* wr = reinterpret_cast<const uint4*>(w + (long long)m * K + hh * d);  // 16-byte aligned: K and d are multiples of 8
     float acc = 0.f;
-    for (int c = 0; c < d; ++c) acc = fmaf(__bfloat162float(wr[c]), st[a * d1 + c], acc);
+    for (int c8 = 0; c8 < d / 8; ++c8) {
+      const uint4 v = __ldg(wr + c8);
+      const uint32_t word[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        acc = fmaf(__uint_as_float(word[e] << 16), st[a * d1 + 8 * c8 + 2 * e], acc);
+        acc = fmaf(__uint_as_float(word[e] & 0xffff0000u), st[a * d1 + 8 * c8 + 2 * e + 1], acc);
+      }
+    }
     M[((long long)b * Cout + m) * K + hh * d + a] = __float2bfloat16_rn(acc);
   }
 }
