@@ -87,25 +87,34 @@ def measured_peaks() -> tuple:
     return FALLBACK_HBM_GBS, "fallback"
 
 
-def kernel_source_hash() -> str:
+# Sources that decide each stage's kernels: the recorded DRAM traffic of a stage stays valid while these are unchanged.
+STAGE_SOURCES = {
+    "project_in": ["gemm_tcgen05.cu", "tcgen05_util.cuh", "tma_host.h", "msla_common.cuh"],
+    "aggregate": ["agg_bf16.cu", "tma_host.h", "msla_common.cuh"],
+    "kv_state": ["core_bf16.cu", "msla_common.cuh"],
+    "apply_project": ["fused_out.cu", "tcgen05_util.cuh", "tma_host.h", "msla_common.cuh"],
+}
+
+
+def kernel_source_hash(stage: str) -> str:
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2205_14756_b200", "csrc")
-    for f in sorted(os.listdir(csrc)):
+    for f in STAGE_SOURCES[stage]:
         h.update(open(os.path.join(csrc, f), "rb").read())
     return h.hexdigest()[:16]
 
 
 def recorded_traffic(stage: str, workload: str):
-    """DRAM bytes per launch from the committed ncu capture, or None when the
-    kernels changed since it was taken."""
+    """DRAM bytes per launch of the stage's kernels from the committed ncu capture, or None when the
+    stage's sources changed since it was taken."""
     p = os.path.join(ROOT, "profiles", "dram_traffic.json")
     if not os.path.exists(p):
         return None
     try:
-        rec = json.load(open(p))
-        if rec.get("csrc_hash") != kernel_source_hash():
+        rec = json.load(open(p)).get("bytes_per_launch", {}).get(workload, {}).get(stage)
+        if not rec or rec.get("source_hash") != kernel_source_hash(stage):
             return None
-        return rec.get("bytes_per_launch", {}).get(workload, {}).get(stage)
+        return rec.get("bytes")
     except Exception:
         return None
 
@@ -273,6 +282,67 @@ def run_reference(args, s: inputs.ModuleShape, rank: int) -> None:
     }))
 
 
+def time_token_sharded(s: inputs.ModuleShape, rank: int, world: int, steps: int, warmup: int, blocks: int = BLOCKS):
+    """ms per forward (each block's, max over ranks) of ONE image of shape `s` cut into `world` bands of rows:
+    halo exchange, steps 1-3 on the band, all-gather of the states, steps 4-5 on the band."""
+    import torch
+    import torch.distributed as dist
+    from paper_2205_14756_b200 import sharded
+    t = inputs.module_inputs(s)                       # the same image on every rank; each keeps its own rows
+    tdt = torch.float32 if s.dtype == "f32" else torch.bfloat16
+    r0, r1 = sharded.band_rows(s.H, world, rank)
+    x_band = torch.from_numpy(np.ascontiguousarray(t["x"][:, :, r0:r1])).to("cuda").to(tdt)
+    wt = [torch.from_numpy(t[n]).to("cuda").to(tdt).contiguous() for n in ("w_qkv", "w_dw", "w_pw", "w_proj")]
+    comp = sharded.CudaBandCompute(*wt, heads=s.heads, d=s.d, eps=s.eps)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(warmup, 3)):
+        sharded.sharded_forward(comp, x_band, rank, world)
+    barrier()
+    res = []
+    for _ in range(blocks):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        a.record(stream)
+        for _ in range(steps):
+            sharded.sharded_forward(comp, x_band, rank, world)
+        b.record(stream)
+        barrier()
+        res.append(a.elapsed_time(b) / steps)
+    return max_over_ranks(res, device="cuda")
+
+
+def run_token_sharded(args, s: inputs.ModuleShape, rank: int, world: int) -> None:
+    """`--shard tokens`: strong scaling of one image over the ranks."""
+    import torch
+    from paper_2205_14756_b200 import binding
+    sampler = ClockSampler(torch.cuda.current_device())
+    if rank == 0:
+        sampler.start()
+    ms = time_token_sharded(s, rank, world, args.steps, args.warmup)
+    clocks = sampler.stop() if rank == 0 else None
+    timeouts = binding.msla_debug_wait_timeouts()
+    if timeouts != 0:
+        raise SystemExit(f"a bounded wait inside a kernel ran out on rank {rank} (flag {timeouts})")
+    if rank != 0:
+        return
+    m = statistics.median(ms)
+    print(json.dumps({
+        "metric": METRIC, "value": s.B * s.N / (m * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": m, "ms_per_step_min": min(ms), "ms_per_step_max": max(ms), "timed_blocks": len(ms), "higher_is_better": True,
+        "scaling": "strong", "vs_baseline": None, "dtype": "bf16" if s.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": s.name, "B": s.B, "C": s.C, "H": s.H, "W": s.W, "heads_per_scale": s.heads, "d": s.d,
+                   "tokens_per_step": s.B * s.N,
+                   "parallelism": f"one image in {world} bands of rows; per forward: halo rows of x by send/recv, one all-gather of "
+                                  f"{s.B * 2 * s.heads * s.d * (s.d + 1) * 4} bytes of partial states per rank, summed in band order"},
+        "clocks": clocks}))
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -282,6 +352,9 @@ def main() -> None:
     ap.add_argument("--workload", default=inputs.CONFIG5[-1].name)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-configs", action="store_true", help="skip the other configurations (the `configs` key)")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "tokens"],
+                    help="N > 1: one image per GPU (weak scaling, the default), or ONE image cut into bands of rows over the GPUs "
+                         "(strong scaling: halo rows by send/recv, one all-gather of the partial states)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -305,6 +378,10 @@ def main() -> None:
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    if args.shard == "tokens":
+        run_token_sharded(args, s, rank, world)
+        return
 
     # every rank runs the same-shaped module on its own image (weak scaling, no collective on the data path)
     shape = rank_shape(s, rank)
@@ -469,6 +546,10 @@ def main() -> None:
         other["cfg4"] = time_module(inputs.CONFIG4)
         # a bf16, d = 16 sibling of config 1's width at 256 x 256 tokens, 384 channels
         other["d16_256x256_c384"] = time_module(inputs.ModuleShape("bf16_d16_256x256_c384", "bf16", 1, 384, 256, 256, 24, 16, seed=7))
+        # the token-sharded path's two band calls on one rank (no halo, one state): what the split itself costs
+        band1 = time_token_sharded(s, 0, 1, steps=10, warmup=3, blocks=5)
+        other["band_calls_one_rank"] = {"workload": s.name, "ms": round(med(band1), 5), "ms_min": round(min(band1), 5),
+                                        "ms_max": round(max(band1), 5)}
         sweep = [time_module(c) for c in inputs.CONFIG5]
         ns = np.array([c["tokens"] for c in sweep], dtype=np.float64)
         ts = np.array([c["ms"] for c in sweep], dtype=np.float64) * 1e3

@@ -188,6 +188,39 @@ size_t msla_forward_host_workspace_bytes(const msla_desc* desc);
 msla_status_t msla_forward_host(const msla_desc* desc, const void* x_host, const msla_weights* weights,
                                 void* out_host, void* stream);
 
+/* The module forward cut into bands of image rows, for one image spread over
+ * several GPUs (the module is linear in the token count, Section 3.1, so
+ * high-resolution inputs are where it is used; Eq. 3's two sums over tokens
+ * are the only coupling between the bands besides the 5x5 window of step 2).
+ * Rank r of R holds a run of whole rows of the image.  desc->H counts the rows
+ * of x_band: the band's own rows plus halo_top rows above and halo_bottom rows
+ * below, copies of the neighbouring bands' edge rows of x (2 each, the reach of
+ * the 5x5 aggregation; 0 where the band touches the image border, which is
+ * where step 2 pads with zeros).  desc->workspace, of
+ * msla_forward_workspace_bytes(desc) bytes, carries the band's multi-scale
+ * tokens from the first call to the second and must not be touched in between.
+ *
+ *   msla_band_states: steps 1 and 2 on x_band [B, C, H, W], step 3 on the
+ *     band's own tokens.  state_out: device fp32 [B][2*heads][d][d+1], entry
+ *     [a][c] = sum over the band's tokens of ReLU(k[a])*v[c], column d = sum of
+ *     ReLU(k[a]) (the band's share of Eq. 3's two sums).
+ *   -- the caller gathers the R states into states[R][B][2*heads][d][d+1],
+ *      band 0 first (an all-gather; every rank must hold the same bytes) --
+ *   msla_band_output: adds the R states in band order (a fixed order, so every
+ *     rank forms the same sums bit for bit), then steps 4 and 5 on the band's
+ *     own tokens.  out_band: device [B, C_out, H - halo_top - halo_bottom, W].
+ *
+ * Both calls enqueue on `stream` and return; pointers are device pointers,
+ * 16-byte aligned, caller-owned, and must not overlap one another or the
+ * workspace.  With R = 1 and no halo the pair computes what msla_forward does
+ * (the state is then summed in a different, still fixed, order).  Errors as
+ * for msla_forward; INVALID_ARG if the halos leave no row. */
+msla_status_t msla_band_states(const msla_desc* desc, const void* x_band, const msla_weights* weights,
+                               int halo_top, int halo_bottom, float* state_out, void* stream);
+msla_status_t msla_band_output(const msla_desc* desc, const msla_weights* weights, int halo_top,
+                               int halo_bottom, const float* states, int n_bands, void* out_band,
+                               void* stream);
+
 /* 1 if msla_forward runs steps 4 and 5 of Section 3.1 (apply and output
  * projection) as one kernel for this descriptor, so that the head concat never
  * goes to device memory; 0 if they run as two kernels; -1 on an invalid

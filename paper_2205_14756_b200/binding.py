@@ -52,6 +52,9 @@ EXPORTS = {
                                       ctypes.POINTER(c_void_p), c_int]),
     "msla_forward_host_workspace_bytes": (c_size_t, [ctypes.POINTER(msla_desc)]),
     "msla_forward_host": (c_int, [ctypes.POINTER(msla_desc), c_void_p, ctypes.POINTER(msla_weights), c_void_p, c_void_p]),
+    "msla_band_states": (c_int, [ctypes.POINTER(msla_desc), c_void_p, ctypes.POINTER(msla_weights), c_int, c_int, c_void_p, c_void_p]),
+    "msla_band_output": (c_int, [ctypes.POINTER(msla_desc), ctypes.POINTER(msla_weights), c_int, c_int, c_void_p, c_int, c_void_p,
+                                 c_void_p]),
     "msla_forward_fuses_apply": (c_int, [ctypes.POINTER(msla_desc)]),
     "msla_kernel_launches": (ctypes.c_ulonglong, []),
     "msla_debug_wait_timeouts": (c_int, []),
@@ -177,6 +180,20 @@ def msla_forward_host(desc: msla_desc, x_host, weights: msla_weights, out_host, 
             raise ValueError("msla_forward_host takes contiguous host tensors")
     _check(lib().msla_forward_host(ctypes.byref(desc), x_host.data_ptr(), ctypes.byref(weights), out_host.data_ptr(),
                                    _stream(stream)))
+
+
+def msla_band_states(desc: msla_desc, x_band, weights: msla_weights, halo_top: int, halo_bottom: int, state_out,
+                     stream=None) -> None:
+    """Steps 1-3 on a band of image rows (desc.H = band rows + halos); state_out: fp32 [B, 2*heads, d, d+1]."""
+    _check(lib().msla_band_states(ctypes.byref(desc), _ptr(x_band), ctypes.byref(weights), halo_top, halo_bottom,
+                                  _ptr(state_out), _stream(stream)))
+
+
+def msla_band_output(desc: msla_desc, weights: msla_weights, halo_top: int, halo_bottom: int, states, n_bands: int,
+                     out_band, stream=None) -> None:
+    """Steps 4-5 on the band's own tokens from the gathered states [n_bands, B, 2*heads, d, d+1]."""
+    _check(lib().msla_band_output(ctypes.byref(desc), ctypes.byref(weights), halo_top, halo_bottom, _ptr(states), n_bands,
+                                  _ptr(out_band), _stream(stream)))
 
 
 def msla_debug_wait_timeouts() -> int:

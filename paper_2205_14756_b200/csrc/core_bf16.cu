@@ -368,7 +368,7 @@ apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf
 
 template <int D>
 msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out, HeadView in, HeadView ov, int B,
-                          int heads, int N, float eps, const CorePlan& p, char* ws, cudaStream_t st, cudaEvent_t mid, bool with_apply) {
+                          int heads, int N, float eps, const CorePlan& p, char* ws, cudaStream_t st, cudaEvent_t mid, int phases) {
   // 4 warps per CTA and 4-deep rings in both kernels; two 16-token MMA tiles per FIFO stage of the apply step
   constexpr int KV_WARPS = 4, KV_STAGES = 4, AP_WARPS = 4, AP_STAGES = 4, AP_U = 2;
   const long long BH = (long long)B * heads;
@@ -378,25 +378,30 @@ msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out
   static std::atomic<unsigned long long> attr_done{0};
   const msla_status_t as = ensure_smem_attr(attr_done, kv_state_mma_kernel<D, KV_WARPS, KV_STAGES>, kv_smem);
   if (as != MSLA_OK) return as;
-  launch_pdl(kv_state_mma_kernel<D, KV_WARPS, KV_STAGES>, dim3((unsigned)BH, p.S), dim3(KV_WARPS * 32), kv_smem, st, k, v, partial, in, heads, N, p.S, p.chunk);
-  if (!with_apply) {  // the caller combines the partial states itself
-    if (mid) cudaEventRecord(mid, st);
-    count_launches(1);
-    return check_launch("attention state kernel (bf16)");
+  int launches = 0;
+  if (phases & CORE_STATE) {
+    launch_pdl(kv_state_mma_kernel<D, KV_WARPS, KV_STAGES>, dim3((unsigned)BH, p.S), dim3(KV_WARPS * 32), kv_smem, st, k, v, partial, in, heads, N, p.S, p.chunk);
+    ++launches;
   }
-  const long long total = BH * p.ne;
-  launch_pdl(kv_combine_bf16path_kernel, dim3((unsigned)ceil_div_ll(total, 256)), dim3(256), 0, st, partial, state, p.S, p.ne, total);
+  if (phases & CORE_COMBINE) {
+    const long long total = BH * p.ne;
+    launch_pdl(kv_combine_bf16path_kernel, dim3((unsigned)ceil_div_ll(total, 256)), dim3(256), 0, st, partial, state, p.S, p.ne, total);
+    ++launches;
+  }
   if (mid) cudaEventRecord(mid, st);
-  if (ov.pair) {  // heads is even here, so a pair never straddles two images
-    const int tok_per_cta = p.apply_tokens / 2;
-    launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, true>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)(BH / 2)),
-               dim3(AP_WARPS * 32), 0, st, q, state, out, in, ov, heads, N, eps, tok_per_cta);
-  } else {
-    const int tok_per_cta = p.apply_tokens;
-    launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, false>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)BH),
-               dim3(AP_WARPS * 32), 0, st, q, state, out, in, ov, heads, N, eps, tok_per_cta);
+  if (phases & CORE_APPLY) {
+    if (ov.pair) {  // heads is even here, so a pair never straddles two images
+      const int tok_per_cta = p.apply_tokens / 2;
+      launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, true>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)(BH / 2)),
+                 dim3(AP_WARPS * 32), 0, st, q, state, out, in, ov, heads, N, eps, tok_per_cta);
+    } else {
+      const int tok_per_cta = p.apply_tokens;
+      launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, false>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)BH),
+                 dim3(AP_WARPS * 32), 0, st, q, state, out, in, ov, heads, N, eps, tok_per_cta);
+    }
+    ++launches;
   }
-  count_launches(3);
+  count_launches(launches);
   return check_launch("attention core kernels (bf16)");
 }
 
@@ -404,10 +409,10 @@ msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out
 
 msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* out, HeadView in, HeadView ov, int B,
                             int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st,
-                            cudaEvent_t mid, bool with_apply) {
+                            cudaEvent_t mid, int phases) {
   if (d == 32)
-    return launch_core<32>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid, with_apply);
-  return launch_core<16>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid, with_apply);
+    return launch_core<32>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid, phases);
+  return launch_core<16>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid, phases);
 }
 
 }  // namespace msla

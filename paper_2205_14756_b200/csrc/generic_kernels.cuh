@@ -213,6 +213,17 @@ kv_combine_kernel(const float* __restrict__ partial, float* __restrict__ state, 
   state[idx] = acc;
 }
 
+// Token-sharded forward: state[i] = states[0][i] + states[1][i] + ... over the R bands of the image in band
+// order (Eq. 3's sums over tokens, cut into bands), the same order on every rank.
+__global__ void __launch_bounds__(256)
+band_state_sum_kernel(const float* __restrict__ states, float* __restrict__ state, int R, long long total) {
+  const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (idx >= total) return;
+  float acc = 0.f;
+  for (int r = 0; r < R; ++r) acc += states[(long long)r * total + idx];
+  state[idx] = acc;
+}
+
 // ---------------------------------------------------------------------------
 // Apply step (Eq. 3): out[i,c] = relu(q[i]) . KV[:,c] / (relu(q[i]) . ks + eps),
 // written at channel offset head*d of the output view (head concat).

@@ -113,17 +113,27 @@ static bool core_shape_ok(int B, int heads, int N, int d) {
 template <typename T>
 static msla_status_t run_core_generic(const T* q, const T* k, const T* v, T* out, HeadView in,
                                       HeadView ov, int B, int heads, int N, int d, float eps,
-                                      const CorePlan& p, char* ws, cudaStream_t st, cudaEvent_t mid) {
+                                      const CorePlan& p, char* ws, cudaStream_t st, cudaEvent_t mid, int phases) {
   const long long BH = (long long)B * heads;
   float* partial = reinterpret_cast<float*>(ws + p.partial_off);
   float* state = reinterpret_cast<float*>(ws + p.state_off);
-  generic::kv_partial_kernel<T><<<dim3((unsigned)BH, p.S), 256, 0, st>>>(k, v, partial, in, heads, N, d, p.S, p.chunk);
-  const long long total = BH * p.ne;
-  generic::kv_combine_kernel<<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>(partial, state, p.S, p.ne, total);
+  int launches = 0;
+  if (phases & CORE_STATE) {
+    generic::kv_partial_kernel<T><<<dim3((unsigned)BH, p.S), 256, 0, st>>>(k, v, partial, in, heads, N, d, p.S, p.chunk);
+    ++launches;
+  }
+  if (phases & CORE_COMBINE) {
+    const long long total = BH * p.ne;
+    generic::kv_combine_kernel<<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>(partial, state, p.S, p.ne, total);
+    ++launches;
+  }
   if (mid) cudaEventRecord(mid, st);
-  generic::apply_kernel<T><<<dim3((unsigned)ceil_div_ll(N, 128), (unsigned)BH), 128, 0, st>>>(
-      q, state, out, in, ov, heads, N, d, eps);
-  count_launches(3);
+  if (phases & CORE_APPLY) {
+    generic::apply_kernel<T><<<dim3((unsigned)ceil_div_ll(N, 128), (unsigned)BH), 128, 0, st>>>(
+        q, state, out, in, ov, heads, N, d, eps);
+    ++launches;
+  }
+  count_launches(launches);
   return check_launch("attention core kernels");
 }
 
@@ -132,21 +142,19 @@ static msla_status_t run_core_generic(const T* q, const T* k, const T* v, T* out
 static msla_status_t run_core(msla_dtype_t dtype, const void* q, const void* k, const void* v,
                               void* out, HeadView in, HeadView ov, int B, int heads, int N, int d,
                               float eps, const CorePlan& p, void* ws, cudaStream_t st,
-                              cudaEvent_t mid = nullptr, bool with_apply = true) {
-  if (!with_apply && dtype != MSLA_BF16) return fail(MSLA_ERR_UNSUPPORTED, "the state-only core exists for bf16 only");
+                              cudaEvent_t mid = nullptr, int phases = CORE_ALL) {
   if (ov.pair && (dtype != MSLA_BF16 || (heads & 1)))  // only the bf16 tensor-core kernels write paired planes
     return fail(MSLA_ERR_UNSUPPORTED, "paired output planes need bf16 and an even number of heads");
   if (dtype == MSLA_F32)
     return run_core_generic<float>((const float*)q, (const float*)k, (const float*)v, (float*)out,
-                                   in, ov, B, heads, N, d, eps, p, (char*)ws, st, mid);
+                                   in, ov, B, heads, N, d, eps, p, (char*)ws, st, mid, phases);
   const bool strides_ok = in.batch % 8 == 0 && in.head % 8 == 0 && in.ld % 8 == 0 && ov.batch % 8 == 0 &&
                           ov.head % 8 == 0 && ov.ld % 8 == 0;
-  if (strides_ok) return run_core_bf16(q, k, v, out, in, ov, B, heads, N, d, eps, p, ws, st, mid, with_apply);
-  if (!with_apply) return fail(MSLA_ERR_UNSUPPORTED, "the state-only core needs strides that are multiples of 8 elements");
+  if (strides_ok) return run_core_bf16(q, k, v, out, in, ov, B, heads, N, d, eps, p, ws, st, mid, phases);
   if (ov.pair) return fail(MSLA_ERR_UNSUPPORTED, "paired output planes need strides that are multiples of 8 elements");
   return run_core_generic<__nv_bfloat16>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
                                          (const __nv_bfloat16*)v, (__nv_bfloat16*)out, in, ov, B,
-                                         heads, N, d, eps, p, (char*)ws, st, mid);
+                                         heads, N, d, eps, p, (char*)ws, st, mid, phases);
 }
 
 static msla_status_t core_entry(msla_dtype_t dtype, const void* q, const void* k, const void* v,
@@ -408,7 +416,7 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   // Steps 4 and 5 run as one kernel when it takes the shape: the head concat then stays in shared memory.
   const bool fused = desc->dtype == MSLA_BF16 && fused_out_bf16_supported(2 * heads, d, desc->C_out, N);
   s = run_core(desc->dtype, ms, ms + (size_t)N * d * e, ms + (size_t)2 * N * d * e, att, in, ov, desc->B, 2 * heads, N, d, desc->eps, p.core,
-               ws + p.core_off, st, events ? (cudaEvent_t)events[3] : nullptr, !fused);
+               ws + p.core_off, st, events ? (cudaEvent_t)events[3] : nullptr, fused ? CORE_STATE : CORE_ALL);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 4, st)) != MSLA_OK) return s;
   // 5. output projection back to NCHW
@@ -428,6 +436,112 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
     }
   }
   return MSLA_OK;
+}
+
+// ------------------------------------------------------- token-sharded forward
+// A band is a run of whole image rows; desc->H counts the band's rows plus halo_top rows above and halo_bottom rows
+// below it.  Steps 1 and 2 run on the band with its halo as if it were an image of its own: the 5x5 window of a band
+// row then sees true neighbours inside the image and zero padding only where the halo is absent, i.e. at the image
+// border.  Steps 3 to 5 read the band's own tokens, which are a contiguous range of every [N][d] plane.
+struct BandPlan {
+  ForwardPlan f;
+  CorePlan core;     // split of the band's tokens
+  int Nb;            // tokens of the band
+  long long tok_off; // first band token inside a plane
+};
+
+static msla_status_t validate_band(const msla_desc* desc, int halo_top, int halo_bottom, BandPlan* b) {
+  msla_status_t s = validate_desc(desc, &b->f);
+  if (s != MSLA_OK) return s;
+  if (halo_top < 0 || halo_bottom < 0 || halo_top + halo_bottom >= desc->H)
+    return fail(MSLA_ERR_INVALID_ARG, "halo rows (%d above, %d below) must be >= 0 and leave at least one of the %d rows", halo_top, halo_bottom, desc->H);
+  b->Nb = (desc->H - halo_top - halo_bottom) * desc->W;
+  b->tok_off = (long long)halo_top * desc->W;
+  b->core = make_core_plan((long long)desc->B * 2 * desc->heads, b->Nb, desc->d);
+  if (b->core.bytes > b->f.core.bytes) return fail(MSLA_ERR_WORKSPACE, "band plan exceeds the forward plan");
+  if (!desc->workspace || desc->workspace_bytes < b->f.bytes)
+    return fail(MSLA_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", b->f.bytes, desc->workspace ? desc->workspace_bytes : (size_t)0);
+  if (!aligned16(desc->workspace)) return fail(MSLA_ERR_ALIGNMENT, "workspace must be 16-byte aligned");
+  return MSLA_OK;
+}
+
+static msla_status_t band_states_impl(const msla_desc* desc, const void* x, const msla_weights* w, int halo_top,
+                                      int halo_bottom, float* state_out, cudaStream_t st) {
+  BandPlan b;
+  msla_status_t s = validate_band(desc, halo_top, halo_bottom, &b);
+  if (s != MSLA_OK) return s;
+  if (!x || !w || !state_out) return fail(MSLA_ERR_INVALID_ARG, "null x, weights or state_out");
+  if (!w->w_qkv || !w->w_dw || !w->w_pw) return fail(MSLA_ERR_INVALID_ARG, "null weight pointer");
+  const void* ptrs[] = {x, w->w_qkv, w->w_dw, w->w_pw, state_out};
+  for (const void* ptr : ptrs)
+    if (!aligned16(ptr)) return fail(MSLA_ERR_ALIGNMENT, "all device pointers must be 16-byte aligned");
+  const ForwardPlan& p = b.f;
+  const size_t e = elem_size(desc->dtype);
+  const size_t xb = (size_t)desc->B * desc->C * p.N * e;
+  const size_t sb = (size_t)desc->B * 2 * desc->heads * b.core.ne * sizeof(float);
+  if (overlaps(x, xb, desc->workspace, p.bytes) || overlaps(state_out, sb, desc->workspace, p.bytes) || overlaps(state_out, sb, x, xb))
+    return fail(MSLA_ERR_INVALID_ARG, "x, state_out and the workspace must not overlap");
+  if ((s = check_arch()) != MSLA_OK) return s;
+  char* ws = (char*)desc->workspace;
+  const int Cp = p.Cp, N = p.N, d = desc->d;
+  const long long ms_sb = 6LL * Cp * N;
+  char* ms = ws + p.ms_off;
+  s = run_project_in(desc->dtype, x, w->w_qkv, ms, desc->B, desc->C, 3 * Cp, N, d, ms_sb, st);
+  if (s != MSLA_OK) return s;
+  s = run_aggregate(desc->dtype, ms, w->w_dw, w->w_pw, ms + (size_t)3 * Cp * N * e, desc->B, desc->H, desc->W, 3 * Cp, d, ms_sb, ms_sb, st);
+  if (s != MSLA_OK) return s;
+  const HeadView in{ms_sb, 3LL * N * d, d};
+  const char* q = ms + (size_t)b.tok_off * d * e;
+  s = run_core(desc->dtype, q, q + (size_t)N * d * e, q + (size_t)2 * N * d * e, nullptr, in, in, desc->B, 2 * desc->heads, b.Nb, d, desc->eps,
+               b.core, ws + p.core_off, st, nullptr, CORE_STATE | CORE_COMBINE);
+  if (s != MSLA_OK) return s;
+  const cudaError_t ce = cudaMemcpyAsync(state_out, ws + p.core_off + b.core.state_off, sb, cudaMemcpyDeviceToDevice, st);
+  if (ce != cudaSuccess) {
+    cudaGetLastError();
+    return fail(MSLA_ERR_CUDA, "copy of the band's state: %s", cudaGetErrorString(ce));
+  }
+  return MSLA_OK;
+}
+
+static msla_status_t band_output_impl(const msla_desc* desc, const msla_weights* w, int halo_top, int halo_bottom,
+                                      const float* states, int R, void* out, cudaStream_t st) {
+  BandPlan b;
+  msla_status_t s = validate_band(desc, halo_top, halo_bottom, &b);
+  if (s != MSLA_OK) return s;
+  if (!w || !states || !out) return fail(MSLA_ERR_INVALID_ARG, "null weights, states or out");
+  if (!w->w_proj) return fail(MSLA_ERR_INVALID_ARG, "null weight pointer");
+  if (R < 1 || R > 4096) return fail(MSLA_ERR_INVALID_ARG, "R = %d bands; 1 .. 4096 are accepted", R);
+  const void* ptrs[] = {w->w_proj, w->b_proj, states, out};
+  for (const void* ptr : ptrs)
+    if (ptr && !aligned16(ptr)) return fail(MSLA_ERR_ALIGNMENT, "all device pointers must be 16-byte aligned");
+  const ForwardPlan& p = b.f;
+  const size_t e = elem_size(desc->dtype);
+  const int Cp = p.Cp, N = p.N, Nb = b.Nb, d = desc->d, heads = desc->heads;
+  const long long total = (long long)desc->B * 2 * heads * b.core.ne;
+  const size_t ob = (size_t)desc->B * desc->C_out * Nb * e, sb = (size_t)R * total * sizeof(float);
+  if (overlaps(out, ob, desc->workspace, p.bytes) || overlaps(states, sb, desc->workspace, p.bytes) || overlaps(out, ob, states, sb))
+    return fail(MSLA_ERR_INVALID_ARG, "out, states and the workspace must not overlap");
+  if ((s = check_arch()) != MSLA_OK) return s;
+  char* ws = (char*)desc->workspace;
+  const long long ms_sb = 6LL * Cp * N, ld_att = 2LL * Cp;
+  char* ms = ws + p.ms_off;
+  char* att = ws + p.att_off;
+  float* state = reinterpret_cast<float*>(ws + p.core_off + b.core.state_off);
+  generic::band_state_sum_kernel<<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>(states, state, R, total);
+  count_launches(1);
+  if ((s = check_launch("sum of the bands' states")) != MSLA_OK) return s;
+  const char* q = ms + (size_t)b.tok_off * d * e;
+  if (desc->dtype == MSLA_BF16 && fused_out_bf16_supported(2 * heads, d, desc->C_out, Nb))
+    return run_fused_out_bf16(q, ms_sb, 3LL * N * d, state, 1, att, w->w_proj, w->b_proj, out, desc->B, 2 * heads, d, Nb, desc->C_out, desc->eps, st);
+  const HeadView in{ms_sb, 3LL * N * d, d};
+  const bool att_planar = desc->dtype == MSLA_BF16 && d == 32 && project_out_planar_bf16_supported(2 * Cp, desc->C_out, Nb);
+  const HeadView ov = att_planar ? HeadView{(long long)Nb * ld_att, (long long)Nb * 2 * d, 2 * d, 1}
+                                 : HeadView{(long long)Nb * ld_att, d, ld_att, 0};
+  s = run_core(desc->dtype, q, q + (size_t)N * d * e, q + (size_t)2 * N * d * e, att, in, ov, desc->B, 2 * heads, Nb, d, desc->eps, b.core,
+               ws + p.core_off, st, nullptr, CORE_APPLY);
+  if (s != MSLA_OK) return s;
+  return att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, out, desc->B, 2 * Cp, desc->C_out, Nb, st)
+                    : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out, desc->B, 2 * Cp, desc->C_out, Nb, st);
 }
 
 }  // namespace msla
@@ -489,6 +603,16 @@ size_t msla_forward_host_workspace_bytes(const msla_desc* desc) {
 
 msla_status_t msla_forward_host(const msla_desc* desc, const void* x_host, const msla_weights* w, void* out_host, void* stream) {
   return forward_impl(desc, x_host, w, out_host, (cudaStream_t)stream, nullptr, true);
+}
+
+msla_status_t msla_band_states(const msla_desc* desc, const void* x_band, const msla_weights* w, int halo_top, int halo_bottom,
+                               float* state_out, void* stream) {
+  return band_states_impl(desc, x_band, w, halo_top, halo_bottom, state_out, (cudaStream_t)stream);
+}
+
+msla_status_t msla_band_output(const msla_desc* desc, const msla_weights* w, int halo_top, int halo_bottom, const float* states,
+                               int n_bands, void* out_band, void* stream) {
+  return band_output_impl(desc, w, halo_top, halo_bottom, states, n_bands, out_band, (cudaStream_t)stream);
 }
 
 int msla_forward_fuses_apply(const msla_desc* desc) {

@@ -94,10 +94,12 @@ inline void launch_pdl_cluster2(void (*kernel)(KArgs...), dim3 grid, dim3 block,
 
 struct HeadView;
 // Tuned bf16 attention core (d in {16, 32}); all view strides must be multiples of 8 elements.
-// with_apply = false stops after the partial states (at ws + p.partial_off, p.S per head); `out` and `ov` are then unused.
+// `phases` selects what runs: CORE_STATE the partial states (at ws + p.partial_off, p.S per head), CORE_COMBINE their
+// fixed-order sum (at ws + p.state_off), CORE_APPLY the apply step reading that sum; without CORE_APPLY `out` and `ov` are unused.
+enum : int { CORE_STATE = 1, CORE_COMBINE = 2, CORE_APPLY = 4, CORE_ALL = 7 };
 msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* out, HeadView in, HeadView ov, int B,
                             int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st,
-                            cudaEvent_t mid, bool with_apply);
+                            cudaEvent_t mid, int phases);
 
 // Apply step and output projection as one GEMM per image (fused_out.cu): bf16, d in {16, 32}, at most 512 attention
 // channels and 256 output channels.  q: planar query matrices [N][d], head h of image b at q + b*q_sb + h*q_sh
