@@ -132,59 +132,67 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
 
 // ---------------------------------------------------------------------------
 // Second level of the state reduction (Eq. 3) and the fold of the state into the projection weights.
-// Grid (B * Ht, ceil(Cout / rows)): a CTA folds `rows` rows of the projection weights with one head's state.  partial: [B*Ht][S][d*(d+1)] fp32, entry [a][c], column d = key sum.
+// Grid (B * Ht, chunks): a CTA takes one head and `da` = d / chunks of its key channels a, i.e. `da` consecutive rows of the
+// head's state.  partial: [B*Ht][S][d*(d+1)] fp32, entry [a][c], column d = key sum.
 //   ks[bh][a]            = sum_s partial[bh][s][a][d]
-//   M[b][m][hh*d + a]    = sum_c w[m][hh*d + c] * (sum_s partial[bh][s][a][c])        (bf16, row stride Kp)
+//   M[b][m][hh*d + a]    = sum_c w[m][hh*d + c] * (sum_s partial[bh][s][a][c])        (bf16, row stride K), all m < Cout
+// Fixed summation order: the S partial states are cut into FOLD_RUNS runs of consecutive indices, each run is summed in
+// index order by its own thread, and the run sums are added in run order.  A thread issues all loads of its run
+// (<= 8 vectors of 16 bytes) before the first add, so the kernel pays one round trip to memory, not S.
 // ---------------------------------------------------------------------------
 constexpr int FOLD_THREADS = 1024;
+constexpr int FOLD_RUNS = 8;       // S <= 64: at most 8 partial states per run
 __global__ void __launch_bounds__(FOLD_THREADS)
 state_fold_kernel(const float* __restrict__ partial, int S, const bf16* __restrict__ w, bf16* __restrict__ M, float* __restrict__ ks,
-                  int Ht, int d, int Cout, int K, int rows) {
-  __shared__ float quarter[4][32 * 33];
+                  int Ht, int d, int Cout, int K, int da) {
+  __shared__ float4 run_sum[FOLD_RUNS][32 * 33 / 4];
   __shared__ float st[32 * 33];
   pdl_launch_dependents();
   pdl_wait();  // the partial states come from the previous kernel
   const int bh = blockIdx.x, b = bh / Ht, hh = bh % Ht;
   const int d1 = d + 1, ne = d * d1;
-  const float* sp = partial + (long long)bh * S * ne;
-  // Fixed summation order: the partial states are cut into four runs of consecutive indices, each run is summed in
-  // index order by its own thread (many loads in flight at once), and the four sums are added in run order.
-  for (int item = threadIdx.x; item < 4 * ne; item += FOLD_THREADS) {
-    const int j = item / ne, e = item - j * ne;
-    const int s0 = (int)((long long)S * j / 4), s1 = (int)((long long)S * (j + 1) / 4);
-    float v = 0.f;
-    int s = s0;
-    for (; s + 4 <= s1; s += 4) {
-      float t[4];
+  const int a0 = blockIdx.y * da;
+  const int nq4 = da * d1 / 4;  // this CTA's rows of the state, in 16-byte vectors (da * d1 is a multiple of 4)
+  const float4* sp = reinterpret_cast<const float4*>(partial + (long long)bh * S * ne + a0 * d1);
+  const int ne4 = ne / 4;
+  for (int item = threadIdx.x; item < FOLD_RUNS * nq4; item += FOLD_THREADS) {
+    const int j = item / nq4, e = item - j * nq4;
+    const int s0 = S * j / FOLD_RUNS, s1 = S * (j + 1) / FOLD_RUNS;
+    float4 t[8];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) t[u] = sp[(long long)(s + u) * ne + e];
+    for (int u = 0; u < 8; ++u) t[u] = s0 + u < s1 ? __ldg(sp + (long long)(s0 + u) * ne4 + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 v = t[0];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) v += t[u];
-    }
-    for (; s < s1; ++s) v += sp[(long long)s * ne + e];
-    quarter[j][e] = v;
+    for (int u = 1; u < 8; ++u) { v.x += t[u].x; v.y += t[u].y; v.z += t[u].z; v.w += t[u].w; }
+    run_sum[j][e] = v;
   }
   __syncthreads();
-  for (int e = threadIdx.x; e < ne; e += FOLD_THREADS) st[e] = ((quarter[0][e] + quarter[1][e]) + quarter[2][e]) + quarter[3][e];
+  for (int e = threadIdx.x; e < nq4; e += FOLD_THREADS) {
+    float4 v = run_sum[0][e];
+#pragma unroll
+    for (int j = 1; j < FOLD_RUNS; ++j) { const float4 r = run_sum[j][e]; v.x += r.x; v.y += r.y; v.z += r.z; v.w += r.w; }
+    reinterpret_cast<float4*>(st)[e] = v;  // st[al * d1 + c], al = a - a0
+  }
   __syncthreads();
-  if (blockIdx.y == 0)
-    for (int a = threadIdx.x; a < d; a += FOLD_THREADS) ks[(long long)bh * d + a] = st[a * d1 + d];
-  const int m0 = blockIdx.y * rows;
-  for (int idx = threadIdx.x; idx < rows * d; idx += FOLD_THREADS) {
-    const int m = m0 + idx / d, a = idx % d;
-    if (m >= Cout) break;
+  for (int al = threadIdx.x; al < da; al += FOLD_THREADS) ks[(long long)bh * d + a0 + al] = st[al * d1 + d];
+  for (int idx = threadIdx.x; idx < Cout * da; idx += FOLD_THREADS) {
+    const int m = idx / da, al = idx - m * da;
     const uint4* wr = reinterpret_cast<const uint4*>(w + (long long)m * K + hh * d);  // 16-byte aligned: K and d are multiples of 8
+    uint4 wv[4];
+#pragma unroll
+    for (int c8 = 0; c8 < 4; ++c8) wv[c8] = c8 < d / 8 ? __ldg(wr + c8) : make_uint4(0u, 0u, 0u, 0u);
     float acc = 0.f;
-    for (int c8 = 0; c8 < d / 8; ++c8) {
-      const uint4 v = __ldg(wr + c8);
-      const uint32_t word[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int c8 = 0; c8 < 4; ++c8) {
+      if (c8 >= d / 8) break;
+      const uint32_t word[4] = {wv[c8].x, wv[c8].y, wv[c8].z, wv[c8].w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        acc = fmaf(__uint_as_float(word[e] << 16), st[a * d1 + 8 * c8 + 2 * e], acc);
-        acc = fmaf(__uint_as_float(word[e] & 0xffff0000u), st[a * d1 + 8 * c8 + 2 * e + 1], acc);
+        acc = fmaf(__uint_as_float(word[e] << 16), st[al * d1 + 8 * c8 + 2 * e], acc);
+        acc = fmaf(__uint_as_float(word[e] & 0xffff0000u), st[al * d1 + 8 * c8 + 2 * e + 1], acc);
       }
     }
-    M[((long long)b * Cout + m) * K + hh * d + a] = __float2bfloat16_rn(acc);
+    M[((long long)b * Cout + m) * K + hh * d + a0 + al] = __float2bfloat16_rn(acc);
   }
 }
 
@@ -479,6 +487,7 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
                                  cudaStream_t st) {
   if (!fused_out_bf16_supported(Ht, d, Cout, N) || q_sb % 8 != 0 || q_sh % 8 != 0)
     return fail(MSLA_ERR_UNSUPPORTED, "fused apply + projection: %d heads of %d channels, %d output channels, %d tokens", Ht, d, Cout, N);
+  if (S < 1 || S > 8 * FOLD_RUNS) return fail(MSLA_ERR_UNSUPPORTED, "fused apply + projection: %d partial states per head (1 .. %d)", S, 8 * FOLD_RUNS);
   const int K = Ht * d;
   // 256-token tiles per pair of CTAs; 128-token tiles for problems so small that half the pairs would have nothing
   // to do (the larger tile is the more efficient one as soon as every pair has work)
@@ -520,12 +529,11 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   long long pairs = sms / 2;
   if (pairs > tiles) pairs = tiles;
   if (pairs < 1) pairs = 1;
-  // about one CTA per SM: few heads -> several CTAs per head (each repeats the short sum over the partial states)
+  // about one CTA per SM: few heads -> up to four CTAs per head, each with a share of the head's key channels
   int fold_chunks = sms / (B * Ht);
-  fold_chunks = fold_chunks < 1 ? 1 : (fold_chunks > 4 ? 4 : fold_chunks);
-  const int fold_rows = (Cout + fold_chunks - 1) / fold_chunks;
-  launch_pdl(state_fold_kernel, dim3((unsigned)(B * Ht), (unsigned)((Cout + fold_rows - 1) / fold_rows)), dim3(FOLD_THREADS), 0, st, partial, S,
-             (const bf16*)w, M, ks, Ht, d, Cout, K, fold_rows);
+  fold_chunks = fold_chunks >= 4 ? 4 : (fold_chunks >= 2 ? 2 : 1);
+  launch_pdl(state_fold_kernel, dim3((unsigned)(B * Ht), (unsigned)fold_chunks), dim3(FOLD_THREADS), 0, st, partial, S,
+             (const bf16*)w, M, ks, Ht, d, Cout, K, d / fold_chunks);
   if (d == 32) launch_pdl_cluster2(fused_out_kernel<32>, dim3((unsigned)(2 * pairs)), dim3(O_THREADS), (size_t)smem, st, tmM, tmQ, tmO, p);
   else launch_pdl_cluster2(fused_out_kernel<16>, dim3((unsigned)(2 * pairs)), dim3(O_THREADS), (size_t)smem, st, tmM, tmQ, tmO, p);
   count_launches(2);
