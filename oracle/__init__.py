@@ -54,6 +54,10 @@ def _load() -> ctypes.CDLL:
         lib.oracle_linattn_relu.restype = None
         lib.oracle_msla_forward.argtypes = [_dp] * 7 + [ctypes.c_int] * 8 + [ctypes.c_double]
         lib.oracle_msla_forward.restype = ctypes.c_int
+        lib.oracle_bias_act.argtypes = [_dp, _dp, ctypes.c_int, ctypes.c_int, ctypes.c_long, ctypes.c_int]
+        lib.oracle_bias_act.restype = None
+        lib.oracle_ffn_dwconv.argtypes = [_dp] * 8 + [ctypes.c_int] * 9
+        lib.oracle_ffn_dwconv.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -139,3 +143,41 @@ def msla_forward(x, w_qkv, w_dw, w_pw, w_proj, b_proj=None, *, heads: int, d: in
     if rc != 0:
         raise MemoryError("oracle_msla_forward: scratch allocation failed")
     return out
+
+
+ACT = {"identity": 0, "relu": 1, "hardswish": 2}
+
+
+def bias_act(y, bias=None, act: str = "identity") -> np.ndarray:
+    """act(y + bias[c]) on y [B, Ch, ...spatial]; returns a new array."""
+    y = _f64(y).copy()
+    B, Ch = y.shape[:2]
+    b = None if bias is None else _f64(bias)
+    _load().oracle_bias_act(_p(y), _p(b), B, Ch, int(np.prod(y.shape[2:])), ACT[act])
+    return y
+
+
+def ffn_dwconv(x, w1, w_dw, w2, b1=None, b_dw=None, b2=None, *, act: str = "hardswish", residual: bool = False) -> np.ndarray:
+    """FFN with a depthwise convolution (Section 3.1, Fig. 2 left) on NCHW x [B, C, H, W] -> [B, C_out, H, W]."""
+    x, w1, w_dw, w2 = map(_f64, (x, w1, w_dw, w2))
+    B, C, H, W = x.shape
+    Ch, k, C_out = w1.shape[0], w_dw.shape[-1], w2.shape[0]
+    assert w1.shape == (Ch, C) and w_dw.shape == (Ch, k, k) and k % 2 == 1 and w2.shape == (C_out, Ch)
+    bs = [None if b is None else _f64(b) for b in (b1, b_dw, b2)]
+    out = np.empty((B, C_out, H, W), dtype=np.float64)
+    rc = _load().oracle_ffn_dwconv(_p(x), _p(w1), _p(bs[0]), _p(w_dw), _p(bs[1]), _p(w2), _p(bs[2]), _p(out),
+                                   B, C, Ch, H, W, k, C_out, ACT[act], int(residual))
+    if rc == -2:
+        raise ValueError("residual needs C_out == C")
+    if rc != 0:
+        raise MemoryError("oracle_ffn_dwconv: scratch allocation failed")
+    return out
+
+
+def evit_block(x, msla_w, ffn_w, *, heads: int, d: int, act: str = "hardswish", eps: float = 1e-15) -> np.ndarray:
+    """The building block of Fig. 2 left: y = x + MSLA(x), out = y + FFN+DWConv(y).
+    msla_w: dict with w_qkv, w_dw, w_pw, w_proj, optional b_proj; ffn_w: dict with w1, w_dw, w2, optional b1, b_dw, b2."""
+    y = _f64(x) + msla_forward(x, msla_w["w_qkv"], msla_w["w_dw"], msla_w["w_pw"], msla_w["w_proj"], msla_w.get("b_proj"),
+                               heads=heads, d=d, eps=eps)
+    return ffn_dwconv(y, ffn_w["w1"], ffn_w["w_dw"], ffn_w["w2"], ffn_w.get("b1"), ffn_w.get("b_dw"), ffn_w.get("b2"),
+                      act=act, residual=True)

@@ -228,3 +228,71 @@ int oracle_msla_forward(const double* x, const double* w_qkv, const double* w_dw
   free(qkv); free(dw); free(agg); free(qh); free(kh); free(vh); free(oh); free(att);
   return rc;
 }
+
+/* ------------------------------------------------------------------------
+ * The other half of the EfficientViT building block (Section 3.1, second
+ * paragraph after Eq. 3, and Fig. 2 left): a feed-forward network with a
+ * depthwise convolution inserted into it (FFN+DWConv), which supplies the
+ * local information that ReLU linear attention lacks.  The paper names
+ * neither the expansion ratio, the activation, the kernel of the depthwise
+ * convolution nor the normalisation; all are arguments here.
+ *
+ * Activation applied after the first linear layer and after the depthwise
+ * convolution: 0 identity, 1 ReLU max(a, 0), 2 hard-swish a * min(max(a + 3, 0), 6) / 6
+ * (Howard et al., "Searching for MobileNetV3", Eq. for h-swish).
+ */
+static double ffn_act(double a, int kind) {
+  if (kind == 1) return a > 0.0 ? a : 0.0;
+  if (kind == 2) {
+    double r = a + 3.0;
+    if (r < 0.0) r = 0.0;
+    if (r > 6.0) r = 6.0;
+    return a * r / 6.0;
+  }
+  return a;
+}
+
+/* y[b,c,n] = act(y[b,c,n] + bias[c]), in place; bias [Ch] or NULL. */
+void oracle_bias_act(double* y, const double* bias, int B, int Ch, long N, int act) {
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int b = 0; b < B; ++b)
+    for (int c = 0; c < Ch; ++c) {
+      double* row = y + ((size_t)b * Ch + c) * N;
+      const double bv = bias ? bias[c] : 0.0;
+      for (long n = 0; n < N; ++n) row[n] = ffn_act(row[n] + bv, act);
+    }
+}
+
+/*
+ * FFN+DWConv on an NCHW feature map:
+ *   h   = act(conv1x1(x, w1) + b1)                 C  -> Ch   (the FFN's first linear layer)
+ *   g   = act(dwconv(h, w_dw) + b_dw)              k x k depthwise, zero padding k/2 (the inserted convolution)
+ *   out = conv1x1(g, w2) + b2 (+ x if residual)    Ch -> C_out (the FFN's second linear layer)
+ * x [B, C, H, W], w1 [Ch, C], w_dw [Ch, k, k], w2 [C_out, Ch], biases [.] or NULL (an inference-time folded
+ * normalisation is a bias), out [B, C_out, H, W].  residual != 0 needs C_out == C.
+ * Returns 0, -1 if a scratch allocation fails, -2 on residual with C_out != C.
+ */
+int oracle_ffn_dwconv(const double* x, const double* w1, const double* b1, const double* w_dw,
+                      const double* b_dw, const double* w2, const double* b2, double* out, int B,
+                      int C, int Ch, int H, int W, int k, int C_out, int act, int residual) {
+  if (residual && C_out != C) return -2;
+  const long N = (long)H * W;
+  const size_t hid = (size_t)B * Ch * N;
+  double* h = (double*)malloc(hid * sizeof(double));
+  double* g = (double*)malloc(hid * sizeof(double));
+  int rc = -1;
+  if (h && g) {
+    oracle_conv1x1(x, w1, b1, h, B, C, Ch, N);
+    oracle_bias_act(h, NULL, B, Ch, N, act);
+    oracle_dwconv(h, w_dw, g, B, Ch, H, W, k);
+    oracle_bias_act(g, b_dw, B, Ch, N, act);
+    oracle_conv1x1(g, w2, b2, out, B, Ch, C_out, N);
+    if (residual) {
+      const size_t total = (size_t)B * C * N;
+      for (size_t i = 0; i < total; ++i) out[i] += x[i];
+    }
+    rc = 0;
+  }
+  free(h); free(g);
+  return rc;
+}
