@@ -221,6 +221,66 @@ msla_status_t msla_band_output(const msla_desc* desc, const msla_weights* weight
                                int halo_bottom, const float* states, int n_bands, void* out_band,
                                void* stream);
 
+/* ---------------------------------------------------------------------------
+ * The other half of the building block (Section 3.1, Fig. 2 left): an FFN with
+ * a depthwise convolution inserted into it (FFN+DWConv), which supplies the
+ * local information ReLU linear attention lacks, and the block itself.
+ *
+ *   h   = act(conv1x1(x, w1) + b1)                  C        -> C_hidden
+ *   g   = act(dwconv3x3(h, w_dw) + b_dw)            depthwise, stride 1, zero padding 1, cross-correlation
+ *   out = conv1x1(g, w2) + b2 (+ x if residual)     C_hidden -> C_out
+ *
+ * The paper fixes neither the expansion ratio, the activation nor the
+ * normalisation: they are fields here (a normalisation folded for inference
+ * is a bias).  dw_kernel must be 3.  residual != 0 needs C_out == C.
+ * ------------------------------------------------------------------------- */
+typedef enum {
+  MSLA_ACT_IDENTITY = 0,
+  MSLA_ACT_RELU = 1,      /* max(a, 0) */
+  MSLA_ACT_HARDSWISH = 2  /* a * min(max(a + 3, 0), 6) / 6 */
+} msla_act_t;
+
+typedef struct {
+  uint32_t struct_size;   /* sizeof(msla_ffn_desc) */
+  int B, C, H, W;         /* input x is [B, C, H, W] */
+  int C_hidden;           /* width between the two linear layers */
+  int C_out;
+  int dw_kernel;          /* 3 */
+  msla_act_t act;         /* after the first linear layer and after the depthwise convolution */
+  int residual;           /* != 0: out += x */
+  msla_dtype_t dtype;     /* type of x, out, weights and biases */
+  void* workspace;        /* device scratch, >= msla_ffn_workspace_bytes(desc) */
+  size_t workspace_bytes;
+} msla_ffn_desc;
+
+typedef struct {
+  const void* w1;    /* [C_hidden, C] */
+  const void* b1;    /* [C_hidden] or NULL */
+  const void* w_dw;  /* [C_hidden, 3, 3] taps [dy][dx]; tap reads pixel (row+dy-1, col+dx-1) */
+  const void* b_dw;  /* [C_hidden] or NULL */
+  const void* w2;    /* [C_out, C_hidden] */
+  const void* b2;    /* [C_out] or NULL */
+} msla_ffn_weights;
+
+/* Scratch bytes msla_ffn_dwconv needs (workspace fields ignored); 0 if the
+ * descriptor is invalid or unsupported. */
+size_t msla_ffn_workspace_bytes(const msla_ffn_desc* desc);
+
+/* x: device [B, C, H, W]; out: device [B, C_out, H, W]; out must not overlap x
+ * or the workspace.  C, C_hidden and C_out must be multiples of 8.  Enqueues
+ * on `stream` and returns.  Errors as for msla_forward. */
+msla_status_t msla_ffn_dwconv(const msla_ffn_desc* desc, const void* x, const msla_ffn_weights* weights,
+                              void* out, void* stream);
+
+/* The building block of Fig. 2 left with its two residual connections:
+ *   y = x + MSLA(x)  (msla_forward),   out = y + FFN+DWConv(y)  (msla_ffn_dwconv with residual).
+ * attn and ffn describe the same B, H, W and dtype with attn->C == attn->C_out
+ * == ffn->C == ffn->C_out; each carries its own workspace; `y`, device
+ * [B, C, H, W], receives the intermediate (caller-owned, no overlap with x,
+ * out or the workspaces).  ffn->residual is taken as 1. */
+msla_status_t msla_evit_block(const msla_desc* attn, const msla_weights* attn_weights, const msla_ffn_desc* ffn,
+                              const msla_ffn_weights* ffn_weights, const void* x, void* y, void* out, void* stream);
+
 /* 1 if msla_forward runs steps 4 and 5 of Section 3.1 (apply and output
  * projection) as one kernel for this descriptor, so that the head concat never
  * goes to device memory; 0 if they run as two kernels; -1 on an invalid

@@ -40,6 +40,20 @@ class msla_weights(ctypes.Structure):
                 ("b_proj", c_void_p)]
 
 
+MSLA_ACT_IDENTITY, MSLA_ACT_RELU, MSLA_ACT_HARDSWISH = 0, 1, 2
+
+
+class msla_ffn_desc(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("B", c_int), ("C", c_int), ("H", c_int), ("W", c_int),
+                ("C_hidden", c_int), ("C_out", c_int), ("dw_kernel", c_int), ("act", c_int), ("residual", c_int),
+                ("dtype", c_int), ("workspace", c_void_p), ("workspace_bytes", c_size_t)]
+
+
+class msla_ffn_weights(ctypes.Structure):
+    _fields_ = [("w1", c_void_p), ("b1", c_void_p), ("w_dw", c_void_p), ("b_dw", c_void_p), ("w2", c_void_p),
+                ("b2", c_void_p)]
+
+
 EXPORTS = {
     "msla_linattn_relu": (c_int, [c_void_p] * 4 + [c_int] * 4 + [c_float, c_void_p]),
     "msla_linattn_relu_f32": (c_int, [c_void_p] * 4 + [c_int] * 4 + [c_float, c_void_p]),
@@ -55,6 +69,10 @@ EXPORTS = {
     "msla_band_states": (c_int, [ctypes.POINTER(msla_desc), c_void_p, ctypes.POINTER(msla_weights), c_int, c_int, c_void_p, c_void_p]),
     "msla_band_output": (c_int, [ctypes.POINTER(msla_desc), ctypes.POINTER(msla_weights), c_int, c_int, c_void_p, c_int, c_void_p,
                                  c_void_p]),
+    "msla_ffn_workspace_bytes": (c_size_t, [ctypes.POINTER(msla_ffn_desc)]),
+    "msla_ffn_dwconv": (c_int, [ctypes.POINTER(msla_ffn_desc), c_void_p, ctypes.POINTER(msla_ffn_weights), c_void_p, c_void_p]),
+    "msla_evit_block": (c_int, [ctypes.POINTER(msla_desc), ctypes.POINTER(msla_weights), ctypes.POINTER(msla_ffn_desc),
+                                ctypes.POINTER(msla_ffn_weights), c_void_p, c_void_p, c_void_p, c_void_p]),
     "msla_forward_fuses_apply": (c_int, [ctypes.POINTER(msla_desc)]),
     "msla_kernel_launches": (ctypes.c_ulonglong, []),
     "msla_debug_wait_timeouts": (c_int, []),
@@ -194,6 +212,37 @@ def msla_band_output(desc: msla_desc, weights: msla_weights, halo_top: int, halo
     """Steps 4-5 on the band's own tokens from the gathered states [n_bands, B, 2*heads, d, d+1]."""
     _check(lib().msla_band_output(ctypes.byref(desc), ctypes.byref(weights), halo_top, halo_bottom, _ptr(states), n_bands,
                                   _ptr(out_band), _stream(stream)))
+
+
+def make_ffn_desc(B, C, H, W, C_hidden, C_out, dtype, act=MSLA_ACT_HARDSWISH, residual=False, dw_kernel=3,
+                  workspace: Optional[torch.Tensor] = None) -> msla_ffn_desc:
+    desc = msla_ffn_desc()
+    desc.struct_size = ctypes.sizeof(msla_ffn_desc)
+    desc.B, desc.C, desc.H, desc.W, desc.C_hidden, desc.C_out = B, C, H, W, C_hidden, C_out
+    desc.dw_kernel, desc.act, desc.residual, desc.dtype = dw_kernel, act, int(residual), dtype
+    desc.workspace = _ptr(workspace) if workspace is not None else None
+    desc.workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    return desc
+
+
+def make_ffn_weights(w1, w_dw, w2, b1=None, b_dw=None, b2=None) -> msla_ffn_weights:
+    w = msla_ffn_weights()
+    w.w1, w.b1, w.w_dw, w.b_dw, w.w2, w.b2 = _ptr(w1), _ptr(b1), _ptr(w_dw), _ptr(b_dw), _ptr(w2), _ptr(b2)
+    return w
+
+
+def msla_ffn_workspace_bytes(desc: msla_ffn_desc) -> int:
+    return lib().msla_ffn_workspace_bytes(ctypes.byref(desc))
+
+
+def msla_ffn_dwconv(desc: msla_ffn_desc, x, weights: msla_ffn_weights, out, stream=None) -> None:
+    _check(lib().msla_ffn_dwconv(ctypes.byref(desc), _ptr(x), ctypes.byref(weights), _ptr(out), _stream(stream)))
+
+
+def msla_evit_block(attn: msla_desc, attn_weights: msla_weights, ffn: msla_ffn_desc, ffn_weights: msla_ffn_weights, x, y, out,
+                    stream=None) -> None:
+    _check(lib().msla_evit_block(ctypes.byref(attn), ctypes.byref(attn_weights), ctypes.byref(ffn), ctypes.byref(ffn_weights),
+                                 _ptr(x), _ptr(y), _ptr(out), _stream(stream)))
 
 
 def msla_debug_wait_timeouts() -> int:

@@ -62,7 +62,16 @@ struct GemmParams {
   bf16* out;
   int tma_store;          // 1: epilogue stages 32x32 blocks in shared memory and writes them with TMA (tmO)
   int planes_per_batch;   // planar output: plane coordinate of (batch, n) = batch*planes_per_batch + n/32
+  int plane_shift;        // log2 of the channels per TMA-stored output plane (5: planes of 32, 6: planes of 64)
+  int act;                // applied to accumulator + bias: 0 none, 1 ReLU, 2 hard-swish
+  const bf16* residual;   // nullptr, or a tensor laid out like the row-major output, added after the activation
 };
+
+__device__ __forceinline__ float epilogue_act(float v, int act) {
+  if (act == 1) return fmaxf(v, 0.f);
+  if (act == 2) return v * __saturatef((v + 3.f) * (1.f / 6.f));  // v * min(max(v + 3, 0), 6) / 6
+  return v;
+}
 
 __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& b, int& mt, int& nt) {
   const int per_batch = p.m_tiles * p.n_tiles;
@@ -82,6 +91,8 @@ constexpr int STAGING_BYTES = 8 * 2048;  // one 32-row x 64-byte block per epilo
 // as the TMA unit's 64B mode expects) and written by one TMA store, which
 // emits whole lines and clips rows and columns outside the tensor.  Without a
 // store map (planes of 16 channels) the lane stores its vectors directly.
+// EPI: the epilogue also applies p.act and adds p.residual (compiled out of the plain projections).
+template <bool EPI>
 __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUtensorMap* tmO, uint32_t stage, int b,
                                                   int mt, int nt, uint32_t tmem_acc, int quarter, int col_half, int lane) {
   const int gs = p.group == 32 ? 5 : 4;  // log2(group) when the output is planar
@@ -96,16 +107,29 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUt
   const uint32_t my_row = stage + lane * 64, sw = (uint32_t)((lane >> 1) & 3);
   uint32_t r[2][32];
   tmem_ld32(taddr, r[0]);
+  // residual: the lane's row of the output-shaped tensor, 32 tokens (64 bytes) per chunk, fetched one chunk ahead
+  const bf16* res_row = (EPI && p.residual && row_ok) ? p.residual + (long long)b * p.out_batch_stride + (long long)m * p.ld_out : nullptr;
+  uint4 rs[2][4];
+  auto load_residual = [&](int c) {
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+      const int n = ncol0 + c * 32 + v * 8;
+      rs[c & 1][v] = (res_row && n < p.N) ? __ldg(reinterpret_cast<const uint4*>(res_row + n)) : make_uint4(0u, 0u, 0u, 0u);
+    }
+  };
+  if (EPI && p.residual) load_residual(0);
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
     tmem_ld_wait();
     if (c + 1 < 4) tmem_ld32(taddr + (c + 1) * 32, r[(c + 1) & 1]);  // next chunk streams in while this one is stored
+    if (EPI && p.residual && c + 1 < 4) load_residual(c + 1);
     const uint32_t(&rc)[32] = r[c & 1];
     const int n0 = ncol0 + c * 32;
     if (n0 >= p.N) continue;  // warp-uniform
     uint32_t w[4][4];
 #pragma unroll
-    for (int v = 0; v < 4; ++v)
+    for (int v = 0; v < 4; ++v) {
+      const uint32_t rw[4] = {rs[c & 1][v].x, rs[c & 1][v].y, rs[c & 1][v].z, rs[c & 1][v].w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         float f0 = __uint_as_float(rc[v * 8 + 2 * e]) + bias_row;
@@ -114,8 +138,11 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUt
           f0 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e]);
           f1 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e + 1]);
         }
+        if (EPI && p.act) { f0 = epilogue_act(f0, p.act); f1 = epilogue_act(f1, p.act); }
+        if (EPI && p.residual) { f0 += __uint_as_float(rw[e] << 16); f1 += __uint_as_float(rw[e] & 0xffff0000u); }
         w[v][e] = pack2(f0, f1);
       }
+    }
     if (p.tma_store) {
       // the previous block must have been read out of the staging buffer
       if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -127,7 +154,7 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUt
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) {
-        if (p.group) tma_store_3d(tmO, stage, 0, row0, b * p.planes_per_batch + (n0 >> 5));
+        if (p.group) tma_store_3d(tmO, stage, n0 & ((1 << p.plane_shift) - 1), row0, b * p.planes_per_batch + (n0 >> p.plane_shift));
         else         tma_store_3d(tmO, stage, n0, row0, b);
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       }
@@ -147,7 +174,7 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUt
 
 // B_PLANAR (output projection with the attention output kept as one [N][64]
 // plane per pair of heads): the 64-wide k-slice kb of B is plane kb of the image.
-template <bool A_MN_MAJOR, bool B_PLANAR>
+template <bool A_MN_MAJOR, bool B_PLANAR, bool EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                          const __grid_constant__ CUtensorMap tmO, GemmParams p) {
@@ -269,7 +296,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      drain_accumulator(p, &tmO, staging + (warp - 2) * 2048, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
+      drain_accumulator<EPI>(p, &tmO, staging + (warp - 2) * 2048, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);  // this warp's share of the accumulator is drained
@@ -308,6 +335,7 @@ constexpr int WS_RING_BYTES = 80 * 1024;
 constexpr int WS_SMEM_BYTES = RES_BYTES + WS_RING_BYTES + STAGING_BYTES + 256 + 1024;
 constexpr int WS_MAX_STAGES = 6;
 
+template <bool EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                             const __grid_constant__ CUtensorMap tmO, GemmParams p, int blocks, int workers) {
@@ -424,7 +452,7 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      drain_accumulator(p, &tmO, staging + (warp - 2) * 2048, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
+      drain_accumulator<EPI>(p, &tmO, staging + (warp - 2) * 2048, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);
@@ -456,32 +484,33 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint
   return tma_make_map_bf16(map, base, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
+template <bool EPI>
 msla_status_t launch_stationary(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO, const GemmParams& p,
                                 int blocks, cudaStream_t st) {
   static std::atomic<unsigned long long> attr_done{0};
-  const msla_status_t as = ensure_smem_attr(attr_done, gemm_bf16_stationary_kernel, WS_SMEM_BYTES);
+  const msla_status_t as = ensure_smem_attr(attr_done, gemm_bf16_stationary_kernel<EPI>, WS_SMEM_BYTES);
   if (as != MSLA_OK) return as;
   const long long stream_total = (long long)p.batches * p.m_tiles;
   long long workers = device_sm_count() / blocks;
   if (workers > stream_total) workers = stream_total;
-  launch_pdl(gemm_bf16_stationary_kernel, dim3((unsigned)(workers * blocks)), dim3(NUM_THREADS), WS_SMEM_BYTES, st, tmA, tmB, tmO, p, blocks, (int)workers);
+  launch_pdl(gemm_bf16_stationary_kernel<EPI>, dim3((unsigned)(workers * blocks)), dim3(NUM_THREADS), WS_SMEM_BYTES, st, tmA, tmB, tmO, p, blocks, (int)workers);
   count_launches(1);
   return check_launch("projection GEMM (tcgen05, stationary weights)");
 }
 
-template <bool A_MN, bool B_PLANAR = false>
+template <bool A_MN, bool B_PLANAR = false, bool EPI = false>
 msla_status_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO, const GemmParams& p, cudaStream_t st) {
   // weight-stationary kernel when the CTA's weight block fits its 128 KB of shared memory
   const int blocks = A_MN ? p.n_tiles : p.m_tiles;
   const int k_iters = (p.K + BK - 1) / BK;
   if (A_MN && k_iters * B_STAGE_BYTES <= RES_BYTES && blocks <= 16 && blocks <= device_sm_count())
-    return launch_stationary(tmA, tmB, tmO, p, blocks, st);
+    return launch_stationary<EPI>(tmA, tmB, tmO, p, blocks, st);
   static std::atomic<unsigned long long> attr_done{0};
-  const msla_status_t as = ensure_smem_attr(attr_done, gemm_bf16_tcgen05_kernel<A_MN, B_PLANAR>, SMEM_BYTES);
+  const msla_status_t as = ensure_smem_attr(attr_done, gemm_bf16_tcgen05_kernel<A_MN, B_PLANAR, EPI>, SMEM_BYTES);
   if (as != MSLA_OK) return as;
   const long long tiles = (long long)p.batches * p.m_tiles * p.n_tiles;
   const int grid = (int)(tiles < device_sm_count() ? tiles : device_sm_count());
-  launch_pdl(gemm_bf16_tcgen05_kernel<A_MN, B_PLANAR>, dim3(grid), dim3(NUM_THREADS), SMEM_BYTES, st, tmA, tmB, tmO, p);
+  launch_pdl(gemm_bf16_tcgen05_kernel<A_MN, B_PLANAR, EPI>, dim3(grid), dim3(NUM_THREADS), SMEM_BYTES, st, tmA, tmB, tmO, p);
   count_launches(1);
   return check_launch("projection GEMM (tcgen05)");
 }
@@ -508,7 +537,7 @@ msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, 
   CUtensorMap tmO = tmA;  // placeholder when the direct-store epilogue is used
   const long long plane_elems = (long long)N * 32;
   if (d == 32 && y_sb % plane_elems == 0) {
-    p.tma_store = 1;
+    p.tma_store = 1; p.plane_shift = 5;
     p.planes_per_batch = (int)(y_sb / plane_elems);
     const cuuint64_t dims[3] = {32, (cuuint64_t)N, (cuuint64_t)B * p.planes_per_batch};
     const cuuint64_t strides[2] = {64, (cuuint64_t)N * 64};
@@ -568,6 +597,54 @@ msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const vo
   p.bias = (const bf16*)bias; p.out = (bf16*)y;
   p.tma_store = 1; p.planes_per_batch = planes;
   return launch<false, true>(tmA, tmB, tmO, p, st);
+}
+
+// ---- the two linear layers of the FFN with a depthwise convolution (Section 3.1, Fig. 2 left)
+bool ffn_bf16_supported(int C, int Ch, int Cout, int N) {
+  return C % 8 == 0 && Ch % 64 == 0 && Cout % 8 == 0 && N % 8 == 0;
+}
+
+// First layer: h[b][o / 64][n][o % 64] = act(sum_c w1[o][c] * x[b][c][n] + b1[o]); x NCHW, h planes of 64 channels.
+msla_status_t run_ffn_expand_bf16(const void* x, const void* w1, const void* b1, void* h, int B, int C, int Ch, int N, int act,
+                                  cudaStream_t st) {
+  CUtensorMap tmA, tmB, tmO;
+  const cuuint64_t dims[3] = {64, (cuuint64_t)N, (cuuint64_t)B * (Ch / 64)};
+  const cuuint64_t strides[2] = {128, (cuuint64_t)N * 128};
+  const cuuint32_t box[3] = {32, 32, 1};  // the epilogue's 32-token x 32-channel blocks: half a plane row each
+  if (!make_map(&tmA, x, (uint64_t)N, (uint64_t)C, (uint64_t)B, (uint64_t)N * 2, (uint64_t)C * N * 2, 64, BK) ||
+      !make_map(&tmB, w1, (uint64_t)C, (uint64_t)Ch, 1, (uint64_t)C * 2, (uint64_t)C * Ch * 2, BK, BN) ||
+      !tma_make_map_bf16(&tmO, h, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B))
+    return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the FFN's first layer");
+  GemmParams p{};
+  p.M = N; p.N = Ch; p.K = C; p.batches = B;
+  p.m_tiles = (N + BM - 1) / BM; p.n_tiles = (Ch + BN - 1) / BN;
+  p.out_batch_stride = (long long)Ch * N; p.ld_out = 0; p.group = 32; p.bias_per_row = 0; p.n_fastest = 1;
+  p.bias = (const bf16*)b1; p.out = (bf16*)h;
+  p.tma_store = 1; p.planes_per_batch = Ch / 64; p.plane_shift = 6;
+  p.act = act; p.residual = nullptr;
+  return launch<true, false, true>(tmA, tmB, tmO, p, st);
+}
+
+// Second layer: y[b][m][n] = sum_j w2[m][j] * g[b][j / 64][n][j % 64] + b2[m] (+ residual[b][m][n]); g planes of 64 channels, y NCHW.
+msla_status_t run_ffn_project_bf16(const void* g, const void* w2, const void* b2, const void* residual, void* y, int B, int Ch,
+                                   int Cout, int N, cudaStream_t st) {
+  CUtensorMap tmA, tmB, tmO;
+  const int planes = Ch / 64;
+  const cuuint64_t dO[3] = {(cuuint64_t)N, (cuuint64_t)Cout, (cuuint64_t)B};
+  const cuuint64_t sO[2] = {(cuuint64_t)N * 2, (cuuint64_t)Cout * N * 2};
+  const cuuint32_t bO[3] = {32, 32, 1};
+  if (!make_map(&tmA, w2, (uint64_t)Ch, (uint64_t)Cout, 1, (uint64_t)Ch * 2, (uint64_t)Ch * Cout * 2, BK, BM) ||
+      !make_map(&tmB, g, 64, (uint64_t)N, (uint64_t)B * planes, 128, (uint64_t)N * 128, BK, BN) ||
+      !tma_make_map_bf16(&tmO, y, 3, dO, sO, bO, CU_TENSOR_MAP_SWIZZLE_64B))
+    return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the FFN's second layer");
+  GemmParams p{};
+  p.M = Cout; p.N = N; p.K = Ch; p.batches = B;
+  p.m_tiles = (Cout + BM - 1) / BM; p.n_tiles = (N + BN - 1) / BN;
+  p.out_batch_stride = (long long)Cout * N; p.ld_out = N; p.group = 0; p.bias_per_row = 1; p.n_fastest = 0;
+  p.bias = (const bf16*)b2; p.out = (bf16*)y;
+  p.tma_store = 1; p.planes_per_batch = planes;
+  p.act = 0; p.residual = (const bf16*)residual;
+  return launch<false, true, true>(tmA, tmB, tmO, p, st);
 }
 
 // Self-test of the bounded wait every kernel of the library relies on: one thread waits, with the given cycle

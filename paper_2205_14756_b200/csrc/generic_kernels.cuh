@@ -22,7 +22,15 @@ struct GemmArgs {
   long long sDb, sDm, sDn, sDg;
   int M, Nc, K;  // tokens, out channels, in channels
   int group;     // out channels per plane (>= Nc: one plane)
+  int act;       // applied to the sum + bias: 0 none, 1 ReLU, 2 hard-swish
+  const void* residual;  // nullptr, or a tensor laid out like D, added after the activation
 };
+
+__device__ __forceinline__ float act_f32(float v, int act) {
+  if (act == 1) return fmaxf(v, 0.f);
+  if (act == 2) return v * fminf(fmaxf(v + 3.f, 0.f), 6.f) / 6.f;
+  return v;
+}
 
 template <typename T>
 __global__ void __launch_bounds__(256)
@@ -82,10 +90,47 @@ gemm_kernel(const T* __restrict__ A, const T* __restrict__ Wt, const T* __restri
     for (int j = 0; j < 4; ++j) {
       const int n = n0 + ni + j;
       if (n >= g.Nc) continue;
-      const float r = acc[i][j] + (bias ? to_f32(bias[n]) : 0.f);
-      Db[(long long)(n / g.group) * g.sDg + m * g.sDm + (long long)(n % g.group) * g.sDn] = from_f32<T>(r);
+      float r = act_f32(acc[i][j] + (bias ? to_f32(bias[n]) : 0.f), g.act);
+      const long long at = (long long)(n / g.group) * g.sDg + m * g.sDm + (long long)(n % g.group) * g.sDn;
+      if (g.residual) r += to_f32(static_cast<const T*>(g.residual)[(long long)b * g.sDb + at]);
+      Db[at] = from_f32<T>(r);
     }
   }
+}
+
+// ---------------------------------------------------------------------------
+// The depthwise 3x3 convolution inside the FFN (Section 3.1, Fig. 2 left) with its bias and activation, on NCHW:
+//   g[b,c,y,x] = act(sum_{dy,dx} w[c,dy,dx] * h[b,c,y+dy-1,x+dx-1] + bias[c]), zero padding 1.  One thread per output.
+// ---------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+ffn_dw3x3_nchw_kernel(const T* __restrict__ h, const T* __restrict__ w, const T* __restrict__ bias, T* __restrict__ g,
+                      int Ch, int H, int W, int act, long long total) {
+  const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (idx >= total) return;
+  const int x = (int)(idx % W), y = (int)((idx / W) % H);
+  const long long bc = idx / ((long long)W * H);
+  const int c = (int)(bc % Ch);
+  const T* hp = h + bc * H * W;
+  float acc = bias ? to_f32(bias[c]) : 0.f;
+  for (int dy = 0; dy < 3; ++dy) {
+    const int yy = y + dy - 1;
+    if (yy < 0 || yy >= H) continue;
+    for (int dx = 0; dx < 3; ++dx) {
+      const int xx = x + dx - 1;
+      if (xx < 0 || xx >= W) continue;
+      acc = fmaf(to_f32(w[(long long)c * 9 + dy * 3 + dx]), to_f32(hp[(long long)yy * W + xx]), acc);
+    }
+  }
+  g[idx] = from_f32<T>(act_f32(acc, act));
+}
+
+// y[i] = a[i] + b[i] (the residual connection around the attention module, Fig. 2 left)
+template <typename T>
+__global__ void __launch_bounds__(256)
+add_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ y, long long total) {
+  const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (idx < total) y[idx] = from_f32<T>(to_f32(a[idx]) + to_f32(b[idx]));
 }
 
 // ---------------------------------------------------------------------------

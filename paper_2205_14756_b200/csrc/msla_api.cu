@@ -544,6 +544,113 @@ static msla_status_t band_output_impl(const msla_desc* desc, const msla_weights*
                     : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out, desc->B, 2 * Cp, desc->C_out, Nb, st);
 }
 
+// ---------------------------------------------------------- FFN with a depthwise convolution
+struct FfnPlan {
+  size_t h_off, g_off, bytes;
+  int N;
+  bool tuned;  // bf16 tensor-core path with the hidden tensor as planes of 64 channels
+};
+
+static msla_status_t validate_ffn(const msla_ffn_desc* d, FfnPlan* plan) {
+  if (!d) return fail(MSLA_ERR_INVALID_ARG, "null descriptor");
+  if (d->struct_size != sizeof(msla_ffn_desc)) return fail(MSLA_ERR_INVALID_ARG, "desc.struct_size = %u, expected %zu", d->struct_size, sizeof(msla_ffn_desc));
+  if (d->dtype != MSLA_F32 && d->dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype %d", (int)d->dtype);
+  if (d->B < 1 || d->C < 1 || d->H < 1 || d->W < 1 || d->C_hidden < 1 || d->C_out < 1)
+    return fail(MSLA_ERR_INVALID_ARG, "B, C, H, W, C_hidden, C_out must be positive");
+  if (d->act != MSLA_ACT_IDENTITY && d->act != MSLA_ACT_RELU && d->act != MSLA_ACT_HARDSWISH)
+    return fail(MSLA_ERR_INVALID_ARG, "unknown activation %d", (int)d->act);
+  if (d->dw_kernel != 3) return fail(MSLA_ERR_UNSUPPORTED, "dw_kernel = %d; only the 3x3 depthwise convolution is supported", d->dw_kernel);
+  if (d->residual && d->C_out != d->C) return fail(MSLA_ERR_INVALID_ARG, "the residual connection needs C_out == C (%d, %d)", d->C_out, d->C);
+  if ((long long)d->H * d->W > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "H*W exceeds 2^31-1");
+  if (d->C % 8 != 0 || d->C_hidden % 8 != 0 || d->C_out % 8 != 0) return fail(MSLA_ERR_UNSUPPORTED, "C, C_hidden and C_out must be multiples of 8");
+  if (d->B > 65535) return fail(MSLA_ERR_UNSUPPORTED, "B exceeds 65535");
+  plan->N = d->H * d->W;
+  plan->tuned = d->dtype == MSLA_BF16 && ffn_bf16_supported(d->C, d->C_hidden, d->C_out, plan->N) &&
+                (long long)d->B * (d->C_hidden / 64) <= 65535;
+  const size_t hid = align_up((size_t)d->B * d->C_hidden * plan->N * elem_size(d->dtype), 256);
+  plan->h_off = 0;
+  plan->g_off = hid;
+  plan->bytes = 2 * hid;
+  return MSLA_OK;
+}
+
+static msla_status_t ffn_impl(const msla_ffn_desc* desc, const void* x, const msla_ffn_weights* w, void* out, bool residual,
+                              cudaStream_t st) {
+  FfnPlan p;
+  msla_status_t s = validate_ffn(desc, &p);
+  if (s != MSLA_OK) return s;
+  if (!x || !out || !w) return fail(MSLA_ERR_INVALID_ARG, "null x, out or weights");
+  if (!w->w1 || !w->w_dw || !w->w2) return fail(MSLA_ERR_INVALID_ARG, "null weight pointer");
+  const void* ptrs[] = {x, out, w->w1, w->b1, w->w_dw, w->b_dw, w->w2, w->b2, desc->workspace};
+  for (const void* ptr : ptrs)
+    if (ptr && !aligned16(ptr)) return fail(MSLA_ERR_ALIGNMENT, "all device pointers must be 16-byte aligned");
+  if (!desc->workspace || desc->workspace_bytes < p.bytes)
+    return fail(MSLA_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", p.bytes, desc->workspace ? desc->workspace_bytes : (size_t)0);
+  const size_t e = elem_size(desc->dtype);
+  const int N = p.N, B = desc->B, C = desc->C, Ch = desc->C_hidden, Co = desc->C_out, act = (int)desc->act;
+  const size_t xb = (size_t)B * C * N * e, ob = (size_t)B * Co * N * e;
+  if (overlaps(out, ob, x, xb) || overlaps(out, ob, desc->workspace, p.bytes) || overlaps(x, xb, desc->workspace, p.bytes))
+    return fail(MSLA_ERR_INVALID_ARG, "x, out and the workspace must not overlap");
+  if ((s = check_arch()) != MSLA_OK) return s;
+  char* ws = (char*)desc->workspace;
+  void* h = ws + p.h_off;
+  void* g = ws + p.g_off;
+  const void* res = residual ? x : nullptr;
+  if (p.tuned) {
+    if ((s = run_ffn_expand_bf16(x, w->w1, w->b1, h, B, C, Ch, N, act, st)) != MSLA_OK) return s;
+    if ((s = run_ffn_dw3x3_bf16(h, w->w_dw, w->b_dw, g, B, Ch, desc->H, desc->W, act, st)) != MSLA_OK) return s;
+    return run_ffn_project_bf16(g, w->w2, w->b2, res, out, B, Ch, Co, N, st);
+  }
+  // plain kernels, hidden tensor NCHW
+  generic::GemmArgs g1{(long long)C * N, 1, N, (long long)Ch * N, 1, N, 0, N, Ch, C, Ch, act, nullptr};
+  generic::GemmArgs g2{(long long)Ch * N, 1, N, (long long)Co * N, 1, N, 0, N, Co, Ch, Co, 0, res};
+  const long long total = (long long)B * Ch * N;
+  if (desc->dtype == MSLA_F32) {
+    launch_gemm<float>((const float*)x, (const float*)w->w1, (const float*)w->b1, (float*)h, g1, B, st);
+    generic::ffn_dw3x3_nchw_kernel<float><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const float*)h, (const float*)w->w_dw, (const float*)w->b_dw,
+                                                                                            (float*)g, Ch, desc->H, desc->W, act, total);
+    launch_gemm<float>((const float*)g, (const float*)w->w2, (const float*)w->b2, (float*)out, g2, B, st);
+  } else {
+    using T = __nv_bfloat16;
+    launch_gemm<T>((const T*)x, (const T*)w->w1, (const T*)w->b1, (T*)h, g1, B, st);
+    generic::ffn_dw3x3_nchw_kernel<T><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const T*)h, (const T*)w->w_dw, (const T*)w->b_dw, (T*)g, Ch,
+                                                                                        desc->H, desc->W, act, total);
+    launch_gemm<T>((const T*)g, (const T*)w->w2, (const T*)w->b2, (T*)out, g2, B, st);
+  }
+  count_launches(1);
+  return check_launch("FFN with a depthwise convolution");
+}
+
+static msla_status_t block_impl(const msla_desc* attn, const msla_weights* aw, const msla_ffn_desc* ffn, const msla_ffn_weights* fw,
+                                const void* x, void* y, void* out, cudaStream_t st) {
+  ForwardPlan ap;
+  FfnPlan fp;
+  msla_status_t s = validate_desc(attn, &ap);
+  if (s != MSLA_OK) return s;
+  if ((s = validate_ffn(ffn, &fp)) != MSLA_OK) return s;
+  if (attn->B != ffn->B || attn->H != ffn->H || attn->W != ffn->W || attn->dtype != ffn->dtype)
+    return fail(MSLA_ERR_INVALID_ARG, "the two halves of the block describe different B, H, W or dtype");
+  if (attn->C != attn->C_out || ffn->C != attn->C || ffn->C_out != attn->C)
+    return fail(MSLA_ERR_INVALID_ARG, "the block's residual connections need one channel count throughout (%d, %d, %d, %d)", attn->C, attn->C_out, ffn->C, ffn->C_out);
+  if (!x || !y || !out) return fail(MSLA_ERR_INVALID_ARG, "null x, y or out");
+  if (!aligned16(y)) return fail(MSLA_ERR_ALIGNMENT, "all device pointers must be 16-byte aligned");
+  const size_t bytes = (size_t)attn->B * attn->C * ap.N * elem_size(attn->dtype);
+  if (overlaps(y, bytes, x, bytes) || overlaps(y, bytes, out, bytes) ||
+      (attn->workspace && overlaps(y, bytes, attn->workspace, ap.bytes)) || (ffn->workspace && overlaps(y, bytes, ffn->workspace, fp.bytes)))
+    return fail(MSLA_ERR_INVALID_ARG, "y overlaps x, out or a workspace");
+  // y = MSLA(x), then y += x
+  if ((s = forward_impl(attn, x, aw, y, st, nullptr, false)) != MSLA_OK) return s;
+  const long long total = (long long)attn->B * attn->C * ap.N;
+  if (attn->dtype == MSLA_F32)
+    generic::add_kernel<float><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const float*)y, (const float*)x, (float*)y, total);
+  else
+    generic::add_kernel<__nv_bfloat16><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const __nv_bfloat16*)y, (const __nv_bfloat16*)x,
+                                                                                         (__nv_bfloat16*)y, total);
+  count_launches(1);
+  if ((s = check_launch("residual connection around the attention module")) != MSLA_OK) return s;
+  return ffn_impl(ffn, y, fw, out, true, st);
+}
+
 }  // namespace msla
 
 using namespace msla;
@@ -613,6 +720,21 @@ msla_status_t msla_band_states(const msla_desc* desc, const void* x_band, const 
 msla_status_t msla_band_output(const msla_desc* desc, const msla_weights* w, int halo_top, int halo_bottom, const float* states,
                                int n_bands, void* out_band, void* stream) {
   return band_output_impl(desc, w, halo_top, halo_bottom, states, n_bands, out_band, (cudaStream_t)stream);
+}
+
+size_t msla_ffn_workspace_bytes(const msla_ffn_desc* desc) {
+  FfnPlan p;
+  if (validate_ffn(desc, &p) != MSLA_OK) return 0;
+  return p.bytes;
+}
+
+msla_status_t msla_ffn_dwconv(const msla_ffn_desc* desc, const void* x, const msla_ffn_weights* w, void* out, void* stream) {
+  return ffn_impl(desc, x, w, out, desc && desc->residual, (cudaStream_t)stream);
+}
+
+msla_status_t msla_evit_block(const msla_desc* attn, const msla_weights* aw, const msla_ffn_desc* ffn, const msla_ffn_weights* fw,
+                              const void* x, void* y, void* out, void* stream) {
+  return block_impl(attn, aw, ffn, fw, x, y, out, (cudaStream_t)stream);
 }
 
 int msla_forward_fuses_apply(const msla_desc* desc) {

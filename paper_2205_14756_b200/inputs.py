@@ -172,3 +172,44 @@ def core_inputs(s: CoreShape) -> Dict[str, np.ndarray]:
         name: quantise(normal(s.seed, stream, n).reshape(shape), s.dtype)
         for stream, name in enumerate(("q", "k", "v"))
     }
+
+
+@dataclass(frozen=True)
+class FfnShape:
+    """One FFN with a depthwise convolution on an NCHW feature map (the second half of the building block)."""
+    name: str
+    dtype: str          # 'f32' | 'bf16'
+    B: int
+    C: int
+    H: int
+    W: int
+    C_hidden: int
+    C_out: int
+    seed: int
+
+    @property
+    def N(self) -> int:
+        return self.H * self.W
+
+
+def ffn_inputs(s: FfnShape, biases: bool = True) -> Dict[str, np.ndarray]:
+    """Activations ~ N(0,1); weights ~ N(0, 1/fan_in); biases ~ N(0, 0.25) (a folded normalisation's shift).
+
+    x [B, C, H, W]; w1 [C_hidden, C] fan_in C; w_dw [C_hidden, 3, 3] fan_in 9; w2 [C_out, C_hidden] fan_in C_hidden;
+    b1, b_dw [C_hidden]; b2 [C_out].  Streams 8.. so that a block's two halves draw different numbers under one seed."""
+    shapes = {
+        "x": ((s.B, s.C, s.H, s.W), 1.0),
+        "w1": ((s.C_hidden, s.C), s.C ** -0.5),
+        "w_dw": ((s.C_hidden, 3, 3), 1.0 / 3.0),
+        "w2": ((s.C_out, s.C_hidden), s.C_hidden ** -0.5),
+        "b1": ((s.C_hidden,), 0.5),
+        "b_dw": ((s.C_hidden,), 0.5),
+        "b2": ((s.C_out,), 0.5),
+    }
+    out = {}
+    for stream, (name, (shape, std)) in enumerate(shapes.items()):
+        if not biases and name.startswith("b"):
+            continue
+        n = int(np.prod(shape))
+        out[name] = quantise(normal(s.seed, 8 + stream, n, std).reshape(shape), s.dtype)
+    return out

@@ -144,3 +144,49 @@ def run_module(s: inputs.ModuleShape, t: dict, bias=None) -> np.ndarray:
     wg.check("module workspace")
     og.check("module output")
     return host(out)
+
+
+ACT_CODE = {"identity": 0, "relu": 1, "hardswish": 2}
+
+
+def run_ffn(s: inputs.FfnShape, t: dict, act: str, residual: bool) -> np.ndarray:
+    """GPU FFN+DWConv through the C ABI on host arrays (guarded output and workspace)."""
+    dt = s.dtype
+    d = {k: dev(v, dt) for k, v in t.items()}
+    desc = binding.make_ffn_desc(s.B, s.C, s.H, s.W, s.C_hidden, s.C_out, CODE[dt], ACT_CODE[act], residual)
+    nbytes = binding.msla_ffn_workspace_bytes(desc)
+    assert nbytes > 0
+    wg = Guarded(nbytes)
+    ws = wg.view(torch.float32, (nbytes // 4,))
+    desc = binding.make_ffn_desc(s.B, s.C, s.H, s.W, s.C_hidden, s.C_out, CODE[dt], ACT_CODE[act], residual, workspace=ws)
+    esz = 4 if dt == "f32" else 2
+    og = Guarded(s.B * s.C_out * s.N * esz)
+    out = og.view(TORCH_DTYPE[dt], (s.B, s.C_out, s.H, s.W))
+    w = binding.make_ffn_weights(d["w1"], d["w_dw"], d["w2"], d.get("b1"), d.get("b_dw"), d.get("b2"))
+    binding.msla_ffn_dwconv(desc, d["x"], w, out)
+    torch.cuda.synchronize()
+    wg.check("FFN workspace")
+    og.check("FFN output")
+    return host(out)
+
+
+def run_block(s: inputs.ModuleShape, t: dict, f: dict, c_hidden: int, act: str) -> np.ndarray:
+    """GPU building block (attention module + FFN, two residual connections) through the C ABI."""
+    dt = s.dtype
+    x, w_qkv, w_dw, w_pw, w_proj = (dev(t[n], dt) for n in ("x", "w_qkv", "w_dw", "w_pw", "w_proj"))
+    fd = {k: dev(v, dt) for k, v in f.items() if k != "x"}
+    a0 = binding.make_desc(s.B, s.C, s.H, s.W, s.heads, s.d, s.C, CODE[dt], s.eps)
+    f0 = binding.make_ffn_desc(s.B, s.C, s.H, s.W, c_hidden, s.C, CODE[dt], ACT_CODE[act], True)
+    ag, fg = Guarded(binding.msla_forward_workspace_bytes(a0)), Guarded(binding.msla_ffn_workspace_bytes(f0))
+    adesc = binding.make_desc(s.B, s.C, s.H, s.W, s.heads, s.d, s.C, CODE[dt], s.eps, workspace=ag.view(torch.uint8, (ag.nbytes,), 0))
+    fdesc = binding.make_ffn_desc(s.B, s.C, s.H, s.W, c_hidden, s.C, CODE[dt], ACT_CODE[act], True,
+                                  workspace=fg.view(torch.uint8, (fg.nbytes,), 0))
+    esz = 4 if dt == "f32" else 2
+    yg, og = Guarded(x.numel() * esz), Guarded(x.numel() * esz)
+    y, out = yg.view(TORCH_DTYPE[dt], x.shape), og.view(TORCH_DTYPE[dt], x.shape)
+    binding.msla_evit_block(adesc, binding.make_weights(w_qkv, w_dw, w_pw, w_proj), fdesc,
+                            binding.make_ffn_weights(fd["w1"], fd["w_dw"], fd["w2"], fd.get("b1"), fd.get("b_dw"), fd.get("b2")), x, y, out)
+    torch.cuda.synchronize()
+    for gd, what in ((ag, "attention workspace"), (fg, "FFN workspace"), (yg, "y"), (og, "block output")):
+        gd.check(what)
+    return host(out)
