@@ -534,6 +534,42 @@ def main() -> None:
                 "module_GBps": round(mbytes / (med(ms) * 1e-3) / 1e9, 1),
                 "l2": "exceeds L2" if mbytes > 4 * 126e6 else "L2-resident", "steps_4_5_fused": fused_m}
 
+    def time_ffn_block(ms_shape: inputs.ModuleShape, c_hidden: int, blocks=5, steps=5):
+        """The other half of the building block at this workload's shape: FFN+DWConv alone (hard-swish, biases,
+        residual) and the whole block (attention module + FFN, both residual connections)."""
+        fs = inputs.FfnShape(f"ffn_{ms_shape.name}", ms_shape.dtype, ms_shape.B, ms_shape.C, ms_shape.H, ms_shape.W, c_hidden, ms_shape.C,
+                             seed=ms_shape.seed)
+        ft = inputs.ffn_inputs(fs)
+        mt = inputs.module_inputs(ms_shape)
+        mdt = torch.float32 if ms_shape.dtype == "f32" else torch.bfloat16
+        mcode = binding.MSLA_F32 if ms_shape.dtype == "f32" else binding.MSLA_BF16
+        fd = {k: torch.from_numpy(v).to("cuda").to(mdt).contiguous() for k, v in ft.items()}
+        md = {k: torch.from_numpy(v).to("cuda").to(mdt).contiguous() for k, v in mt.items()}
+        B, C, H, W = ms_shape.B, ms_shape.C, ms_shape.H, ms_shape.W
+        f0 = binding.make_ffn_desc(B, C, H, W, c_hidden, C, mcode, binding.MSLA_ACT_HARDSWISH, True)
+        fws = torch.empty(binding.msla_ffn_workspace_bytes(f0), dtype=torch.uint8, device="cuda")
+        fdesc = binding.make_ffn_desc(B, C, H, W, c_hidden, C, mcode, binding.MSLA_ACT_HARDSWISH, True, workspace=fws)
+        fw = binding.make_ffn_weights(fd["w1"], fd["w_dw"], fd["w2"], fd["b1"], fd["b_dw"], fd["b2"])
+        a0 = binding.make_desc(B, C, H, W, ms_shape.heads, ms_shape.d, C, mcode, ms_shape.eps)
+        aws = torch.empty(binding.msla_forward_workspace_bytes(a0), dtype=torch.uint8, device="cuda")
+        adesc = binding.make_desc(B, C, H, W, ms_shape.heads, ms_shape.d, C, mcode, ms_shape.eps, workspace=aws)
+        aw = binding.make_weights(md["w_qkv"], md["w_dw"], md["w_pw"], md["w_proj"])
+        y, o = torch.empty_like(md["x"]), torch.empty_like(md["x"])
+        res = {}
+        e = 2 if ms_shape.dtype == "bf16" else 4
+        tokens = B * ms_shape.N
+        # bytes with materialised intermediates: first layer C + Ch, depthwise 2 Ch, second layer Ch + 2 C (residual read, output)
+        ffn_bytes = (4 * c_hidden + 4 * C) * e * tokens
+        for name, call in (("ffn_dwconv", lambda i: binding.msla_ffn_dwconv(fdesc, md["x"], fw, o, stream)),
+                           ("evit_block", lambda i: binding.msla_evit_block(adesc, aw, fdesc, fw, md["x"], y, o, stream))):
+            for i in range(3):
+                call(i)
+            ms = [m / steps for m in timed_blocks(call, blocks=blocks, steps=steps)]
+            res[name] = {"workload": f"{ms_shape.name}_hidden{c_hidden}", "tokens": tokens, "ms": round(med(ms), 5),
+                         "ms_min": round(min(ms), 5), "ms_max": round(max(ms), 5), "tokens_per_s": tokens / (med(ms) * 1e-3)}
+        res["ffn_dwconv"]["GBps_of_materialised_plan"] = round(ffn_bytes / (res["ffn_dwconv"]["ms"] * 1e-3) / 1e9, 1)
+        return res
+
     other = None
     if rank == 0 and world == 1 and not args.no_configs:
         other = {}
@@ -550,6 +586,8 @@ def main() -> None:
         band1 = time_token_sharded(s, 0, 1, steps=10, warmup=3, blocks=5)
         other["band_calls_one_rank"] = {"workload": s.name, "ms": round(med(band1), 5), "ms_min": round(min(band1), 5),
                                         "ms_max": round(max(band1), 5)}
+        # the rest of the building block (FFN with a depthwise convolution, expansion 4) at the bench workload's shape
+        other.update(time_ffn_block(s, 4 * s.C))
         sweep = [time_module(c) for c in inputs.CONFIG5]
         ns = np.array([c["tokens"] for c in sweep], dtype=np.float64)
         ts = np.array([c["ms"] for c in sweep], dtype=np.float64) * 1e3

@@ -4,16 +4,27 @@
 //
 //   g[b][c][y][x] = act( sum_{dy,dx} w[c][dy][dx] * h[b][c][y+dy-1][x+dx-1] + bias[c] ),   3x3, zero padding 1
 //
-// on the hidden tensor kept as planes of 64 channels, h[b][c / 64][y*W + x][c % 64]: what the first linear layer's
-// epilogue writes and what the second one's tile loads want (128-byte token rows).
+// Input: the hidden tensor as planes of 32 channels, h[b][c / 32][y*W + x][c % 32] (what the first linear layer's
+// epilogue writes: dense 64-byte token rows); output: planes of 64 channels, g[b][c / 64][y*W + x][c % 64] (what the
+// second linear layer's tile loads want: 128-byte token rows).  The change of plane width costs nothing here.
 //
 // The filter has no contraction over channels, so there is nothing for the tensor cores: at 9 multiply-adds per
-// element read and written (2.25 MAC per byte) the step is bound by HBM as long as the loads stay low.  A thread owns
-// 8 channels (16 bytes) of one pixel column and walks R rows with the three filter rows' partial sums in registers:
-// every input row is loaded once per column triple (3 vectors per output instead of 9), a warp's loads and stores
-// are 512 contiguous bytes, and the 72 filter taps of the thread's channels sit in registers as fp32.
+// element read and written (2.25 MAC per byte) the step is bound by HBM if enough bytes are in flight and every
+// input element is touched few times.  Persistent CTAs, one per SM, each with a contiguous run of 32 x 8 pixel tiles:
+//   warp 8      TMA producer: two 4-D boxes [32 channels][34 px][10 rows] per tile, one per input plane (the tile with
+//               its halo; rows and columns outside the image are zero-filled by the TMA unit = the zero padding),
+//               64B swizzle, 4-deep ring
+//   warps 0-15  a thread owns 4 channels (8 bytes) of one pixel column and walks the tile's rows with the three
+//               filter rows' partial sums in registers: 3 shared-memory loads per output instead of 9; the 36 taps
+//               of its channels sit in registers as fp32; bias, activation, bf16, one 8-byte store per output
+//               (a warp writes 256 contiguous bytes).  With 8 channels per thread the registers allow 8 warps only,
+//               too few to hide the latencies of the dependent load -> multiply-add -> store chain.
+// Every mbarrier wait is bounded; on time-out the CTA raises a flag and all roles leave their loops.
+#include <cuda.h>
+
 #include "msla_common.cuh"
 #include "msla_host.h"
+#include "tma_host.h"
 #include "tcgen05_util.cuh"
 
 namespace msla {
@@ -21,9 +32,20 @@ namespace {
 
 using bf16 = __nv_bfloat16;
 
-constexpr int DW_PX = 32;      // pixel columns per CTA
-constexpr int DW_ROWS = 8;     // output rows per CTA
-constexpr int DW_THREADS = DW_PX * 8;
+constexpr int DW_PX = 32;      // output pixel columns per tile
+constexpr int DW_ROWS = 8;     // output rows per tile
+constexpr int DW_BOX_PX = DW_PX + 2, DW_BOX_ROWS = DW_ROWS + 2;
+constexpr int DW_HALF_BYTES = DW_BOX_ROWS * DW_BOX_PX * 64;                // one input plane's box: 21 760
+constexpr int DW_HALF_STRIDE = (DW_HALF_BYTES + 511) / 512 * 512;          // 64B-swizzle atoms (8 rows) need 512-byte alignment
+constexpr int DW_TILE_BYTES = 2 * DW_HALF_BYTES;
+constexpr int DW_STAGE_BYTES = (2 * DW_HALF_STRIDE + 1023) / 1024 * 1024;
+constexpr int DW_STAGES = 4;
+constexpr int DW_CPT = 4;                                                  // channels per thread
+constexpr int DW_CONSUMERS = DW_PX * (64 / DW_CPT);                        // 512 threads: 16 warps to hide the latencies
+constexpr int DW_THREADS = DW_CONSUMERS + 32;
+constexpr int DW_SMEM = DW_STAGES * DW_STAGE_BYTES + 256 + 1024;
+
+__device__ int g_dw_timeout_flag = 0;
 
 __device__ __forceinline__ float dw_act(float v, int act) {
   if (act == 1) return fmaxf(v, 0.f);
@@ -31,97 +53,180 @@ __device__ __forceinline__ float dw_act(float v, int act) {
   return v;
 }
 
-__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
-  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    f[2 * e] = __uint_as_float(w[e] << 16);
-    f[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
-  }
+__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 
-// grid: (ceil(W / DW_PX), ceil(H / DW_ROWS), B * planes); planes = Ch / 64
-__global__ void __launch_bounds__(DW_THREADS)
-ffn_dw3x3_kernel(const bf16* __restrict__ h, const bf16* __restrict__ w_dw, const bf16* __restrict__ b_dw, bf16* __restrict__ g,
-                 int H, int W, int planes, int act) {
-  __shared__ float wsh[9][64];
-  __shared__ float bsh[64];
+struct DwParams {
+  const bf16* w_dw;  // [Ch][3][3]
+  const bf16* b_dw;  // [Ch] or nullptr
+  bf16* g;
+  int H, W, planes, act;
+  int tiles_x, tiles_y;
+  long long num_tiles;
+};
+
+__global__ void __launch_bounds__(DW_THREADS, 1)
+ffn_dw3x3_kernel(const __grid_constant__ CUtensorMap tmH, DwParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bars = ring + DW_STAGES * DW_STAGE_BYTES;
+  const uint32_t full_bar = bars, empty_bar = bars + 8 * DW_STAGES;
+  __shared__ int abort_flag;
   pdl_launch_dependents();
-  const int plane = blockIdx.z % planes;
-  for (int i = threadIdx.x; i < 9 * 64; i += DW_THREADS) {  // weights do not come from the previous kernel
-    const int c = i / 9, t = i - c * 9;
-    wsh[t][c] = __bfloat162float(w_dw[(long long)(plane * 64 + c) * 9 + t]);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < DW_STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, DW_CONSUMERS / 32); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int i = threadIdx.x; i < 64; i += DW_THREADS) bsh[i] = b_dw ? __bfloat162float(b_dw[plane * 64 + i]) : 0.f;
   __syncthreads();
-  const int c8 = threadIdx.x & 7, x = blockIdx.x * DW_PX + (threadIdx.x >> 3);
-  float wt[9][8], bias[8];
-#pragma unroll
-  for (int t = 0; t < 9; ++t)
-#pragma unroll
-    for (int i = 0; i < 8; ++i) wt[t][i] = wsh[t][c8 * 8 + i];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) bias[i] = bsh[c8 * 8 + i];
-  pdl_wait();  // h is the previous kernel's output
-  if (x >= W) return;
-  const long long base = (long long)blockIdx.z * H * W * 64 + c8 * 8;
-  const bf16* hp = h + base;
-  bf16* gp = g + base;
-  const int y0 = blockIdx.y * DW_ROWS;
-  const bool has_l = x > 0, has_r = x + 1 < W;
-  float acc[3][8];  // acc[o % 3]: output row o under construction
-#pragma unroll
-  for (int r = 0; r < DW_ROWS + 2; ++r) {  // input row y0 - 1 + r feeds output rows y0 + r - 2 .. y0 + r
-    const int yi = y0 - 1 + r;
-    const bool row_in = yi >= 0 && yi < H;
-    float in[3][8];
-    {
-      const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-      const bf16* rp = hp + ((long long)yi * W + x) * 64;
-      const uint4 vl = (row_in && has_l) ? __ldg(reinterpret_cast<const uint4*>(rp - 64)) : z;
-      const uint4 vc = row_in ? __ldg(reinterpret_cast<const uint4*>(rp)) : z;
-      const uint4 vr = (row_in && has_r) ? __ldg(reinterpret_cast<const uint4*>(rp + 64)) : z;
-      unpack8(vl, in[0]); unpack8(vc, in[1]); unpack8(vr, in[2]);
-    }
-#pragma unroll
-    for (int dy = 0; dy < 3; ++dy) {       // this input row is filter row dy of output row o = r - dy (relative to y0)
-      const int o = r - dy;
-      if (o < 0 || o >= DW_ROWS) continue;
-      float (&a)[8] = acc[o % 3];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        float v = dy == 0 ? bias[i] : a[i];  // filter row 0 opens the accumulator
-        v = fmaf(wt[dy * 3 + 0][i], in[0][i], v);
-        v = fmaf(wt[dy * 3 + 1][i], in[1][i], v);
-        v = fmaf(wt[dy * 3 + 2][i], in[2][i], v);
-        a[i] = v;
+  // contiguous run of tiles: x fastest, then rows, then (image, plane)
+  const long long t_first = p.num_tiles * blockIdx.x / gridDim.x, t_end = p.num_tiles * (blockIdx.x + 1) / gridDim.x;
+  const int per_z = p.tiles_x * p.tiles_y;
+  pdl_wait();  // h is the previous kernel's output; g may still be read by an earlier one
+
+  if (warp == DW_CONSUMERS / 32) {
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tmH) : "memory");
+      uint32_t it = 0;
+      for (long long t = t_first; t < t_end; ++t, ++it) {
+        const uint32_t s = it % DW_STAGES, ph = (it / DW_STAGES) & 1;
+        if (!mbar_wait(empty_bar + 8 * s, ph ^ 1, &abort_flag)) break;
+        const int z = (int)(t / per_z), r = (int)(t % per_z);
+        const int ty = r / p.tiles_x, tx = r % p.tiles_x;
+        mbar_expect_tx(full_bar + 8 * s, DW_TILE_BYTES);
+        tma_load_tile(ring + s * DW_STAGE_BYTES, &tmH, full_bar + 8 * s, 0, tx * DW_PX - 1, ty * DW_ROWS - 1, 2 * z);
+        tma_load_tile(ring + s * DW_STAGE_BYTES + DW_HALF_STRIDE, &tmH, full_bar + 8 * s, 0, tx * DW_PX - 1, ty * DW_ROWS - 1, 2 * z + 1);
       }
     }
-    const int od = r - 2;                  // output row completed by this input row
-    if (od >= 0 && y0 + od < H) {
-      const float (&a)[8] = acc[od % 3];
-      uint4 out;
-      out.x = pack2(dw_act(a[0], act), dw_act(a[1], act));
-      out.y = pack2(dw_act(a[2], act), dw_act(a[3], act));
-      out.z = pack2(dw_act(a[4], act), dw_act(a[5], act));
-      out.w = pack2(dw_act(a[6], act), dw_act(a[7], act));
-      *reinterpret_cast<uint4*>(gp + ((long long)(y0 + od) * W + x) * 64) = out;
+  } else {
+    // lane bits: [2:0] 8-byte piece (4 channels) of the plane's 64-byte row, [3] pixel bit 0, [4] input plane of the
+    // pair: sixteen consecutive lanes read 128 contiguous bytes of shared memory, a warp writes 256 contiguous bytes
+    const int piece = lane & 7, side = lane >> 4;
+    const int ch = side * 32 + piece * 4;       // first of the thread's 4 channels inside the 64-channel output plane
+    const int px = warp * 2 + ((lane >> 3) & 1);
+    float wt[9][4], bias[4];
+    int plane_loaded = -1;
+    uint32_t it = 0;
+    bool ok = true;
+    for (long long t = t_first; ok && t < t_end; ++t, ++it) {
+      const uint32_t s = it % DW_STAGES, ph = (it / DW_STAGES) & 1;
+      const int z = (int)(t / per_z), r0 = (int)(t % per_z);
+      const int ty = r0 / p.tiles_x, tx = r0 % p.tiles_x;
+      const int plane = z % p.planes;
+      if (plane != plane_loaded) {  // the thread's 4 channels x 9 taps: 72 contiguous bytes of the weight tensor
+        const uint2* wp = reinterpret_cast<const uint2*>(p.w_dw + (long long)(plane * 64 + ch) * 9);
+        uint32_t raw[18];
+#pragma unroll
+        for (int v = 0; v < 9; ++v) {
+          const uint2 q = __ldg(wp + v);
+          raw[2 * v] = q.x; raw[2 * v + 1] = q.y;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int tp = 0; tp < 9; ++tp) {
+            const int e = i * 9 + tp;  // element e of the 36: upper or lower half of word e / 2
+            wt[tp][i] = __uint_as_float((e & 1) ? (raw[e >> 1] & 0xffff0000u) : (raw[e >> 1] << 16));
+          }
+        if (p.b_dw) {
+          const uint2 q = __ldg(reinterpret_cast<const uint2*>(p.b_dw + plane * 64 + ch));
+          bias[0] = __uint_as_float(q.x << 16); bias[1] = __uint_as_float(q.x & 0xffff0000u);
+          bias[2] = __uint_as_float(q.y << 16); bias[3] = __uint_as_float(q.y & 0xffff0000u);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) bias[i] = 0.f;
+        }
+        plane_loaded = plane;
+      }
+      ok = mbar_wait(full_bar + 8 * s, ph, &abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      const uint32_t tile = ring + s * DW_STAGE_BYTES + side * DW_HALF_STRIDE;
+      const int x = tx * DW_PX + px, y0 = ty * DW_ROWS;
+      bf16* gp = p.g + ((long long)z * p.H * p.W) * 64 + ch;
+      float acc[3][4];  // acc[o % 3]: output row o under construction
+#pragma unroll
+      for (int r = 0; r < DW_BOX_ROWS; ++r) {  // box row r = image row y0 - 1 + r: filter row dy of output row r - dy
+        float in[3][4];
+#pragma unroll
+        for (int dx = 0; dx < 3; ++dx) {
+          const uint32_t row = (uint32_t)(r * DW_BOX_PX + px + dx);
+          uint2 v;  // 64B swizzle: 16-byte chunk index XOR bits 1-2 of the row
+          asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y)
+                       : "r"(tile + row * 64 + ((((uint32_t)piece >> 1) ^ ((row >> 1) & 3u)) << 4) + (((uint32_t)piece & 1u) << 3)));
+          in[dx][0] = __uint_as_float(v.x << 16); in[dx][1] = __uint_as_float(v.x & 0xffff0000u);
+          in[dx][2] = __uint_as_float(v.y << 16); in[dx][3] = __uint_as_float(v.y & 0xffff0000u);
+        }
+#pragma unroll
+        for (int dy = 0; dy < 3; ++dy) {
+          const int o = r - dy;
+          if (o < 0 || o >= DW_ROWS) continue;
+          float (&a)[4] = acc[o % 3];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            float v = dy == 0 ? bias[i] : a[i];  // filter row 0 opens the accumulator
+            v = fmaf(wt[dy * 3 + 0][i], in[0][i], v);
+            v = fmaf(wt[dy * 3 + 1][i], in[1][i], v);
+            v = fmaf(wt[dy * 3 + 2][i], in[2][i], v);
+            a[i] = v;
+          }
+        }
+        const int od = r - 2;  // output row completed by this box row
+        if (od >= 0 && y0 + od < p.H && x < p.W) {
+          const float (&a)[4] = acc[od % 3];
+          uint2 out;
+          out.x = pack2(dw_act(a[0], p.act), dw_act(a[1], p.act));
+          out.y = pack2(dw_act(a[2], p.act), dw_act(a[3], p.act));
+          *reinterpret_cast<uint2*>(gp + ((long long)(y0 + od) * p.W + x) * 64) = out;
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_bar + 8 * s);  // the warp has read all it needs of this stage
     }
   }
+  __syncthreads();
+  if (abort_flag && threadIdx.x == 0) atomicExch(&g_dw_timeout_flag, 1);
 }
 
 }  // namespace
 
-// h, g: [B][Ch / 64][H * W][64] bf16; w_dw [Ch][3][3]; b_dw [Ch] or nullptr.
+// h: [B][Ch / 32][H * W][32], g: [B][Ch / 64][H * W][64] bf16; w_dw [Ch][3][3]; b_dw [Ch] or nullptr.
 msla_status_t run_ffn_dw3x3_bf16(const void* h, const void* w_dw, const void* b_dw, void* g, int B, int Ch, int H, int W, int act,
                                  cudaStream_t st) {
   const long long z = (long long)B * (Ch / 64);
-  if (Ch % 64 != 0 || z > 65535 || (H + DW_ROWS - 1) / DW_ROWS > 65535)
-    return fail(MSLA_ERR_UNSUPPORTED, "FFN depthwise convolution: %d hidden channels, batch %d, %d rows", Ch, B, H);
-  launch_pdl(ffn_dw3x3_kernel, dim3((unsigned)((W + DW_PX - 1) / DW_PX), (unsigned)((H + DW_ROWS - 1) / DW_ROWS), (unsigned)z),
-             dim3(DW_THREADS), 0, st, (const bf16*)h, (const bf16*)w_dw, (const bf16*)b_dw, (bf16*)g, H, W, Ch / 64, act);
+  if (Ch % 64 != 0 || z > 0x7fffffffLL)
+    return fail(MSLA_ERR_UNSUPPORTED, "FFN depthwise convolution: %d hidden channels, batch %d", Ch, B);
+  CUtensorMap tmH;
+  const cuuint64_t dims[4] = {32, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)(2 * z)};
+  const cuuint64_t strides[3] = {64, (cuuint64_t)W * 64, (cuuint64_t)H * W * 64};
+  const cuuint32_t box[4] = {32, DW_BOX_PX, DW_BOX_ROWS, 1};
+  if (!tma_make_map_bf16(&tmH, h, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B))
+    return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the FFN's depthwise convolution");
+  DwParams p{};
+  p.w_dw = (const bf16*)w_dw; p.b_dw = (const bf16*)b_dw; p.g = (bf16*)g;
+  p.H = H; p.W = W; p.planes = Ch / 64; p.act = act;
+  p.tiles_x = (W + DW_PX - 1) / DW_PX; p.tiles_y = (H + DW_ROWS - 1) / DW_ROWS;
+  p.num_tiles = z * p.tiles_x * p.tiles_y;
+  static std::atomic<unsigned long long> attr_done{0};
+  const msla_status_t as = ensure_smem_attr(attr_done, ffn_dw3x3_kernel, DW_SMEM);
+  if (as != MSLA_OK) return as;
+  const long long grid = p.num_tiles < device_sm_count() ? p.num_tiles : device_sm_count();
+  launch_pdl(ffn_dw3x3_kernel, dim3((unsigned)grid), dim3(DW_THREADS), DW_SMEM, st, tmH, p);
   count_launches(1);
   return check_launch("FFN depthwise convolution (bf16)");
+}
+
+int dw_timeout_flag() {
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, g_dw_timeout_flag, sizeof(int)) != cudaSuccess) {
+    cudaGetLastError();
+    return -1;
+  }
+  return v;
 }
 
 }  // namespace msla

@@ -63,15 +63,9 @@ struct GemmParams {
   int tma_store;          // 1: epilogue stages 32x32 blocks in shared memory and writes them with TMA (tmO)
   int planes_per_batch;   // planar output: plane coordinate of (batch, n) = batch*planes_per_batch + n/32
   int plane_shift;        // log2 of the channels per TMA-stored output plane (5: planes of 32, 6: planes of 64)
-  int act;                // applied to accumulator + bias: 0 none, 1 ReLU, 2 hard-swish
-  const bf16* residual;   // nullptr, or a tensor laid out like the row-major output, added after the activation
+  float act_a, act_b;     // EPI 1: act(v) = v * sat(v * act_a + act_b)
+  const bf16* residual;   // EPI 2: a tensor laid out like the row-major output, added after the bias
 };
-
-__device__ __forceinline__ float epilogue_act(float v, int act) {
-  if (act == 1) return fmaxf(v, 0.f);
-  if (act == 2) return v * __saturatef((v + 3.f) * (1.f / 6.f));  // v * min(max(v + 3, 0), 6) / 6
-  return v;
-}
 
 __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& b, int& mt, int& nt) {
   const int per_batch = p.m_tiles * p.n_tiles;
@@ -91,24 +85,31 @@ constexpr int STAGING_BYTES = 8 * 2048;  // one 32-row x 64-byte block per epilo
 // as the TMA unit's 64B mode expects) and written by one TMA store, which
 // emits whole lines and clips rows and columns outside the tensor.  Without a
 // store map (planes of 16 channels) the lane stores its vectors directly.
-// EPI: the epilogue also applies p.act and adds p.residual (compiled out of the plain projections).
-template <bool EPI>
+// EPI selects what else the epilogue does (compiled out of the plain projections):
+//   0  nothing
+//   1  column biases read from shared memory (bias_sm: the tile's 256 columns as fp32) and the activation
+//      act(v) = v * sat(v * p.act_a + p.act_b), which is the identity for (0, 1), hard-swish for (1/6, 1/2) and ReLU
+//      for (1e30, 0); the staging block is double-buffered (NBUF = 2) so that this arithmetic overlaps the previous
+//      block's TMA store instead of lengthening the chain tmem load -> convert -> stage -> store
+//   2  adds p.residual (laid out like the row-major output) after the bias
+template <int EPI, int NBUF = 1>
 __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUtensorMap* tmO, uint32_t stage, int b,
-                                                  int mt, int nt, uint32_t tmem_acc, int quarter, int col_half, int lane) {
+                                                  int mt, int nt, uint32_t tmem_acc, int quarter, int col_half, int lane,
+                                                  const float* bias_sm = nullptr) {
   const int gs = p.group == 32 ? 5 : 4;  // log2(group) when the output is planar
   const int row0 = mt * BM + quarter * 32;
   const int m = row0 + lane;
   const bool row_ok = m < p.M;
   bf16* obase = p.out + (long long)b * p.out_batch_stride;
-  const float bias_row = (p.bias && p.bias_per_row && row_ok) ? __bfloat162float(p.bias[m]) : 0.f;
-  const bool bias_col = p.bias && !p.bias_per_row;
+  const float bias_row = (EPI != 1 && p.bias && p.bias_per_row && row_ok) ? __bfloat162float(p.bias[m]) : 0.f;
+  const bool bias_col = EPI != 1 && p.bias && !p.bias_per_row;
   const int ncol0 = nt * BN + col_half * 128;
   const uint32_t taddr = tmem_acc + col_half * 128 + ((uint32_t)(quarter * 32) << 16);
-  const uint32_t my_row = stage + lane * 64, sw = (uint32_t)((lane >> 1) & 3);
+  const uint32_t sw = (uint32_t)((lane >> 1) & 3);
   uint32_t r[2][32];
   tmem_ld32(taddr, r[0]);
   // residual: the lane's row of the output-shaped tensor, 32 tokens (64 bytes) per chunk, fetched one chunk ahead
-  const bf16* res_row = (EPI && p.residual && row_ok) ? p.residual + (long long)b * p.out_batch_stride + (long long)m * p.ld_out : nullptr;
+  const bf16* res_row = (EPI == 2 && p.residual && row_ok) ? p.residual + (long long)b * p.out_batch_stride + (long long)m * p.ld_out : nullptr;
   uint4 rs[2][4];
   auto load_residual = [&](int c) {
 #pragma unroll
@@ -117,45 +118,65 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUt
       rs[c & 1][v] = (res_row && n < p.N) ? __ldg(reinterpret_cast<const uint4*>(res_row + n)) : make_uint4(0u, 0u, 0u, 0u);
     }
   };
-  if (EPI && p.residual) load_residual(0);
+  if (EPI == 2) load_residual(0);
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
     tmem_ld_wait();
     if (c + 1 < 4) tmem_ld32(taddr + (c + 1) * 32, r[(c + 1) & 1]);  // next chunk streams in while this one is stored
-    if (EPI && p.residual && c + 1 < 4) load_residual(c + 1);
+    if (EPI == 2 && c + 1 < 4) load_residual(c + 1);
     const uint32_t(&rc)[32] = r[c & 1];
     const int n0 = ncol0 + c * 32;
     if (n0 >= p.N) continue;  // warp-uniform
     uint32_t w[4][4];
 #pragma unroll
     for (int v = 0; v < 4; ++v) {
-      const uint32_t rw[4] = {rs[c & 1][v].x, rs[c & 1][v].y, rs[c & 1][v].z, rs[c & 1][v].w};
+      float bc[8];
+      if (EPI == 1 && bias_sm) {  // same address in every lane: broadcast reads
+        const float4 b0 = *reinterpret_cast<const float4*>(bias_sm + col_half * 128 + c * 32 + v * 8);
+        const float4 b1 = *reinterpret_cast<const float4*>(bias_sm + col_half * 128 + c * 32 + v * 8 + 4);
+        bc[0] = b0.x; bc[1] = b0.y; bc[2] = b0.z; bc[3] = b0.w; bc[4] = b1.x; bc[5] = b1.y; bc[6] = b1.z; bc[7] = b1.w;
+      } else if (EPI == 1) {      // no staged copy (the kernel whose CTAs change weight block from tile to tile)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) bc[i] = (p.bias && n0 + v * 8 < p.N) ? __bfloat162float(p.bias[n0 + v * 8 + i]) : 0.f;
+      }
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        float f0 = __uint_as_float(rc[v * 8 + 2 * e]) + bias_row;
-        float f1 = __uint_as_float(rc[v * 8 + 2 * e + 1]) + bias_row;
-        if (bias_col && n0 + v * 8 < p.N) {
-          f0 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e]);
-          f1 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e + 1]);
+        float f0 = __uint_as_float(rc[v * 8 + 2 * e]), f1 = __uint_as_float(rc[v * 8 + 2 * e + 1]);
+        if (EPI == 1) {
+          f0 += bc[2 * e]; f1 += bc[2 * e + 1];
+          f0 *= __saturatef(fmaf(f0, p.act_a, p.act_b));
+          f1 *= __saturatef(fmaf(f1, p.act_a, p.act_b));
+        } else {
+          f0 += bias_row; f1 += bias_row;
+          if (bias_col && n0 + v * 8 < p.N) {
+            f0 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e]);
+            f1 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e + 1]);
+          }
         }
-        if (EPI && p.act) { f0 = epilogue_act(f0, p.act); f1 = epilogue_act(f1, p.act); }
-        if (EPI && p.residual) { f0 += __uint_as_float(rw[e] << 16); f1 += __uint_as_float(rw[e] & 0xffff0000u); }
+        if (EPI == 2) {
+          const uint32_t rw = e == 0 ? rs[c & 1][v].x : e == 1 ? rs[c & 1][v].y : e == 2 ? rs[c & 1][v].z : rs[c & 1][v].w;
+          f0 += __uint_as_float(rw << 16); f1 += __uint_as_float(rw & 0xffff0000u);
+        }
         w[v][e] = pack2(f0, f1);
       }
     }
     if (p.tma_store) {
-      // the previous block must have been read out of the staging buffer
-      if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      const uint32_t buf = stage + (NBUF == 2 ? (uint32_t)(c & 1) * 2048u : 0u);
+      // the block stored from this buffer before must have been read out of it
+      if (lane == 0) {
+        if (NBUF == 2) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        else           asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      }
       __syncwarp();
 #pragma unroll
       for (int v = 0; v < 4; ++v)
-        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(my_row + (((uint32_t)v ^ sw) << 4)), "r"(w[v][0]),
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(buf + lane * 64 + (((uint32_t)v ^ sw) << 4)), "r"(w[v][0]),
                      "r"(w[v][1]), "r"(w[v][2]), "r"(w[v][3]) : "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) {
-        if (p.group) tma_store_3d(tmO, stage, n0 & ((1 << p.plane_shift) - 1), row0, b * p.planes_per_batch + (n0 >> p.plane_shift));
-        else         tma_store_3d(tmO, stage, n0, row0, b);
+        if (p.group) tma_store_3d(tmO, buf, n0 & ((1 << p.plane_shift) - 1), row0, b * p.planes_per_batch + (n0 >> p.plane_shift));
+        else         tma_store_3d(tmO, buf, n0, row0, b);
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       }
     } else if (row_ok) {
@@ -174,7 +195,7 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUt
 
 // B_PLANAR (output projection with the attention output kept as one [N][64]
 // plane per pair of heads): the 64-wide k-slice kb of B is plane kb of the image.
-template <bool A_MN_MAJOR, bool B_PLANAR, bool EPI>
+template <bool A_MN_MAJOR, bool B_PLANAR, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                          const __grid_constant__ CUtensorMap tmO, GemmParams p) {
@@ -335,28 +356,37 @@ constexpr int WS_RING_BYTES = 80 * 1024;
 constexpr int WS_SMEM_BYTES = RES_BYTES + WS_RING_BYTES + STAGING_BYTES + 256 + 1024;
 constexpr int WS_MAX_STAGES = 6;
 
-template <bool EPI>
+template <int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                             const __grid_constant__ CUtensorMap tmO, GemmParams p, int blocks, int workers) {
   constexpr int STREAM_BYTES = A_STAGE_BYTES;             // one k-slice of the streamed operand (the x tile)
-  constexpr int NSTAGE = WS_RING_BYTES / STREAM_BYTES;    // 5
+  constexpr int NBUF = EPI == 1 ? 2 : 1;                  // staging blocks per epilogue warp
+  constexpr int RING_BYTES = WS_RING_BYTES - (NBUF - 1) * STAGING_BYTES;  // the second staging block comes out of the ring
+  constexpr int NSTAGE = RING_BYTES / STREAM_BYTES;       // 5 (4 with double-buffered staging)
   constexpr int RES_SLICE = B_STAGE_BYTES;                // one k-slice of the resident operand (256 weight rows)
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t res_base = smem_base, ring_base = smem_base + RES_BYTES;
-  const uint32_t staging = ring_base + WS_RING_BYTES;
-  const uint32_t bars = staging + STAGING_BYTES;
+  const uint32_t staging = ring_base + RING_BYTES;
+  const uint32_t bars = staging + NBUF * STAGING_BYTES;
   const uint32_t full_bar = bars, empty_bar = bars + 8 * WS_MAX_STAGES;
   const uint32_t tfull_bar = bars + 16 * WS_MAX_STAGES, tempty_bar = tfull_bar + 16;
   const uint32_t res_bar = tempty_bar + 16, tmem_slot = res_bar + 8;
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_sh;
+  __shared__ __align__(16) float bias_sm[EPI == 1 ? BN : 4];  // the CTA's 256 column biases (weights: not the previous kernel's output)
 
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int k_iters = (p.K + BK - 1) / BK;
   const int blk = blockIdx.x % blocks, worker = blockIdx.x / blocks;
+  if (EPI == 1) {
+    for (int i = threadIdx.x; i < BN; i += NUM_THREADS) {
+      const int n = blk * BN + i;
+      bias_sm[i] = (p.bias && !p.bias_per_row && n < p.N) ? __bfloat162float(p.bias[n]) : 0.f;
+    }
+  }
   const int stream_per_batch = p.m_tiles;
   const int stream_total = p.batches * stream_per_batch;
 
@@ -452,7 +482,7 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      drain_accumulator<EPI>(p, &tmO, staging + (warp - 2) * 2048, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
+      drain_accumulator<EPI, NBUF>(p, &tmO, staging + (warp - 2) * 2048 * NBUF, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane, bias_sm);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);
@@ -484,7 +514,7 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint
   return tma_make_map_bf16(map, base, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
-template <bool EPI>
+template <int EPI>
 msla_status_t launch_stationary(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO, const GemmParams& p,
                                 int blocks, cudaStream_t st) {
   static std::atomic<unsigned long long> attr_done{0};
@@ -498,7 +528,7 @@ msla_status_t launch_stationary(const CUtensorMap& tmA, const CUtensorMap& tmB, 
   return check_launch("projection GEMM (tcgen05, stationary weights)");
 }
 
-template <bool A_MN, bool B_PLANAR = false, bool EPI = false>
+template <bool A_MN, bool B_PLANAR = false, int EPI = 0>
 msla_status_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO, const GemmParams& p, cudaStream_t st) {
   // weight-stationary kernel when the CTA's weight block fits its 128 KB of shared memory
   const int blocks = A_MN ? p.n_tiles : p.m_tiles;
@@ -604,13 +634,14 @@ bool ffn_bf16_supported(int C, int Ch, int Cout, int N) {
   return C % 8 == 0 && Ch % 64 == 0 && Cout % 8 == 0 && N % 8 == 0;
 }
 
-// First layer: h[b][o / 64][n][o % 64] = act(sum_c w1[o][c] * x[b][c][n] + b1[o]); x NCHW, h planes of 64 channels.
+// First layer: h[b][o / 32][n][o % 32] = act(sum_c w1[o][c] * x[b][c][n] + b1[o]); x NCHW, h planes of 32 channels
+// (dense 2 KB per 32 tokens for the epilogue's TMA stores: half-line stores into 64-channel planes cost this GEMM 2x).
 msla_status_t run_ffn_expand_bf16(const void* x, const void* w1, const void* b1, void* h, int B, int C, int Ch, int N, int act,
                                   cudaStream_t st) {
   CUtensorMap tmA, tmB, tmO;
-  const cuuint64_t dims[3] = {64, (cuuint64_t)N, (cuuint64_t)B * (Ch / 64)};
-  const cuuint64_t strides[2] = {128, (cuuint64_t)N * 128};
-  const cuuint32_t box[3] = {32, 32, 1};  // the epilogue's 32-token x 32-channel blocks: half a plane row each
+  const cuuint64_t dims[3] = {32, (cuuint64_t)N, (cuuint64_t)B * (Ch / 32)};
+  const cuuint64_t strides[2] = {64, (cuuint64_t)N * 64};
+  const cuuint32_t box[3] = {32, 32, 1};
   if (!make_map(&tmA, x, (uint64_t)N, (uint64_t)C, (uint64_t)B, (uint64_t)N * 2, (uint64_t)C * N * 2, 64, BK) ||
       !make_map(&tmB, w1, (uint64_t)C, (uint64_t)Ch, 1, (uint64_t)C * 2, (uint64_t)C * Ch * 2, BK, BN) ||
       !tma_make_map_bf16(&tmO, h, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B))
@@ -620,9 +651,11 @@ msla_status_t run_ffn_expand_bf16(const void* x, const void* w1, const void* b1,
   p.m_tiles = (N + BM - 1) / BM; p.n_tiles = (Ch + BN - 1) / BN;
   p.out_batch_stride = (long long)Ch * N; p.ld_out = 0; p.group = 32; p.bias_per_row = 0; p.n_fastest = 1;
   p.bias = (const bf16*)b1; p.out = (bf16*)h;
-  p.tma_store = 1; p.planes_per_batch = Ch / 64; p.plane_shift = 6;
-  p.act = act; p.residual = nullptr;
-  return launch<true, false, true>(tmA, tmB, tmO, p, st);
+  p.tma_store = 1; p.planes_per_batch = Ch / 32; p.plane_shift = 5;
+  p.act_a = act == 2 ? 1.f / 6.f : (act == 1 ? 1e30f : 0.f);  // act(v) = v * sat(v * act_a + act_b)
+  p.act_b = act == 2 ? 0.5f : (act == 1 ? 0.f : 1.f);
+  p.residual = nullptr;
+  return launch<true, false, 1>(tmA, tmB, tmO, p, st);
 }
 
 // Second layer: y[b][m][n] = sum_j w2[m][j] * g[b][j / 64][n][j % 64] + b2[m] (+ residual[b][m][n]); g planes of 64 channels, y NCHW.
@@ -643,8 +676,8 @@ msla_status_t run_ffn_project_bf16(const void* g, const void* w2, const void* b2
   p.out_batch_stride = (long long)Cout * N; p.ld_out = N; p.group = 0; p.bias_per_row = 1; p.n_fastest = 0;
   p.bias = (const bf16*)b2; p.out = (bf16*)y;
   p.tma_store = 1; p.planes_per_batch = planes;
-  p.act = 0; p.residual = (const bf16*)residual;
-  return launch<false, true, true>(tmA, tmB, tmO, p, st);
+  p.residual = (const bf16*)residual;
+  return launch<false, true, 2>(tmA, tmB, tmO, p, st);
 }
 
 // Self-test of the bounded wait every kernel of the library relies on: one thread waits, with the given cycle

@@ -643,9 +643,8 @@ static msla_status_t block_impl(const msla_desc* attn, const msla_weights* aw, c
   const long long total = (long long)attn->B * attn->C * ap.N;
   if (attn->dtype == MSLA_F32)
     generic::add_kernel<float><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const float*)y, (const float*)x, (float*)y, total);
-  else
-    generic::add_kernel<__nv_bfloat16><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const __nv_bfloat16*)y, (const __nv_bfloat16*)x,
-                                                                                         (__nv_bfloat16*)y, total);
+  else  // C is a multiple of 8, so is the element count
+    generic::add_bf16x8_kernel<<<(unsigned)ceil_div_ll(total / 8, 256), 256, 0, st>>>((const uint4*)y, (const uint4*)x, (uint4*)y, total / 8);
   count_launches(1);
   if ((s = check_launch("residual connection around the attention module")) != MSLA_OK) return s;
   return ffn_impl(ffn, y, fw, out, true, st);
@@ -746,8 +745,8 @@ int msla_forward_fuses_apply(const msla_desc* desc) {
 unsigned long long msla_kernel_launches(void) { return g_launches; }
 
 int msla_debug_wait_timeouts(void) {
-  const int a = gemm_timeout_flag(), b = agg_timeout_flag(), c = fused_timeout_flag();
-  return (a < 0 || b < 0 || c < 0) ? -1 : (a | b | c);
+  const int a = gemm_timeout_flag(), b = agg_timeout_flag(), c = fused_timeout_flag(), e = dw_timeout_flag();
+  return (a < 0 || b < 0 || c < 0 || e < 0) ? -1 : (a | b | c | e);
 }
 
 int msla_debug_wait_selftest(long long limit_cycles, void* scratch, void* stream) {

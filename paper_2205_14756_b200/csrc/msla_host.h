@@ -101,8 +101,9 @@ msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* o
                             int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st,
                             cudaEvent_t mid, int phases);
 
-// FFN with a depthwise convolution (gemm_tcgen05.cu, ffn_dw_bf16.cu): bf16, hidden tensor as planes of 64 channels
-// [B][Ch / 64][N][64].  act: 0 none, 1 ReLU, 2 hard-swish.
+// FFN with a depthwise convolution (gemm_tcgen05.cu, ffn_dw_bf16.cu): bf16; the hidden tensor is planes of 32 channels
+// [B][Ch / 32][N][32] after the first layer, planes of 64 channels [B][Ch / 64][N][64] after the depthwise convolution.
+// act: 0 none, 1 ReLU, 2 hard-swish.
 bool ffn_bf16_supported(int C, int Ch, int Cout, int N);
 msla_status_t run_ffn_expand_bf16(const void* x, const void* w1, const void* b1, void* h, int B, int C, int Ch, int N, int act,
                                   cudaStream_t st);
@@ -120,6 +121,7 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
                                  const void* w, const void* bias, void* y, int B, int Ht, int d, int N, int Cout, float eps,
                                  cudaStream_t st);
 int fused_timeout_flag();
+int dw_timeout_flag();
 
 // bf16 projections on tcgen05 tensor cores (gemm_tcgen05.cu).
 bool project_in_bf16_supported(int C, int Cout, int N, int d);
