@@ -142,14 +142,23 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
 // ---------------------------------------------------------------------------
 constexpr int FOLD_THREADS = 1024;
 constexpr int FOLD_RUNS = 8;       // S <= 64: at most 8 partial states per run
+constexpr int FOLD_RUN_BYTES = FOLD_RUNS * 32 * 33 * 4, FOLD_ST_BYTES = 32 * 33 * 4;
+constexpr int FOLD_SMEM = FOLD_RUN_BYTES + FOLD_ST_BYTES + 256 * 32 * 2;  // + the head's [Cout <= 256][d <= 32] weight columns
 __global__ void __launch_bounds__(FOLD_THREADS)
 state_fold_kernel(const float* __restrict__ partial, int S, const bf16* __restrict__ w, bf16* __restrict__ M, float* __restrict__ ks,
                   int Ht, int d, int Cout, int K, int da) {
-  __shared__ float4 run_sum[FOLD_RUNS][32 * 33 / 4];
-  __shared__ float st[32 * 33];
+  extern __shared__ __align__(16) unsigned char fold_smem[];
+  float4 (*run_sum)[32 * 33 / 4] = reinterpret_cast<float4 (*)[32 * 33 / 4]>(fold_smem);
+  float* st = reinterpret_cast<float*>(fold_smem + FOLD_RUN_BYTES);
+  uint4* wtile = reinterpret_cast<uint4*>(fold_smem + FOLD_RUN_BYTES + FOLD_ST_BYTES);  // the head's columns of w: [Cout][d] bf16
   pdl_launch_dependents();
-  pdl_wait();  // the partial states come from the previous kernel
   const int bh = blockIdx.x, b = bh / Ht, hh = bh % Ht;
+  // the projection weights do not come from the previous kernel: staged while it drains
+  for (int i = threadIdx.x; i < Cout * (d / 8); i += FOLD_THREADS) {
+    const int m = i / (d / 8), c8 = i - m * (d / 8);
+    wtile[i] = __ldg(reinterpret_cast<const uint4*>(w + (long long)m * K + hh * d) + c8);  // 16-byte aligned: K and d are multiples of 8
+  }
+  pdl_wait();  // the partial states come from the previous kernel
   const int d1 = d + 1, ne = d * d1;
   const int a0 = blockIdx.y * da;
   const int nq4 = da * d1 / 4;  // this CTA's rows of the state, in 16-byte vectors (da * d1 is a multiple of 4)
@@ -175,21 +184,25 @@ state_fold_kernel(const float* __restrict__ partial, int S, const bf16* __restri
   }
   __syncthreads();
   for (int al = threadIdx.x; al < da; al += FOLD_THREADS) ks[(long long)bh * d + a0 + al] = st[al * d1 + d];
-  for (int idx = threadIdx.x; idx < Cout * da; idx += FOLD_THREADS) {
-    const int m = idx / da, al = idx - m * da;
-    const uint4* wr = reinterpret_cast<const uint4*>(w + (long long)m * K + hh * d);  // 16-byte aligned: K and d are multiples of 8
+  // M: a thread keeps key channel al = threadIdx.x % da (FOLD_THREADS is a multiple of da), i.e. one row of the state,
+  // in registers and walks the output channels m = threadIdx.x / da, + FOLD_THREADS / da, ...
+  const int al = threadIdx.x % da;
+  float srow[32];
+#pragma unroll
+  for (int c = 0; c < 32; ++c) srow[c] = c < d ? st[al * d1 + c] : 0.f;
+  for (int m = threadIdx.x / da; m < Cout; m += FOLD_THREADS / da) {
+    const uint4* wr = wtile + m * (d / 8);
     uint4 wv[4];
 #pragma unroll
-    for (int c8 = 0; c8 < 4; ++c8) wv[c8] = c8 < d / 8 ? __ldg(wr + c8) : make_uint4(0u, 0u, 0u, 0u);
+    for (int c8 = 0; c8 < 4; ++c8) wv[c8] = c8 < d / 8 ? wr[c8] : make_uint4(0u, 0u, 0u, 0u);
     float acc = 0.f;
 #pragma unroll
     for (int c8 = 0; c8 < 4; ++c8) {
-      if (c8 >= d / 8) break;
       const uint32_t word[4] = {wv[c8].x, wv[c8].y, wv[c8].z, wv[c8].w};
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        acc = fmaf(__uint_as_float(word[e] << 16), st[al * d1 + 8 * c8 + 2 * e], acc);
-        acc = fmaf(__uint_as_float(word[e] & 0xffff0000u), st[al * d1 + 8 * c8 + 2 * e + 1], acc);
+      for (int e = 0; e < 4; ++e) {  // channels beyond d carry zeros on both sides
+        acc = fmaf(__uint_as_float(word[e] << 16), srow[8 * c8 + 2 * e], acc);
+        acc = fmaf(__uint_as_float(word[e] & 0xffff0000u), srow[8 * c8 + 2 * e + 1], acc);
       }
     }
     M[((long long)b * Cout + m) * K + hh * d + a0 + al] = __float2bfloat16_rn(acc);
@@ -532,7 +545,9 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   // about one CTA per SM: few heads -> up to four CTAs per head, each with a share of the head's key channels
   int fold_chunks = sms / (B * Ht);
   fold_chunks = fold_chunks >= 4 ? 4 : (fold_chunks >= 2 ? 2 : 1);
-  launch_pdl(state_fold_kernel, dim3((unsigned)(B * Ht), (unsigned)fold_chunks), dim3(FOLD_THREADS), 0, st, partial, S,
+  static std::atomic<unsigned long long> attr_fold{0};
+  if ((s = ensure_smem_attr(attr_fold, state_fold_kernel, FOLD_SMEM)) != MSLA_OK) return s;
+  launch_pdl(state_fold_kernel, dim3((unsigned)(B * Ht), (unsigned)fold_chunks), dim3(FOLD_THREADS), FOLD_SMEM, st, partial, S,
              (const bf16*)w, M, ks, Ht, d, Cout, K, d / fold_chunks);
   if (d == 32) launch_pdl_cluster2(fused_out_kernel<32>, dim3((unsigned)(2 * pairs)), dim3(O_THREADS), (size_t)smem, st, tmM, tmQ, tmO, p);
   else launch_pdl_cluster2(fused_out_kernel<16>, dim3((unsigned)(2 * pairs)), dim3(O_THREADS), (size_t)smem, st, tmM, tmQ, tmO, p);
