@@ -11,9 +11,10 @@
 // The filter has no contraction over channels, so there is nothing for the tensor cores: at 9 multiply-adds per
 // element read and written (2.25 MAC per byte) the step is bound by HBM if enough bytes are in flight and every
 // input element is touched few times.  Persistent CTAs, one per SM, each with a contiguous run of 32 x 8 pixel tiles:
-//   warp 8      TMA producer: two 4-D boxes [32 channels][34 px][10 rows] per tile, one per input plane (the tile with
-//               its halo; rows and columns outside the image are zero-filled by the TMA unit = the zero padding),
-//               64B swizzle, 4-deep ring
+//   warp 16     TMA producer: per tile, image row and input plane one 4-D box [32 channels][34 px] (the tile with its
+//               halo; rows and columns outside the image are zero-filled by the TMA unit = the zero padding), 64B
+//               swizzle, each into a 40-pixel slot so that a pixel's swizzle phase is the same in every row and the
+//               consumers' addresses are constants plus a per-thread offset; 4-deep ring
 //   warps 0-15  a thread owns 4 channels (8 bytes) of one pixel column and walks the tile's rows with the three
 //               filter rows' partial sums in registers: 3 shared-memory loads per output instead of 9; the 36 taps
 //               of its channels sit in registers as fp32; bias, activation, bf16, one 8-byte store per output
@@ -35,10 +36,12 @@ using bf16 = __nv_bfloat16;
 constexpr int DW_PX = 32;      // output pixel columns per tile
 constexpr int DW_ROWS = 8;     // output rows per tile
 constexpr int DW_BOX_PX = DW_PX + 2, DW_BOX_ROWS = DW_ROWS + 2;
-constexpr int DW_HALF_BYTES = DW_BOX_ROWS * DW_BOX_PX * 64;                // one input plane's box: 21 760
-constexpr int DW_HALF_STRIDE = (DW_HALF_BYTES + 511) / 512 * 512;          // 64B-swizzle atoms (8 rows) need 512-byte alignment
-constexpr int DW_TILE_BYTES = 2 * DW_HALF_BYTES;
-constexpr int DW_STAGE_BYTES = (2 * DW_HALF_STRIDE + 1023) / 1024 * 1024;
+constexpr int DW_ROW_BYTES = DW_BOX_PX * 64;                               // one image row of one input plane's box: 2 176
+constexpr int DW_ROW_PITCH = 40 * 64;                                      // its slot: a multiple of the 64B-swizzle atom (8 pixels =
+                                                                           // 512 bytes), so the swizzle phase of a pixel does not depend on the row
+constexpr int DW_HALF_STRIDE = DW_BOX_ROWS * DW_ROW_PITCH;                 // one input plane's rows: 25 600
+constexpr int DW_TILE_BYTES = 2 * DW_BOX_ROWS * DW_ROW_BYTES;              // bytes the TMA unit delivers per tile
+constexpr int DW_STAGE_BYTES = 2 * DW_HALF_STRIDE;                         // 51 200
 constexpr int DW_STAGES = 4;
 constexpr int DW_CPT = 4;                                                  // channels per thread
 constexpr int DW_CONSUMERS = DW_PX * (64 / DW_CPT);                        // 512 threads: 16 warps to hide the latencies
@@ -47,11 +50,6 @@ constexpr int DW_SMEM = DW_STAGES * DW_STAGE_BYTES + 256 + 1024;
 
 __device__ int g_dw_timeout_flag = 0;
 
-__device__ __forceinline__ float dw_act(float v, int act) {
-  if (act == 1) return fmaxf(v, 0.f);
-  if (act == 2) return v * __saturatef((v + 3.f) * (1.f / 6.f));  // v * min(max(v + 3, 0), 6) / 6
-  return v;
-}
 
 __device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
   asm volatile(
@@ -63,7 +61,8 @@ struct DwParams {
   const bf16* w_dw;  // [Ch][3][3]
   const bf16* b_dw;  // [Ch] or nullptr
   bf16* g;
-  int H, W, planes, act;
+  int H, W, planes;
+  float act_a, act_b;  // act(v) = v * sat(v * act_a + act_b): identity (0, 1), hard-swish (1/6, 1/2), ReLU (1e30, 0)
   int tiles_x, tiles_y;
   long long num_tiles;
 };
@@ -83,7 +82,8 @@ ffn_dw3x3_kernel(const __grid_constant__ CUtensorMap tmH, DwParams p) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  // contiguous run of tiles: x fastest, then rows, then (image, plane)
+  // contiguous run of tiles: down a column of tiles first (the two halo rows a tile shares with the one above were
+  // loaded a moment ago), then the next column, then the next (image, plane)
   const long long t_first = p.num_tiles * blockIdx.x / gridDim.x, t_end = p.num_tiles * (blockIdx.x + 1) / gridDim.x;
   const int per_z = p.tiles_x * p.tiles_y;
   pdl_wait();  // h is the previous kernel's output; g may still be read by an earlier one
@@ -96,10 +96,13 @@ ffn_dw3x3_kernel(const __grid_constant__ CUtensorMap tmH, DwParams p) {
         const uint32_t s = it % DW_STAGES, ph = (it / DW_STAGES) & 1;
         if (!mbar_wait(empty_bar + 8 * s, ph ^ 1, &abort_flag)) break;
         const int z = (int)(t / per_z), r = (int)(t % per_z);
-        const int ty = r / p.tiles_x, tx = r % p.tiles_x;
+        const int tx = r / p.tiles_y, ty = r % p.tiles_y;
         mbar_expect_tx(full_bar + 8 * s, DW_TILE_BYTES);
-        tma_load_tile(ring + s * DW_STAGE_BYTES, &tmH, full_bar + 8 * s, 0, tx * DW_PX - 1, ty * DW_ROWS - 1, 2 * z);
-        tma_load_tile(ring + s * DW_STAGE_BYTES + DW_HALF_STRIDE, &tmH, full_bar + 8 * s, 0, tx * DW_PX - 1, ty * DW_ROWS - 1, 2 * z + 1);
+        for (int row = 0; row < DW_BOX_ROWS; ++row) {  // one box per image row and input plane, each into its own slot
+          const uint32_t dst = ring + s * DW_STAGE_BYTES + row * DW_ROW_PITCH;
+          tma_load_tile(dst, &tmH, full_bar + 8 * s, 0, tx * DW_PX - 1, ty * DW_ROWS - 1 + row, 2 * z);
+          tma_load_tile(dst + DW_HALF_STRIDE, &tmH, full_bar + 8 * s, 0, tx * DW_PX - 1, ty * DW_ROWS - 1 + row, 2 * z + 1);
+        }
       }
     }
   } else {
@@ -108,6 +111,10 @@ ffn_dw3x3_kernel(const __grid_constant__ CUtensorMap tmH, DwParams p) {
     const int piece = lane & 7, side = lane >> 4;
     const int ch = side * 32 + piece * 4;       // first of the thread's 4 channels inside the 64-channel output plane
     const int px = warp * 2 + ((lane >> 3) & 1);
+    uint32_t pre[3];  // offset of the thread's 8 bytes of pixel px + dx inside a row slot (64B swizzle: 16-byte chunk XOR pixel bits 1-2)
+#pragma unroll
+    for (int dx = 0; dx < 3; ++dx)
+      pre[dx] = (uint32_t)(px + dx) * 64u + ((((uint32_t)piece >> 1) ^ (((uint32_t)(px + dx) >> 1) & 3u)) << 4) + (((uint32_t)piece & 1u) << 3);
     float wt[9][4], bias[4];
     int plane_loaded = -1;
     uint32_t it = 0;
@@ -115,7 +122,7 @@ ffn_dw3x3_kernel(const __grid_constant__ CUtensorMap tmH, DwParams p) {
     for (long long t = t_first; ok && t < t_end; ++t, ++it) {
       const uint32_t s = it % DW_STAGES, ph = (it / DW_STAGES) & 1;
       const int z = (int)(t / per_z), r0 = (int)(t % per_z);
-      const int ty = r0 / p.tiles_x, tx = r0 % p.tiles_x;
+      const int tx = r0 / p.tiles_y, ty = r0 % p.tiles_y;
       const int plane = z % p.planes;
       if (plane != plane_loaded) {  // the thread's 4 channels x 9 taps: 72 contiguous bytes of the weight tensor
         const uint2* wp = reinterpret_cast<const uint2*>(p.w_dw + (long long)(plane * 64 + ch) * 9);
@@ -154,10 +161,8 @@ ffn_dw3x3_kernel(const __grid_constant__ CUtensorMap tmH, DwParams p) {
         float in[3][4];
 #pragma unroll
         for (int dx = 0; dx < 3; ++dx) {
-          const uint32_t row = (uint32_t)(r * DW_BOX_PX + px + dx);
-          uint2 v;  // 64B swizzle: 16-byte chunk index XOR bits 1-2 of the row
-          asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y)
-                       : "r"(tile + row * 64 + ((((uint32_t)piece >> 1) ^ ((row >> 1) & 3u)) << 4) + (((uint32_t)piece & 1u) << 3)));
+          uint2 v;
+          asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(tile + r * DW_ROW_PITCH + pre[dx]));
           in[dx][0] = __uint_as_float(v.x << 16); in[dx][1] = __uint_as_float(v.x & 0xffff0000u);
           in[dx][2] = __uint_as_float(v.y << 16); in[dx][3] = __uint_as_float(v.y & 0xffff0000u);
         }
@@ -179,8 +184,11 @@ ffn_dw3x3_kernel(const __grid_constant__ CUtensorMap tmH, DwParams p) {
         if (od >= 0 && y0 + od < p.H && x < p.W) {
           const float (&a)[4] = acc[od % 3];
           uint2 out;
-          out.x = pack2(dw_act(a[0], p.act), dw_act(a[1], p.act));
-          out.y = pack2(dw_act(a[2], p.act), dw_act(a[3], p.act));
+          float o4[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) o4[i] = a[i] * __saturatef(fmaf(a[i], p.act_a, p.act_b));
+          out.x = pack2(o4[0], o4[1]);
+          out.y = pack2(o4[2], o4[3]);
           *reinterpret_cast<uint2*>(gp + ((long long)(y0 + od) * p.W + x) * 64) = out;
         }
       }
@@ -203,12 +211,14 @@ msla_status_t run_ffn_dw3x3_bf16(const void* h, const void* w_dw, const void* b_
   CUtensorMap tmH;
   const cuuint64_t dims[4] = {32, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)(2 * z)};
   const cuuint64_t strides[3] = {64, (cuuint64_t)W * 64, (cuuint64_t)H * W * 64};
-  const cuuint32_t box[4] = {32, DW_BOX_PX, DW_BOX_ROWS, 1};
+  const cuuint32_t box[4] = {32, DW_BOX_PX, 1, 1};  // one image row of a tile with its halo columns
   if (!tma_make_map_bf16(&tmH, h, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B))
     return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the FFN's depthwise convolution");
   DwParams p{};
   p.w_dw = (const bf16*)w_dw; p.b_dw = (const bf16*)b_dw; p.g = (bf16*)g;
-  p.H = H; p.W = W; p.planes = Ch / 64; p.act = act;
+  p.H = H; p.W = W; p.planes = Ch / 64;
+  p.act_a = act == 2 ? 1.f / 6.f : (act == 1 ? 1e30f : 0.f);
+  p.act_b = act == 2 ? 0.5f : (act == 1 ? 0.f : 1.f);
   p.tiles_x = (W + DW_PX - 1) / DW_PX; p.tiles_y = (H + DW_ROWS - 1) / DW_ROWS;
   p.num_tiles = z * p.tiles_x * p.tiles_y;
   static std::atomic<unsigned long long> attr_done{0};
