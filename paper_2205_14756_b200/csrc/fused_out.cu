@@ -60,6 +60,7 @@ __device__ int g_fused_timeout_flag = 0;
 struct OutParams {
   const float* ks;   // [B][Ht][d] key sums
   const bf16* bias;  // [Cout] or nullptr
+  const bf16* residual;  // RES kernels: [B][Cout][N], added to the output (the residual connection around the module)
   int B, N, Cout, Ht, d;
   int kslices;       // 64-wide k-slices of M: ceil(Ht * d / 64)
   int ot;            // tokens per CTA and tile: 128 or 64
@@ -209,7 +210,7 @@ state_fold_kernel(const float* __restrict__ partial, int S, const bf16* __restri
   }
 }
 
-template <int D>
+template <int D, bool RES>
 __global__ void __launch_bounds__(O_THREADS, 1)
 fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmQ,
                  const __grid_constant__ CUtensorMap tmO, OutParams p) {
@@ -427,11 +428,23 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
       uint32_t r[2][32];
       tmem_ld32(taddr, r[0]);
       const int chunks = (2 * p.ot) / 32;  // the accumulator's columns are the pair's tokens
+      // RES: the lane's channel row of the residual, 32 tokens (64 bytes) per chunk, fetched one chunk ahead
+      const bf16* res_row = (RES && row0 + lane < p.Cout) ? p.residual + ((long long)b * p.Cout + row0 + lane) * p.N : nullptr;
+      uint4 rs[2][4];
+      auto load_residual = [&](int c) {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          const int n = nt * (2 * p.ot) + c * 32 + v * 8;
+          rs[c & 1][v] = (res_row && n < p.N) ? __ldg(reinterpret_cast<const uint4*>(res_row + n)) : make_uint4(0u, 0u, 0u, 0u);
+        }
+      };
+      if (RES) load_residual(0);
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         if (c >= chunks) break;
         tmem_ld_wait();
         if (c + 1 < chunks) tmem_ld32(taddr + (c + 1) * 32, r[(c + 1) & 1]);  // next chunk streams in meanwhile
+        if (RES && c + 1 < chunks) load_residual(c + 1);
         const uint32_t(&rc)[32] = r[c & 1];
         const int n0 = nt * (2 * p.ot) + (c >> 1) * 64;  // first token of the 64-token block
         if (n0 >= p.N || row0 >= p.Cout) continue;    // warp-uniform
@@ -443,8 +456,14 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
         for (int v = 0; v < 4; ++v) {
           uint32_t w[4];
 #pragma unroll
-          for (int e = 0; e < 4; ++e)
-            w[e] = pack2(__uint_as_float(rc[v * 8 + 2 * e]) + bias, __uint_as_float(rc[v * 8 + 2 * e + 1]) + bias);
+          for (int e = 0; e < 4; ++e) {
+            float f0 = __uint_as_float(rc[v * 8 + 2 * e]) + bias, f1 = __uint_as_float(rc[v * 8 + 2 * e + 1]) + bias;
+            if (RES) {
+              const uint32_t rw = e == 0 ? rs[c & 1][v].x : e == 1 ? rs[c & 1][v].y : e == 2 ? rs[c & 1][v].z : rs[c & 1][v].w;
+              f0 += __uint_as_float(rw << 16); f1 += __uint_as_float(rw & 0xffff0000u);
+            }
+            w[e] = pack2(f0, f1);
+          }
           const uint32_t pc = (uint32_t)((c & 1) * 4 + v);
           asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(my_row + ((pc ^ sw) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]),
                        "r"(w[3]) : "memory");
@@ -496,8 +515,8 @@ size_t fused_out_scratch_bytes(int B, int Ht, int d, int Cout) { return fused_ou
 // column d).  q: planar bf16 query matrices [N][d], head h of image b at q + b*q_sb + h*q_sh (elements); y: NCHW
 // [B, Cout, N].
 msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, const float* partial, int S, void* scratch,
-                                 const void* w, const void* bias, void* y, int B, int Ht, int d, int N, int Cout, float eps,
-                                 cudaStream_t st) {
+                                 const void* w, const void* bias, const void* residual, void* y, int B, int Ht, int d, int N, int Cout,
+                                 float eps, cudaStream_t st) {
   if (!fused_out_bf16_supported(Ht, d, Cout, N) || q_sb % 8 != 0 || q_sh % 8 != 0)
     return fail(MSLA_ERR_UNSUPPORTED, "fused apply + projection: %d heads of %d channels, %d output channels, %d tokens", Ht, d, Cout, N);
   if (S < 1 || S > 8 * FOLD_RUNS) return fail(MSLA_ERR_UNSUPPORTED, "fused apply + projection: %d partial states per head (1 .. %d)", S, 8 * FOLD_RUNS);
@@ -525,7 +544,7 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
       return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the fused apply + output projection");
   }
   OutParams p{};
-  p.ks = ks; p.bias = (const bf16*)bias;
+  p.ks = ks; p.bias = (const bf16*)bias; p.residual = (const bf16*)residual;
   p.B = B; p.N = N; p.Cout = Cout; p.Ht = Ht; p.d = d; p.eps = eps;
   p.kslices = (K + OKS - 1) / OKS;
   p.ot = ot;
@@ -534,10 +553,12 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   if (tiles > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many token tiles");
   p.num_tiles = (int)tiles;
   const int smem = p.kslices * O_A_SLICE + O_STAGES * (OT * d * 2) + O_STAGING + O_BAR_BYTES + 1024;
-  static std::atomic<unsigned long long> attr_done{0}, attr_done16{0};
+  static std::atomic<unsigned long long> attr_done{0}, attr_done16{0}, attr_res{0}, attr_res16{0};
   constexpr int smem_max = O_SMEM_MAX;
-  msla_status_t s = ensure_smem_attr(attr_done, fused_out_kernel<32>, smem_max);
-  if (s == MSLA_OK) s = ensure_smem_attr(attr_done16, fused_out_kernel<16>, smem_max);
+  msla_status_t s = ensure_smem_attr(attr_done, fused_out_kernel<32, false>, smem_max);
+  if (s == MSLA_OK) s = ensure_smem_attr(attr_done16, fused_out_kernel<16, false>, smem_max);
+  if (s == MSLA_OK && residual) s = ensure_smem_attr(attr_res, fused_out_kernel<32, true>, smem_max);
+  if (s == MSLA_OK && residual) s = ensure_smem_attr(attr_res16, fused_out_kernel<16, true>, smem_max);
   if (s != MSLA_OK) return s;
   long long pairs = sms / 2;
   if (pairs > tiles) pairs = tiles;
@@ -549,8 +570,11 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   if ((s = ensure_smem_attr(attr_fold, state_fold_kernel, FOLD_SMEM)) != MSLA_OK) return s;
   launch_pdl(state_fold_kernel, dim3((unsigned)(B * Ht), (unsigned)fold_chunks), dim3(FOLD_THREADS), FOLD_SMEM, st, partial, S,
              (const bf16*)w, M, ks, Ht, d, Cout, K, d / fold_chunks);
-  if (d == 32) launch_pdl_cluster2(fused_out_kernel<32>, dim3((unsigned)(2 * pairs)), dim3(O_THREADS), (size_t)smem, st, tmM, tmQ, tmO, p);
-  else launch_pdl_cluster2(fused_out_kernel<16>, dim3((unsigned)(2 * pairs)), dim3(O_THREADS), (size_t)smem, st, tmM, tmQ, tmO, p);
+  const dim3 grid((unsigned)(2 * pairs)), block(O_THREADS);
+  if (d == 32 && !residual) launch_pdl_cluster2(fused_out_kernel<32, false>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, p);
+  else if (d == 32) launch_pdl_cluster2(fused_out_kernel<32, true>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, p);
+  else if (!residual) launch_pdl_cluster2(fused_out_kernel<16, false>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, p);
+  else launch_pdl_cluster2(fused_out_kernel<16, true>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, p);
   count_launches(2);
   return check_launch("fused apply + output projection (tcgen05, paired CTAs)");
 }

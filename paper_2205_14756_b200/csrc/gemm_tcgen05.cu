@@ -581,8 +581,8 @@ msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, 
 bool project_out_bf16_supported(int Cin, int Cout, int N) { return Cin % 8 == 0 && N % 8 == 0 && Cout >= 1; }
 
 // y[b][m][n] = sum_j w[m][j] * a[b][n][j] + bias[m];  a token-major [B, N, Cin], y NCHW [B, Cout, N].
-msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin, int Cout,
-                                   int N, cudaStream_t st) {
+msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bias, const void* residual, void* y, int B, int Cin,
+                                   int Cout, int N, cudaStream_t st) {
   CUtensorMap tmA, tmB;
   if (!make_map(&tmA, w, (uint64_t)Cin, (uint64_t)Cout, 1, (uint64_t)Cin * 2, (uint64_t)Cin * Cout * 2, BK, BM) ||
       !make_map(&tmB, a, (uint64_t)Cin, (uint64_t)N, (uint64_t)B, (uint64_t)Cin * 2, (uint64_t)N * Cin * 2, BK, BN))
@@ -601,14 +601,15 @@ msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bia
     if (!tma_make_map_bf16(&tmO, y, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B))
       return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the output projection's output");
   }
-  return launch<false>(tmA, tmB, tmO, p, st);
+  p.residual = (const bf16*)residual;
+  return residual ? launch<false, false, 2>(tmA, tmB, tmO, p, st) : launch<false>(tmA, tmB, tmO, p, st);
 }
 
 bool project_out_planar_bf16_supported(int Cin, int Cout, int N) { return Cin % 64 == 0 && N % 8 == 0 && Cout >= 1; }
 
 // Same product with the attention output kept planar: a[b][j / 64][n][j % 64] (one [N][64] plane per pair of heads).
-msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin,
-                                          int Cout, int N, cudaStream_t st) {
+msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const void* bias, const void* residual, void* y, int B,
+                                          int Cin, int Cout, int N, cudaStream_t st) {
   CUtensorMap tmA, tmB, tmO;
   const int planes = Cin / 64;
   {
@@ -626,7 +627,8 @@ msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const vo
   p.out_batch_stride = (long long)Cout * N; p.ld_out = N; p.group = 0; p.bias_per_row = 1; p.n_fastest = 0;
   p.bias = (const bf16*)bias; p.out = (bf16*)y;
   p.tma_store = 1; p.planes_per_batch = planes;
-  return launch<false, true>(tmA, tmB, tmO, p, st);
+  p.residual = (const bf16*)residual;
+  return residual ? launch<false, true, 2>(tmA, tmB, tmO, p, st) : launch<false, true>(tmA, tmB, tmO, p, st);
 }
 
 // ---- the two linear layers of the FFN with a depthwise convolution (Section 3.1, Fig. 2 left)

@@ -125,31 +125,6 @@ ffn_dw3x3_nchw_kernel(const T* __restrict__ h, const T* __restrict__ w, const T*
   g[idx] = from_f32<T>(act_f32(acc, act));
 }
 
-// y[i] = a[i] + b[i] (the residual connection around the attention module, Fig. 2 left)
-template <typename T>
-__global__ void __launch_bounds__(256)
-add_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ y, long long total) {
-  const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
-  if (idx < total) y[idx] = from_f32<T>(to_f32(a[idx]) + to_f32(b[idx]));
-}
-// bf16, 8 elements (16 bytes) per thread; total8 = elements / 8.  a may alias y.
-__global__ void __launch_bounds__(256)
-add_bf16x8_kernel(const uint4* a, const uint4* __restrict__ b, uint4* y, long long total8) {
-  const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
-  if (idx >= total8) return;
-  const uint4 va = a[idx], vb = __ldg(b + idx);
-  const uint32_t wa[4] = {va.x, va.y, va.z, va.w}, wb[4] = {vb.x, vb.y, vb.z, vb.w};
-  uint32_t r[4];
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const float lo = __uint_as_float(wa[e] << 16) + __uint_as_float(wb[e] << 16);
-    const float hi = __uint_as_float(wa[e] & 0xffff0000u) + __uint_as_float(wb[e] & 0xffff0000u);
-    const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
-    r[e] = *reinterpret_cast<const uint32_t*>(&p);
-  }
-  y[idx] = make_uint4(r[0], r[1], r[2], r[3]);
-}
-
 // ---------------------------------------------------------------------------
 // Multi-scale token aggregation (Section 3.1): 5x5 depthwise convolution
 // (cross-correlation, zero padding 2) followed by the grouped 1x1 convolution,

@@ -303,9 +303,9 @@ static msla_status_t run_project_in(msla_dtype_t dt, const void* x, const void* 
 }
 
 static msla_status_t run_project_out(msla_dtype_t dt, const void* a, const void* w, const void* bias,
-                                     void* y, int B, int Cin, int Cout, int N, cudaStream_t st) {
-  if (dt == MSLA_BF16 && project_out_bf16_supported(Cin, Cout, N)) return run_project_out_bf16(a, w, bias, y, B, Cin, Cout, N, st);
-  generic::GemmArgs g{(long long)N * Cin, Cin, 1, (long long)Cout * N, 1, N, 0, N, Cout, Cin, Cout};
+                                     void* y, int B, int Cin, int Cout, int N, cudaStream_t st, const void* residual = nullptr) {
+  if (dt == MSLA_BF16 && project_out_bf16_supported(Cin, Cout, N)) return run_project_out_bf16(a, w, bias, residual, y, B, Cin, Cout, N, st);
+  generic::GemmArgs g{(long long)N * Cin, Cin, 1, (long long)Cout * N, 1, N, 0, N, Cout, Cin, Cout, 0, residual};
   if (dt == MSLA_F32) launch_gemm<float>((const float*)a, (const float*)w, (const float*)bias, (float*)y, g, B, st);
   else launch_gemm<__nv_bfloat16>((const __nv_bfloat16*)a, (const __nv_bfloat16*)w, (const __nv_bfloat16*)bias, (__nv_bfloat16*)y, g, B, st);
   return check_launch("output projection");
@@ -356,8 +356,9 @@ static msla_status_t record(void* const* events, int i, cudaStream_t st) {
 }
 
 // host_io: x and out are host pointers staged through the tail of the workspace.
+// residual: nullptr, or a device tensor shaped like out that the output projection adds (the block's first residual connection).
 static msla_status_t forward_impl(const msla_desc* desc, const void* x, const msla_weights* w, void* out,
-                                  cudaStream_t st, void* const* events, bool host_io) {
+                                  cudaStream_t st, void* const* events, bool host_io, const void* residual = nullptr) {
   ForwardPlan p;
   msla_status_t s = validate_desc(desc, &p);
   if (s != MSLA_OK) return s;
@@ -422,10 +423,10 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   // 5. output projection back to NCHW
   if (fused)
     s = run_fused_out_bf16(ms, ms_sb, 3LL * N * d, reinterpret_cast<const float*>(ws + p.core_off + p.core.partial_off), p.core.S, att, w->w_proj,
-                           w->b_proj, out_dev, desc->B, 2 * heads, d, N, desc->C_out, desc->eps, st);
+                           w->b_proj, residual, out_dev, desc->B, 2 * heads, d, N, desc->C_out, desc->eps, st);
   else
-    s = att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st)
-                   : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st);
+    s = att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, residual, out_dev, desc->B, 2 * Cp, desc->C_out, N, st)
+                   : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st, residual);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 5, st)) != MSLA_OK) return s;
   if (host_io) {
@@ -532,7 +533,7 @@ static msla_status_t band_output_impl(const msla_desc* desc, const msla_weights*
   if ((s = check_launch("sum of the bands' states")) != MSLA_OK) return s;
   const char* q = ms + (size_t)b.tok_off * d * e;
   if (desc->dtype == MSLA_BF16 && fused_out_bf16_supported(2 * heads, d, desc->C_out, Nb))
-    return run_fused_out_bf16(q, ms_sb, 3LL * N * d, state, 1, att, w->w_proj, w->b_proj, out, desc->B, 2 * heads, d, Nb, desc->C_out, desc->eps, st);
+    return run_fused_out_bf16(q, ms_sb, 3LL * N * d, state, 1, att, w->w_proj, w->b_proj, nullptr, out, desc->B, 2 * heads, d, Nb, desc->C_out, desc->eps, st);
   const HeadView in{ms_sb, 3LL * N * d, d};
   const bool att_planar = desc->dtype == MSLA_BF16 && d == 32 && project_out_planar_bf16_supported(2 * Cp, desc->C_out, Nb);
   const HeadView ov = att_planar ? HeadView{(long long)Nb * ld_att, (long long)Nb * 2 * d, 2 * d, 1}
@@ -540,7 +541,7 @@ static msla_status_t band_output_impl(const msla_desc* desc, const msla_weights*
   s = run_core(desc->dtype, q, q + (size_t)N * d * e, q + (size_t)2 * N * d * e, att, in, ov, desc->B, 2 * heads, Nb, d, desc->eps, b.core,
                ws + p.core_off, st, nullptr, CORE_APPLY);
   if (s != MSLA_OK) return s;
-  return att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, out, desc->B, 2 * Cp, desc->C_out, Nb, st)
+  return att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, nullptr, out, desc->B, 2 * Cp, desc->C_out, Nb, st)
                     : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out, desc->B, 2 * Cp, desc->C_out, Nb, st);
 }
 
@@ -638,15 +639,8 @@ static msla_status_t block_impl(const msla_desc* attn, const msla_weights* aw, c
   if (overlaps(y, bytes, x, bytes) || overlaps(y, bytes, out, bytes) ||
       (attn->workspace && overlaps(y, bytes, attn->workspace, ap.bytes)) || (ffn->workspace && overlaps(y, bytes, ffn->workspace, fp.bytes)))
     return fail(MSLA_ERR_INVALID_ARG, "y overlaps x, out or a workspace");
-  // y = MSLA(x), then y += x
-  if ((s = forward_impl(attn, x, aw, y, st, nullptr, false)) != MSLA_OK) return s;
-  const long long total = (long long)attn->B * attn->C * ap.N;
-  if (attn->dtype == MSLA_F32)
-    generic::add_kernel<float><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const float*)y, (const float*)x, (float*)y, total);
-  else  // C is a multiple of 8, so is the element count
-    generic::add_bf16x8_kernel<<<(unsigned)ceil_div_ll(total / 8, 256), 256, 0, st>>>((const uint4*)y, (const uint4*)x, (uint4*)y, total / 8);
-  count_launches(1);
-  if ((s = check_launch("residual connection around the attention module")) != MSLA_OK) return s;
+  // y = MSLA(x) + x: the output projection's epilogue adds the residual
+  if ((s = forward_impl(attn, x, aw, y, st, nullptr, false, x)) != MSLA_OK) return s;
   return ffn_impl(ffn, y, fw, out, true, st);
 }
 

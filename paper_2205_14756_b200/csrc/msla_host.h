@@ -118,8 +118,8 @@ msla_status_t run_ffn_project_bf16(const void* g, const void* w2, const void* b2
 bool fused_out_bf16_supported(int Ht, int d, int Cout, int N);
 size_t fused_out_scratch_bytes(int B, int Ht, int d, int Cout);
 msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, const float* partial, int S, void* scratch,
-                                 const void* w, const void* bias, void* y, int B, int Ht, int d, int N, int Cout, float eps,
-                                 cudaStream_t st);
+                                 const void* w, const void* bias, const void* residual, void* y, int B, int Ht, int d, int N, int Cout,
+                                 float eps, cudaStream_t st);
 int fused_timeout_flag();
 int dw_timeout_flag();
 
@@ -128,11 +128,12 @@ bool project_in_bf16_supported(int C, int Cout, int N, int d);
 msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d,
                                   long long y_batch_stride, cudaStream_t st);
 bool project_out_bf16_supported(int Cin, int Cout, int N);
-msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin, int Cout,
-                                   int N, cudaStream_t st);
+// residual: nullptr, or a tensor shaped like y that is added to it
+msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bias, const void* residual, void* y, int B, int Cin,
+                                   int Cout, int N, cudaStream_t st);
 bool project_out_planar_bf16_supported(int Cin, int Cout, int N);
-msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const void* bias, void* y, int B, int Cin,
-                                          int Cout, int N, cudaStream_t st);
+msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const void* bias, const void* residual, void* y, int B,
+                                          int Cin, int Cout, int N, cudaStream_t st);
 int gemm_timeout_flag();
 int run_wait_selftest(long long limit_cycles, int* scratch, cudaStream_t st);
 
