@@ -127,7 +127,8 @@ msla_status_t msla_linattn_relu_noalloc(msla_dtype_t dtype, const void* q, const
  *      out = 1x1 conv (att, w_proj) (+ b_proj)      2C' -> C_out
  *
  * with C' = heads*d.  Section 4.1 fixes two branches and 5x5 aggregation;
- * n_scales must be 2 and agg_kernel must be 5.  No bias, normalisation or
+ * n_scales must be 2; agg_kernel is 5, or 3 (another small kernel in the sense
+ * of Section 3.1; it runs through the same kernels).  No bias, normalisation or
  * activation sits between the stages; the residual connection around the
  * module is the caller's.
  * ------------------------------------------------------------------------- */
@@ -136,7 +137,7 @@ typedef struct {
   int B, C, H, W;         /* input x is [B, C, H, W] */
   int heads, d;           /* heads per scale and channels per head; d in {16, 32} */
   int n_scales;           /* 2 */
-  int agg_kernel;         /* 5 */
+  int agg_kernel;         /* 5 (Section 4.1) or 3 */
   int C_out;              /* output channels */
   msla_dtype_t dtype;     /* type of x, out and all weights */
   float eps;              /* added to the attention denominator */

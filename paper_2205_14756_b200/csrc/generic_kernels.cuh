@@ -125,6 +125,18 @@ ffn_dw3x3_nchw_kernel(const T* __restrict__ h, const T* __restrict__ w, const T*
   g[idx] = from_f32<T>(act_f32(acc, act));
 }
 
+// 3x3 depthwise taps embedded in a 5x5 filter with a ring of zeros: w5[c][r][s] = w3[c][r-1][s-1] inside, 0 outside.
+template <typename T>
+__global__ void __launch_bounds__(256)
+embed_taps_kernel(const T* __restrict__ w3, T* __restrict__ w5, long long total) {
+  const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (idx >= total) return;
+  const long long c = idx / 25;
+  const int r = (int)(idx % 25) / 5, s = (int)(idx % 5);
+  const bool inside = r >= 1 && r <= 3 && s >= 1 && s <= 3;
+  w5[idx] = inside ? w3[c * 9 + (r - 1) * 3 + (s - 1)] : from_f32<T>(0.f);
+}
+
 // ---------------------------------------------------------------------------
 // Multi-scale token aggregation (Section 3.1): 5x5 depthwise convolution
 // (cross-correlation, zero padding 2) followed by the grouped 1x1 convolution,

@@ -251,7 +251,7 @@ static msla_status_t core_entry_noalloc(msla_dtype_t dtype, const void* q, const
 
 // ------------------------------------------------------------- module plan
 struct ForwardPlan {
-  size_t ms_off, att_off, core_off, bytes;
+  size_t ms_off, att_off, core_off, wpad_off, bytes;  // wpad: 3x3 aggregation taps embedded in 5x5 (agg_kernel == 3)
   CorePlan core;
   int Cp, N;
 };
@@ -264,7 +264,8 @@ static msla_status_t validate_desc(const msla_desc* d, ForwardPlan* plan) {
     return fail(MSLA_ERR_INVALID_ARG, "B, C, H, W, heads, d, C_out must be positive");
   if (!(d->eps >= 0.f)) return fail(MSLA_ERR_INVALID_ARG, "eps must be >= 0");
   if (d->n_scales != 2) return fail(MSLA_ERR_UNSUPPORTED, "n_scales = %d; the module has two branches", d->n_scales);
-  if (d->agg_kernel != 5) return fail(MSLA_ERR_UNSUPPORTED, "agg_kernel = %d; only 5x5 aggregation is supported", d->agg_kernel);
+  if (d->agg_kernel != 5 && d->agg_kernel != 3)
+    return fail(MSLA_ERR_UNSUPPORTED, "agg_kernel = %d; 5x5 and 3x3 aggregation are supported", d->agg_kernel);
   if (d->d != 16 && d->d != 32) return fail(MSLA_ERR_UNSUPPORTED, "d = %d; only 16 and 32 are supported", d->d);
   if ((long long)d->H * d->W > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "H*W exceeds 2^31-1");
   if (d->C % 8 != 0 || d->C_out % 8 != 0) return fail(MSLA_ERR_UNSUPPORTED, "C and C_out must be multiples of 8");
@@ -281,7 +282,8 @@ static msla_status_t validate_desc(const msla_desc* d, ForwardPlan* plan) {
   const size_t fused_scratch = fused_out_bf16_supported(2 * d->heads, d->d, d->C_out, plan->N) ? fused_out_scratch_bytes(d->B, 2 * d->heads, d->d, d->C_out) : 0;
   if (att_bytes < fused_scratch) att_bytes = fused_scratch;
   plan->core_off = plan->att_off + align_up(att_bytes, 256);
-  plan->bytes = plan->core_off + plan->core.bytes;
+  plan->wpad_off = plan->core_off + plan->core.bytes;
+  plan->bytes = plan->wpad_off + (d->agg_kernel == 3 ? align_up((size_t)3 * plan->Cp * 25 * e, 256) : 0);
   return MSLA_OK;
 }
 
@@ -345,6 +347,20 @@ static msla_status_t run_aggregate(msla_dtype_t dt, const void* src, const void*
   return check_launch("token aggregation");
 }
 
+// The aggregation kernels are 5x5.  A 3x3 depthwise filter (another of Section 3.1's small kernels) is the same
+// filter with a ring of zero taps around it: w5[c][dy+1][dx+1] = w3[c][dy][dx].  Returns the taps to use.
+static const void* aggregation_taps(const msla_desc* desc, const msla_weights* w, const ForwardPlan& p, cudaStream_t st) {
+  if (desc->agg_kernel == 5) return w->w_dw;
+  void* w5 = (char*)desc->workspace + p.wpad_off;
+  const long long total = 3LL * p.Cp * 25;
+  if (desc->dtype == MSLA_F32)
+    generic::embed_taps_kernel<float><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const float*)w->w_dw, (float*)w5, total);
+  else
+    generic::embed_taps_kernel<__nv_bfloat16><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const __nv_bfloat16*)w->w_dw, (__nv_bfloat16*)w5, total);
+  count_launches(1);
+  return w5;
+}
+
 static msla_status_t record(void* const* events, int i, cudaStream_t st) {
   if (!events) return MSLA_OK;
   const cudaError_t e = cudaEventRecord((cudaEvent_t)events[i], st);
@@ -403,7 +419,7 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   if (s != MSLA_OK) return s;
   if ((s = record(events, 1, st)) != MSLA_OK) return s;
   // 2. aggregation of every scale-0 plane into the matching scale-1 plane
-  s = run_aggregate(desc->dtype, ms, w->w_dw, w->w_pw, ms + (size_t)3 * Cp * N * e, desc->B, desc->H, desc->W, 3 * Cp, d, ms_sb, ms_sb, st);
+  s = run_aggregate(desc->dtype, ms, aggregation_taps(desc, w, p, st), w->w_pw, ms + (size_t)3 * Cp * N * e, desc->B, desc->H, desc->W, 3 * Cp, d, ms_sb, ms_sb, st);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 2, st)) != MSLA_OK) return s;
   // 3+4. attention over 2*heads heads of [q|k|v]; outputs land at channel head*d (concat)
@@ -489,7 +505,7 @@ static msla_status_t band_states_impl(const msla_desc* desc, const void* x, cons
   char* ms = ws + p.ms_off;
   s = run_project_in(desc->dtype, x, w->w_qkv, ms, desc->B, desc->C, 3 * Cp, N, d, ms_sb, st);
   if (s != MSLA_OK) return s;
-  s = run_aggregate(desc->dtype, ms, w->w_dw, w->w_pw, ms + (size_t)3 * Cp * N * e, desc->B, desc->H, desc->W, 3 * Cp, d, ms_sb, ms_sb, st);
+  s = run_aggregate(desc->dtype, ms, aggregation_taps(desc, w, p, st), w->w_pw, ms + (size_t)3 * Cp * N * e, desc->B, desc->H, desc->W, 3 * Cp, d, ms_sb, ms_sb, st);
   if (s != MSLA_OK) return s;
   const HeadView in{ms_sb, 3LL * N * d, d};
   const char* q = ms + (size_t)b.tok_off * d * e;

@@ -67,6 +67,15 @@ def test_module_with_bias_and_different_c_out(B, C, H, W, heads, d, c_out, with_
     assert binding.msla_debug_wait_timeouts() == 0
 
 
+# A 3x3 aggregation filter (another of Section 3.1's small kernels): same kernels, taps embedded in 5x5.
+@pytest.mark.parametrize("dtype,B,C,H,W,heads,d", [("f32", 1, 32, 9, 11, 2, 16), ("bf16", 2, 64, 24, 40, 2, 32), ("bf16", 1, 96, 16, 16, 6, 16)])
+def test_module_with_3x3_aggregation(dtype, B, C, H, W, heads, d):
+    s = inputs.ModuleShape("agg3", dtype, B, C, H, W, heads, d, seed=41, agg_kernel=3)
+    t = inputs.module_inputs(s)
+    assert t["w_dw"].shape[-2:] == (3, 3)
+    util.assert_close(util.run_module(s, t), _ref(s, t), dtype, "3x3 aggregation", block=util.MODULE_BLOCK if dtype == "bf16" else None)
+
+
 def test_config3_bf16():
     s = inputs.CONFIG3
     t = inputs.module_inputs(s)

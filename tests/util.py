@@ -129,12 +129,12 @@ def run_module(s: inputs.ModuleShape, t: dict, bias=None) -> np.ndarray:
     x, w_qkv, w_dw, w_pw, w_proj = (dev(t[n], dt) for n in ("x", "w_qkv", "w_dw", "w_pw", "w_proj"))
     b = dev(bias, dt) if bias is not None else None
     c_out = t["w_proj"].shape[0]
-    desc = binding.make_desc(s.B, s.C, s.H, s.W, s.heads, s.d, c_out, CODE[dt], s.eps)
+    desc = binding.make_desc(s.B, s.C, s.H, s.W, s.heads, s.d, c_out, CODE[dt], s.eps, agg_kernel=s.agg_kernel)
     nbytes = binding.msla_forward_workspace_bytes(desc)
     assert nbytes > 0
     wg = Guarded(nbytes)
     ws = wg.view(torch.float32, (nbytes // 4,))
-    desc = binding.make_desc(s.B, s.C, s.H, s.W, s.heads, s.d, c_out, CODE[dt], s.eps, workspace=ws)
+    desc = binding.make_desc(s.B, s.C, s.H, s.W, s.heads, s.d, c_out, CODE[dt], s.eps, agg_kernel=s.agg_kernel, workspace=ws)
     esz = 4 if dt == "f32" else 2
     og = Guarded(s.B * c_out * s.H * s.W * esz)
     out = og.view(TORCH_DTYPE[dt], (s.B, c_out, s.H, s.W))
