@@ -54,6 +54,8 @@ def _load() -> ctypes.CDLL:
         lib.oracle_linattn_relu.restype = None
         lib.oracle_msla_forward.argtypes = [_dp] * 7 + [ctypes.c_int] * 8 + [ctypes.c_double]
         lib.oracle_msla_forward.restype = ctypes.c_int
+        lib.oracle_msla_forward3.argtypes = [_dp] * 9 + [ctypes.c_int] * 9 + [ctypes.c_double]
+        lib.oracle_msla_forward3.restype = ctypes.c_int
         lib.oracle_bias_act.argtypes = [_dp, _dp, ctypes.c_int, ctypes.c_int, ctypes.c_long, ctypes.c_int]
         lib.oracle_bias_act.restype = None
         lib.oracle_ffn_dwconv.argtypes = [_dp] * 8 + [ctypes.c_int] * 9
@@ -142,6 +144,22 @@ def msla_forward(x, w_qkv, w_dw, w_pw, w_proj, b_proj=None, *, heads: int, d: in
                                      _p(out), B, C, H, W, heads, d, k, C_out, float(eps))
     if rc != 0:
         raise MemoryError("oracle_msla_forward: scratch allocation failed")
+    return out
+
+
+def msla_forward3(x, w_qkv, w_dw, w_pw, w_dw2, w_pw2, w_proj, b_proj=None, *, heads: int, d: int, eps: float = 1e-15) -> np.ndarray:
+    """The module with three branches (projected tokens and two aggregated copies) on NCHW x -> [B, C_out, H, W]."""
+    x, w_qkv, w_dw, w_pw, w_dw2, w_pw2, w_proj = map(_f64, (x, w_qkv, w_dw, w_pw, w_dw2, w_pw2, w_proj))
+    B, C, H, W = x.shape
+    Cp, k1, k2, C_out = heads * d, w_dw.shape[-1], w_dw2.shape[-1], w_proj.shape[0]
+    assert w_qkv.shape == (3 * Cp, C) and w_dw.shape == (3 * Cp, k1, k1) and w_dw2.shape == (3 * Cp, k2, k2)
+    assert w_pw.shape == (3 * Cp, d) and w_pw2.shape == (3 * Cp, d) and w_proj.shape == (C_out, 3 * Cp)
+    b = None if b_proj is None else _f64(b_proj)
+    out = np.empty((B, C_out, H, W), dtype=np.float64)
+    rc = _load().oracle_msla_forward3(_p(x), _p(w_qkv), _p(w_dw), _p(w_pw), _p(w_dw2), _p(w_pw2), _p(w_proj), _p(b), _p(out),
+                                      B, C, H, W, heads, d, k1, k2, C_out, float(eps))
+    if rc != 0:
+        raise MemoryError("oracle_msla_forward3: scratch allocation failed")
     return out
 
 

@@ -296,3 +296,65 @@ int oracle_ffn_dwconv(const double* x, const double* w1, const double* b1, const
   free(h); free(g);
   return rc;
 }
+
+/* ------------------------------------------------------------------------
+ * The module with THREE branches (Section 3.1 builds multi-scale tokens by
+ * aggregating nearby tokens with several small kernels; Section 4.1 then
+ * settles on two branches, which is oracle_msla_forward above): the projected
+ * tokens, and two aggregated copies of them, each through its own depthwise
+ * k x k convolution and grouped 1x1 convolution.  Heads: all heads of branch
+ * 0, then branch 1, then branch 2; w_proj is [C_out, 3C'].  Written out in
+ * full rather than folded into the two-branch function so that each can be
+ * read against the text on its own.  Returns 0, or -1 if an allocation fails.
+ */
+int oracle_msla_forward3(const double* x, const double* w_qkv, const double* w_dw1,
+                         const double* w_pw1, const double* w_dw2, const double* w_pw2,
+                         const double* w_proj, const double* b_proj, double* out, int B, int C,
+                         int H, int W, int heads, int d, int k1, int k2, int C_out, double eps) {
+  const long N = (long)H * W;
+  const int Cp = heads * d;
+  const int C3 = 3 * Cp;
+  const int Ht = 3 * heads;
+  const size_t plane = (size_t)B * C3 * N;
+  double* qkv = (double*)malloc(plane * sizeof(double));
+  double* dw = (double*)malloc(plane * sizeof(double));
+  double* agg1 = (double*)malloc(plane * sizeof(double));
+  double* agg2 = (double*)malloc(plane * sizeof(double));
+  const size_t hsz = (size_t)B * Ht * N * d;
+  double* qh = (double*)malloc(hsz * sizeof(double));
+  double* kh = (double*)malloc(hsz * sizeof(double));
+  double* vh = (double*)malloc(hsz * sizeof(double));
+  double* oh = (double*)malloc(hsz * sizeof(double));
+  double* att = (double*)malloc((size_t)B * 3 * Cp * N * sizeof(double));
+  int rc = -1;
+  if (qkv && dw && agg1 && agg2 && qh && kh && vh && oh && att) {
+    oracle_conv1x1(x, w_qkv, NULL, qkv, B, C, C3, N);
+    oracle_dwconv(qkv, w_dw1, dw, B, C3, H, W, k1);
+    oracle_group1x1(dw, w_pw1, agg1, B, C3, d, N);
+    oracle_dwconv(qkv, w_dw2, dw, B, C3, H, W, k2);
+    oracle_group1x1(dw, w_pw2, agg2, B, C3, d, N);
+    for (int b = 0; b < B; ++b)
+      for (int hh = 0; hh < Ht; ++hh) {
+        const int branch = hh / heads, hs = hh % heads; /* head index inside its branch */
+        const double* src = (branch == 0 ? qkv : branch == 1 ? agg1 : agg2) + (size_t)b * C3 * N;
+        for (long n = 0; n < N; ++n)
+          for (int i = 0; i < d; ++i) {
+            const size_t dst = (((size_t)b * Ht + hh) * N + n) * d + i;
+            qh[dst] = src[((size_t)hs * 3 * d + 0 * d + i) * N + n];
+            kh[dst] = src[((size_t)hs * 3 * d + 1 * d + i) * N + n];
+            vh[dst] = src[((size_t)hs * 3 * d + 2 * d + i) * N + n];
+          }
+      }
+    oracle_linattn_relu(qh, kh, vh, oh, B, Ht, N, d, eps);
+    for (int b = 0; b < B; ++b)
+      for (int hh = 0; hh < Ht; ++hh)
+        for (long n = 0; n < N; ++n)
+          for (int c = 0; c < d; ++c)
+            att[((size_t)b * 3 * Cp + (size_t)hh * d + c) * N + n] =
+                oh[(((size_t)b * Ht + hh) * N + n) * d + c];
+    oracle_conv1x1(att, w_proj, b_proj, out, B, 3 * Cp, C_out, N);
+    rc = 0;
+  }
+  free(qkv); free(dw); free(agg1); free(agg2); free(qh); free(kh); free(vh); free(oh); free(att);
+  return rc;
+}
