@@ -126,9 +126,12 @@ msla_status_t msla_linattn_relu_noalloc(msla_dtype_t dtype, const void* q, const
  *      scale first, then the aggregated scale), then
  *      out = 1x1 conv (att, w_proj) (+ b_proj)      2C' -> C_out
  *
- * with C' = heads*d.  Section 4.1 fixes two branches and 5x5 aggregation;
- * n_scales must be 2; agg_kernel is 5, or 3 (another small kernel in the sense
- * of Section 3.1; it runs through the same kernels).  No bias, normalisation or
+ * with C' = heads*d.  Section 4.1 fixes two branches and 5x5 aggregation:
+ * n_scales = 2, agg_kernel = 5.  Also accepted, in the sense of Section 3.1's
+ * "small kernels" and multi-scale tokens: agg_kernel = 3, and n_scales = 3, a
+ * second aggregated branch with its own filters (w_dw2, w_pw2, agg_kernel2);
+ * the heads of branch 0 come first in the concat, then branch 1, then branch
+ * 2, and w_proj is [C_out, n_scales*C'].  No bias, normalisation or
  * activation sits between the stages; the residual connection around the
  * module is the caller's.
  * ------------------------------------------------------------------------- */
@@ -136,21 +139,24 @@ typedef struct {
   uint32_t struct_size;   /* sizeof(msla_desc), for versioning */
   int B, C, H, W;         /* input x is [B, C, H, W] */
   int heads, d;           /* heads per scale and channels per head; d in {16, 32} */
-  int n_scales;           /* 2 */
+  int n_scales;           /* 2 (Section 4.1), or 3: a second aggregated branch */
   int agg_kernel;         /* 5 (Section 4.1) or 3 */
   int C_out;              /* output channels */
   msla_dtype_t dtype;     /* type of x, out and all weights */
   float eps;              /* added to the attention denominator */
   void* workspace;        /* device scratch, >= msla_forward_workspace_bytes(desc) */
   size_t workspace_bytes;
+  int agg_kernel2;        /* n_scales == 3: filter size of the second aggregated branch, 5 or 3; else ignored */
 } msla_desc;
 
 typedef struct {
   const void* w_qkv;  /* [3C', C]     row o = output channel (h*3 + t)*d + i, t: 0 q, 1 k, 2 v */
   const void* w_dw;   /* [3C', k, k]  taps [dy][dx]; tap reads pixel (row+dy-k/2, col+dx-k/2) */
   const void* w_pw;   /* [3C', d]     out channel o reads in channels (o/d)*d .. (o/d)*d + d-1 */
-  const void* w_proj; /* [C_out, 2C'] column j = att channel head*d + c */
+  const void* w_proj; /* [C_out, n_scales*C'] column j = att channel head*d + c */
   const void* b_proj; /* [C_out] or NULL */
+  const void* w_dw2;  /* n_scales == 3: [3C', k2, k2] and [3C', d] of the second aggregated branch; else ignored */
+  const void* w_pw2;
 } msla_weights;
 
 /* Scratch bytes msla_forward needs for this descriptor (workspace fields are

@@ -32,12 +32,12 @@ class msla_desc(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_uint32), ("B", c_int), ("C", c_int), ("H", c_int), ("W", c_int),
                 ("heads", c_int), ("d", c_int), ("n_scales", c_int), ("agg_kernel", c_int),
                 ("C_out", c_int), ("dtype", c_int), ("eps", c_float), ("workspace", c_void_p),
-                ("workspace_bytes", c_size_t)]
+                ("workspace_bytes", c_size_t), ("agg_kernel2", c_int)]
 
 
 class msla_weights(ctypes.Structure):
     _fields_ = [("w_qkv", c_void_p), ("w_dw", c_void_p), ("w_pw", c_void_p), ("w_proj", c_void_p),
-                ("b_proj", c_void_p)]
+                ("b_proj", c_void_p), ("w_dw2", c_void_p), ("w_pw2", c_void_p)]
 
 
 MSLA_ACT_IDENTITY, MSLA_ACT_RELU, MSLA_ACT_HARDSWISH = 0, 1, 2
@@ -160,13 +160,14 @@ def msla_linattn_relu_noalloc(dtype, q, k, v, out, B, heads, N, d, eps=1e-15, st
 
 
 def make_desc(B, C, H, W, heads, d, C_out, dtype, eps=1e-15, n_scales=2, agg_kernel=5,
-              workspace: Optional[torch.Tensor] = None) -> msla_desc:
+              workspace: Optional[torch.Tensor] = None, agg_kernel2=3) -> msla_desc:
     desc = msla_desc()
     desc.struct_size = ctypes.sizeof(msla_desc)
     desc.B, desc.C, desc.H, desc.W = B, C, H, W
     desc.heads, desc.d, desc.n_scales, desc.agg_kernel, desc.C_out = heads, d, n_scales, agg_kernel, C_out
     desc.dtype = dtype
     desc.eps = eps
+    desc.agg_kernel2 = agg_kernel2
     desc.workspace = _ptr(workspace) if workspace is not None else None
     desc.workspace_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
     return desc
@@ -262,9 +263,10 @@ def msla_kernel_launches() -> int:
     return lib().msla_kernel_launches()
 
 
-def make_weights(w_qkv, w_dw, w_pw, w_proj, b_proj=None) -> msla_weights:
+def make_weights(w_qkv, w_dw, w_pw, w_proj, b_proj=None, w_dw2=None, w_pw2=None) -> msla_weights:
     w = msla_weights()
     w.w_qkv, w.w_dw, w.w_pw, w.w_proj, w.b_proj = _ptr(w_qkv), _ptr(w_dw), _ptr(w_pw), _ptr(w_proj), _ptr(b_proj)
+    w.w_dw2, w.w_pw2 = _ptr(w_dw2), _ptr(w_pw2)
     return w
 
 

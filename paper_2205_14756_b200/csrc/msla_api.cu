@@ -254,6 +254,8 @@ struct ForwardPlan {
   size_t ms_off, att_off, core_off, wpad_off, bytes;  // wpad: 3x3 aggregation taps embedded in 5x5 (agg_kernel == 3)
   CorePlan core;
   int Cp, N;
+  int S;              // branches: the projected tokens and S - 1 aggregated copies
+  size_t wpad2_off;   // embedded taps of the second aggregated branch
 };
 
 static msla_status_t validate_desc(const msla_desc* d, ForwardPlan* plan) {
@@ -263,27 +265,32 @@ static msla_status_t validate_desc(const msla_desc* d, ForwardPlan* plan) {
   if (d->B < 1 || d->C < 1 || d->H < 1 || d->W < 1 || d->heads < 1 || d->d < 1 || d->C_out < 1)
     return fail(MSLA_ERR_INVALID_ARG, "B, C, H, W, heads, d, C_out must be positive");
   if (!(d->eps >= 0.f)) return fail(MSLA_ERR_INVALID_ARG, "eps must be >= 0");
-  if (d->n_scales != 2) return fail(MSLA_ERR_UNSUPPORTED, "n_scales = %d; the module has two branches", d->n_scales);
+  if (d->n_scales != 2 && d->n_scales != 3) return fail(MSLA_ERR_UNSUPPORTED, "n_scales = %d; two or three branches are supported", d->n_scales);
   if (d->agg_kernel != 5 && d->agg_kernel != 3)
     return fail(MSLA_ERR_UNSUPPORTED, "agg_kernel = %d; 5x5 and 3x3 aggregation are supported", d->agg_kernel);
+  if (d->n_scales == 3 && d->agg_kernel2 != 5 && d->agg_kernel2 != 3)
+    return fail(MSLA_ERR_UNSUPPORTED, "agg_kernel2 = %d; 5x5 and 3x3 aggregation are supported", d->agg_kernel2);
   if (d->d != 16 && d->d != 32) return fail(MSLA_ERR_UNSUPPORTED, "d = %d; only 16 and 32 are supported", d->d);
   if ((long long)d->H * d->W > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "H*W exceeds 2^31-1");
   if (d->C % 8 != 0 || d->C_out % 8 != 0) return fail(MSLA_ERR_UNSUPPORTED, "C and C_out must be multiples of 8");
-  if ((long long)d->B * 2 * d->heads > 65535 || d->B > 65535) return fail(MSLA_ERR_UNSUPPORTED, "B*2*heads exceeds 65535");
+  const int S = d->n_scales;
+  if ((long long)d->B * S * d->heads > 65535 || d->B > 65535) return fail(MSLA_ERR_UNSUPPORTED, "B*n_scales*heads exceeds 65535");
+  plan->S = S;
   plan->Cp = d->heads * d->d;
   plan->N = d->H * d->W;
   const size_t e = elem_size(d->dtype);
   const size_t tokens = (size_t)d->B * plan->N;
-  plan->core = make_core_plan((long long)d->B * 2 * d->heads, plan->N, d->d);
+  plan->core = make_core_plan((long long)d->B * S * d->heads, plan->N, d->d);
   plan->ms_off = 0;
-  plan->att_off = align_up(tokens * 6 * plan->Cp * e, 256);
+  plan->att_off = align_up(tokens * 3 * S * plan->Cp * e, 256);
   // the attention output's region doubles as scratch of the fused apply + projection kernel, which writes no attention output
-  size_t att_bytes = tokens * 2 * plan->Cp * e;
-  const size_t fused_scratch = fused_out_bf16_supported(2 * d->heads, d->d, d->C_out, plan->N) ? fused_out_scratch_bytes(d->B, 2 * d->heads, d->d, d->C_out) : 0;
+  size_t att_bytes = tokens * S * plan->Cp * e;
+  const size_t fused_scratch = fused_out_bf16_supported(S * d->heads, d->d, d->C_out, plan->N) ? fused_out_scratch_bytes(d->B, S * d->heads, d->d, d->C_out) : 0;
   if (att_bytes < fused_scratch) att_bytes = fused_scratch;
   plan->core_off = plan->att_off + align_up(att_bytes, 256);
   plan->wpad_off = plan->core_off + plan->core.bytes;
-  plan->bytes = plan->wpad_off + (d->agg_kernel == 3 ? align_up((size_t)3 * plan->Cp * 25 * e, 256) : 0);
+  plan->wpad2_off = plan->wpad_off + (d->agg_kernel == 3 ? align_up((size_t)3 * plan->Cp * 25 * e, 256) : 0);
+  plan->bytes = plan->wpad2_off + (S == 3 && d->agg_kernel2 == 3 ? align_up((size_t)3 * plan->Cp * 25 * e, 256) : 0);
   return MSLA_OK;
 }
 
@@ -349,16 +356,28 @@ static msla_status_t run_aggregate(msla_dtype_t dt, const void* src, const void*
 
 // The aggregation kernels are 5x5.  A 3x3 depthwise filter (another of Section 3.1's small kernels) is the same
 // filter with a ring of zero taps around it: w5[c][dy+1][dx+1] = w3[c][dy][dx].  Returns the taps to use.
-static const void* aggregation_taps(const msla_desc* desc, const msla_weights* w, const ForwardPlan& p, cudaStream_t st) {
-  if (desc->agg_kernel == 5) return w->w_dw;
-  void* w5 = (char*)desc->workspace + p.wpad_off;
+static const void* aggregation_taps(const msla_desc* desc, const msla_weights* w, const ForwardPlan& p, int branch, cudaStream_t st) {
+  const void* w_dw = branch == 1 ? w->w_dw : w->w_dw2;
+  if ((branch == 1 ? desc->agg_kernel : desc->agg_kernel2) == 5) return w_dw;
+  void* w5 = (char*)desc->workspace + (branch == 1 ? p.wpad_off : p.wpad2_off);
   const long long total = 3LL * p.Cp * 25;
   if (desc->dtype == MSLA_F32)
-    generic::embed_taps_kernel<float><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const float*)w->w_dw, (float*)w5, total);
+    generic::embed_taps_kernel<float><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const float*)w_dw, (float*)w5, total);
   else
-    generic::embed_taps_kernel<__nv_bfloat16><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const __nv_bfloat16*)w->w_dw, (__nv_bfloat16*)w5, total);
+    generic::embed_taps_kernel<__nv_bfloat16><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const __nv_bfloat16*)w_dw, (__nv_bfloat16*)w5, total);
   count_launches(1);
   return w5;
+}
+
+// Step 2 for every aggregated branch: the scale-0 planes through that branch's filters into the branch's planes.
+static msla_status_t run_branches(const msla_desc* desc, const msla_weights* w, const ForwardPlan& p, char* ms, long long ms_sb, cudaStream_t st) {
+  const size_t branch_bytes = (size_t)3 * p.Cp * p.N * elem_size(desc->dtype);
+  for (int br = 1; br < p.S; ++br) {
+    const msla_status_t s = run_aggregate(desc->dtype, ms, aggregation_taps(desc, w, p, br, st), br == 1 ? w->w_pw : w->w_pw2, ms + br * branch_bytes,
+                                          desc->B, desc->H, desc->W, 3 * p.Cp, desc->d, ms_sb, ms_sb, st);
+    if (s != MSLA_OK) return s;
+  }
+  return MSLA_OK;
 }
 
 static msla_status_t record(void* const* events, int i, cudaStream_t st) {
@@ -380,7 +399,9 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   if (s != MSLA_OK) return s;
   if (!x || !out || !w) return fail(MSLA_ERR_INVALID_ARG, "null x, out or weights");
   if (!w->w_qkv || !w->w_dw || !w->w_pw || !w->w_proj) return fail(MSLA_ERR_INVALID_ARG, "null weight pointer");
-  const void* ptrs[] = {host_io ? nullptr : x, host_io ? nullptr : out, w->w_qkv, w->w_dw, w->w_pw, w->w_proj, w->b_proj, desc->workspace};
+  if (p.S == 3 && (!w->w_dw2 || !w->w_pw2)) return fail(MSLA_ERR_INVALID_ARG, "three branches need w_dw2 and w_pw2");
+  const void* ptrs[] = {host_io ? nullptr : x, host_io ? nullptr : out, w->w_qkv, w->w_dw, w->w_pw, w->w_proj, w->b_proj, desc->workspace,
+                        p.S == 3 ? w->w_dw2 : nullptr, p.S == 3 ? w->w_pw2 : nullptr};
   for (const void* ptr : ptrs)
     if (ptr && !aligned16(ptr)) return fail(MSLA_ERR_ALIGNMENT, "all device pointers must be 16-byte aligned");
   const size_t e = elem_size(desc->dtype);
@@ -407,8 +428,9 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
     }
   }
   const int Cp = p.Cp, N = p.N, d = desc->d, heads = desc->heads;
-  const long long ld_att = 2LL * Cp;
-  const long long ms_sb = 6LL * Cp * N;  // elements per image of the multi-scale buffer
+  const int S = p.S, Ht = S * heads;
+  const long long ld_att = (long long)S * Cp;
+  const long long ms_sb = 3LL * S * Cp * N;  // elements per image of the multi-scale buffer
   // ms: planar [B][6*heads planes][N][d]; plane (s*heads + h)*3 + t holds q (t=0), k (1) or v (2)
   // of head h at scale s (0: projected tokens, 1: aggregated tokens).
   char* ms = ws + p.ms_off;
@@ -419,30 +441,29 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   if (s != MSLA_OK) return s;
   if ((s = record(events, 1, st)) != MSLA_OK) return s;
   // 2. aggregation of every scale-0 plane into the matching scale-1 plane
-  s = run_aggregate(desc->dtype, ms, aggregation_taps(desc, w, p, st), w->w_pw, ms + (size_t)3 * Cp * N * e, desc->B, desc->H, desc->W, 3 * Cp, d, ms_sb, ms_sb, st);
-  if (s != MSLA_OK) return s;
+  if ((s = run_branches(desc, w, p, ms, ms_sb, st)) != MSLA_OK) return s;
   if ((s = record(events, 2, st)) != MSLA_OK) return s;
   // 3+4. attention over 2*heads heads of [q|k|v]; outputs land at channel head*d (concat)
   const HeadView in{ms_sb, 3LL * N * d, d};
   // Attention output: one [N][2d] plane per pair of heads when the tcgen05 output projection can
   // take it (dense 128-byte rows for the apply kernel's stores and the GEMM's tile loads),
   // otherwise token-major [N][2C'].
-  const bool att_planar = desc->dtype == MSLA_BF16 && d == 32 && project_out_planar_bf16_supported(2 * Cp, desc->C_out, N);
+  const bool att_planar = desc->dtype == MSLA_BF16 && d == 32 && Ht % 2 == 0 && project_out_planar_bf16_supported(S * Cp, desc->C_out, N);
   const HeadView ov = att_planar ? HeadView{(long long)N * ld_att, (long long)N * 2 * d, 2 * d, 1}
                                  : HeadView{(long long)N * ld_att, d, ld_att, 0};
   // Steps 4 and 5 run as one kernel when it takes the shape: the head concat then stays in shared memory.
-  const bool fused = desc->dtype == MSLA_BF16 && fused_out_bf16_supported(2 * heads, d, desc->C_out, N);
-  s = run_core(desc->dtype, ms, ms + (size_t)N * d * e, ms + (size_t)2 * N * d * e, att, in, ov, desc->B, 2 * heads, N, d, desc->eps, p.core,
+  const bool fused = desc->dtype == MSLA_BF16 && fused_out_bf16_supported(Ht, d, desc->C_out, N);
+  s = run_core(desc->dtype, ms, ms + (size_t)N * d * e, ms + (size_t)2 * N * d * e, att, in, ov, desc->B, Ht, N, d, desc->eps, p.core,
                ws + p.core_off, st, events ? (cudaEvent_t)events[3] : nullptr, fused ? CORE_STATE : CORE_ALL);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 4, st)) != MSLA_OK) return s;
   // 5. output projection back to NCHW
   if (fused)
     s = run_fused_out_bf16(ms, ms_sb, 3LL * N * d, reinterpret_cast<const float*>(ws + p.core_off + p.core.partial_off), p.core.S, att, w->w_proj,
-                           w->b_proj, residual, out_dev, desc->B, 2 * heads, d, N, desc->C_out, desc->eps, st);
+                           w->b_proj, residual, out_dev, desc->B, Ht, d, N, desc->C_out, desc->eps, st);
   else
-    s = att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, residual, out_dev, desc->B, 2 * Cp, desc->C_out, N, st)
-                   : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out_dev, desc->B, 2 * Cp, desc->C_out, N, st, residual);
+    s = att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, residual, out_dev, desc->B, S * Cp, desc->C_out, N, st)
+                   : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out_dev, desc->B, S * Cp, desc->C_out, N, st, residual);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 5, st)) != MSLA_OK) return s;
   if (host_io) {
@@ -474,7 +495,7 @@ static msla_status_t validate_band(const msla_desc* desc, int halo_top, int halo
     return fail(MSLA_ERR_INVALID_ARG, "halo rows (%d above, %d below) must be >= 0 and leave at least one of the %d rows", halo_top, halo_bottom, desc->H);
   b->Nb = (desc->H - halo_top - halo_bottom) * desc->W;
   b->tok_off = (long long)halo_top * desc->W;
-  b->core = make_core_plan((long long)desc->B * 2 * desc->heads, b->Nb, desc->d);
+  b->core = make_core_plan((long long)desc->B * b->f.S * desc->heads, b->Nb, desc->d);
   if (b->core.bytes > b->f.core.bytes) return fail(MSLA_ERR_WORKSPACE, "band plan exceeds the forward plan");
   if (!desc->workspace || desc->workspace_bytes < b->f.bytes)
     return fail(MSLA_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", b->f.bytes, desc->workspace ? desc->workspace_bytes : (size_t)0);
@@ -489,27 +510,27 @@ static msla_status_t band_states_impl(const msla_desc* desc, const void* x, cons
   if (s != MSLA_OK) return s;
   if (!x || !w || !state_out) return fail(MSLA_ERR_INVALID_ARG, "null x, weights or state_out");
   if (!w->w_qkv || !w->w_dw || !w->w_pw) return fail(MSLA_ERR_INVALID_ARG, "null weight pointer");
-  const void* ptrs[] = {x, w->w_qkv, w->w_dw, w->w_pw, state_out};
+  if (b.f.S == 3 && (!w->w_dw2 || !w->w_pw2)) return fail(MSLA_ERR_INVALID_ARG, "three branches need w_dw2 and w_pw2");
+  const void* ptrs[] = {x, w->w_qkv, w->w_dw, w->w_pw, state_out, b.f.S == 3 ? w->w_dw2 : x, b.f.S == 3 ? w->w_pw2 : x};
   for (const void* ptr : ptrs)
     if (!aligned16(ptr)) return fail(MSLA_ERR_ALIGNMENT, "all device pointers must be 16-byte aligned");
   const ForwardPlan& p = b.f;
   const size_t e = elem_size(desc->dtype);
   const size_t xb = (size_t)desc->B * desc->C * p.N * e;
-  const size_t sb = (size_t)desc->B * 2 * desc->heads * b.core.ne * sizeof(float);
+  const size_t sb = (size_t)desc->B * p.S * desc->heads * b.core.ne * sizeof(float);
   if (overlaps(x, xb, desc->workspace, p.bytes) || overlaps(state_out, sb, desc->workspace, p.bytes) || overlaps(state_out, sb, x, xb))
     return fail(MSLA_ERR_INVALID_ARG, "x, state_out and the workspace must not overlap");
   if ((s = check_arch()) != MSLA_OK) return s;
   char* ws = (char*)desc->workspace;
   const int Cp = p.Cp, N = p.N, d = desc->d;
-  const long long ms_sb = 6LL * Cp * N;
+  const long long ms_sb = 3LL * p.S * Cp * N;
   char* ms = ws + p.ms_off;
   s = run_project_in(desc->dtype, x, w->w_qkv, ms, desc->B, desc->C, 3 * Cp, N, d, ms_sb, st);
   if (s != MSLA_OK) return s;
-  s = run_aggregate(desc->dtype, ms, aggregation_taps(desc, w, p, st), w->w_pw, ms + (size_t)3 * Cp * N * e, desc->B, desc->H, desc->W, 3 * Cp, d, ms_sb, ms_sb, st);
-  if (s != MSLA_OK) return s;
+  if ((s = run_branches(desc, w, p, ms, ms_sb, st)) != MSLA_OK) return s;
   const HeadView in{ms_sb, 3LL * N * d, d};
   const char* q = ms + (size_t)b.tok_off * d * e;
-  s = run_core(desc->dtype, q, q + (size_t)N * d * e, q + (size_t)2 * N * d * e, nullptr, in, in, desc->B, 2 * desc->heads, b.Nb, d, desc->eps,
+  s = run_core(desc->dtype, q, q + (size_t)N * d * e, q + (size_t)2 * N * d * e, nullptr, in, in, desc->B, p.S * desc->heads, b.Nb, d, desc->eps,
                b.core, ws + p.core_off, st, nullptr, CORE_STATE | CORE_COMBINE);
   if (s != MSLA_OK) return s;
   const cudaError_t ce = cudaMemcpyAsync(state_out, ws + p.core_off + b.core.state_off, sb, cudaMemcpyDeviceToDevice, st);
@@ -534,13 +555,14 @@ static msla_status_t band_output_impl(const msla_desc* desc, const msla_weights*
   const ForwardPlan& p = b.f;
   const size_t e = elem_size(desc->dtype);
   const int Cp = p.Cp, N = p.N, Nb = b.Nb, d = desc->d, heads = desc->heads;
-  const long long total = (long long)desc->B * 2 * heads * b.core.ne;
+  const int Ht = p.S * heads;
+  const long long total = (long long)desc->B * Ht * b.core.ne;
   const size_t ob = (size_t)desc->B * desc->C_out * Nb * e, sb = (size_t)R * total * sizeof(float);
   if (overlaps(out, ob, desc->workspace, p.bytes) || overlaps(states, sb, desc->workspace, p.bytes) || overlaps(out, ob, states, sb))
     return fail(MSLA_ERR_INVALID_ARG, "out, states and the workspace must not overlap");
   if ((s = check_arch()) != MSLA_OK) return s;
   char* ws = (char*)desc->workspace;
-  const long long ms_sb = 6LL * Cp * N, ld_att = 2LL * Cp;
+  const long long ms_sb = 3LL * p.S * Cp * N, ld_att = (long long)p.S * Cp;
   char* ms = ws + p.ms_off;
   char* att = ws + p.att_off;
   float* state = reinterpret_cast<float*>(ws + p.core_off + b.core.state_off);
@@ -548,17 +570,17 @@ static msla_status_t band_output_impl(const msla_desc* desc, const msla_weights*
   count_launches(1);
   if ((s = check_launch("sum of the bands' states")) != MSLA_OK) return s;
   const char* q = ms + (size_t)b.tok_off * d * e;
-  if (desc->dtype == MSLA_BF16 && fused_out_bf16_supported(2 * heads, d, desc->C_out, Nb))
-    return run_fused_out_bf16(q, ms_sb, 3LL * N * d, state, 1, att, w->w_proj, w->b_proj, nullptr, out, desc->B, 2 * heads, d, Nb, desc->C_out, desc->eps, st);
+  if (desc->dtype == MSLA_BF16 && fused_out_bf16_supported(Ht, d, desc->C_out, Nb))
+    return run_fused_out_bf16(q, ms_sb, 3LL * N * d, state, 1, att, w->w_proj, w->b_proj, nullptr, out, desc->B, Ht, d, Nb, desc->C_out, desc->eps, st);
   const HeadView in{ms_sb, 3LL * N * d, d};
-  const bool att_planar = desc->dtype == MSLA_BF16 && d == 32 && project_out_planar_bf16_supported(2 * Cp, desc->C_out, Nb);
+  const bool att_planar = desc->dtype == MSLA_BF16 && d == 32 && Ht % 2 == 0 && project_out_planar_bf16_supported(p.S * Cp, desc->C_out, Nb);
   const HeadView ov = att_planar ? HeadView{(long long)Nb * ld_att, (long long)Nb * 2 * d, 2 * d, 1}
                                  : HeadView{(long long)Nb * ld_att, d, ld_att, 0};
-  s = run_core(desc->dtype, q, q + (size_t)N * d * e, q + (size_t)2 * N * d * e, att, in, ov, desc->B, 2 * heads, Nb, d, desc->eps, b.core,
+  s = run_core(desc->dtype, q, q + (size_t)N * d * e, q + (size_t)2 * N * d * e, att, in, ov, desc->B, Ht, Nb, d, desc->eps, b.core,
                ws + p.core_off, st, nullptr, CORE_APPLY);
   if (s != MSLA_OK) return s;
-  return att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, nullptr, out, desc->B, 2 * Cp, desc->C_out, Nb, st)
-                    : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out, desc->B, 2 * Cp, desc->C_out, Nb, st);
+  return att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, nullptr, out, desc->B, p.S * Cp, desc->C_out, Nb, st)
+                    : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out, desc->B, p.S * Cp, desc->C_out, Nb, st);
 }
 
 // ---------------------------------------------------------- FFN with a depthwise convolution
@@ -749,7 +771,7 @@ msla_status_t msla_evit_block(const msla_desc* attn, const msla_weights* aw, con
 int msla_forward_fuses_apply(const msla_desc* desc) {
   ForwardPlan p;
   if (validate_desc(desc, &p) != MSLA_OK) return -1;
-  return desc->dtype == MSLA_BF16 && fused_out_bf16_supported(2 * desc->heads, desc->d, desc->C_out, p.N) ? 1 : 0;
+  return desc->dtype == MSLA_BF16 && fused_out_bf16_supported(p.S * desc->heads, desc->d, desc->C_out, p.N) ? 1 : 0;
 }
 
 unsigned long long msla_kernel_launches(void) { return g_launches; }

@@ -100,6 +100,7 @@ class ModuleShape:
     n_scales: int = 2   # identity branch + one 5x5-aggregated branch
     agg_kernel: int = 5
     eps: float = 1e-15
+    agg_kernel2: int = 3  # filter of the second aggregated branch when n_scales == 3
 
     @property
     def N(self) -> int:
@@ -161,6 +162,10 @@ def module_inputs(s: ModuleShape) -> Dict[str, np.ndarray]:
     for stream, (name, (shape, std)) in enumerate(shapes.items()):
         n = int(np.prod(shape))
         out[name] = quantise(normal(s.seed, stream, n, std).reshape(shape), s.dtype)
+    if s.n_scales == 3:  # the second aggregated branch's filters: streams 5 and 6
+        k2 = s.agg_kernel2
+        out["w_dw2"] = quantise(normal(s.seed, 5, 3 * Cp * k2 * k2, 1.0 / k2).reshape(3 * Cp, k2, k2), s.dtype)
+        out["w_pw2"] = quantise(normal(s.seed, 6, 3 * Cp * s.d, s.d ** -0.5).reshape(3 * Cp, s.d), s.dtype)
     return out
 
 

@@ -77,7 +77,7 @@ def test_forward_descriptor_validation():
     need = binding.msla_forward_workspace_bytes(ok)
     # at least the multi-scale buffer (6C') and the attention output (2C')
     assert need >= 256 * (6 * 64 + 2 * 64) * 4
-    for field, value in [("n_scales", 3), ("agg_kernel", 7), ("agg_kernel", 4), ("d", 20), ("heads", 0), ("struct_size", 8), ("C", 60)]:
+    for field, value in [("n_scales", 4), ("n_scales", 1), ("agg_kernel", 7), ("agg_kernel", 4), ("d", 20), ("heads", 0), ("struct_size", 8), ("C", 60)]:
         bad = binding.make_desc(1, 64, 16, 16, 4, 16, 64, binding.MSLA_F32)
         setattr(bad, field, value)
         assert binding.msla_forward_workspace_bytes(bad) == 0, field

@@ -76,6 +76,24 @@ def test_module_with_3x3_aggregation(dtype, B, C, H, W, heads, d):
     util.assert_close(util.run_module(s, t), _ref(s, t), dtype, "3x3 aggregation", block=util.MODULE_BLOCK if dtype == "bf16" else None)
 
 
+# Three branches (Section 3.1's multi-scale tokens with a second aggregated copy): 5x5 + 3x3 and 3x3 + 5x5 filters;
+# fp32 on the plain kernels, bf16 with 3C' <= 512 through the fused output kernel, with 3C' = 768 and with an odd
+# number of heads through the apply kernel and a projection GEMM.
+@pytest.mark.parametrize("dtype,B,C,H,W,heads,d,k1,k2,fused", [("f32", 1, 32, 7, 9, 2, 16, 5, 3, 0), ("bf16", 2, 64, 24, 40, 2, 32, 5, 3, 1),
+                                                              ("bf16", 1, 128, 16, 24, 4, 32, 3, 5, 1), ("bf16", 1, 256, 16, 16, 8, 32, 5, 3, 0),
+                                                              ("bf16", 1, 32, 12, 12, 1, 32, 5, 5, 1), ("bf16", 1, 96, 16, 16, 6, 16, 5, 3, 1)])
+def test_module_with_three_branches(dtype, B, C, H, W, heads, d, k1, k2, fused):
+    s = inputs.ModuleShape("three", dtype, B, C, H, W, heads, d, seed=43, n_scales=3, agg_kernel=k1, agg_kernel2=k2)
+    t = inputs.module_inputs(s)
+    assert t["w_proj"].shape == (C, 3 * heads * d) and t["w_dw2"].shape[-1] == k2
+    desc = binding.make_desc(B, C, H, W, heads, d, C, binding.MSLA_BF16 if dtype == "bf16" else binding.MSLA_F32, n_scales=3,
+                             agg_kernel=k1, agg_kernel2=k2)
+    assert binding.msla_forward_fuses_apply(desc) == fused
+    ref = oracle.msla_forward3(t["x"], t["w_qkv"], t["w_dw"], t["w_pw"], t["w_dw2"], t["w_pw2"], t["w_proj"], heads=heads, d=d)
+    util.assert_close(util.run_module(s, t), ref, dtype, "three branches", block=util.MODULE_BLOCK if dtype == "bf16" else None)
+    assert binding.msla_debug_wait_timeouts() == 0
+
+
 def test_config3_bf16():
     s = inputs.CONFIG3
     t = inputs.module_inputs(s)

@@ -129,16 +129,17 @@ def run_module(s: inputs.ModuleShape, t: dict, bias=None) -> np.ndarray:
     x, w_qkv, w_dw, w_pw, w_proj = (dev(t[n], dt) for n in ("x", "w_qkv", "w_dw", "w_pw", "w_proj"))
     b = dev(bias, dt) if bias is not None else None
     c_out = t["w_proj"].shape[0]
-    desc = binding.make_desc(s.B, s.C, s.H, s.W, s.heads, s.d, c_out, CODE[dt], s.eps, agg_kernel=s.agg_kernel)
+    desc = binding.make_desc(s.B, s.C, s.H, s.W, s.heads, s.d, c_out, CODE[dt], s.eps, n_scales=s.n_scales, agg_kernel=s.agg_kernel, agg_kernel2=s.agg_kernel2)
     nbytes = binding.msla_forward_workspace_bytes(desc)
     assert nbytes > 0
     wg = Guarded(nbytes)
     ws = wg.view(torch.float32, (nbytes // 4,))
-    desc = binding.make_desc(s.B, s.C, s.H, s.W, s.heads, s.d, c_out, CODE[dt], s.eps, agg_kernel=s.agg_kernel, workspace=ws)
+    desc = binding.make_desc(s.B, s.C, s.H, s.W, s.heads, s.d, c_out, CODE[dt], s.eps, n_scales=s.n_scales, agg_kernel=s.agg_kernel, agg_kernel2=s.agg_kernel2, workspace=ws)
     esz = 4 if dt == "f32" else 2
     og = Guarded(s.B * c_out * s.H * s.W * esz)
     out = og.view(TORCH_DTYPE[dt], (s.B, c_out, s.H, s.W))
-    w = binding.make_weights(w_qkv, w_dw, w_pw, w_proj, b)
+    extra = [dev(t[n], dt) for n in ("w_dw2", "w_pw2")] if s.n_scales == 3 else [None, None]
+    w = binding.make_weights(w_qkv, w_dw, w_pw, w_proj, b, *extra)
     binding.msla_forward(desc, x, w, out)
     torch.cuda.synchronize()
     wg.check("module workspace")
