@@ -54,6 +54,28 @@ def test_ffn_at_the_bench_width_256x256():
     assert binding.msla_debug_wait_timeouts() == 0
 
 
+def test_ffn_at_the_bench_shape_on_sampled_pixels():
+    """[1, 256, 512, 512], expansion 4: the shape and launch configuration the benchmark times.  The oracle computes
+    sampled output pixels one by one from the 3x3 neighbourhood each depends on (image corners and edges included)."""
+    s = inputs.FfnShape("ffn_c256_512x512", "bf16", 1, 256, 512, 512, 1024, 256, seed=36)
+    t = inputs.ffn_inputs(s)
+    got = util.run_ffn(s, t, "hardswish", True)
+    rng = np.random.default_rng(36)
+    pts = [(0, 0), (0, 511), (511, 0), (511, 511), (0, 200), (300, 511), (255, 256), (31, 32), (8, 7)]
+    pts += [(int(a), int(b)) for a, b in zip(rng.integers(0, 512, 40), rng.integers(0, 512, 40))]
+    ref, val = [], []
+    for (y, x) in pts:
+        y0, y1, x0, x1 = max(y - 1, 0), min(y + 2, 512), max(x - 1, 0), min(x + 2, 512)
+        crop = dict(t, x=np.ascontiguousarray(t["x"][:, :, y0:y1, x0:x1]))
+        ref.append(_ref(crop, "hardswish", True)[0, :, y - y0, x - x0])
+        val.append(got[0, :, y, x])
+    ref, val = np.stack(ref), np.stack(val)
+    assert np.linalg.norm(val - ref) <= util.TOL_BF16_RELL2 * np.linalg.norm(ref)
+    assert np.abs(val - ref).max() <= util.TOL_BF16_MAXABS * np.abs(ref).max()
+    assert np.isfinite(got).all()
+    assert binding.msla_debug_wait_timeouts() == 0
+
+
 @pytest.mark.parametrize("dtype,B,C,H,W,heads,d,Ch", [("f32", 1, 32, 8, 8, 2, 16, 64), ("bf16", 2, 64, 16, 24, 2, 32, 256),
                                                       ("bf16", 1, 256, 64, 64, 8, 32, 1024)])
 def test_block_matches_the_oracle(dtype, B, C, H, W, heads, d, Ch):
