@@ -213,7 +213,7 @@ state_fold_kernel(const float* __restrict__ partial, int S, const bf16* __restri
 template <int D, bool RES>
 __global__ void __launch_bounds__(O_THREADS, 1)
 fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmQ,
-                 const __grid_constant__ CUtensorMap tmO, OutParams p) {
+                 const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmR, OutParams p) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
   const uint32_t a_base = smem_base;                                  // resident rows of M: kslices x 16 KB
@@ -221,7 +221,8 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
   constexpr int ROWB = D * 2;                                          // bytes per token row = the swizzle span
   const uint32_t ring = a_base + (uint32_t)p.kslices * O_A_SLICE;
   const uint32_t staging = ring + O_STAGES * SLICE;
-  const uint32_t bars = staging + O_STAGING;
+  const uint32_t resbuf = staging + O_STAGING;           // RES: one 32-channel x 64-token block of the residual per epilogue warp
+  const uint32_t bars = resbuf + (RES ? O_STAGING : 0);
   const uint32_t full_bar = bars;                        // [stage] TMA landed (own CTA)
   const uint32_t empty_bar = bars + 8 * O_STAGES;        // [stage] MMAs have read the slice (commit, both CTAs)
   const uint32_t ready_bar = bars + 16 * O_STAGES;       // [stage] both CTAs' slices transformed (leader only)
@@ -230,6 +231,7 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
   const uint32_t res_bar = tempty_bar + 16;              // rows of M landed (own CTA)
   const uint32_t peer_res_bar = res_bar + 8;             // the peer's rows of M landed (leader only)
   const uint32_t tmem_slot = peer_res_bar + 8;
+  const uint32_t resid_bar = bars + 256;                 // [epilogue warp] RES: the warp's residual block landed
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_sh;
 
@@ -251,6 +253,8 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar + 8 * a, 1); mbar_init(tempty_bar + 8 * a, 2 * 4); }
     mbar_init(res_bar, 1);
     mbar_init(peer_res_bar, 1);
+    if (RES)
+      for (int w = 0; w < 4; ++w) mbar_init(resid_bar + 8 * w, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {  // one warp of each CTA of the pair: all 512 tensor-memory columns in both
@@ -415,6 +419,15 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     const int row0 = (int)rank * OM + quarter * 32;
     const float bias = (p.bias && row0 + lane < p.Cout) ? __bfloat162float(p.bias[row0 + lane]) : 0.f;
     const uint32_t tempty_remote = map_to_cta(tempty_bar, 0);
+    // RES: the residual arrives by TMA, one 32-channel x 64-token block per warp and request, a block ahead of its use
+    const uint32_t my_resid_bar = resid_bar + 8 * (uint32_t)(warp - 2 - O_XWARPS);
+    const uint32_t my_res = resbuf + (uint32_t)(warp - 2 - O_XWARPS) * O_STAGING_WARP, my_res_row = my_res + lane * 128;
+    uint32_t res_count = 0;
+    auto request_residual = [&](int t2, int j2) {  // one lane
+      mbar_expect_tx(my_resid_bar, O_STAGING_WARP);
+      tma_load_3d(my_res, &tmR, my_resid_bar, (t2 % p.tiles_per_image) * (2 * p.ot) + j2 * 64, row0, t2 / p.tiles_per_image);
+    };
+    if (RES && lane == 0 && row0 < p.Cout && tile_first < tile_end) request_residual(tile_first, 0);
     uint32_t local = 0;
     bool ok = true;
     for (int tile = tile_first; ok && tile < tile_end; ++tile, ++local) {
@@ -428,52 +441,51 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
       uint32_t r[2][32];
       tmem_ld32(taddr, r[0]);
       const int chunks = (2 * p.ot) / 32;  // the accumulator's columns are the pair's tokens
-      // RES: the lane's channel row of the residual, 32 tokens (64 bytes) per chunk, fetched one chunk ahead
-      const bf16* res_row = (RES && row0 + lane < p.Cout) ? p.residual + ((long long)b * p.Cout + row0 + lane) * p.N : nullptr;
-      uint4 rs[2][4];
-      auto load_residual = [&](int c) {
-#pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          const int n = nt * (2 * p.ot) + c * 32 + v * 8;
-          rs[c & 1][v] = (res_row && n < p.N) ? __ldg(reinterpret_cast<const uint4*>(res_row + n)) : make_uint4(0u, 0u, 0u, 0u);
-        }
-      };
-      if (RES) load_residual(0);
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         if (c >= chunks) break;
         tmem_ld_wait();
         if (c + 1 < chunks) tmem_ld32(taddr + (c + 1) * 32, r[(c + 1) & 1]);  // next chunk streams in meanwhile
-        if (RES && c + 1 < chunks) load_residual(c + 1);
         const uint32_t(&rc)[32] = r[c & 1];
         const int n0 = nt * (2 * p.ot) + (c >> 1) * 64;  // first token of the 64-token block
         if (n0 >= p.N || row0 >= p.Cout) continue;    // warp-uniform
         if ((c & 1) == 0) {  // the previous block must have been read out of the staging buffer
           if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
           __syncwarp();
+          if (RES) {           // this block of the residual was requested one block ago
+            ok = mbar_wait(my_resid_bar, res_count & 1, &abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            ++res_count;
+          }
         }
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
+          const uint32_t pc = (uint32_t)((c & 1) * 4 + v);
+          uint4 rv = make_uint4(0u, 0u, 0u, 0u);  // the same 16-byte piece of the lane's row in the residual block (same box, same swizzle)
+          if (RES) asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(rv.x), "=r"(rv.y), "=r"(rv.z), "=r"(rv.w) : "r"(my_res_row + ((pc ^ sw) << 4)));
+          const uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w};
           uint32_t w[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             float f0 = __uint_as_float(rc[v * 8 + 2 * e]) + bias, f1 = __uint_as_float(rc[v * 8 + 2 * e + 1]) + bias;
-            if (RES) {
-              const uint32_t rw = e == 0 ? rs[c & 1][v].x : e == 1 ? rs[c & 1][v].y : e == 2 ? rs[c & 1][v].z : rs[c & 1][v].w;
-              f0 += __uint_as_float(rw << 16); f1 += __uint_as_float(rw & 0xffff0000u);
-            }
+            if (RES) { f0 += __uint_as_float(rw[e] << 16); f1 += __uint_as_float(rw[e] & 0xffff0000u); }
             w[e] = pack2(f0, f1);
           }
-          const uint32_t pc = (uint32_t)((c & 1) * 4 + v);
           asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(my_row + ((pc ^ sw) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]),
                        "r"(w[3]) : "memory");
         }
         if (c & 1) {
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // also orders the reads of the residual block before its refill
           __syncwarp();
           if (lane == 0) {
             tma_store_3d(&tmO, stage, n0, row0, b);
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            if (RES) {  // request the next block this warp will drain: the next 64 tokens of this tile, else the next tile's first
+              int t2 = tile, j2 = (c >> 1) + 1;
+              if (j2 * 64 >= 2 * p.ot || (t2 % p.tiles_per_image) * (2 * p.ot) + j2 * 64 >= p.N) { ++t2; j2 = 0; }
+              if (t2 < tile_end) request_residual(t2, j2);
+            }
           }
         }
       }
@@ -527,7 +539,7 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   const int ot = 2LL * B * ((N + 2 * OT - 1) / (2 * OT)) <= sms / 2 ? OT / 2 : OT;
   bf16* M = (bf16*)scratch;
   float* ks = (float*)((char*)scratch + fused_out_m_bytes(B, Ht, d, Cout));
-  CUtensorMap tmM, tmQ, tmO;
+  CUtensorMap tmM, tmQ, tmO, tmR;
   {
     const cuuint64_t dM[3] = {(cuuint64_t)K, (cuuint64_t)Cout, (cuuint64_t)B};
     const cuuint64_t sM[2] = {(cuuint64_t)K * 2, (cuuint64_t)K * Cout * 2};
@@ -540,7 +552,8 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
     const cuuint32_t bO[3] = {64, 32, 1};
     if (!tma_make_map_bf16(&tmM, M, 3, dM, sM, bM, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !tma_make_map_bf16(&tmQ, q, 4, dQ, sQ, bQ, d == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B) ||
-        !tma_make_map_bf16(&tmO, y, 3, dO, sO, bO, CU_TENSOR_MAP_SWIZZLE_128B))
+        !tma_make_map_bf16(&tmO, y, 3, dO, sO, bO, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !tma_make_map_bf16(&tmR, residual ? residual : y, 3, dO, sO, bO, CU_TENSOR_MAP_SWIZZLE_128B))
       return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the fused apply + output projection");
   }
   OutParams p{};
@@ -552,13 +565,13 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   const long long tiles = (long long)B * p.tiles_per_image;
   if (tiles > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many token tiles");
   p.num_tiles = (int)tiles;
-  const int smem = p.kslices * O_A_SLICE + O_STAGES * (OT * d * 2) + O_STAGING + O_BAR_BYTES + 1024;
+  const int smem = p.kslices * O_A_SLICE + O_STAGES * (OT * d * 2) + O_STAGING + (residual ? O_STAGING : 0) + O_BAR_BYTES + 1024;
   static std::atomic<unsigned long long> attr_done{0}, attr_done16{0}, attr_res{0}, attr_res16{0};
   constexpr int smem_max = O_SMEM_MAX;
   msla_status_t s = ensure_smem_attr(attr_done, fused_out_kernel<32, false>, smem_max);
   if (s == MSLA_OK) s = ensure_smem_attr(attr_done16, fused_out_kernel<16, false>, smem_max);
-  if (s == MSLA_OK && residual) s = ensure_smem_attr(attr_res, fused_out_kernel<32, true>, smem_max);
-  if (s == MSLA_OK && residual) s = ensure_smem_attr(attr_res16, fused_out_kernel<16, true>, smem_max);
+  if (s == MSLA_OK && residual) s = ensure_smem_attr(attr_res, fused_out_kernel<32, true>, smem_max + O_STAGING);
+  if (s == MSLA_OK && residual) s = ensure_smem_attr(attr_res16, fused_out_kernel<16, true>, smem_max + O_STAGING);
   if (s != MSLA_OK) return s;
   long long pairs = sms / 2;
   if (pairs > tiles) pairs = tiles;
@@ -571,10 +584,10 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   launch_pdl(state_fold_kernel, dim3((unsigned)(B * Ht), (unsigned)fold_chunks), dim3(FOLD_THREADS), FOLD_SMEM, st, partial, S,
              (const bf16*)w, M, ks, Ht, d, Cout, K, d / fold_chunks);
   const dim3 grid((unsigned)(2 * pairs)), block(O_THREADS);
-  if (d == 32 && !residual) launch_pdl_cluster2(fused_out_kernel<32, false>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, p);
-  else if (d == 32) launch_pdl_cluster2(fused_out_kernel<32, true>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, p);
-  else if (!residual) launch_pdl_cluster2(fused_out_kernel<16, false>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, p);
-  else launch_pdl_cluster2(fused_out_kernel<16, true>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, p);
+  if (d == 32 && !residual) launch_pdl_cluster2(fused_out_kernel<32, false>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, tmR, p);
+  else if (d == 32) launch_pdl_cluster2(fused_out_kernel<32, true>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, tmR, p);
+  else if (!residual) launch_pdl_cluster2(fused_out_kernel<16, false>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, tmR, p);
+  else launch_pdl_cluster2(fused_out_kernel<16, true>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, tmR, p);
   count_launches(2);
   return check_launch("fused apply + output projection (tcgen05, paired CTAs)");
 }
