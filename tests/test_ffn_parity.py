@@ -31,6 +31,10 @@ def test_ffn_f32_plain_kernels(act):
     (1, 128, 24, 40, 512, 128, "identity", True, False),
     (1, 320, 8, 24, 640, 320, "hardswish", True, True),
     (3, 64, 5, 3, 64, 64, "relu", False, False),
+    (1, 64, 8, 12, 128, 64, "hardswish", True, True),       # W not a multiple of 8
+    (2, 64, 13, 24, 192, 72, "hardswish", False, True),     # ragged tiles in both directions, C_out not a multiple of 32
+    (1, 256, 40, 48, 1024, 256, "relu", True, True),
+    (1, 64, 16, 16, 1088, 64, "hardswish", True, False),    # 17 hidden planes of 64 channels
 ])
 def test_ffn_bf16_tensor_core_path(B, C, H, W, Ch, Cout, act, residual, biases):
     s = inputs.FfnShape("ffn_bf16", "bf16", B, C, H, W, Ch, Cout, seed=32)
