@@ -26,6 +26,8 @@
 //                  K-major, fp32 accumulators in both CTAs' tensor memory
 //     warps 10-13  drain the accumulators: TMEM -> bf16 (+ bias) -> swizzled staging -> TMA
 //                  stores of 32-channel x 64-token blocks into the NCHW output
+//                  (RES kernels: the same block of a residual tensor, fetched by TMA into a block of its own one
+//                  block ahead of its use, is added before the conversion: the residual connection around the module)
 //   Two accumulator sets (2 x 256 TMEM columns) let the drain of a tile overlap the next.
 // No TMA load is multicast: each CTA loads its own operands; only tcgen05.commit signals
 // both CTAs' barriers.  Every mbarrier wait is bounded as in the GEMM.
