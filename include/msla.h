@@ -43,7 +43,11 @@ typedef enum {
   MSLA_ERR_CUDA = 6         /* a CUDA runtime call or launch failed; see msla_last_error() */
 } msla_status_t;
 
-typedef enum { MSLA_F32 = 0, MSLA_BF16 = 1 } msla_dtype_t;
+/* Storage type of activations and weights.  Arithmetic and the attention state are fp32 for all three.  MSLA_F16
+ * (the paper's deployment precision, Section 4.1) runs on the library's plain kernels; the tensor-core kernels are
+ * bf16.  MSLA_F16 is accepted wherever a dtype is taken (msla_linattn_relu_ws and _noalloc, msla_forward*, the band
+ * pair, the stage entry points, msla_ffn_dwconv, msla_evit_block). */
+typedef enum { MSLA_F32 = 0, MSLA_BF16 = 1, MSLA_F16 = 2 } msla_dtype_t;
 
 /* ------------------------------------------------------------------------- *
  * Attention core: ReLU linear attention, Eq. 3 of the paper (the linear-time

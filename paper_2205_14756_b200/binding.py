@@ -16,8 +16,8 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("MSLA_LIBRARY_PATH") or os.path.join(_PKG, "libmsla.so")
 
-MSLA_F32, MSLA_BF16 = 0, 1
-_DTYPES = {torch.float32: MSLA_F32, torch.bfloat16: MSLA_BF16}
+MSLA_F32, MSLA_BF16, MSLA_F16 = 0, 1, 2
+_DTYPES = {torch.float32: MSLA_F32, torch.bfloat16: MSLA_BF16, torch.float16: MSLA_F16}
 
 c_int, c_float, c_size_t, c_void_p = ctypes.c_int, ctypes.c_float, ctypes.c_size_t, ctypes.c_void_p
 

@@ -3,6 +3,7 @@
 
 #include <atomic>
 #include <cstdarg>
+#include <type_traits>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
@@ -82,6 +83,7 @@ static bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
 }
 
 static size_t elem_size(msla_dtype_t t) { return t == MSLA_F32 ? 4 : 2; }
+static bool known_dtype(msla_dtype_t t) { return t == MSLA_F32 || t == MSLA_BF16 || t == MSLA_F16; }
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // ----------------------------------------------------------------- core plan
@@ -148,6 +150,9 @@ static msla_status_t run_core(msla_dtype_t dtype, const void* q, const void* k, 
   if (dtype == MSLA_F32)
     return run_core_generic<float>((const float*)q, (const float*)k, (const float*)v, (float*)out,
                                    in, ov, B, heads, N, d, eps, p, (char*)ws, st, mid, phases);
+  if (dtype == MSLA_F16)  // fp16 storage runs on the plain kernels (fp32 arithmetic, one rounding per stored value)
+    return run_core_generic<__half>((const __half*)q, (const __half*)k, (const __half*)v, (__half*)out,
+                                    in, ov, B, heads, N, d, eps, p, (char*)ws, st, mid, phases);
   const bool strides_ok = in.batch % 8 == 0 && in.head % 8 == 0 && in.ld % 8 == 0 && ov.batch % 8 == 0 &&
                           ov.head % 8 == 0 && ov.ld % 8 == 0;
   if (strides_ok) return run_core_bf16(q, k, v, out, in, ov, B, heads, N, d, eps, p, ws, st, mid, phases);
@@ -160,7 +165,7 @@ static msla_status_t run_core(msla_dtype_t dtype, const void* q, const void* k, 
 static msla_status_t core_entry(msla_dtype_t dtype, const void* q, const void* k, const void* v,
                                 void* out, int B, int heads, int N, int d, float eps, void* ws,
                                 size_t ws_bytes, bool own_ws, cudaStream_t st) {
-  if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype %d", (int)dtype);
+  if (!known_dtype(dtype)) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype %d", (int)dtype);
   if (!q || !k || !v || !out) return fail(MSLA_ERR_INVALID_ARG, "null tensor pointer");
   if (B < 1 || heads < 1 || N < 1 || d < 1) return fail(MSLA_ERR_INVALID_ARG, "B, heads, N, d must be positive (got %d, %d, %d, %d)", B, heads, N, d);
   if (!(eps >= 0.f)) return fail(MSLA_ERR_INVALID_ARG, "eps must be >= 0");
@@ -225,7 +230,7 @@ static msla_status_t noalloc_scratch(void** out_ptr) {
 
 static msla_status_t core_entry_noalloc(msla_dtype_t dtype, const void* q, const void* k, const void* v,
                                         void* out, int B, int heads, int N, int d, float eps, cudaStream_t st) {
-  if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype %d", (int)dtype);
+  if (!known_dtype(dtype)) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype %d", (int)dtype);
   if (!q || !k || !v || !out) return fail(MSLA_ERR_INVALID_ARG, "null tensor pointer");
   if (B < 1 || heads < 1 || N < 1 || d < 1) return fail(MSLA_ERR_INVALID_ARG, "B, heads, N, d must be positive (got %d, %d, %d, %d)", B, heads, N, d);
   if (!(eps >= 0.f)) return fail(MSLA_ERR_INVALID_ARG, "eps must be >= 0");
@@ -261,7 +266,7 @@ struct ForwardPlan {
 static msla_status_t validate_desc(const msla_desc* d, ForwardPlan* plan) {
   if (!d) return fail(MSLA_ERR_INVALID_ARG, "null descriptor");
   if (d->struct_size != sizeof(msla_desc)) return fail(MSLA_ERR_INVALID_ARG, "desc.struct_size = %u, expected %zu", d->struct_size, sizeof(msla_desc));
-  if (d->dtype != MSLA_F32 && d->dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype %d", (int)d->dtype);
+  if (!known_dtype(d->dtype)) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype %d", (int)d->dtype);
   if (d->B < 1 || d->C < 1 || d->H < 1 || d->W < 1 || d->heads < 1 || d->d < 1 || d->C_out < 1)
     return fail(MSLA_ERR_INVALID_ARG, "B, C, H, W, heads, d, C_out must be positive");
   if (!(d->eps >= 0.f)) return fail(MSLA_ERR_INVALID_ARG, "eps must be >= 0");
@@ -307,6 +312,7 @@ static msla_status_t run_project_in(msla_dtype_t dt, const void* x, const void* 
   if (dt == MSLA_BF16 && project_in_bf16_supported(C, Cout, N, d)) return run_project_in_bf16(x, w, y, B, C, Cout, N, d, y_sb, st);
   generic::GemmArgs g{(long long)C * N, 1, N, y_sb, d, 1, (long long)N * d, N, Cout, C, d};
   if (dt == MSLA_F32) launch_gemm<float>((const float*)x, (const float*)w, nullptr, (float*)y, g, B, st);
+  else if (dt == MSLA_F16) launch_gemm<__half>((const __half*)x, (const __half*)w, nullptr, (__half*)y, g, B, st);
   else launch_gemm<__nv_bfloat16>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w, nullptr, (__nv_bfloat16*)y, g, B, st);
   return check_launch("input projection");
 }
@@ -316,6 +322,7 @@ static msla_status_t run_project_out(msla_dtype_t dt, const void* a, const void*
   if (dt == MSLA_BF16 && project_out_bf16_supported(Cin, Cout, N)) return run_project_out_bf16(a, w, bias, residual, y, B, Cin, Cout, N, st);
   generic::GemmArgs g{(long long)N * Cin, Cin, 1, (long long)Cout * N, 1, N, 0, N, Cout, Cin, Cout, 0, residual};
   if (dt == MSLA_F32) launch_gemm<float>((const float*)a, (const float*)w, (const float*)bias, (float*)y, g, B, st);
+  else if (dt == MSLA_F16) launch_gemm<__half>((const __half*)a, (const __half*)w, (const __half*)bias, (__half*)y, g, B, st);
   else launch_gemm<__nv_bfloat16>((const __nv_bfloat16*)a, (const __nv_bfloat16*)w, (const __nv_bfloat16*)bias, (__nv_bfloat16*)y, g, B, st);
   return check_launch("output projection");
 }
@@ -346,6 +353,9 @@ static msla_status_t run_aggregate(msla_dtype_t dt, const void* src, const void*
   if (dt == MSLA_F32)
     generic::aggregate_kernel<float><<<grid, 256, 0, st>>>((const float*)src, (const float*)w_dw, (const float*)w_pw,
                                                            (float*)dst, H, W, d, src_sb, dst_sb);
+  else if (dt == MSLA_F16)
+    generic::aggregate_kernel<__half><<<grid, 256, 0, st>>>((const __half*)src, (const __half*)w_dw, (const __half*)w_pw,
+                                                            (__half*)dst, H, W, d, src_sb, dst_sb);
   else
     generic::aggregate_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)src, (const __nv_bfloat16*)w_dw,
                                                                    (const __nv_bfloat16*)w_pw, (__nv_bfloat16*)dst, H, W, d,
@@ -363,7 +373,7 @@ static const void* aggregation_taps(const msla_desc* desc, const msla_weights* w
   const long long total = 3LL * p.Cp * 25;
   if (desc->dtype == MSLA_F32)
     generic::embed_taps_kernel<float><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const float*)w_dw, (float*)w5, total);
-  else
+  else  // 16-bit patterns are copied as they are: bf16 and fp16 alike (zero is all bits clear in both)
     generic::embed_taps_kernel<__nv_bfloat16><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const __nv_bfloat16*)w_dw, (__nv_bfloat16*)w5, total);
   count_launches(1);
   return w5;
@@ -593,7 +603,7 @@ struct FfnPlan {
 static msla_status_t validate_ffn(const msla_ffn_desc* d, FfnPlan* plan) {
   if (!d) return fail(MSLA_ERR_INVALID_ARG, "null descriptor");
   if (d->struct_size != sizeof(msla_ffn_desc)) return fail(MSLA_ERR_INVALID_ARG, "desc.struct_size = %u, expected %zu", d->struct_size, sizeof(msla_ffn_desc));
-  if (d->dtype != MSLA_F32 && d->dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype %d", (int)d->dtype);
+  if (!known_dtype(d->dtype)) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype %d", (int)d->dtype);
   if (d->B < 1 || d->C < 1 || d->H < 1 || d->W < 1 || d->C_hidden < 1 || d->C_out < 1)
     return fail(MSLA_ERR_INVALID_ARG, "B, C, H, W, C_hidden, C_out must be positive");
   if (d->act != MSLA_ACT_IDENTITY && d->act != MSLA_ACT_RELU && d->act != MSLA_ACT_HARDSWISH)
@@ -644,18 +654,16 @@ static msla_status_t ffn_impl(const msla_ffn_desc* desc, const void* x, const ms
   generic::GemmArgs g1{(long long)C * N, 1, N, (long long)Ch * N, 1, N, 0, N, Ch, C, Ch, act, nullptr};
   generic::GemmArgs g2{(long long)Ch * N, 1, N, (long long)Co * N, 1, N, 0, N, Co, Ch, Co, 0, res};
   const long long total = (long long)B * Ch * N;
-  if (desc->dtype == MSLA_F32) {
-    launch_gemm<float>((const float*)x, (const float*)w->w1, (const float*)w->b1, (float*)h, g1, B, st);
-    generic::ffn_dw3x3_nchw_kernel<float><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const float*)h, (const float*)w->w_dw, (const float*)w->b_dw,
-                                                                                            (float*)g, Ch, desc->H, desc->W, act, total);
-    launch_gemm<float>((const float*)g, (const float*)w->w2, (const float*)w->b2, (float*)out, g2, B, st);
-  } else {
-    using T = __nv_bfloat16;
+  auto plain = [&](auto* tag) {
+    using T = std::remove_pointer_t<decltype(tag)>;
     launch_gemm<T>((const T*)x, (const T*)w->w1, (const T*)w->b1, (T*)h, g1, B, st);
     generic::ffn_dw3x3_nchw_kernel<T><<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>((const T*)h, (const T*)w->w_dw, (const T*)w->b_dw, (T*)g, Ch,
                                                                                         desc->H, desc->W, act, total);
     launch_gemm<T>((const T*)g, (const T*)w->w2, (const T*)w->b2, (T*)out, g2, B, st);
-  }
+  };
+  if (desc->dtype == MSLA_F32) plain((float*)nullptr);
+  else if (desc->dtype == MSLA_F16) plain((__half*)nullptr);
+  else plain((__nv_bfloat16*)nullptr);
   count_launches(1);
   return check_launch("FFN with a depthwise convolution");
 }
@@ -788,7 +796,7 @@ int msla_debug_wait_selftest(long long limit_cycles, void* scratch, void* stream
 }
 
 msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d, void* stream) {
-  if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");
+  if (!known_dtype(dtype)) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");
   if (!x || !w || !y) return fail(MSLA_ERR_INVALID_ARG, "null pointer");
   if (B < 1 || C < 1 || Cout < 1 || N < 1 || B > 65535) return fail(MSLA_ERR_INVALID_ARG, "sizes must be positive (B <= 65535)");
   if (C % 8 || Cout % 8) return fail(MSLA_ERR_UNSUPPORTED, "C and Cout must be multiples of 8");
@@ -801,7 +809,7 @@ msla_status_t msla_project_in(msla_dtype_t dtype, const void* x, const void* w, 
 }
 
 msla_status_t msla_aggregate(msla_dtype_t dtype, const void* t, const void* w_dw, const void* w_pw, void* y, int B, int H, int W, int Ch, int d, void* stream) {
-  if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");
+  if (!known_dtype(dtype)) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");
   if (!t || !w_dw || !w_pw || !y) return fail(MSLA_ERR_INVALID_ARG, "null pointer");
   if (B < 1 || H < 1 || W < 1 || Ch < 1 || d < 1 || B > 65535) return fail(MSLA_ERR_INVALID_ARG, "sizes must be positive (B <= 65535)");
   if ((long long)H * W > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "H*W exceeds 2^31-1");
@@ -817,7 +825,7 @@ msla_status_t msla_aggregate(msla_dtype_t dtype, const void* t, const void* w_dw
 }
 
 msla_status_t msla_project_out(msla_dtype_t dtype, const void* a, const void* w, const void* bias, void* y, int B, int Cin, int Cout, int N, void* stream) {
-  if (dtype != MSLA_F32 && dtype != MSLA_BF16) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");
+  if (!known_dtype(dtype)) return fail(MSLA_ERR_INVALID_ARG, "unknown dtype");
   if (!a || !w || !y) return fail(MSLA_ERR_INVALID_ARG, "null pointer");
   if (B < 1 || Cin < 1 || Cout < 1 || N < 1 || B > 65535) return fail(MSLA_ERR_INVALID_ARG, "sizes must be positive (B <= 65535)");
   if (Cin % 8 || Cout % 8) return fail(MSLA_ERR_UNSUPPORTED, "Cin and Cout must be multiples of 8");

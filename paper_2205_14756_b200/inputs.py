@@ -76,12 +76,14 @@ def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
 
 
 def quantise(a: np.ndarray, dtype: str) -> np.ndarray:
-    """Round ``a`` to the storage type of a config ('f32' or 'bf16') and return
+    """Round ``a`` to the storage type of a config ('f32', 'bf16' or 'f16') and return
     it widened back to float32.  Both implementations consume these values."""
     if dtype == "f32":
         return np.ascontiguousarray(a, dtype=np.float32)
     if dtype == "bf16":
         return bf16_bits_to_f32(round_to_bf16_bits(a)).reshape(a.shape)
+    if dtype == "f16":  # IEEE binary16, round to nearest even (numpy's conversion)
+        return np.ascontiguousarray(a, dtype=np.float32).astype(np.float16).astype(np.float32)
     raise ValueError(dtype)
 
 

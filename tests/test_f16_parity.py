@@ -1,0 +1,56 @@
+"""fp16 storage (the paper's deployment precision, Section 4.1's TensorRT fp16 runs) through the C ABI: every entry
+point with dtype MSLA_F16, element by element against the fp64 oracle on inputs rounded to fp16.  fp16 runs on the
+library's plain kernels: fp32 arithmetic and state, one rounding per stored value."""
+import numpy as np
+import pytest
+
+import oracle
+import util
+from paper_2205_14756_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("B,heads,N,d", [(2, 3, 300, 32), (1, 4, 4096, 16), (1, 2, 7, 32)])
+def test_core_f16(B, heads, N, d):
+    s = inputs.CoreShape("core_f16", "f16", B, heads, N, d, seed=51)
+    t = inputs.core_inputs(s)
+    got = util.run_core(t, "f16")
+    util.assert_close(got, oracle.linattn_relu(t["q"], t["k"], t["v"]), "f16", "core fp16", block=util.CORE_BLOCK)
+
+
+@pytest.mark.parametrize("B,C,H,W,heads,d,n_scales,k1", [(1, 64, 16, 16, 4, 16, 2, 5), (2, 64, 9, 20, 2, 32, 2, 3), (1, 96, 12, 12, 3, 32, 3, 5)])
+def test_module_f16(B, C, H, W, heads, d, n_scales, k1):
+    s = inputs.ModuleShape("module_f16", "f16", B, C, H, W, heads, d, seed=52, n_scales=n_scales, agg_kernel=k1)
+    t = inputs.module_inputs(s)
+    if n_scales == 3:
+        ref = oracle.msla_forward3(t["x"], t["w_qkv"], t["w_dw"], t["w_pw"], t["w_dw2"], t["w_pw2"], t["w_proj"], heads=heads, d=d)
+    else:
+        ref = oracle.msla_forward(t["x"], t["w_qkv"], t["w_dw"], t["w_pw"], t["w_proj"], heads=heads, d=d)
+    util.assert_close(util.run_module(s, t), ref, "f16", "module fp16", block=util.MODULE_BLOCK)
+
+
+def test_many_tokens_do_not_overflow_f16():
+    """The state sums over all tokens (here 16 384 per head: entries of the order of 10^4) and stays in fp32; only
+    the quotient of Eq. 3, which is of the order of the values, is stored in 16 bits."""
+    s = inputs.ModuleShape("module_f16_128x128", "f16", 1, 32, 128, 128, 1, 32, seed=53)
+    t = inputs.module_inputs(s)
+    ref = oracle.msla_forward(t["x"], t["w_qkv"], t["w_dw"], t["w_pw"], t["w_proj"], heads=1, d=32)
+    util.assert_close(util.run_module(s, t), ref, "f16", "fp16, 16384 tokens", block=util.MODULE_BLOCK)
+
+
+def test_ffn_and_block_f16():
+    fs = inputs.FfnShape("ffn_f16", "f16", 2, 32, 9, 12, 96, 32, seed=54)
+    ft = inputs.ffn_inputs(fs)
+    ref = oracle.ffn_dwconv(ft["x"], ft["w1"], ft["w_dw"], ft["w2"], ft["b1"], ft["b_dw"], ft["b2"], act="hardswish", residual=True)
+    util.assert_close(util.run_ffn(fs, ft, "hardswish", True), ref, "f16", "FFN fp16", block=util.MODULE_BLOCK)
+    s = inputs.ModuleShape("block_f16", "f16", 1, 64, 12, 16, 2, 32, seed=55)
+    t = inputs.module_inputs(s)
+    f = inputs.ffn_inputs(inputs.FfnShape("block_ffn_f16", "f16", 1, 64, 12, 16, 128, 64, seed=55))
+    ref = oracle.evit_block(t["x"], t, f, heads=2, d=32, act="hardswish")
+    util.assert_close(util.run_block(s, t, f, 128, "hardswish"), ref, "f16", "block fp16", block=util.MODULE_BLOCK)
+
+
+def test_f16_never_takes_the_fused_bf16_kernels():
+    desc = binding.make_desc(1, 256, 64, 64, 8, 32, 256, binding.MSLA_F16)
+    assert binding.msla_forward_workspace_bytes(desc) > 0 and binding.msla_forward_fuses_apply(desc) == 0

@@ -4,8 +4,8 @@ import torch
 
 from paper_2205_14756_b200 import binding, inputs
 
-TORCH_DTYPE = {"f32": torch.float32, "bf16": torch.bfloat16}
-CODE = {"f32": binding.MSLA_F32, "bf16": binding.MSLA_BF16}
+TORCH_DTYPE = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}
+CODE = {"f32": binding.MSLA_F32, "bf16": binding.MSLA_BF16, "f16": binding.MSLA_F16}
 
 # Acceptance bounds: fp32 storage -> max-abs error over max |ref| <= 1e-4;
 # bf16 storage with fp32 accumulation -> relative L2 error <= 1e-2.
@@ -41,6 +41,10 @@ def rel_l2(got: np.ndarray, ref: np.ndarray) -> float:
 MODULE_BLOCK = (1, 32, 16, 16)
 CORE_BLOCK = (1, 1, 256, 0)   # 0 = the whole axis
 TOL_BF16_MAXABS = 3e-2
+# fp16 storage (fp32 arithmetic, one rounding per stored value): the bf16 bounds scaled by the ratio of the unit
+# roundoffs, 2^-11 / 2^-8 = 1/8.
+TOL_F16_RELL2 = 1.25e-3
+TOL_F16_MAXABS = 3.75e-3
 
 
 def worst_block(got: np.ndarray, ref: np.ndarray, block) -> tuple:
@@ -66,13 +70,14 @@ def assert_close(got: np.ndarray, ref: np.ndarray, dtype: str, what: str = "", b
         err = max_abs_rel(got, ref)
         assert err <= TOL_F32_MAXABS, f"{what}: max-abs/max|ref| = {err:.3e} > {TOL_F32_MAXABS}"
     else:
+        tol_l2, tol_max = (TOL_F16_RELL2, TOL_F16_MAXABS) if dtype == "f16" else (TOL_BF16_RELL2, TOL_BF16_MAXABS)
         err = rel_l2(got, ref)
-        assert err <= TOL_BF16_RELL2, f"{what}: rel-L2 = {err:.3e} > {TOL_BF16_RELL2}"
+        assert err <= tol_l2, f"{what}: rel-L2 = {err:.3e} > {tol_l2}"
         mx = max_abs_rel(got, ref)
-        assert mx <= TOL_BF16_MAXABS, f"{what}: max-abs/max|ref| = {mx:.3e} > {TOL_BF16_MAXABS}"
+        assert mx <= tol_max, f"{what}: max-abs/max|ref| = {mx:.3e} > {tol_max}"
         if block is not None:
             w, where = worst_block(got, ref, block)
-            assert w <= TOL_BF16_RELL2, f"{what}: block {where} has rel-L2 = {w:.3e} > {TOL_BF16_RELL2}"
+            assert w <= tol_l2, f"{what}: block {where} has rel-L2 = {w:.3e} > {tol_l2}"
 
 
 # Guard regions: every output and workspace handed to the library sits inside a larger allocation whose 4 KB on
