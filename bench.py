@@ -492,11 +492,13 @@ def main() -> None:
     def time_core(cs: inputs.CoreShape, blocks=BLOCKS, steps=K):
         """Stand-alone attention core (steps 3 + 4) on seeded q, k, v: (median ms per call, min, max, bytes)."""
         ct = inputs.core_inputs(cs)
-        q, k, v = (torch.from_numpy(ct[n]).to("cuda").to(tdt).contiguous() for n in ("q", "k", "v"))
+        cdt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[cs.dtype]
+        ccode = {"f32": binding.MSLA_F32, "bf16": binding.MSLA_BF16, "f16": binding.MSLA_F16}[cs.dtype]
+        q, k, v = (torch.from_numpy(ct[n]).to("cuda").to(cdt).contiguous() for n in ("q", "k", "v"))
         o = torch.empty_like(q)
         nb = binding.msla_linattn_relu_workspace_bytes(cs.B, cs.heads, cs.N, cs.d)
         cws = torch.empty(nb, dtype=torch.uint8, device="cuda")
-        call = lambda i: binding.msla_linattn_relu_ws(code, q, k, v, o, cs.B, cs.heads, cs.N, cs.d, cs.eps, cws, nb)
+        call = lambda i: binding.msla_linattn_relu_ws(ccode, q, k, v, o, cs.B, cs.heads, cs.N, cs.d, cs.eps, cws, nb)
         for i in range(3):
             call(i)
         ms = [m / steps for m in timed_blocks(call, blocks=blocks, steps=steps)]
@@ -578,6 +580,10 @@ def main() -> None:
         other["cfg2_core"] = {"workload": c2.name, "ms": round(m2, 5), "ms_min": round(lo2, 5), "ms_max": round(hi2, 5),
                               "token_heads_per_s": c2.B * c2.heads * c2.N / (m2 * 1e-3), "GBps": round(b2 / (m2 * 1e-3) / 1e9, 1),
                               "l2": "L2-resident (134 MB in and out)"}
+        m2h, lo2h, hi2h, b2h = time_core(inputs.CoreShape(c2.name.replace("bf16", "f16"), "f16", c2.B, c2.heads, c2.N, c2.d, c2.seed), blocks=5, steps=10)
+        other["cfg2_core_f16"] = {"workload": c2.name.replace("bf16", "f16"), "ms": round(m2h, 5), "ms_min": round(lo2h, 5), "ms_max": round(hi2h, 5),
+                                  "token_heads_per_s": c2.B * c2.heads * c2.N / (m2h * 1e-3), "GBps": round(b2h / (m2h * 1e-3) / 1e9, 1),
+                                  "l2": "L2-resident (134 MB in and out)"}
         other["cfg3"] = time_module(inputs.CONFIG3)
         other["cfg4"] = time_module(inputs.CONFIG4)
         # a bf16, d = 16 sibling of config 1's width at 256 x 256 tokens, 384 channels

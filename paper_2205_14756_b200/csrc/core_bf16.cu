@@ -1,4 +1,4 @@
-// Tuned bf16 attention core (Eq. 3): KV-state reduction and apply step on
+// Tuned 16-bit (bf16, and fp16) attention core (Eq. 3): KV-state reduction and apply step on
 // warp-level tensor-core MMAs with fp32 accumulation.
 //
 // Both steps are HBM-bound only if their small contractions (d x (d+1) per
@@ -17,15 +17,24 @@ namespace {
 
 using bf16 = __nv_bfloat16;
 
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+// F16 selects the 16-bit storage type of the operands: IEEE binary16 instead of bfloat16.  Accumulators are fp32 in both.
+template <bool F16>
+__device__ __forceinline__ void mma16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  if constexpr (F16)
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+  else
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ uint32_t relu2(uint32_t x) {  // packed bf16x2 max(x, 0)
+template <bool F16>
+__device__ __forceinline__ uint32_t relu2(uint32_t x) {  // packed max(x, 0) on two 16-bit values
   uint32_t r;
-  asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(0u));
+  if constexpr (F16) asm("max.f16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(0u));
+  else asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(0u));
   return r;
 }
 
@@ -37,10 +46,18 @@ __device__ __forceinline__ void stg(void* p, const uint32_t (&r)[4]) {
   asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
 }
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+template <bool F16>
+__device__ __forceinline__ uint32_t pack16(float lo, float hi) {
   uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  if constexpr (F16) asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  else asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
+}
+// v rounded to the 16-bit type and widened again
+template <bool F16>
+__device__ __forceinline__ float round16(float v) {
+  if constexpr (F16) return __half2float(__float2half_rn(v));
+  else return __bfloat162float(__float2bfloat16_rn(v));
 }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -79,7 +96,7 @@ __device__ __forceinline__ void lds64(uint32_t (&r)[2], uint32_t addr) {
 // occupancy); no block-wide barrier is taken inside the loop.  An extra B tile
 // of bf16 ones yields sum relu(k).
 // ---------------------------------------------------------------------------
-template <int D, int NWARPS, int STAGES>
+template <int D, int NWARPS, int STAGES, bool F16>
 __global__ void __launch_bounds__(NWARPS * 32)
 kv_state_mma_kernel(const bf16* __restrict__ k, const bf16* __restrict__ v, float* __restrict__ partial,
                     HeadView kv, int heads, int N, int S, int chunk) {
@@ -160,7 +177,7 @@ kv_state_mma_kernel(const bf16* __restrict__ k, const bf16* __restrict__ v, floa
         const int c = 2 * i + (lm & 1);
         ldsm_x4_trans(A[i], tK + r * ROWB + ((c ^ ((r >> SW_SHIFT) & (CH - 1))) << 4));
 #pragma unroll
-        for (int e = 0; e < 4; ++e) A[i][e] = relu2(A[i][e]);
+        for (int e = 0; e < 4; ++e) A[i][e] = relu2<F16>(A[i][e]);
       }
 #pragma unroll
       for (int j = 0; j < NT; j += 2) {
@@ -174,8 +191,8 @@ kv_state_mma_kernel(const bf16* __restrict__ k, const bf16* __restrict__ v, floa
 #pragma unroll
       for (int i = 0; i < MT; ++i) {
 #pragma unroll
-        for (int j = 0; j < NT; ++j) mma_bf16(acc[i][j], A[i], Bt[j][0], Bt[j][1]);
-        mma_bf16(acc[i][NT], A[i], 0x3F803F80u, 0x3F803F80u);  // bf16 ones
+        for (int j = 0; j < NT; ++j) mma16<F16>(acc[i][j], A[i], Bt[j][0], Bt[j][1]);
+        mma16<F16>(acc[i][NT], A[i], F16 ? 0x3C003C00u : 0x3F803F80u, F16 ? 0x3C003C00u : 0x3F803F80u);  // ones
       }
     }
     __syncwarp();  // all lanes done with this stage before a later issue() overwrites it
@@ -237,10 +254,13 @@ kv_combine_bf16path_kernel(const float* __restrict__ partial, float* __restrict_
 // PAIR: one CTA serves heads 2p (even warps) and 2p+1 (odd warps) of a paired
 // output view, so that the two 64-byte halves of each 128-byte output row are
 // written at nearly the same time.
-template <int D, int NWARPS, int STAGES, int U, bool PAIR>
+// state_scale: the state (numerator and denominator columns alike) and eps are multiplied by it before they are cut
+// into 16-bit pieces; the quotient of Eq. 3 does not change.  1 for bf16 (its exponent range is fp32's); for fp16 a
+// power of two near 1/N, so that sums over N tokens fit the format.
+template <int D, int NWARPS, int STAGES, int U, bool PAIR, bool F16>
 __global__ void __launch_bounds__(NWARPS * 32)
 apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf16* __restrict__ out,
-                 HeadView qv, HeadView ov, int heads, int N, float eps, int tok_per_cta) {
+                 HeadView qv, HeadView ov, int heads, int N, float eps, int tok_per_cta, float state_scale) {
   constexpr int KS = D / 16;   // MMA steps over the channel contraction
   constexpr int NT = D / 8;    // output tiles, + 1 for the denominator
   constexpr int CPT = D / 4;   // channels per lane per token
@@ -301,10 +321,9 @@ apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf
         for (int r = 0; r < 2; ++r) {
           const int a0 = CPT * t + 4 * ks + 2 * r;
           const int c = j < NT ? (g >> 1) * CPT + 2 * j + (g & 1) : D;
-          const float v0 = st[a0 * (D + 1) + c], v1 = st[(a0 + 1) * (D + 1) + c];
-          const bf16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
-          bhi[ks][j][r] = pack_bf16(v0, v1);
-          blo[ks][j][r] = pack_bf16(v0 - __bfloat162float(h0), v1 - __bfloat162float(h1));
+          const float v0 = st[a0 * (D + 1) + c] * state_scale, v1 = st[(a0 + 1) * (D + 1) + c] * state_scale;
+          bhi[ks][j][r] = pack16<F16>(v0, v1);
+          blo[ks][j][r] = pack16<F16>(v0 - round16<F16>(v0), v1 - round16<F16>(v1));
         }
   }
 
@@ -337,17 +356,17 @@ apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf
       uint32_t A[U][4];
 #pragma unroll
       for (int u = 0; u < U; ++u) {
-        A[u][0] = relu2(qa[u][2 * ks]); A[u][1] = relu2(qb[u][2 * ks]);
-        A[u][2] = relu2(qa[u][2 * ks + 1]); A[u][3] = relu2(qb[u][2 * ks + 1]);
+        A[u][0] = relu2<F16>(qa[u][2 * ks]); A[u][1] = relu2<F16>(qb[u][2 * ks]);
+        A[u][2] = relu2<F16>(qa[u][2 * ks + 1]); A[u][3] = relu2<F16>(qb[u][2 * ks + 1]);
       }
 #pragma unroll
       for (int j = 0; j <= NT; ++j)
 #pragma unroll
-        for (int u = 0; u < U; ++u) mma_bf16(acc[u][j], A[u], bhi[ks][j][0], bhi[ks][j][1]);
+        for (int u = 0; u < U; ++u) mma16<F16>(acc[u][j], A[u], bhi[ks][j][0], bhi[ks][j][1]);
 #pragma unroll
       for (int j = 0; j <= NT; ++j)
 #pragma unroll
-        for (int u = 0; u < U; ++u) mma_bf16(acc[u][j], A[u], blo[ks][j][0], blo[ks][j][1]);
+        for (int u = 0; u < U; ++u) mma16<F16>(acc[u][j], A[u], blo[ks][j][0], blo[ks][j][1]);
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -355,8 +374,8 @@ apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf
       uint32_t oa[WQ], ob[WQ];
 #pragma unroll
       for (int j = 0; j < NT; ++j) {
-        oa[j] = pack_bf16(acc[u][j][0] * inv_a, acc[u][j][1] * inv_a);
-        ob[j] = pack_bf16(acc[u][j][2] * inv_b, acc[u][j][3] * inv_b);
+        oa[j] = pack16<F16>(acc[u][j][0] * inv_a, acc[u][j][1] * inv_a);
+        ob[j] = pack16<F16>(acc[u][j][2] * inv_b, acc[u][j][3] * inv_b);
       }
       const int na = n0 + u * 16 + g, nb = na + 8;
       if (na < n_end) stg(out + obase + (long long)na * ov.ld, oa);
@@ -366,7 +385,7 @@ apply_mma_kernel(const bf16* __restrict__ q, const float* __restrict__ state, bf
   cp_async_wait<0>();
 }
 
-template <int D>
+template <int D, bool F16>
 msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out, HeadView in, HeadView ov, int B,
                           int heads, int N, float eps, const CorePlan& p, char* ws, cudaStream_t st, cudaEvent_t mid, int phases) {
   // 4 warps per CTA and 4-deep rings in both kernels; two 16-token MMA tiles per FIFO stage of the apply step
@@ -376,11 +395,11 @@ msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out
   float* state = reinterpret_cast<float*>(ws + p.state_off);
   constexpr int kv_smem = KV_WARPS * KV_STAGES * 2 * 32 * D * 2;
   static std::atomic<unsigned long long> attr_done{0};
-  const msla_status_t as = ensure_smem_attr(attr_done, kv_state_mma_kernel<D, KV_WARPS, KV_STAGES>, kv_smem);
+  const msla_status_t as = ensure_smem_attr(attr_done, kv_state_mma_kernel<D, KV_WARPS, KV_STAGES, F16>, kv_smem);
   if (as != MSLA_OK) return as;
   int launches = 0;
   if (phases & CORE_STATE) {
-    launch_pdl(kv_state_mma_kernel<D, KV_WARPS, KV_STAGES>, dim3((unsigned)BH, p.S), dim3(KV_WARPS * 32), kv_smem, st, k, v, partial, in, heads, N, p.S, p.chunk);
+    launch_pdl(kv_state_mma_kernel<D, KV_WARPS, KV_STAGES, F16>, dim3((unsigned)BH, p.S), dim3(KV_WARPS * 32), kv_smem, st, k, v, partial, in, heads, N, p.S, p.chunk);
     ++launches;
   }
   if (phases & CORE_COMBINE) {
@@ -390,29 +409,38 @@ msla_status_t launch_core(const bf16* q, const bf16* k, const bf16* v, bf16* out
   }
   if (mid) cudaEventRecord(mid, st);
   if (phases & CORE_APPLY) {
+    // fp16 pieces of the state must fit the format: a sum over N tokens is scaled by the power of two just above 1/N
+    float state_scale = 1.f;
+    if (F16) for (long long n = 1; n < N; n *= 2) state_scale *= 0.5f;
+    eps *= state_scale;
     if (ov.pair) {  // heads is even here, so a pair never straddles two images
       const int tok_per_cta = p.apply_tokens / 2;
-      launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, true>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)(BH / 2)),
-                 dim3(AP_WARPS * 32), 0, st, q, state, out, in, ov, heads, N, eps, tok_per_cta);
+      launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, true, F16>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)(BH / 2)),
+                 dim3(AP_WARPS * 32), 0, st, q, state, out, in, ov, heads, N, eps, tok_per_cta, state_scale);
     } else {
       const int tok_per_cta = p.apply_tokens;
-      launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, false>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)BH),
-                 dim3(AP_WARPS * 32), 0, st, q, state, out, in, ov, heads, N, eps, tok_per_cta);
+      launch_pdl(apply_mma_kernel<D, AP_WARPS, AP_STAGES, AP_U, false, F16>, dim3((unsigned)ceil_div_ll(N, tok_per_cta), (unsigned)BH),
+                 dim3(AP_WARPS * 32), 0, st, q, state, out, in, ov, heads, N, eps, tok_per_cta, state_scale);
     }
     ++launches;
   }
   count_launches(launches);
-  return check_launch("attention core kernels (bf16)");
+  return check_launch(F16 ? "attention core kernels (fp16)" : "attention core kernels (bf16)");
 }
 
 }  // namespace
 
 msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* out, HeadView in, HeadView ov, int B,
                             int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st,
-                            cudaEvent_t mid, int phases) {
-  if (d == 32)
-    return launch_core<32>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid, phases);
-  return launch_core<16>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid, phases);
+                            cudaEvent_t mid, int phases, bool f16) {
+  // the kernels move 16-bit values untyped; only the MMA, ReLU and conversion instructions depend on the format
+  const bf16 *q16 = (const bf16*)q, *k16 = (const bf16*)k, *v16 = (const bf16*)v;
+  if (f16) {
+    if (d == 32) return launch_core<32, true>(q16, k16, v16, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid, phases);
+    return launch_core<16, true>(q16, k16, v16, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid, phases);
+  }
+  if (d == 32) return launch_core<32, false>(q16, k16, v16, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid, phases);
+  return launch_core<16, false>(q16, k16, v16, (bf16*)out, in, ov, B, heads, N, eps, p, (char*)ws, st, mid, phases);
 }
 
 }  // namespace msla

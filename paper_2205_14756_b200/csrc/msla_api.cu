@@ -150,9 +150,12 @@ static msla_status_t run_core(msla_dtype_t dtype, const void* q, const void* k, 
   if (dtype == MSLA_F32)
     return run_core_generic<float>((const float*)q, (const float*)k, (const float*)v, (float*)out,
                                    in, ov, B, heads, N, d, eps, p, (char*)ws, st, mid, phases);
-  if (dtype == MSLA_F16)  // fp16 storage runs on the plain kernels (fp32 arithmetic, one rounding per stored value)
+  if (dtype == MSLA_F16) {  // the tensor-core kernels take fp16 too; other strides run on the plain kernels
+    const bool ok16 = !ov.pair && in.batch % 8 == 0 && in.head % 8 == 0 && in.ld % 8 == 0 && ov.batch % 8 == 0 && ov.head % 8 == 0 && ov.ld % 8 == 0;
+    if (ok16) return run_core_bf16(q, k, v, out, in, ov, B, heads, N, d, eps, p, ws, st, mid, phases, true);
     return run_core_generic<__half>((const __half*)q, (const __half*)k, (const __half*)v, (__half*)out,
                                     in, ov, B, heads, N, d, eps, p, (char*)ws, st, mid, phases);
+  }
   const bool strides_ok = in.batch % 8 == 0 && in.head % 8 == 0 && in.ld % 8 == 0 && ov.batch % 8 == 0 &&
                           ov.head % 8 == 0 && ov.ld % 8 == 0;
   if (strides_ok) return run_core_bf16(q, k, v, out, in, ov, B, heads, N, d, eps, p, ws, st, mid, phases);

@@ -93,13 +93,13 @@ inline void launch_pdl_cluster2(void (*kernel)(KArgs...), dim3 grid, dim3 block,
 }
 
 struct HeadView;
-// Tuned bf16 attention core (d in {16, 32}); all view strides must be multiples of 8 elements.
+// Tuned attention core for 16-bit storage, bf16 or (f16 = true) fp16 (d in {16, 32}); all view strides must be multiples of 8 elements.
 // `phases` selects what runs: CORE_STATE the partial states (at ws + p.partial_off, p.S per head), CORE_COMBINE their
 // fixed-order sum (at ws + p.state_off), CORE_APPLY the apply step reading that sum; without CORE_APPLY `out` and `ov` are unused.
 enum : int { CORE_STATE = 1, CORE_COMBINE = 2, CORE_APPLY = 4, CORE_ALL = 7 };
 msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* out, HeadView in, HeadView ov, int B,
                             int heads, int N, int d, float eps, const CorePlan& p, void* ws, cudaStream_t st,
-                            cudaEvent_t mid, int phases);
+                            cudaEvent_t mid, int phases, bool f16 = false);
 
 // FFN with a depthwise convolution (gemm_tcgen05.cu, ffn_dw_bf16.cu): bf16; the hidden tensor is planes of 32 channels
 // [B][Ch / 32][N][32] after the first layer, planes of 64 channels [B][Ch / 64][N][64] after the depthwise convolution.
