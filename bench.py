@@ -513,8 +513,8 @@ def main() -> None:
     def time_module(ms_shape: inputs.ModuleShape, blocks=5, steps=10):
         """Plain msla_forward on another configuration: dict with ms per step, tokens/s and module GB/s."""
         mt = inputs.module_inputs(ms_shape)
-        mdt = torch.float32 if ms_shape.dtype == "f32" else torch.bfloat16
-        mcode = binding.MSLA_F32 if ms_shape.dtype == "f32" else binding.MSLA_BF16
+        mdt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[ms_shape.dtype]
+        mcode = {"f32": binding.MSLA_F32, "bf16": binding.MSLA_BF16, "f16": binding.MSLA_F16}[ms_shape.dtype]
         mx = torch.from_numpy(mt["x"]).to("cuda").to(mdt).contiguous()
         mw = [torch.from_numpy(mt[n]).to("cuda").to(mdt).contiguous() for n in ("w_qkv", "w_dw", "w_pw", "w_proj")]
         mweights = binding.make_weights(*mw)
@@ -588,6 +588,9 @@ def main() -> None:
         other["cfg4"] = time_module(inputs.CONFIG4)
         # a bf16, d = 16 sibling of config 1's width at 256 x 256 tokens, 384 channels
         other["d16_256x256_c384"] = time_module(inputs.ModuleShape("bf16_d16_256x256_c384", "bf16", 1, 384, 256, 256, 24, 16, seed=7))
+        # fp16 storage at the bench workload's shape: projections, aggregation and attention core on their f16
+        # tensor-core instantiations, steps 4 and 5 as two kernels
+        other["cfg5_512x512_f16"] = time_module(inputs.ModuleShape(s.name.replace("bf16", "f16"), "f16", s.B, s.C, s.H, s.W, s.heads, s.d, seed=s.seed))
         # the token-sharded path's two band calls on one rank (no halo, one state): what the split itself costs
         band1 = time_token_sharded(s, 0, 1, steps=10, warmup=3, blocks=5)
         other["band_calls_one_rank"] = {"workload": s.name, "ms": round(med(band1), 5), "ms_min": round(min(band1), 5),

@@ -69,15 +69,25 @@ static_assert(BOX_ROW % 512 == 0, "the 64B swizzle pattern must restart with eve
 __device__ int g_aggt_timeout_flag = 0;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+// F16: the 16-bit storage type is IEEE binary16 instead of bfloat16 (activations and weights alike); the kernel moves
+// 16-bit values untyped, only the conversions and the MMA operand type differ.  Accumulators are fp32 in both.
+template <bool F16>
+__device__ __forceinline__ uint32_t pack_x2(float lo, float hi) {
   uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  if constexpr (F16) asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  else asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
-__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+template <bool F16>
+__device__ __forceinline__ void mma_16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  if constexpr (F16)
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  else
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ void ldsm_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3, uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -101,7 +111,7 @@ struct ToeplitzParams {
   long long units_per_cta;
 };
 
-template <bool D16>
+template <bool D16, bool F16>
 __global__ void __launch_bounds__(T_THREADS, 2)
 aggregate_toeplitz_kernel(const __grid_constant__ CUtensorMap tm_src, const __grid_constant__ CUtensorMap tm_dst, ToeplitzParams p) {
   extern __shared__ unsigned char smem_raw[];
@@ -294,14 +304,14 @@ aggregate_toeplitz_kernel(const __grid_constant__ CUtensorMap tm_src, const __gr
       for (int dy = 0; dy < 5; ++dy)
 #pragma unroll
         for (int nb = 0; nb < 2; ++nb)
-          mma_bf16(acc[nb], R[dy][nb], R[dy + 1][nb], R[dy][nb + 1], R[dy + 1][nb + 1], bt[cc][dy][0], bt[cc][dy][1]);
+          mma_16<F16>(acc[nb], R[dy][nb], R[dy + 1][nb], R[dy][nb + 1], R[dy + 1][nb + 1], bt[cc][dy][0], bt[cc][dy][1]);
       // pixel pair (row 2g + half, columns 8nb + 2t, +1) goes to word (2nb + half) * 32 + lane of the channel's row
       const uint32_t o = dwo + (uint32_t)(c * DWO_CH + lane * 4);
 #pragma unroll
       for (int nb = 0; nb < 2; ++nb)
 #pragma unroll
         for (int half = 0; half < 2; ++half)
-          sts32(o + (uint32_t)((2 * nb + half) * 128), pack_bf16x2(acc[nb][2 * half], acc[nb][2 * half + 1]));
+          sts32(o + (uint32_t)((2 * nb + half) * 128), pack_x2<F16>(acc[nb][2 * half], acc[nb][2 * half + 1]));
     }
     __syncthreads();
 
@@ -324,14 +334,14 @@ aggregate_toeplitz_kernel(const __grid_constant__ CUtensorMap tm_src, const __gr
         uint32_t a0, a1, a2, a3;  // rows = pixels of block qa / qa+8, contraction = channels 16ks .. 16ks+15
         ldsm_x4_trans(a0, a1, a2, a3, dwo + (uint32_t)((16 * ks + 8 * (mi >> 1) + (lane & 7)) * DWO_CH + (qa + 8 * (mi & 1)) * 16));
 #pragma unroll
-        for (int jn = 0; jn < 4; ++jn) mma_bf16(c[jn], a0, a1, a2, a3, bw[ks][jn][0], bw[ks][jn][1]);
+        for (int jn = 0; jn < 4; ++jn) mma_16<F16>(c[jn], a0, a1, a2, a3, bw[ks][jn][0], bw[ks][jn][1]);
       }
 #pragma unroll
       for (int half = 0; half < 2; ++half)  // staging: [row 2mb + half][pixel g][channels 8t .. 8t+7]; d = 16: one such block of 16 channels per plane
         asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(my_out + (D16 ? (uint32_t)((t >> 1) * (OUT_WARP_BYTES / 2) + ((2 * mb + half) * 8 + g) * 32 + (t & 1) * 16)
                                                                                         : (uint32_t)(((2 * mb + half) * 8 + g) * 64 + t * 16))),
-                     "r"(pack_bf16x2(c[0][2 * half], c[0][2 * half + 1])), "r"(pack_bf16x2(c[1][2 * half], c[1][2 * half + 1])),
-                     "r"(pack_bf16x2(c[2][2 * half], c[2][2 * half + 1])), "r"(pack_bf16x2(c[3][2 * half], c[3][2 * half + 1]))
+                     "r"(pack_x2<F16>(c[0][2 * half], c[0][2 * half + 1])), "r"(pack_x2<F16>(c[1][2 * half], c[1][2 * half + 1])),
+                     "r"(pack_x2<F16>(c[2][2 * half], c[2][2 * half + 1])), "r"(pack_x2<F16>(c[3][2 * half], c[3][2 * half + 1]))
                      : "memory");
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -356,7 +366,7 @@ aggregate_toeplitz_kernel(const __grid_constant__ CUtensorMap tm_src, const __gr
 bool aggregate_bf16_supported(int H, int W, int Ch, int d) { return (d == 32 || d == 16) && Ch % TD == 0 && H >= 1 && W >= 1; }
 
 namespace {
-template <bool D16>
+template <bool D16, bool F16>
 msla_status_t launch_toeplitz(const void* src, long long src_planes_total, int src_ppb, const void* w_dw, const void* w_pw,
                               void* dst, long long dst_planes_total, int dst_ppb, int B, int H, int W, int Ch, cudaStream_t st) {
   constexpr int DP = D16 ? 16 : 32;  // channels per plane
@@ -387,11 +397,11 @@ msla_status_t launch_toeplitz(const void* src, long long src_planes_total, int s
   if (p.units_per_cta > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many aggregation tiles");
   const unsigned grid = (unsigned)((p.units + p.units_per_cta - 1) / p.units_per_cta);
   static std::atomic<unsigned long long> attr_done{0};
-  const msla_status_t as = ensure_smem_attr(attr_done, aggregate_toeplitz_kernel<D16>, T_SMEM_BYTES);
+  const msla_status_t as = ensure_smem_attr(attr_done, aggregate_toeplitz_kernel<D16, F16>, T_SMEM_BYTES);
   if (as != MSLA_OK) return as;
-  launch_pdl(aggregate_toeplitz_kernel<D16>, dim3(grid), dim3(T_THREADS), T_SMEM_BYTES, st, tm_src, tm_dst, p);
+  launch_pdl(aggregate_toeplitz_kernel<D16, F16>, dim3(grid), dim3(T_THREADS), T_SMEM_BYTES, st, tm_src, tm_dst, p);
   count_launches(1);
-  return check_launch("token aggregation (bf16)");
+  return check_launch(F16 ? "token aggregation (fp16)" : "token aggregation (bf16)");
 }
 }  // namespace
 
@@ -400,13 +410,16 @@ msla_status_t launch_toeplitz(const void* src, long long src_planes_total, int s
 // the plane size).
 msla_status_t run_aggregate_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
                                  const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch, int d,
-                                 cudaStream_t st) {
+                                 cudaStream_t st, bool f16) {
   const long long plane = (long long)H * W * d;
   if (!aggregate_bf16_supported(H, W, Ch, d) || dst_sb % plane != 0)
     return fail(MSLA_ERR_UNSUPPORTED, "aggregation: d = %d, %d channels, output batch stride %lld elements", d, Ch, dst_sb);
   const long long dst_ppb = dst_sb / plane, dst_total = (B - 1) * dst_ppb + Ch / d;
-  return d == 16 ? launch_toeplitz<true>(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_total, (int)dst_ppb, B, H, W, Ch, st)
-                 : launch_toeplitz<false>(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_total, (int)dst_ppb, B, H, W, Ch, st);
+  if (f16)
+    return d == 16 ? launch_toeplitz<true, true>(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_total, (int)dst_ppb, B, H, W, Ch, st)
+                   : launch_toeplitz<false, true>(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_total, (int)dst_ppb, B, H, W, Ch, st);
+  return d == 16 ? launch_toeplitz<true, false>(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_total, (int)dst_ppb, B, H, W, Ch, st)
+                 : launch_toeplitz<false, false>(src, src_planes_total, src_ppb, w_dw, w_pw, dst, dst_total, (int)dst_ppb, B, H, W, Ch, st);
 }
 
 int agg_timeout_flag() {

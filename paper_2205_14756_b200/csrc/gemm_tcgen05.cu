@@ -92,7 +92,32 @@ constexpr int STAGING_BYTES = 8 * 2048;  // one 32-row x 64-byte block per epilo
 //      for (1e30, 0); the staging block is double-buffered (NBUF = 2) so that this arithmetic overlaps the previous
 //      block's TMA store instead of lengthening the chain tmem load -> convert -> stage -> store
 //   2  adds p.residual (laid out like the row-major output) after the bias
-template <int EPI, int NBUF = 1>
+// F16: operands and output are IEEE binary16 instead of bfloat16 (16-bit values travel untyped; the MMA's operand
+// format bits and the conversions differ).
+template <bool F16> __device__ __forceinline__ float ld16(const bf16* p) {
+  if constexpr (F16) return __half2float(*reinterpret_cast<const __half*>(p));
+  else return __bfloat162float(*p);
+}
+template <bool F16> __device__ __forceinline__ uint32_t pack16(float lo, float hi) {
+  if constexpr (F16) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+  } else {
+    return pack2(lo, hi);
+  }
+}
+template <bool F16> __device__ __forceinline__ void unpack16(uint32_t w, float& lo, float& hi) {
+  if constexpr (F16) {
+    const __half2 h = *reinterpret_cast<const __half2*>(&w);
+    lo = __low2float(h); hi = __high2float(h);
+  } else {
+    lo = __uint_as_float(w << 16); hi = __uint_as_float(w & 0xffff0000u);
+  }
+}
+template <bool F16> __device__ __forceinline__ constexpr uint32_t operand_format_bits() { return F16 ? 0u : ((1u << 7) | (1u << 10)); }
+
+template <int EPI, int NBUF = 1, bool F16 = false>
 __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUtensorMap* tmO, uint32_t stage, int b,
                                                   int mt, int nt, uint32_t tmem_acc, int quarter, int col_half, int lane,
                                                   const float* bias_sm = nullptr) {
@@ -101,7 +126,7 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUt
   const int m = row0 + lane;
   const bool row_ok = m < p.M;
   bf16* obase = p.out + (long long)b * p.out_batch_stride;
-  const float bias_row = (EPI != 1 && p.bias && p.bias_per_row && row_ok) ? __bfloat162float(p.bias[m]) : 0.f;
+  const float bias_row = (EPI != 1 && p.bias && p.bias_per_row && row_ok) ? ld16<F16>(p.bias + m) : 0.f;
   const bool bias_col = EPI != 1 && p.bias && !p.bias_per_row;
   const int ncol0 = nt * BN + col_half * 128;
   const uint32_t taddr = tmem_acc + col_half * 128 + ((uint32_t)(quarter * 32) << 16);
@@ -137,7 +162,7 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUt
         bc[0] = b0.x; bc[1] = b0.y; bc[2] = b0.z; bc[3] = b0.w; bc[4] = b1.x; bc[5] = b1.y; bc[6] = b1.z; bc[7] = b1.w;
       } else if (EPI == 1) {      // no staged copy (the kernel whose CTAs change weight block from tile to tile)
 #pragma unroll
-        for (int i = 0; i < 8; ++i) bc[i] = (p.bias && n0 + v * 8 < p.N) ? __bfloat162float(p.bias[n0 + v * 8 + i]) : 0.f;
+        for (int i = 0; i < 8; ++i) bc[i] = (p.bias && n0 + v * 8 < p.N) ? ld16<F16>(p.bias + n0 + v * 8 + i) : 0.f;
       }
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
@@ -149,15 +174,17 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUt
         } else {
           f0 += bias_row; f1 += bias_row;
           if (bias_col && n0 + v * 8 < p.N) {
-            f0 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e]);
-            f1 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e + 1]);
+            f0 += ld16<F16>(p.bias + n0 + v * 8 + 2 * e);
+            f1 += ld16<F16>(p.bias + n0 + v * 8 + 2 * e + 1);
           }
         }
         if (EPI == 2) {
           const uint32_t rw = e == 0 ? rs[c & 1][v].x : e == 1 ? rs[c & 1][v].y : e == 2 ? rs[c & 1][v].z : rs[c & 1][v].w;
-          f0 += __uint_as_float(rw << 16); f1 += __uint_as_float(rw & 0xffff0000u);
+          float r0f, r1f;
+          unpack16<F16>(rw, r0f, r1f);
+          f0 += r0f; f1 += r1f;
         }
-        w[v][e] = pack2(f0, f1);
+        w[v][e] = pack16<F16>(f0, f1);
       }
     }
     if (p.tma_store) {
@@ -195,7 +222,7 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUt
 
 // B_PLANAR (output projection with the attention output kept as one [N][64]
 // plane per pair of heads): the 64-wide k-slice kb of B is plane kb of the image.
-template <bool A_MN_MAJOR, bool B_PLANAR, int EPI>
+template <bool A_MN_MAJOR, bool B_PLANAR, int EPI, bool F16>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                          const __grid_constant__ CUtensorMap tmO, GemmParams p) {
@@ -271,7 +298,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       // instruction descriptor: D = f32, A = B = bf16, A major, B K-major, N = 256, M = 128
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN_MAJOR ? 1u : 0u) << 15) |
+      const uint32_t idesc = (1u << 4) | operand_format_bits<F16>() | ((A_MN_MAJOR ? 1u : 0u) << 15) |
                              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
       uint32_t it = 0, local = 0;
       bool ok = true;
@@ -317,7 +344,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      drain_accumulator<EPI>(p, &tmO, staging + (warp - 2) * 2048, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
+      drain_accumulator<EPI, 1, F16>(p, &tmO, staging + (warp - 2) * 2048, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);  // this warp's share of the accumulator is drained
@@ -356,7 +383,7 @@ constexpr int WS_RING_BYTES = 80 * 1024;
 constexpr int WS_SMEM_BYTES = RES_BYTES + WS_RING_BYTES + STAGING_BYTES + 256 + 1024;
 constexpr int WS_MAX_STAGES = 6;
 
-template <int EPI>
+template <int EPI, bool F16>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                             const __grid_constant__ CUtensorMap tmO, GemmParams p, int blocks, int workers) {
@@ -384,7 +411,7 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
   if (EPI == 1) {
     for (int i = threadIdx.x; i < BN; i += NUM_THREADS) {
       const int n = blk * BN + i;
-      bias_sm[i] = (p.bias && !p.bias_per_row && n < p.N) ? __bfloat162float(p.bias[n]) : 0.f;
+      bias_sm[i] = (p.bias && !p.bias_per_row && n < p.N) ? ld16<F16>(p.bias + n) : 0.f;
     }
   }
   const int stream_per_batch = p.m_tiles;
@@ -440,7 +467,7 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) |
+      const uint32_t idesc = (1u << 4) | operand_format_bits<F16>() | (1u << 15) |
                              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
       uint32_t it = 0, local = 0;
       bool ok = mbar_wait(res_bar, 0, &abort_flag);
@@ -482,7 +509,7 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      drain_accumulator<EPI, NBUF>(p, &tmO, staging + (warp - 2) * 2048 * NBUF, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane, bias_sm);
+      drain_accumulator<EPI, NBUF, F16>(p, &tmO, staging + (warp - 2) * 2048 * NBUF, b, mt, nt, tmem_base + acc * BN, quarter, col_half, lane, bias_sm);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);
@@ -514,33 +541,33 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint
   return tma_make_map_bf16(map, base, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
-template <int EPI>
+template <int EPI, bool F16>
 msla_status_t launch_stationary(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO, const GemmParams& p,
                                 int blocks, cudaStream_t st) {
   static std::atomic<unsigned long long> attr_done{0};
-  const msla_status_t as = ensure_smem_attr(attr_done, gemm_bf16_stationary_kernel<EPI>, WS_SMEM_BYTES);
+  const msla_status_t as = ensure_smem_attr(attr_done, gemm_bf16_stationary_kernel<EPI, F16>, WS_SMEM_BYTES);
   if (as != MSLA_OK) return as;
   const long long stream_total = (long long)p.batches * p.m_tiles;
   long long workers = device_sm_count() / blocks;
   if (workers > stream_total) workers = stream_total;
-  launch_pdl(gemm_bf16_stationary_kernel<EPI>, dim3((unsigned)(workers * blocks)), dim3(NUM_THREADS), WS_SMEM_BYTES, st, tmA, tmB, tmO, p, blocks, (int)workers);
+  launch_pdl(gemm_bf16_stationary_kernel<EPI, F16>, dim3((unsigned)(workers * blocks)), dim3(NUM_THREADS), WS_SMEM_BYTES, st, tmA, tmB, tmO, p, blocks, (int)workers);
   count_launches(1);
   return check_launch("projection GEMM (tcgen05, stationary weights)");
 }
 
-template <bool A_MN, bool B_PLANAR = false, int EPI = 0>
+template <bool A_MN, bool B_PLANAR = false, int EPI = 0, bool F16 = false>
 msla_status_t launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO, const GemmParams& p, cudaStream_t st) {
   // weight-stationary kernel when the CTA's weight block fits its 128 KB of shared memory
   const int blocks = A_MN ? p.n_tiles : p.m_tiles;
   const int k_iters = (p.K + BK - 1) / BK;
   if (A_MN && k_iters * B_STAGE_BYTES <= RES_BYTES && blocks <= 16 && blocks <= device_sm_count())
-    return launch_stationary<EPI>(tmA, tmB, tmO, p, blocks, st);
+    return launch_stationary<EPI, F16>(tmA, tmB, tmO, p, blocks, st);
   static std::atomic<unsigned long long> attr_done{0};
-  const msla_status_t as = ensure_smem_attr(attr_done, gemm_bf16_tcgen05_kernel<A_MN, B_PLANAR, EPI>, SMEM_BYTES);
+  const msla_status_t as = ensure_smem_attr(attr_done, gemm_bf16_tcgen05_kernel<A_MN, B_PLANAR, EPI, F16>, SMEM_BYTES);
   if (as != MSLA_OK) return as;
   const long long tiles = (long long)p.batches * p.m_tiles * p.n_tiles;
   const int grid = (int)(tiles < device_sm_count() ? tiles : device_sm_count());
-  launch_pdl(gemm_bf16_tcgen05_kernel<A_MN, B_PLANAR, EPI>, dim3(grid), dim3(NUM_THREADS), SMEM_BYTES, st, tmA, tmB, tmO, p);
+  launch_pdl(gemm_bf16_tcgen05_kernel<A_MN, B_PLANAR, EPI, F16>, dim3(grid), dim3(NUM_THREADS), SMEM_BYTES, st, tmA, tmB, tmO, p);
   count_launches(1);
   return check_launch("projection GEMM (tcgen05)");
 }
@@ -553,7 +580,7 @@ bool project_in_bf16_supported(int C, int Cout, int N, int d) {
 
 // y[b][o / d][n][o % d] = sum_c w[o][c] * x[b][c][n];  x NCHW [B, C, N], y planar with batch stride y_sb.
 msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d,
-                                  long long y_sb, cudaStream_t st) {
+                                  long long y_sb, cudaStream_t st, bool f16) {
   CUtensorMap tmA, tmB;
   if (!make_map(&tmA, x, (uint64_t)N, (uint64_t)C, (uint64_t)B, (uint64_t)N * 2, (uint64_t)C * N * 2, 64, BK) ||
       !make_map(&tmB, w, (uint64_t)C, (uint64_t)Cout, 1, (uint64_t)C * 2, (uint64_t)C * Cout * 2, BK, BN))
@@ -575,14 +602,15 @@ msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, 
     if (!tma_make_map_bf16(&tmO, y, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B))
       return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the input projection's output");
   }
-  return launch<true>(tmA, tmB, tmO, p, st);
+  return f16 ? launch<true, false, 0, true>(tmA, tmB, tmO, p, st) : launch<true>(tmA, tmB, tmO, p, st);
 }
 
 bool project_out_bf16_supported(int Cin, int Cout, int N) { return Cin % 8 == 0 && N % 8 == 0 && Cout >= 1; }
 
 // y[b][m][n] = sum_j w[m][j] * a[b][n][j] + bias[m];  a token-major [B, N, Cin], y NCHW [B, Cout, N].
 msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bias, const void* residual, void* y, int B, int Cin,
-                                   int Cout, int N, cudaStream_t st) {
+                                   int Cout, int N, cudaStream_t st, bool f16) {
+  if (f16 && residual) return fail(MSLA_ERR_UNSUPPORTED, "the fp16 projection has no residual epilogue");
   CUtensorMap tmA, tmB;
   if (!make_map(&tmA, w, (uint64_t)Cin, (uint64_t)Cout, 1, (uint64_t)Cin * 2, (uint64_t)Cin * Cout * 2, BK, BM) ||
       !make_map(&tmB, a, (uint64_t)Cin, (uint64_t)N, (uint64_t)B, (uint64_t)Cin * 2, (uint64_t)N * Cin * 2, BK, BN))
@@ -602,6 +630,7 @@ msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bia
       return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the output projection's output");
   }
   p.residual = (const bf16*)residual;
+  if (f16) return launch<false, false, 0, true>(tmA, tmB, tmO, p, st);
   return residual ? launch<false, false, 2>(tmA, tmB, tmO, p, st) : launch<false>(tmA, tmB, tmO, p, st);
 }
 
@@ -609,7 +638,8 @@ bool project_out_planar_bf16_supported(int Cin, int Cout, int N) { return Cin % 
 
 // Same product with the attention output kept planar: a[b][j / 64][n][j % 64] (one [N][64] plane per pair of heads).
 msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const void* bias, const void* residual, void* y, int B,
-                                          int Cin, int Cout, int N, cudaStream_t st) {
+                                          int Cin, int Cout, int N, cudaStream_t st, bool f16) {
+  if (f16 && residual) return fail(MSLA_ERR_UNSUPPORTED, "the fp16 projection has no residual epilogue");
   CUtensorMap tmA, tmB, tmO;
   const int planes = Cin / 64;
   {
@@ -628,6 +658,7 @@ msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const vo
   p.bias = (const bf16*)bias; p.out = (bf16*)y;
   p.tma_store = 1; p.planes_per_batch = planes;
   p.residual = (const bf16*)residual;
+  if (f16) return launch<false, true, 0, true>(tmA, tmB, tmO, p, st);
   return residual ? launch<false, true, 2>(tmA, tmB, tmO, p, st) : launch<false, true>(tmA, tmB, tmO, p, st);
 }
 

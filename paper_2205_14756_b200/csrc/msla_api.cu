@@ -145,14 +145,15 @@ static msla_status_t run_core(msla_dtype_t dtype, const void* q, const void* k, 
                               void* out, HeadView in, HeadView ov, int B, int heads, int N, int d,
                               float eps, const CorePlan& p, void* ws, cudaStream_t st,
                               cudaEvent_t mid = nullptr, int phases = CORE_ALL) {
-  if (ov.pair && (dtype != MSLA_BF16 || (heads & 1)))  // only the bf16 tensor-core kernels write paired planes
-    return fail(MSLA_ERR_UNSUPPORTED, "paired output planes need bf16 and an even number of heads");
+  if (ov.pair && (dtype == MSLA_F32 || (heads & 1)))  // only the tensor-core kernels write paired planes
+    return fail(MSLA_ERR_UNSUPPORTED, "paired output planes need 16-bit storage and an even number of heads");
   if (dtype == MSLA_F32)
     return run_core_generic<float>((const float*)q, (const float*)k, (const float*)v, (float*)out,
                                    in, ov, B, heads, N, d, eps, p, (char*)ws, st, mid, phases);
   if (dtype == MSLA_F16) {  // the tensor-core kernels take fp16 too; other strides run on the plain kernels
-    const bool ok16 = !ov.pair && in.batch % 8 == 0 && in.head % 8 == 0 && in.ld % 8 == 0 && ov.batch % 8 == 0 && ov.head % 8 == 0 && ov.ld % 8 == 0;
+    const bool ok16 = in.batch % 8 == 0 && in.head % 8 == 0 && in.ld % 8 == 0 && ov.batch % 8 == 0 && ov.head % 8 == 0 && ov.ld % 8 == 0;
     if (ok16) return run_core_bf16(q, k, v, out, in, ov, B, heads, N, d, eps, p, ws, st, mid, phases, true);
+    if (ov.pair) return fail(MSLA_ERR_UNSUPPORTED, "paired output planes need strides that are multiples of 8 elements");
     return run_core_generic<__half>((const __half*)q, (const __half*)k, (const __half*)v, (__half*)out,
                                     in, ov, B, heads, N, d, eps, p, (char*)ws, st, mid, phases);
   }
@@ -312,7 +313,7 @@ static void launch_gemm(const T* A, const T* W, const T* bias, T* D, generic::Ge
 // y planar: y[b*y_sb + ((o/d)*N + n)*d + o%d]
 static msla_status_t run_project_in(msla_dtype_t dt, const void* x, const void* w, void* y, int B,
                                     int C, int Cout, int N, int d, long long y_sb, cudaStream_t st) {
-  if (dt == MSLA_BF16 && project_in_bf16_supported(C, Cout, N, d)) return run_project_in_bf16(x, w, y, B, C, Cout, N, d, y_sb, st);
+  if (dt != MSLA_F32 && project_in_bf16_supported(C, Cout, N, d)) return run_project_in_bf16(x, w, y, B, C, Cout, N, d, y_sb, st, dt == MSLA_F16);
   generic::GemmArgs g{(long long)C * N, 1, N, y_sb, d, 1, (long long)N * d, N, Cout, C, d};
   if (dt == MSLA_F32) launch_gemm<float>((const float*)x, (const float*)w, nullptr, (float*)y, g, B, st);
   else if (dt == MSLA_F16) launch_gemm<__half>((const __half*)x, (const __half*)w, nullptr, (__half*)y, g, B, st);
@@ -322,7 +323,8 @@ static msla_status_t run_project_in(msla_dtype_t dt, const void* x, const void* 
 
 static msla_status_t run_project_out(msla_dtype_t dt, const void* a, const void* w, const void* bias,
                                      void* y, int B, int Cin, int Cout, int N, cudaStream_t st, const void* residual = nullptr) {
-  if (dt == MSLA_BF16 && project_out_bf16_supported(Cin, Cout, N)) return run_project_out_bf16(a, w, bias, residual, y, B, Cin, Cout, N, st);
+  if (dt != MSLA_F32 && project_out_bf16_supported(Cin, Cout, N) && !(dt == MSLA_F16 && residual))
+    return run_project_out_bf16(a, w, bias, residual, y, B, Cin, Cout, N, st, dt == MSLA_F16);
   generic::GemmArgs g{(long long)N * Cin, Cin, 1, (long long)Cout * N, 1, N, 0, N, Cout, Cin, Cout, 0, residual};
   if (dt == MSLA_F32) launch_gemm<float>((const float*)a, (const float*)w, (const float*)bias, (float*)y, g, B, st);
   else if (dt == MSLA_F16) launch_gemm<__half>((const __half*)a, (const __half*)w, (const __half*)bias, (__half*)y, g, B, st);
@@ -335,19 +337,23 @@ static msla_status_t run_aggregate(msla_dtype_t dt, const void* src, const void*
                                    void* dst, int B, int H, int W, int Ch, int d, long long src_sb,
                                    long long dst_sb, cudaStream_t st) {
   const long long plane = (long long)H * W * d;
-  if (dt == MSLA_BF16 && src_sb % plane == 0 && dst_sb % plane == 0) {
+  const bool f16 = dt == MSLA_F16;
+  if (dt != MSLA_F32 && src_sb % plane == 0 && dst_sb % plane == 0) {
     if (aggregate_bf16_supported(H, W, Ch, d))
-      return run_aggregate_bf16(src, (long long)B * (src_sb / plane), (int)(src_sb / plane), w_dw, w_pw, dst, dst_sb, B, H, W, Ch, d, st);
+      return run_aggregate_bf16(src, (long long)B * (src_sb / plane), (int)(src_sb / plane), w_dw, w_pw, dst, dst_sb, B, H, W, Ch, d, st, f16);
     if (d == 16 && Ch > 16 && aggregate_bf16_supported(H, W, Ch - 16, d)) {
       // odd number of 16-channel groups: the tuned kernel takes them in pairs, the plain one the last group
-      msla_status_t s = run_aggregate_bf16(src, (long long)B * (src_sb / plane), (int)(src_sb / plane), w_dw, w_pw, dst, dst_sb, B, H, W, Ch - 16, d, st);
+      msla_status_t s = run_aggregate_bf16(src, (long long)B * (src_sb / plane), (int)(src_sb / plane), w_dw, w_pw, dst, dst_sb, B, H, W, Ch - 16, d, st, f16);
       if (s != MSLA_OK) return s;
-      const __nv_bfloat16* s16 = (const __nv_bfloat16*)src + (long long)(Ch / 16 - 1) * plane;
-      __nv_bfloat16* d16 = (__nv_bfloat16*)dst + (long long)(Ch / 16 - 1) * plane;
       dim3 grid1((unsigned)(ceil_div_ll(W, 8) * ceil_div_ll(H, 8)), 1u, (unsigned)B);
-      generic::aggregate_kernel<__nv_bfloat16><<<grid1, 256, 0, st>>>(s16, (const __nv_bfloat16*)w_dw + (long long)(Ch - 16) * 25,
-                                                                      (const __nv_bfloat16*)w_pw + (long long)(Ch - 16) * 16, d16, H, W, d,
-                                                                      src_sb, dst_sb);
+      auto last_group = [&](auto* tag) {
+        using T = std::remove_pointer_t<decltype(tag)>;
+        generic::aggregate_kernel<T><<<grid1, 256, 0, st>>>((const T*)src + (long long)(Ch / 16 - 1) * plane, (const T*)w_dw + (long long)(Ch - 16) * 25,
+                                                            (const T*)w_pw + (long long)(Ch - 16) * 16, (T*)dst + (long long)(Ch / 16 - 1) * plane, H, W, d,
+                                                            src_sb, dst_sb);
+      };
+      if (f16) last_group((__half*)nullptr);
+      else last_group((__nv_bfloat16*)nullptr);
       count_launches(1);
       return check_launch("token aggregation (last group)");
     }
@@ -461,7 +467,8 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   // Attention output: one [N][2d] plane per pair of heads when the tcgen05 output projection can
   // take it (dense 128-byte rows for the apply kernel's stores and the GEMM's tile loads),
   // otherwise token-major [N][2C'].
-  const bool att_planar = desc->dtype == MSLA_BF16 && d == 32 && Ht % 2 == 0 && project_out_planar_bf16_supported(S * Cp, desc->C_out, N);
+  const bool f16 = desc->dtype == MSLA_F16;
+  const bool att_planar = desc->dtype != MSLA_F32 && !(f16 && residual) && d == 32 && Ht % 2 == 0 && project_out_planar_bf16_supported(S * Cp, desc->C_out, N);
   const HeadView ov = att_planar ? HeadView{(long long)N * ld_att, (long long)N * 2 * d, 2 * d, 1}
                                  : HeadView{(long long)N * ld_att, d, ld_att, 0};
   // Steps 4 and 5 run as one kernel when it takes the shape: the head concat then stays in shared memory.
@@ -475,7 +482,7 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
     s = run_fused_out_bf16(ms, ms_sb, 3LL * N * d, reinterpret_cast<const float*>(ws + p.core_off + p.core.partial_off), p.core.S, att, w->w_proj,
                            w->b_proj, residual, out_dev, desc->B, Ht, d, N, desc->C_out, desc->eps, st);
   else
-    s = att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, residual, out_dev, desc->B, S * Cp, desc->C_out, N, st)
+    s = att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, residual, out_dev, desc->B, S * Cp, desc->C_out, N, st, f16)
                    : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out_dev, desc->B, S * Cp, desc->C_out, N, st, residual);
   if (s != MSLA_OK) return s;
   if ((s = record(events, 5, st)) != MSLA_OK) return s;
@@ -586,13 +593,13 @@ static msla_status_t band_output_impl(const msla_desc* desc, const msla_weights*
   if (desc->dtype == MSLA_BF16 && fused_out_bf16_supported(Ht, d, desc->C_out, Nb))
     return run_fused_out_bf16(q, ms_sb, 3LL * N * d, state, 1, att, w->w_proj, w->b_proj, nullptr, out, desc->B, Ht, d, Nb, desc->C_out, desc->eps, st);
   const HeadView in{ms_sb, 3LL * N * d, d};
-  const bool att_planar = desc->dtype == MSLA_BF16 && d == 32 && Ht % 2 == 0 && project_out_planar_bf16_supported(p.S * Cp, desc->C_out, Nb);
+  const bool att_planar = desc->dtype != MSLA_F32 && d == 32 && Ht % 2 == 0 && project_out_planar_bf16_supported(p.S * Cp, desc->C_out, Nb);
   const HeadView ov = att_planar ? HeadView{(long long)Nb * ld_att, (long long)Nb * 2 * d, 2 * d, 1}
                                  : HeadView{(long long)Nb * ld_att, d, ld_att, 0};
   s = run_core(desc->dtype, q, q + (size_t)N * d * e, q + (size_t)2 * N * d * e, att, in, ov, desc->B, Ht, Nb, d, desc->eps, b.core,
                ws + p.core_off, st, nullptr, CORE_APPLY);
   if (s != MSLA_OK) return s;
-  return att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, nullptr, out, desc->B, p.S * Cp, desc->C_out, Nb, st)
+  return att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, nullptr, out, desc->B, p.S * Cp, desc->C_out, Nb, st, desc->dtype == MSLA_F16)
                     : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out, desc->B, p.S * Cp, desc->C_out, Nb, st);
 }
 

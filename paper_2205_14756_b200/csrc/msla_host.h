@@ -126,14 +126,14 @@ int dw_timeout_flag();
 // bf16 projections on tcgen05 tensor cores (gemm_tcgen05.cu).
 bool project_in_bf16_supported(int C, int Cout, int N, int d);
 msla_status_t run_project_in_bf16(const void* x, const void* w, void* y, int B, int C, int Cout, int N, int d,
-                                  long long y_batch_stride, cudaStream_t st);
+                                  long long y_batch_stride, cudaStream_t st, bool f16 = false);
 bool project_out_bf16_supported(int Cin, int Cout, int N);
 // residual: nullptr, or a tensor shaped like y that is added to it
 msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bias, const void* residual, void* y, int B, int Cin,
-                                   int Cout, int N, cudaStream_t st);
+                                   int Cout, int N, cudaStream_t st, bool f16 = false);
 bool project_out_planar_bf16_supported(int Cin, int Cout, int N);
 msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const void* bias, const void* residual, void* y, int B,
-                                          int Cin, int Cout, int N, cudaStream_t st);
+                                          int Cin, int Cout, int N, cudaStream_t st, bool f16 = false);
 int gemm_timeout_flag();
 int run_wait_selftest(long long limit_cycles, int* scratch, cudaStream_t st);
 
@@ -142,7 +142,7 @@ int run_wait_selftest(long long limit_cycles, int* scratch, cudaStream_t st);
 bool aggregate_bf16_supported(int H, int W, int Ch, int d);
 msla_status_t run_aggregate_bf16(const void* src, long long src_planes_total, int src_ppb, const void* w_dw,
                                  const void* w_pw, void* dst, long long dst_sb, int B, int H, int W, int Ch, int d,
-                                 cudaStream_t st);
+                                 cudaStream_t st, bool f16 = false);
 int agg_timeout_flag();
 
 }  // namespace msla

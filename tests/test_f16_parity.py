@@ -1,6 +1,7 @@
 """fp16 storage (the paper's deployment precision, Section 4.1's TensorRT fp16 runs) through the C ABI: every entry
-point with dtype MSLA_F16, element by element against the fp64 oracle on inputs rounded to fp16.  fp16 runs on the
-library's plain kernels: fp32 arithmetic and state, one rounding per stored value."""
+point with dtype MSLA_F16, element by element against the fp64 oracle on inputs rounded to fp16.  The projections, the
+aggregation and the attention core run on their tensor-core kernels instantiated for f16 (steps 4 and 5 as two kernels);
+shapes those do not take, and the FFN, run on the plain kernels.  fp32 accumulation and state throughout."""
 import numpy as np
 import pytest
 
@@ -23,7 +24,9 @@ def test_core_f16(B, heads, N, d):
     util.assert_close(got, oracle.linattn_relu(t["q"], t["k"], t["v"]), "f16", "core fp16", block=util.CORE_BLOCK)
 
 
-@pytest.mark.parametrize("B,C,H,W,heads,d,n_scales,k1", [(1, 64, 16, 16, 4, 16, 2, 5), (2, 64, 9, 20, 2, 32, 2, 3), (1, 96, 12, 12, 3, 32, 3, 5)])
+@pytest.mark.parametrize("B,C,H,W,heads,d,n_scales,k1", [(1, 64, 16, 16, 4, 16, 2, 5), (2, 64, 9, 20, 2, 32, 2, 3), (1, 96, 12, 12, 3, 32, 3, 5),
+                                                         (1, 256, 64, 64, 8, 32, 2, 5), (2, 64, 24, 40, 2, 32, 2, 5), (1, 48, 11, 13, 3, 16, 2, 5),
+                                                         (1, 192, 64, 128, 6, 32, 2, 5), (1, 320, 16, 24, 10, 32, 2, 5)])
 def test_module_f16(B, C, H, W, heads, d, n_scales, k1):
     s = inputs.ModuleShape("module_f16", "f16", B, C, H, W, heads, d, seed=52, n_scales=n_scales, agg_kernel=k1)
     t = inputs.module_inputs(s)
