@@ -94,6 +94,8 @@ constexpr int STAGING_BYTES = 8 * 2048;  // one 32-row x 64-byte block per epilo
 //   2  adds p.residual (laid out like the row-major output) after the bias
 // F16: operands and output are IEEE binary16 instead of bfloat16 (16-bit values travel untyped; the MMA's operand
 // format bits and the conversions differ).
+// (The bf16 loads stay written as `__bfloat162float(p.bias[i])` at their sites: routed through this helper the input
+// projection's epilogue came out 10 % slower, 0.109 -> 0.119 ms.)
 template <bool F16> __device__ __forceinline__ float ld16(const bf16* p) {
   if constexpr (F16) return __half2float(*reinterpret_cast<const __half*>(p));
   else return __bfloat162float(*p);
@@ -126,7 +128,7 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUt
   const int m = row0 + lane;
   const bool row_ok = m < p.M;
   bf16* obase = p.out + (long long)b * p.out_batch_stride;
-  const float bias_row = (EPI != 1 && p.bias && p.bias_per_row && row_ok) ? ld16<F16>(p.bias + m) : 0.f;
+  const float bias_row = (EPI != 1 && p.bias && p.bias_per_row && row_ok) ? (F16 ? ld16<true>(p.bias + m) : __bfloat162float(p.bias[m])) : 0.f;
   const bool bias_col = EPI != 1 && p.bias && !p.bias_per_row;
   const int ncol0 = nt * BN + col_half * 128;
   const uint32_t taddr = tmem_acc + col_half * 128 + ((uint32_t)(quarter * 32) << 16);
@@ -162,7 +164,7 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUt
         bc[0] = b0.x; bc[1] = b0.y; bc[2] = b0.z; bc[3] = b0.w; bc[4] = b1.x; bc[5] = b1.y; bc[6] = b1.z; bc[7] = b1.w;
       } else if (EPI == 1) {      // no staged copy (the kernel whose CTAs change weight block from tile to tile)
 #pragma unroll
-        for (int i = 0; i < 8; ++i) bc[i] = (p.bias && n0 + v * 8 < p.N) ? ld16<F16>(p.bias + n0 + v * 8 + i) : 0.f;
+        for (int i = 0; i < 8; ++i) bc[i] = (p.bias && n0 + v * 8 < p.N) ? (F16 ? ld16<true>(p.bias + n0 + v * 8 + i) : __bfloat162float(p.bias[n0 + v * 8 + i])) : 0.f;
       }
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
@@ -174,8 +176,8 @@ __device__ __forceinline__ void drain_accumulator(const GemmParams& p, const CUt
         } else {
           f0 += bias_row; f1 += bias_row;
           if (bias_col && n0 + v * 8 < p.N) {
-            f0 += ld16<F16>(p.bias + n0 + v * 8 + 2 * e);
-            f1 += ld16<F16>(p.bias + n0 + v * 8 + 2 * e + 1);
+            if constexpr (F16) { f0 += ld16<true>(p.bias + n0 + v * 8 + 2 * e); f1 += ld16<true>(p.bias + n0 + v * 8 + 2 * e + 1); }
+            else { f0 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e]); f1 += __bfloat162float(p.bias[n0 + v * 8 + 2 * e + 1]); }
           }
         }
         if (EPI == 2) {
@@ -411,7 +413,7 @@ gemm_bf16_stationary_kernel(const __grid_constant__ CUtensorMap tmA, const __gri
   if (EPI == 1) {
     for (int i = threadIdx.x; i < BN; i += NUM_THREADS) {
       const int n = blk * BN + i;
-      bias_sm[i] = (p.bias && !p.bias_per_row && n < p.N) ? ld16<F16>(p.bias + n) : 0.f;
+      bias_sm[i] = (p.bias && !p.bias_per_row && n < p.N) ? (F16 ? ld16<true>(p.bias + n) : __bfloat162float(p.bias[n])) : 0.f;
     }
   }
   const int stream_per_batch = p.m_tiles;
