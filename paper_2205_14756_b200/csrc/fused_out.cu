@@ -49,13 +49,15 @@ constexpr int OKS = 64;                  // k-extent of one resident slice of M 
 constexpr int O_A_SLICE = OM * OKS * 2;  // 16 KB: 128 rows of M x 64 k
 constexpr int O_MAX_KS = 8;              // K = 2C' <= 512
 constexpr int O_SLICE_MAX = OT * 32 * 2; // 8 KB: 128 tokens x 32 channels (d = 16: half of it is used)
-constexpr int O_STAGES = 8;
-constexpr int O_XWARPS = 8;              // transform warps: two groups of four, alternating slices
+constexpr int O_MIN_STAGES = 4, O_MAX_STAGES = 16;  // query ring: as many slots as shared memory holds (the host decides)
+constexpr int O_XWARPS = 12;             // transform warps: three groups of four, each taking every third slice
 constexpr int O_THREADS = 32 * (2 + O_XWARPS + 4);
 constexpr int O_STAGING_WARP = 32 * 128;
 constexpr int O_STAGING = 4 * O_STAGING_WARP;
 constexpr int O_BAR_BYTES = 512;
-constexpr int O_SMEM_MAX = O_MAX_KS * O_A_SLICE + O_STAGES * O_SLICE_MAX + O_STAGING + O_BAR_BYTES + 1024;
+constexpr int O_SMEM_FIXED = O_STAGING + O_BAR_BYTES + 1024;  // besides the rows of M, the ring and the residual blocks
+constexpr int O_SMEM_LIMIT = 226 * 1024;                     // dynamic shared memory of a CTA (1 KB of the 227 left to static data)
+static_assert(24 * O_MAX_STAGES + 16 + 16 + 8 + 8 + 8 + 4 * 8 <= O_BAR_BYTES, "barrier block");
 
 __device__ int g_fused_timeout_flag = 0;
 
@@ -66,6 +68,7 @@ struct OutParams {
   int B, N, Cout, Ht, d;
   int kslices;       // 64-wide k-slices of M: ceil(Ht * d / 64)
   int ot;            // tokens per CTA and tile: 128 or 64
+  int stages;        // slots of the query ring
   int tiles_per_image, num_tiles;  // tiles of 2 * ot tokens
   float eps;
 };
@@ -222,18 +225,18 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
   constexpr int SLICE = OT * D * 2;                                    // ring slot: one head's queries of this CTA's (up to) 128 tokens
   constexpr int ROWB = D * 2;                                          // bytes per token row = the swizzle span
   const uint32_t ring = a_base + (uint32_t)p.kslices * O_A_SLICE;
-  const uint32_t staging = ring + O_STAGES * SLICE;
+  const uint32_t staging = ring + (uint32_t)p.stages * SLICE;
   const uint32_t resbuf = staging + O_STAGING;           // RES: one 32-channel x 64-token block of the residual per epilogue warp
   const uint32_t bars = resbuf + (RES ? O_STAGING : 0);
   const uint32_t full_bar = bars;                        // [stage] TMA landed (own CTA)
-  const uint32_t empty_bar = bars + 8 * O_STAGES;        // [stage] MMAs have read the slice (commit, both CTAs)
-  const uint32_t ready_bar = bars + 16 * O_STAGES;       // [stage] both CTAs' slices transformed (leader only)
-  const uint32_t tfull_bar = bars + 24 * O_STAGES;       // [acc] accumulator complete (commit, both CTAs)
+  const uint32_t empty_bar = bars + 8 * O_MAX_STAGES;        // [stage] MMAs have read the slice (commit, both CTAs)
+  const uint32_t ready_bar = bars + 16 * O_MAX_STAGES;       // [stage] both CTAs' slices transformed (leader only)
+  const uint32_t tfull_bar = bars + 24 * O_MAX_STAGES;       // [acc] accumulator complete (commit, both CTAs)
   const uint32_t tempty_bar = tfull_bar + 16;            // [acc] both CTAs' epilogues have drained it (leader only)
   const uint32_t res_bar = tempty_bar + 16;              // rows of M landed (own CTA)
   const uint32_t peer_res_bar = res_bar + 8;             // the peer's rows of M landed (leader only)
   const uint32_t tmem_slot = peer_res_bar + 8;
-  const uint32_t resid_bar = bars + 256;                 // [epilogue warp] RES: the warp's residual block landed
+  const uint32_t resid_bar = tmem_slot + 8;              // [epilogue warp] RES: the warp's residual block landed
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_sh;
 
@@ -247,10 +250,10 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
-    for (int s = 0; s < O_STAGES; ++s) {
+    for (int s = 0; s < p.stages; ++s) {
       mbar_init(full_bar + 8 * s, 1);
       mbar_init(empty_bar + 8 * s, 1);
-      mbar_init(ready_bar + 8 * s, 2 * (O_XWARPS / 2));
+      mbar_init(ready_bar + 8 * s, 2 * 4);  // the four warps of one transform group, in both CTAs
     }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar + 8 * a, 1); mbar_init(tempty_bar + 8 * a, 2 * 4); }
     mbar_init(res_bar, 1);
@@ -280,7 +283,7 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tmM) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tmQ) : "memory");
-      uint32_t it = 0, local = 0;
+      uint32_t local = 0, s = 0, ph = 0;  // ring slot and the parity of its current use
       int cur_b = -1;
       bool ok = true;
       for (int tile = tile_first; ok && tile < tile_end; ++tile, ++local) {
@@ -297,12 +300,12 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
             tma_load_3d(a_base + ks * O_A_SLICE, &tmM, res_bar, ks * OKS, (int)rank * OM, b);
         }
         const int n0 = nt * (2 * p.ot) + (int)rank * p.ot;
-        for (int h = 0; ok && h < p.Ht; ++h, ++it) {
-          const uint32_t s = it % O_STAGES, ph = (it / O_STAGES) & 1;
+        for (int h = 0; ok && h < p.Ht; ++h) {
           ok = mbar_wait_cluster(empty_bar + 8 * s, ph ^ 1, &abort_flag);
           if (!ok) break;
           mbar_expect_tx(full_bar + 8 * s, (uint32_t)(p.ot * ROWB));
           tma_load_4d(ring + s * SLICE, &tmQ, full_bar + 8 * s, 0, n0, h, b);  // rows past the last token are filled with zeros
+          if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
         }
       }
     }
@@ -312,7 +315,11 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
       // instruction descriptor: D = f32, A = B = bf16, both K-major, N = 256, M = 256 (pair)
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * p.ot) >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
       const uint32_t peer_res_remote = map_to_cta(peer_res_bar, 0);
-      uint32_t it = 0, local = 0, res_ph = 0;
+      uint32_t local = 0, res_ph = 0, s = 0, ph = 0;  // s, ph: ring slot and the parity of its current use
+      // Matrix descriptors: the high words are constants; the low words carry the start address in 16-byte units
+      // (A: the 128B-swizzled rows of M; B: the slice, K-major, the swizzle span being the token row).
+      const uint64_t a_hi = make_desc(0, 1, 1024 >> 4), b_hi = make_desc_kmajor(0, (8 * ROWB) >> 4, D == 32 ? 4ull : 6ull);
+      const uint32_t a_lo0 = (a_base & 0x3FFFFu) >> 4, b_lo0 = (ring & 0x3FFFFu) >> 4;
       int cur_b = -1;
       bool ok = true;
       for (int tile = tile_first; ok && tile < tile_end; ++tile, ++local) {
@@ -335,26 +342,28 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * 256;
-        for (int h = 0; ok && h < p.Ht; ++h, ++it) {
-          const uint32_t s = it % O_STAGES, ph = (it / O_STAGES) & 1;
+        uint32_t a_lo = a_lo0;  // walks the columns of M: 32 bytes per 16 columns, 64-column slices O_A_SLICE apart
+        int col = 0;
+        for (int h = 0; ok && h < p.Ht; ++h) {
           ok = mbar_wait_cluster(ready_bar + 8 * s, ph, &abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t sb = ring + s * SLICE;
+          const uint32_t b_lo = b_lo0 + s * (uint32_t)(SLICE >> 4);
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {
-            const int k0 = h * D + 16 * kk;  // column of M: 64-wide slices 16 KB apart, 32 bytes per 16 columns inside a slice
-            umma2_bf16(d_tmem, make_desc(a_base + (uint32_t)((k0 >> 6) * O_A_SLICE + (k0 & 63) * 2), 1, 1024 >> 4),
-                       make_desc_kmajor(sb + kk * 32, (8 * ROWB) >> 4, D == 32 ? 4ull : 6ull), idesc, (h > 0 || kk > 0) ? 1u : 0u);
+            umma2_bf16(d_tmem, a_hi | a_lo, b_hi | (b_lo + 2 * kk), idesc, (h > 0 || kk > 0) ? 1u : 0u);
+            col += 16;
+            a_lo += (col & 63) ? 2u : (uint32_t)((O_A_SLICE - 96) >> 4);
           }
           umma2_commit_both(empty_bar + 8 * s);  // both CTAs may refill the slice once these MMAs have read it
+          if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
         }
         if (ok) umma2_commit_both(tfull_bar + 8 * acc);
       }
     }
   } else if (warp < 2 + O_XWARPS) {
     // ------------------------------------------------------------ transform warps: q -> relu(q) / den, in place
-    // Group xg of four warps takes the slices with (slice counter & 1) == xg; its 128 lanes own one token
+    // Group xg of four warps takes every third slice, starting with slice xg; its 128 lanes own one token
     // row each (d channels: 64 or 32 bytes, 16-byte pieces XOR-swizzled with the row as the TMA unit
     // wrote them and as the MMA reads them; eight consecutive rows cover all banks once).
     constexpr int PCS = D / 8;     // 16-byte pieces per token row
@@ -363,12 +372,16 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     const uint32_t row = (uint32_t)(wig * 32 + lane);
     const uint32_t swz = D == 32 ? (row >> 1) & 3u : (row >> 2) & 1u;
     const uint32_t row_off = row * ROWB;
-    uint32_t it = 0;
+    uint32_t s = 0, ph = 0, turn = 0;  // ring slot, the parity of its current use, and the group whose slice it holds
+    auto next_slice = [&]() {
+      if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
+      if (++turn == O_XWARPS / 4) turn = 0;
+    };
     bool ok = true;
     for (int tile = tile_first; ok && tile < tile_end; ++tile) {
       const int b = tile / p.tiles_per_image;
-      for (int h = 0; ok && h < p.Ht; ++h, ++it) {
-        if ((int)(it & 1) != xg) continue;
+      for (int h = 0; ok && h < p.Ht; ++h, next_slice()) {
+        if ((int)turn != xg) continue;
         const bool has_row = (int)row < p.ot;  // with 64-token tiles only the first two warps of a group own rows
         // the head's key sums, fetched before the wait so that their latency hides behind it
         float kk[D];
@@ -378,7 +391,6 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
           const float4 v = __ldg(ksp + a4);
           kk[4 * a4] = v.x; kk[4 * a4 + 1] = v.y; kk[4 * a4 + 2] = v.z; kk[4 * a4 + 3] = v.w;
         }
-        const uint32_t s = it % O_STAGES, ph = (it / O_STAGES) & 1;
         ok = mbar_wait(full_bar + 8 * s, ph, &abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -567,13 +579,18 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   const long long tiles = (long long)B * p.tiles_per_image;
   if (tiles > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many token tiles");
   p.num_tiles = (int)tiles;
-  const int smem = p.kslices * O_A_SLICE + O_STAGES * (OT * d * 2) + O_STAGING + (residual ? O_STAGING : 0) + O_BAR_BYTES + 1024;
+  // the query ring takes what shared memory is left beside the rows of M (and the residual blocks)
+  const int smem_fixed = p.kslices * O_A_SLICE + O_SMEM_FIXED + (residual ? O_STAGING : 0), slot = OT * d * 2;
+  p.stages = (O_SMEM_LIMIT - smem_fixed) / slot;
+  if (p.stages > O_MAX_STAGES) p.stages = O_MAX_STAGES;
+  if (p.stages < O_MIN_STAGES) return fail(MSLA_ERR_UNSUPPORTED, "fused apply + projection: no room for the query ring (%d slots)", p.stages);
+  const int smem = smem_fixed + p.stages * slot;
   static std::atomic<unsigned long long> attr_done{0}, attr_done16{0}, attr_res{0}, attr_res16{0};
-  constexpr int smem_max = O_SMEM_MAX;
+  constexpr int smem_max = O_SMEM_LIMIT;
   msla_status_t s = ensure_smem_attr(attr_done, fused_out_kernel<32, false>, smem_max);
   if (s == MSLA_OK) s = ensure_smem_attr(attr_done16, fused_out_kernel<16, false>, smem_max);
-  if (s == MSLA_OK && residual) s = ensure_smem_attr(attr_res, fused_out_kernel<32, true>, smem_max + O_STAGING);
-  if (s == MSLA_OK && residual) s = ensure_smem_attr(attr_res16, fused_out_kernel<16, true>, smem_max + O_STAGING);
+  if (s == MSLA_OK && residual) s = ensure_smem_attr(attr_res, fused_out_kernel<32, true>, smem_max);
+  if (s == MSLA_OK && residual) s = ensure_smem_attr(attr_res16, fused_out_kernel<16, true>, smem_max);
   if (s != MSLA_OK) return s;
   long long pairs = sms / 2;
   if (pairs > tiles) pairs = tiles;
