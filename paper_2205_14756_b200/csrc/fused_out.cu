@@ -18,13 +18,16 @@
 //                     is reproducible bit for bit), writes ks and M (fp32 accumulate, bf16 out).
 // fused_out_kernel  : clusters of two CTAs, paired tensor-core MMAs (cta_group::2, M = 256).
 //   Each CTA keeps its 128 rows of M (<= 128 KB) in shared memory while the image lasts and
-//   owns 128 of the pair's 256 tokens per tile.  Per head (one slice of d query channels):
-//     warp 0       TMA: one box of 128 tokens x d channels of the head's planar [N][d] query
-//                  matrix (one contiguous 8 KB piece for d = 32; swizzle span = the row)
-//     warps 2-9    turn q into qt in place (normaliser on the fp32 pipes, one token per lane)
+//   owns 128 of the pair's 256 tokens per tile.  The unit handed from role to role is a pair of
+//   heads (two slices of d query channels in one ring slot, one set of barriers): the thread that
+//   issues the MMAs pays a wait and a commit per unit, and its serial chain is what bounds the kernel.
+//     warp 0       TMA: per head one box of 128 tokens x d channels of the head's planar [N][d]
+//                  query matrix (one contiguous 8 KB piece for d = 32; swizzle span = the row)
+//     warps 2-13   turn q into qt in place (normaliser on the fp32 pipes, one token per lane);
+//                  three groups of four warps, each taking every third slice
 //     warp 1       (leader CTA only) issues tcgen05.mma 256 x 256 x 16: A = M, B = qt, both
 //                  K-major, fp32 accumulators in both CTAs' tensor memory
-//     warps 10-13  drain the accumulators: TMEM -> bf16 (+ bias) -> swizzled staging -> TMA
+//     warps 14-17  drain the accumulators: TMEM -> bf16 (+ bias) -> swizzled staging -> TMA
 //                  stores of 32-channel x 64-token blocks into the NCHW output
 //                  (RES kernels: the same block of a residual tensor, fetched by TMA into a block of its own one
 //                  block ahead of its use, is added before the conversion: the residual connection around the module)
@@ -49,7 +52,7 @@ constexpr int OKS = 64;                  // k-extent of one resident slice of M 
 constexpr int O_A_SLICE = OM * OKS * 2;  // 16 KB: 128 rows of M x 64 k
 constexpr int O_MAX_KS = 8;              // K = 2C' <= 512
 constexpr int O_SLICE_MAX = OT * 32 * 2; // 8 KB: 128 tokens x 32 channels (d = 16: half of it is used)
-constexpr int O_MIN_STAGES = 4, O_MAX_STAGES = 16;  // query ring: as many slots as shared memory holds (the host decides)
+constexpr int O_MIN_STAGES = 2, O_MAX_STAGES = 16;  // query ring: as many slots (of two slices each) as shared memory holds (the host decides)
 constexpr int O_XWARPS = 12;             // transform warps: three groups of four, each taking every third slice
 constexpr int O_THREADS = 32 * (2 + O_XWARPS + 4);
 constexpr int O_STAGING_WARP = 32 * 128;
@@ -68,7 +71,7 @@ struct OutParams {
   int B, N, Cout, Ht, d;
   int kslices;       // 64-wide k-slices of M: ceil(Ht * d / 64)
   int ot;            // tokens per CTA and tile: 128 or 64
-  int stages;        // slots of the query ring
+  int stages;        // slots of the query ring (a slot holds the slices of two consecutive heads)
   int tiles_per_image, num_tiles;  // tiles of 2 * ot tokens
   float eps;
 };
@@ -222,13 +225,14 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024-byte alignment
   const uint32_t a_base = smem_base;                                  // resident rows of M: kslices x 16 KB
-  constexpr int SLICE = OT * D * 2;                                    // ring slot: one head's queries of this CTA's (up to) 128 tokens
+  constexpr int SLICE = OT * D * 2;                                    // one head's queries of this CTA's (up to) 128 tokens
+  constexpr int SLOT = 2 * SLICE;                                      // ring slot: two consecutive heads
   constexpr int ROWB = D * 2;                                          // bytes per token row = the swizzle span
   const uint32_t ring = a_base + (uint32_t)p.kslices * O_A_SLICE;
-  const uint32_t staging = ring + (uint32_t)p.stages * SLICE;
+  const uint32_t staging = ring + (uint32_t)p.stages * SLOT;
   const uint32_t resbuf = staging + O_STAGING;           // RES: one 32-channel x 64-token block of the residual per epilogue warp
   const uint32_t bars = resbuf + (RES ? O_STAGING : 0);
-  const uint32_t full_bar = bars;                        // [stage] TMA landed (own CTA)
+  const uint32_t full_bar = bars;                        // [stage] both heads' boxes landed (own CTA)
   const uint32_t empty_bar = bars + 8 * O_MAX_STAGES;        // [stage] MMAs have read the slice (commit, both CTAs)
   const uint32_t ready_bar = bars + 16 * O_MAX_STAGES;       // [stage] both CTAs' slices transformed (leader only)
   const uint32_t tfull_bar = bars + 24 * O_MAX_STAGES;       // [acc] accumulator complete (commit, both CTAs)
@@ -253,7 +257,7 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(full_bar + 8 * s, 1);
       mbar_init(empty_bar + 8 * s, 1);
-      mbar_init(ready_bar + 8 * s, 2 * 4);  // the four warps of one transform group, in both CTAs
+      mbar_init(ready_bar + 8 * s, 2 * 2 * 4);  // per head the four warps of one transform group, in both CTAs
     }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar + 8 * a, 1); mbar_init(tempty_bar + 8 * a, 2 * 4); }
     mbar_init(res_bar, 1);
@@ -300,11 +304,13 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
             tma_load_3d(a_base + ks * O_A_SLICE, &tmM, res_bar, ks * OKS, (int)rank * OM, b);
         }
         const int n0 = nt * (2 * p.ot) + (int)rank * p.ot;
-        for (int h = 0; ok && h < p.Ht; ++h) {
+        for (int h = 0; ok && h < p.Ht; h += 2) {
           ok = mbar_wait_cluster(empty_bar + 8 * s, ph ^ 1, &abort_flag);
           if (!ok) break;
-          mbar_expect_tx(full_bar + 8 * s, (uint32_t)(p.ot * ROWB));
-          tma_load_4d(ring + s * SLICE, &tmQ, full_bar + 8 * s, 0, n0, h, b);  // rows past the last token are filled with zeros
+          const bool two = h + 1 < p.Ht;  // an odd head count leaves the last slot half used
+          mbar_expect_tx(full_bar + 8 * s, (uint32_t)((two ? 2 : 1) * p.ot * ROWB));
+          tma_load_4d(ring + s * SLOT, &tmQ, full_bar + 8 * s, 0, n0, h, b);  // rows past the last token are filled with zeros
+          if (two) tma_load_4d(ring + s * SLOT + SLICE, &tmQ, full_bar + 8 * s, 0, n0, h + 1, b);
           if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
         }
       }
@@ -344,18 +350,22 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
         const uint32_t d_tmem = tmem_base + acc * 256;
         uint32_t a_lo = a_lo0;  // walks the columns of M: 32 bytes per 16 columns, 64-column slices O_A_SLICE apart
         int col = 0;
-        for (int h = 0; ok && h < p.Ht; ++h) {
+        for (int h = 0; ok && h < p.Ht; h += 2) {
           ok = mbar_wait_cluster(ready_bar + 8 * s, ph, &abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t b_lo = b_lo0 + s * (uint32_t)(SLICE >> 4);
+          const uint32_t b_lo = b_lo0 + s * (uint32_t)(SLOT >> 4);
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            umma2_bf16(d_tmem, a_hi | a_lo, b_hi | (b_lo + 2 * kk), idesc, (h > 0 || kk > 0) ? 1u : 0u);
-            col += 16;
-            a_lo += (col & 63) ? 2u : (uint32_t)((O_A_SLICE - 96) >> 4);
+          for (int j = 0; j < 2; ++j) {
+            if (h + j >= p.Ht) break;
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+              umma2_bf16(d_tmem, a_hi | a_lo, b_hi | (b_lo + (uint32_t)(j * (SLICE >> 4) + 2 * kk)), idesc, (h > 0 || j > 0 || kk > 0) ? 1u : 0u);
+              col += 16;
+              a_lo += (col & 63) ? 2u : (uint32_t)((O_A_SLICE - 96) >> 4);
+            }
           }
-          umma2_commit_both(empty_bar + 8 * s);  // both CTAs may refill the slice once these MMAs have read it
+          umma2_commit_both(empty_bar + 8 * s);  // both CTAs may refill the slot once these MMAs have read it
           if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
         }
         if (ok) umma2_commit_both(tfull_bar + 8 * acc);
@@ -372,31 +382,33 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     const uint32_t row = (uint32_t)(wig * 32 + lane);
     const uint32_t swz = D == 32 ? (row >> 1) & 3u : (row >> 2) & 1u;
     const uint32_t row_off = row * ROWB;
-    uint32_t s = 0, ph = 0, turn = 0;  // ring slot, the parity of its current use, and the group whose slice it holds
-    auto next_slice = [&]() {
-      if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
-      if (++turn == O_XWARPS / 4) turn = 0;
-    };
+    uint32_t s = 0, ph = 0, turn = 0;  // ring slot, the parity of its current use, and the group whose turn it is
+    const int h_end = (p.Ht + 1) & ~1;  // an odd head count: the empty half of the last slot still has to be signed off
     bool ok = true;
     for (int tile = tile_first; ok && tile < tile_end; ++tile) {
       const int b = tile / p.tiles_per_image;
-      for (int h = 0; ok && h < p.Ht; ++h, next_slice()) {
-        if ((int)turn != xg) continue;
-        const bool has_row = (int)row < p.ot;  // with 64-token tiles only the first two warps of a group own rows
+      for (int h = 0; ok && h < h_end; ++h) {
+        const uint32_t cs = s, cph = ph;  // this slice's slot; the counters move on to the next slice
+        const bool mine = (int)turn == xg;
+        if (h & 1) { if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; } }
+        if (++turn == O_XWARPS / 4) turn = 0;
+        if (!mine) continue;
+        // with 64-token tiles only the first two warps of a group own rows; past the last head there is nothing to do
+        const bool has_row = (int)row < p.ot && h < p.Ht;
         // the head's key sums, fetched before the wait so that their latency hides behind it
         float kk[D];
-        const float4* ksp = reinterpret_cast<const float4*>(p.ks + ((long long)b * p.Ht + h) * D);
+        const float4* ksp = reinterpret_cast<const float4*>(p.ks + ((long long)b * p.Ht + min(h, p.Ht - 1)) * D);
 #pragma unroll
         for (int a4 = 0; a4 < D / 4; ++a4) {
           const float4 v = __ldg(ksp + a4);
           kk[4 * a4] = v.x; kk[4 * a4 + 1] = v.y; kk[4 * a4 + 2] = v.z; kk[4 * a4 + 3] = v.w;
         }
-        ok = mbar_wait(full_bar + 8 * s, ph, &abort_flag);
+        ok = mbar_wait(full_bar + 8 * cs, cph, &abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
-        const uint32_t rbase = ring + s * SLICE + row_off;
+        const uint32_t rbase = ring + cs * SLOT + (uint32_t)(h & 1) * SLICE + row_off;
         if (!has_row) {  // warp-uniform
-          if (lane == 0) mbar_arrive_cluster(ready_remote + 8 * s);
+          if (lane == 0) mbar_arrive_cluster(ready_remote + 8 * cs);
           continue;
         }
         uint32_t q[D / 2];  // word w = channels 2w (low half), 2w+1 (high half)
@@ -420,7 +432,7 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
                        "r"(q[4 * c + 2]), "r"(q[4 * c + 3]) : "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the tensor cores read what was just written
         __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(ready_remote + 8 * s);
+        if (lane == 0) mbar_arrive_cluster(ready_remote + 8 * cs);
       }
     }
   } else {
@@ -580,7 +592,7 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   if (tiles > 0x7fffffffLL) return fail(MSLA_ERR_UNSUPPORTED, "too many token tiles");
   p.num_tiles = (int)tiles;
   // the query ring takes what shared memory is left beside the rows of M (and the residual blocks)
-  const int smem_fixed = p.kslices * O_A_SLICE + O_SMEM_FIXED + (residual ? O_STAGING : 0), slot = OT * d * 2;
+  const int smem_fixed = p.kslices * O_A_SLICE + O_SMEM_FIXED + (residual ? O_STAGING : 0), slot = 2 * OT * d * 2;
   p.stages = (O_SMEM_LIMIT - smem_fixed) / slot;
   if (p.stages > O_MAX_STAGES) p.stages = O_MAX_STAGES;
   if (p.stages < O_MIN_STAGES) return fail(MSLA_ERR_UNSUPPORTED, "fused apply + projection: no room for the query ring (%d slots)", p.stages);
