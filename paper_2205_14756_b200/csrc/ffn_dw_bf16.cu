@@ -57,6 +57,25 @@ __device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* m
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 
+// F16: the 16-bit storage type is IEEE binary16 instead of bfloat16 (values travel untyped; only the conversions differ).
+template <bool F16> __device__ __forceinline__ void unpack16(uint32_t w, float& lo, float& hi) {
+  if constexpr (F16) {
+    const __half2 h = *reinterpret_cast<const __half2*>(&w);
+    lo = __low2float(h); hi = __high2float(h);
+  } else {
+    lo = __uint_as_float(w << 16); hi = __uint_as_float(w & 0xffff0000u);
+  }
+}
+template <bool F16> __device__ __forceinline__ uint32_t pack16(float lo, float hi) {
+  if constexpr (F16) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+  } else {
+    return pack2(lo, hi);
+  }
+}
+
 struct DwParams {
   const bf16* w_dw;  // [Ch][3][3]
   const bf16* b_dw;  // [Ch] or nullptr
@@ -67,6 +86,7 @@ struct DwParams {
   long long num_tiles;
 };
 
+template <bool F16>
 __global__ void __launch_bounds__(DW_THREADS, 1)
 ffn_dw3x3_kernel(const __grid_constant__ CUtensorMap tmH, DwParams p) {
   extern __shared__ unsigned char smem_raw[];
@@ -126,23 +146,21 @@ ffn_dw3x3_kernel(const __grid_constant__ CUtensorMap tmH, DwParams p) {
       const int plane = z % p.planes;
       if (plane != plane_loaded) {  // the thread's 4 channels x 9 taps: 72 contiguous bytes of the weight tensor
         const uint2* wp = reinterpret_cast<const uint2*>(p.w_dw + (long long)(plane * 64 + ch) * 9);
-        uint32_t raw[18];
+        float flat[36];  // element e = channel e / 9, tap e % 9
 #pragma unroll
         for (int v = 0; v < 9; ++v) {
           const uint2 q = __ldg(wp + v);
-          raw[2 * v] = q.x; raw[2 * v + 1] = q.y;
+          unpack16<F16>(q.x, flat[4 * v], flat[4 * v + 1]);
+          unpack16<F16>(q.y, flat[4 * v + 2], flat[4 * v + 3]);
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i)
 #pragma unroll
-          for (int tp = 0; tp < 9; ++tp) {
-            const int e = i * 9 + tp;  // element e of the 36: upper or lower half of word e / 2
-            wt[tp][i] = __uint_as_float((e & 1) ? (raw[e >> 1] & 0xffff0000u) : (raw[e >> 1] << 16));
-          }
+          for (int tp = 0; tp < 9; ++tp) wt[tp][i] = flat[i * 9 + tp];
         if (p.b_dw) {
           const uint2 q = __ldg(reinterpret_cast<const uint2*>(p.b_dw + plane * 64 + ch));
-          bias[0] = __uint_as_float(q.x << 16); bias[1] = __uint_as_float(q.x & 0xffff0000u);
-          bias[2] = __uint_as_float(q.y << 16); bias[3] = __uint_as_float(q.y & 0xffff0000u);
+          unpack16<F16>(q.x, bias[0], bias[1]);
+          unpack16<F16>(q.y, bias[2], bias[3]);
         } else {
 #pragma unroll
           for (int i = 0; i < 4; ++i) bias[i] = 0.f;
@@ -163,8 +181,8 @@ ffn_dw3x3_kernel(const __grid_constant__ CUtensorMap tmH, DwParams p) {
         for (int dx = 0; dx < 3; ++dx) {
           uint2 v;
           asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(tile + r * DW_ROW_PITCH + pre[dx]));
-          in[dx][0] = __uint_as_float(v.x << 16); in[dx][1] = __uint_as_float(v.x & 0xffff0000u);
-          in[dx][2] = __uint_as_float(v.y << 16); in[dx][3] = __uint_as_float(v.y & 0xffff0000u);
+          unpack16<F16>(v.x, in[dx][0], in[dx][1]);
+          unpack16<F16>(v.y, in[dx][2], in[dx][3]);
         }
 #pragma unroll
         for (int dy = 0; dy < 3; ++dy) {
@@ -187,8 +205,8 @@ ffn_dw3x3_kernel(const __grid_constant__ CUtensorMap tmH, DwParams p) {
           float o4[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) o4[i] = a[i] * __saturatef(fmaf(a[i], p.act_a, p.act_b));
-          out.x = pack2(o4[0], o4[1]);
-          out.y = pack2(o4[2], o4[3]);
+          out.x = pack16<F16>(o4[0], o4[1]);
+          out.y = pack16<F16>(o4[2], o4[3]);
           *reinterpret_cast<uint2*>(gp + ((long long)(y0 + od) * p.W + x) * 64) = out;
         }
       }
@@ -202,9 +220,9 @@ ffn_dw3x3_kernel(const __grid_constant__ CUtensorMap tmH, DwParams p) {
 
 }  // namespace
 
-// h: [B][Ch / 32][H * W][32], g: [B][Ch / 64][H * W][64] bf16; w_dw [Ch][3][3]; b_dw [Ch] or nullptr.
+// h: [B][Ch / 32][H * W][32], g: [B][Ch / 64][H * W][64] bf16 (f16: binary16); w_dw [Ch][3][3]; b_dw [Ch] or nullptr.
 msla_status_t run_ffn_dw3x3_bf16(const void* h, const void* w_dw, const void* b_dw, void* g, int B, int Ch, int H, int W, int act,
-                                 cudaStream_t st) {
+                                 cudaStream_t st, bool f16) {
   const long long z = (long long)B * (Ch / 64);
   if (Ch % 64 != 0 || z > 0x7fffffffLL)
     return fail(MSLA_ERR_UNSUPPORTED, "FFN depthwise convolution: %d hidden channels, batch %d", Ch, B);
@@ -221,13 +239,14 @@ msla_status_t run_ffn_dw3x3_bf16(const void* h, const void* w_dw, const void* b_
   p.act_b = act == 2 ? 0.5f : (act == 1 ? 0.f : 1.f);
   p.tiles_x = (W + DW_PX - 1) / DW_PX; p.tiles_y = (H + DW_ROWS - 1) / DW_ROWS;
   p.num_tiles = z * p.tiles_x * p.tiles_y;
-  static std::atomic<unsigned long long> attr_done{0};
-  const msla_status_t as = ensure_smem_attr(attr_done, ffn_dw3x3_kernel, DW_SMEM);
+  static std::atomic<unsigned long long> attr_done{0}, attr_done16{0};
+  const msla_status_t as = f16 ? ensure_smem_attr(attr_done16, ffn_dw3x3_kernel<true>, DW_SMEM) : ensure_smem_attr(attr_done, ffn_dw3x3_kernel<false>, DW_SMEM);
   if (as != MSLA_OK) return as;
   const long long grid = p.num_tiles < device_sm_count() ? p.num_tiles : device_sm_count();
-  launch_pdl(ffn_dw3x3_kernel, dim3((unsigned)grid), dim3(DW_THREADS), DW_SMEM, st, tmH, p);
+  if (f16) launch_pdl(ffn_dw3x3_kernel<true>, dim3((unsigned)grid), dim3(DW_THREADS), DW_SMEM, st, tmH, p);
+  else launch_pdl(ffn_dw3x3_kernel<false>, dim3((unsigned)grid), dim3(DW_THREADS), DW_SMEM, st, tmH, p);
   count_launches(1);
-  return check_launch("FFN depthwise convolution (bf16)");
+  return check_launch(f16 ? "FFN depthwise convolution (fp16)" : "FFN depthwise convolution (bf16)");
 }
 
 int dw_timeout_flag() {

@@ -612,7 +612,6 @@ bool project_out_bf16_supported(int Cin, int Cout, int N) { return Cin % 8 == 0 
 // y[b][m][n] = sum_j w[m][j] * a[b][n][j] + bias[m];  a token-major [B, N, Cin], y NCHW [B, Cout, N].
 msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bias, const void* residual, void* y, int B, int Cin,
                                    int Cout, int N, cudaStream_t st, bool f16) {
-  if (f16 && residual) return fail(MSLA_ERR_UNSUPPORTED, "the fp16 projection has no residual epilogue");
   CUtensorMap tmA, tmB;
   if (!make_map(&tmA, w, (uint64_t)Cin, (uint64_t)Cout, 1, (uint64_t)Cin * 2, (uint64_t)Cin * Cout * 2, BK, BM) ||
       !make_map(&tmB, a, (uint64_t)Cin, (uint64_t)N, (uint64_t)B, (uint64_t)Cin * 2, (uint64_t)N * Cin * 2, BK, BN))
@@ -632,7 +631,7 @@ msla_status_t run_project_out_bf16(const void* a, const void* w, const void* bia
       return fail(MSLA_ERR_CUDA, "cuTensorMapEncodeTiled failed for the output projection's output");
   }
   p.residual = (const bf16*)residual;
-  if (f16) return launch<false, false, 0, true>(tmA, tmB, tmO, p, st);
+  if (f16) return residual ? launch<false, false, 2, true>(tmA, tmB, tmO, p, st) : launch<false, false, 0, true>(tmA, tmB, tmO, p, st);
   return residual ? launch<false, false, 2>(tmA, tmB, tmO, p, st) : launch<false>(tmA, tmB, tmO, p, st);
 }
 
@@ -641,7 +640,6 @@ bool project_out_planar_bf16_supported(int Cin, int Cout, int N) { return Cin % 
 // Same product with the attention output kept planar: a[b][j / 64][n][j % 64] (one [N][64] plane per pair of heads).
 msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const void* bias, const void* residual, void* y, int B,
                                           int Cin, int Cout, int N, cudaStream_t st, bool f16) {
-  if (f16 && residual) return fail(MSLA_ERR_UNSUPPORTED, "the fp16 projection has no residual epilogue");
   CUtensorMap tmA, tmB, tmO;
   const int planes = Cin / 64;
   {
@@ -660,7 +658,7 @@ msla_status_t run_project_out_planar_bf16(const void* a, const void* w, const vo
   p.bias = (const bf16*)bias; p.out = (bf16*)y;
   p.tma_store = 1; p.planes_per_batch = planes;
   p.residual = (const bf16*)residual;
-  if (f16) return launch<false, true, 0, true>(tmA, tmB, tmO, p, st);
+  if (f16) return residual ? launch<false, true, 2, true>(tmA, tmB, tmO, p, st) : launch<false, true, 0, true>(tmA, tmB, tmO, p, st);
   return residual ? launch<false, true, 2>(tmA, tmB, tmO, p, st) : launch<false, true>(tmA, tmB, tmO, p, st);
 }
 
@@ -672,7 +670,7 @@ bool ffn_bf16_supported(int C, int Ch, int Cout, int N) {
 // First layer: h[b][o / 32][n][o % 32] = act(sum_c w1[o][c] * x[b][c][n] + b1[o]); x NCHW, h planes of 32 channels
 // (dense 2 KB per 32 tokens for the epilogue's TMA stores: half-line stores into 64-channel planes cost this GEMM 2x).
 msla_status_t run_ffn_expand_bf16(const void* x, const void* w1, const void* b1, void* h, int B, int C, int Ch, int N, int act,
-                                  cudaStream_t st) {
+                                  cudaStream_t st, bool f16) {
   CUtensorMap tmA, tmB, tmO;
   const cuuint64_t dims[3] = {32, (cuuint64_t)N, (cuuint64_t)B * (Ch / 32)};
   const cuuint64_t strides[2] = {64, (cuuint64_t)N * 64};
@@ -690,12 +688,12 @@ msla_status_t run_ffn_expand_bf16(const void* x, const void* w1, const void* b1,
   p.act_a = act == 2 ? 1.f / 6.f : (act == 1 ? 1e30f : 0.f);  // act(v) = v * sat(v * act_a + act_b)
   p.act_b = act == 2 ? 0.5f : (act == 1 ? 0.f : 1.f);
   p.residual = nullptr;
-  return launch<true, false, 1>(tmA, tmB, tmO, p, st);
+  return f16 ? launch<true, false, 1, true>(tmA, tmB, tmO, p, st) : launch<true, false, 1>(tmA, tmB, tmO, p, st);
 }
 
 // Second layer: y[b][m][n] = sum_j w2[m][j] * g[b][j / 64][n][j % 64] + b2[m] (+ residual[b][m][n]); g planes of 64 channels, y NCHW.
 msla_status_t run_ffn_project_bf16(const void* g, const void* w2, const void* b2, const void* residual, void* y, int B, int Ch,
-                                   int Cout, int N, cudaStream_t st) {
+                                   int Cout, int N, cudaStream_t st, bool f16) {
   CUtensorMap tmA, tmB, tmO;
   const int planes = Ch / 64;
   const cuuint64_t dO[3] = {(cuuint64_t)N, (cuuint64_t)Cout, (cuuint64_t)B};
@@ -712,7 +710,7 @@ msla_status_t run_ffn_project_bf16(const void* g, const void* w2, const void* b2
   p.bias = (const bf16*)b2; p.out = (bf16*)y;
   p.tma_store = 1; p.planes_per_batch = planes;
   p.residual = (const bf16*)residual;
-  return launch<false, true, 2>(tmA, tmB, tmO, p, st);
+  return f16 ? launch<false, true, 2, true>(tmA, tmB, tmO, p, st) : launch<false, true, 2>(tmA, tmB, tmO, p, st);
 }
 
 // Self-test of the bounded wait every kernel of the library relies on: one thread waits, with the given cycle

@@ -323,7 +323,7 @@ static msla_status_t run_project_in(msla_dtype_t dt, const void* x, const void* 
 
 static msla_status_t run_project_out(msla_dtype_t dt, const void* a, const void* w, const void* bias,
                                      void* y, int B, int Cin, int Cout, int N, cudaStream_t st, const void* residual = nullptr) {
-  if (dt != MSLA_F32 && project_out_bf16_supported(Cin, Cout, N) && !(dt == MSLA_F16 && residual))
+  if (dt != MSLA_F32 && project_out_bf16_supported(Cin, Cout, N))
     return run_project_out_bf16(a, w, bias, residual, y, B, Cin, Cout, N, st, dt == MSLA_F16);
   generic::GemmArgs g{(long long)N * Cin, Cin, 1, (long long)Cout * N, 1, N, 0, N, Cout, Cin, Cout, 0, residual};
   if (dt == MSLA_F32) launch_gemm<float>((const float*)a, (const float*)w, (const float*)bias, (float*)y, g, B, st);
@@ -468,7 +468,7 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   // take it (dense 128-byte rows for the apply kernel's stores and the GEMM's tile loads),
   // otherwise token-major [N][2C'].
   const bool f16 = desc->dtype == MSLA_F16;
-  const bool att_planar = desc->dtype != MSLA_F32 && !(f16 && residual) && d == 32 && Ht % 2 == 0 && project_out_planar_bf16_supported(S * Cp, desc->C_out, N);
+  const bool att_planar = desc->dtype != MSLA_F32 && d == 32 && Ht % 2 == 0 && project_out_planar_bf16_supported(S * Cp, desc->C_out, N);
   const HeadView ov = att_planar ? HeadView{(long long)N * ld_att, (long long)N * 2 * d, 2 * d, 1}
                                  : HeadView{(long long)N * ld_att, d, ld_att, 0};
   // Steps 4 and 5 run as one kernel when it takes the shape: the head concat then stays in shared memory.
@@ -607,7 +607,7 @@ static msla_status_t band_output_impl(const msla_desc* desc, const msla_weights*
 struct FfnPlan {
   size_t h_off, g_off, bytes;
   int N;
-  bool tuned;  // bf16 tensor-core path with the hidden tensor as planes of 64 channels
+  bool tuned;  // bf16 / fp16 tensor-core path with the hidden tensor as planes of 64 channels
 };
 
 static msla_status_t validate_ffn(const msla_ffn_desc* d, FfnPlan* plan) {
@@ -624,7 +624,7 @@ static msla_status_t validate_ffn(const msla_ffn_desc* d, FfnPlan* plan) {
   if (d->C % 8 != 0 || d->C_hidden % 8 != 0 || d->C_out % 8 != 0) return fail(MSLA_ERR_UNSUPPORTED, "C, C_hidden and C_out must be multiples of 8");
   if (d->B > 65535) return fail(MSLA_ERR_UNSUPPORTED, "B exceeds 65535");
   plan->N = d->H * d->W;
-  plan->tuned = d->dtype == MSLA_BF16 && ffn_bf16_supported(d->C, d->C_hidden, d->C_out, plan->N) &&
+  plan->tuned = d->dtype != MSLA_F32 && ffn_bf16_supported(d->C, d->C_hidden, d->C_out, plan->N) &&
                 (long long)d->B * (d->C_hidden / 64) <= 65535;
   const size_t hid = align_up((size_t)d->B * d->C_hidden * plan->N * elem_size(d->dtype), 256);
   plan->h_off = 0;
@@ -656,9 +656,10 @@ static msla_status_t ffn_impl(const msla_ffn_desc* desc, const void* x, const ms
   void* g = ws + p.g_off;
   const void* res = residual ? x : nullptr;
   if (p.tuned) {
-    if ((s = run_ffn_expand_bf16(x, w->w1, w->b1, h, B, C, Ch, N, act, st)) != MSLA_OK) return s;
-    if ((s = run_ffn_dw3x3_bf16(h, w->w_dw, w->b_dw, g, B, Ch, desc->H, desc->W, act, st)) != MSLA_OK) return s;
-    return run_ffn_project_bf16(g, w->w2, w->b2, res, out, B, Ch, Co, N, st);
+    const bool f16 = desc->dtype == MSLA_F16;
+    if ((s = run_ffn_expand_bf16(x, w->w1, w->b1, h, B, C, Ch, N, act, st, f16)) != MSLA_OK) return s;
+    if ((s = run_ffn_dw3x3_bf16(h, w->w_dw, w->b_dw, g, B, Ch, desc->H, desc->W, act, st, f16)) != MSLA_OK) return s;
+    return run_ffn_project_bf16(g, w->w2, w->b2, res, out, B, Ch, Co, N, st, f16);
   }
   // plain kernels, hidden tensor NCHW
   generic::GemmArgs g1{(long long)C * N, 1, N, (long long)Ch * N, 1, N, 0, N, Ch, C, Ch, act, nullptr};

@@ -106,11 +106,11 @@ msla_status_t run_core_bf16(const void* q, const void* k, const void* v, void* o
 // act: 0 none, 1 ReLU, 2 hard-swish.
 bool ffn_bf16_supported(int C, int Ch, int Cout, int N);
 msla_status_t run_ffn_expand_bf16(const void* x, const void* w1, const void* b1, void* h, int B, int C, int Ch, int N, int act,
-                                  cudaStream_t st);
+                                  cudaStream_t st, bool f16 = false);
 msla_status_t run_ffn_dw3x3_bf16(const void* h, const void* w_dw, const void* b_dw, void* g, int B, int Ch, int H, int W, int act,
-                                 cudaStream_t st);
+                                 cudaStream_t st, bool f16 = false);
 msla_status_t run_ffn_project_bf16(const void* g, const void* w2, const void* b2, const void* residual, void* y, int B, int Ch,
-                                   int Cout, int N, cudaStream_t st);
+                                   int Cout, int N, cudaStream_t st, bool f16 = false);
 
 // Apply step and output projection as one GEMM per image (fused_out.cu): bf16, d in {16, 32}, at most 512 attention
 // channels and 256 output channels.  q: planar query matrices [N][d], head h of image b at q + b*q_sb + h*q_sh

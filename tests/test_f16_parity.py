@@ -1,7 +1,8 @@
 """fp16 storage (the paper's deployment precision, Section 4.1's TensorRT fp16 runs) through the C ABI: every entry
 point with dtype MSLA_F16, element by element against the fp64 oracle on inputs rounded to fp16.  The projections, the
-aggregation and the attention core run on their tensor-core kernels instantiated for f16 (steps 4 and 5 as two kernels);
-shapes those do not take, and the FFN, run on the plain kernels.  fp32 accumulation and state throughout."""
+aggregation, the attention core and the FFN (both linear layers, the depthwise convolution, the residual epilogues)
+run on their tensor-core kernels instantiated for f16 (steps 4 and 5 as two kernels); shapes those do not take run on
+the plain kernels.  fp32 accumulation and state throughout."""
 import numpy as np
 import pytest
 
@@ -61,3 +62,14 @@ def test_ffn_and_block_f16():
 def test_f16_never_takes_the_fused_bf16_kernels():
     desc = binding.make_desc(1, 256, 64, 64, 8, 32, 256, binding.MSLA_F16)
     assert binding.msla_forward_workspace_bytes(desc) > 0 and binding.msla_forward_fuses_apply(desc) == 0
+
+
+# fp16 FFN on the tensor-core kernels (C_hidden a multiple of 64, H*W a multiple of 8): ragged tiles in both
+# directions, every activation, with and without the residual connection.
+@pytest.mark.parametrize("B,C,H,W,Ch,act,residual", [(1, 64, 20, 36, 128, "hardswish", True), (2, 32, 9, 16, 64, "relu", False),
+                                                     (1, 128, 33, 40, 256, "identity", True), (3, 64, 8, 8, 192, "hardswish", False)])
+def test_ffn_f16_tensor_core_shapes(B, C, H, W, Ch, act, residual):
+    fs = inputs.FfnShape("ffn_f16_tc", "f16", B, C, H, W, Ch, C, seed=56)
+    ft = inputs.ffn_inputs(fs)
+    ref = oracle.ffn_dwconv(ft["x"], ft["w1"], ft["w_dw"], ft["w2"], ft["b1"], ft["b_dw"], ft["b2"], act=act, residual=residual)
+    util.assert_close(util.run_ffn(fs, ft, act, residual), ref, "f16", "FFN fp16 (tensor cores)", block=util.MODULE_BLOCK)
