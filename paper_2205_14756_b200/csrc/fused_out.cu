@@ -139,6 +139,26 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
                ::"r"(bar), "h"((unsigned short)3) : "memory");
 }
 
+// F16 kernels: the 16-bit storage type is IEEE binary16 instead of bfloat16.  The values travel untyped; the conversions,
+// the packed maximum and the MMA's operand format differ.
+template <bool F16> __device__ __forceinline__ float lo16(uint32_t w) {
+  if constexpr (F16) return __low2float(*reinterpret_cast<const __half2*>(&w));
+  else return __uint_as_float(w << 16);
+}
+template <bool F16> __device__ __forceinline__ float hi16(uint32_t w) {
+  if constexpr (F16) return __high2float(*reinterpret_cast<const __half2*>(&w));
+  else return __uint_as_float(w & 0xffff0000u);
+}
+template <bool F16> __device__ __forceinline__ uint32_t pack16(float lo, float hi) {
+  if constexpr (F16) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+  } else {
+    return pack2(lo, hi);
+  }
+}
+
 // ---------------------------------------------------------------------------
 // Second level of the state reduction (Eq. 3) and the fold of the state into the projection weights.
 // Grid (B * Ht, chunks): a CTA takes one head and `da` = d / chunks of its key channels a, i.e. `da` consecutive rows of the
@@ -153,9 +173,12 @@ constexpr int FOLD_THREADS = 1024;
 constexpr int FOLD_RUNS = 8;       // S <= 64: at most 8 partial states per run
 constexpr int FOLD_RUN_BYTES = FOLD_RUNS * 32 * 33 * 4, FOLD_ST_BYTES = 32 * 33 * 4;
 constexpr int FOLD_SMEM = FOLD_RUN_BYTES + FOLD_ST_BYTES + 256 * 32 * 2;  // + the head's [Cout <= 256][d <= 32] weight columns
+// F16: M and ks are multiplied by `scale`, a power of two near 1 / N (the output kernel scales eps alike, so Eq. 3's quotient is
+// unchanged): sums over N tokens then stay inside binary16's range.
+template <bool F16>
 __global__ void __launch_bounds__(FOLD_THREADS)
 state_fold_kernel(const float* __restrict__ partial, int S, const bf16* __restrict__ w, bf16* __restrict__ M, float* __restrict__ ks,
-                  int Ht, int d, int Cout, int K, int da) {
+                  int Ht, int d, int Cout, int K, int da, float scale) {
   extern __shared__ __align__(16) unsigned char fold_smem[];
   float4 (*run_sum)[32 * 33 / 4] = reinterpret_cast<float4 (*)[32 * 33 / 4]>(fold_smem);
   float* st = reinterpret_cast<float*>(fold_smem + FOLD_RUN_BYTES);
@@ -192,7 +215,7 @@ state_fold_kernel(const float* __restrict__ partial, int S, const bf16* __restri
     reinterpret_cast<float4*>(st)[e] = v;  // st[al * d1 + c], al = a - a0
   }
   __syncthreads();
-  for (int al = threadIdx.x; al < da; al += FOLD_THREADS) ks[(long long)bh * d + a0 + al] = st[al * d1 + d];
+  for (int al = threadIdx.x; al < da; al += FOLD_THREADS) ks[(long long)bh * d + a0 + al] = F16 ? st[al * d1 + d] * scale : st[al * d1 + d];
   // M: a thread keeps key channel al = threadIdx.x % da (FOLD_THREADS is a multiple of da), i.e. one row of the state,
   // in registers and walks the output channels m = threadIdx.x / da, + FOLD_THREADS / da, ...
   const int al = threadIdx.x % da;
@@ -210,15 +233,17 @@ state_fold_kernel(const float* __restrict__ partial, int S, const bf16* __restri
       const uint32_t word[4] = {wv[c8].x, wv[c8].y, wv[c8].z, wv[c8].w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {  // channels beyond d carry zeros on both sides
-        acc = fmaf(__uint_as_float(word[e] << 16), srow[8 * c8 + 2 * e], acc);
-        acc = fmaf(__uint_as_float(word[e] & 0xffff0000u), srow[8 * c8 + 2 * e + 1], acc);
+        acc = fmaf(lo16<F16>(word[e]), srow[8 * c8 + 2 * e], acc);
+        acc = fmaf(hi16<F16>(word[e]), srow[8 * c8 + 2 * e + 1], acc);
       }
     }
-    M[((long long)b * Cout + m) * K + hh * d + a0 + al] = __float2bfloat16_rn(acc);
+    bf16* mp = M + ((long long)b * Cout + m) * K + hh * d + a0 + al;
+    if constexpr (F16) *reinterpret_cast<__half*>(mp) = __float2half_rn(acc * scale);
+    else *mp = __float2bfloat16_rn(acc);
   }
 }
 
-template <int D, bool RES>
+template <int D, bool RES, bool F16>
 __global__ void __launch_bounds__(O_THREADS, 1)
 fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmQ,
                  const __grid_constant__ CUtensorMap tmO, const __grid_constant__ CUtensorMap tmR, OutParams p) {
@@ -319,7 +344,7 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     // ------------------------------------------------------------ MMA issuer (leader) / M hand-shake (peer)
     if (lane == 0) {
       // instruction descriptor: D = f32, A = B = bf16, both K-major, N = 256, M = 256 (pair)
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * p.ot) >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+      const uint32_t idesc = (1u << 4) | (F16 ? 0u : ((1u << 7) | (1u << 10))) | ((uint32_t)((2 * p.ot) >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
       const uint32_t peer_res_remote = map_to_cta(peer_res_bar, 0);
       uint32_t local = 0, res_ph = 0, s = 0, ph = 0;  // s, ph: ring slot and the parity of its current use
       // Matrix descriptors: the high words are constants; the low words carry the start address in 16-byte units
@@ -419,13 +444,14 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
         float den[4] = {0.f, 0.f, 0.f, 0.f};  // four chains
 #pragma unroll
         for (int w = 0; w < D / 2; ++w) {
-          asm("max.bf16x2 %0, %1, %2;" : "=r"(q[w]) : "r"(q[w]), "r"(0u));
-          den[2 * (w & 1)] = fmaf(__uint_as_float(q[w] << 16), kk[2 * w], den[2 * (w & 1)]);
-          den[2 * (w & 1) + 1] = fmaf(__uint_as_float(q[w] & 0xffff0000u), kk[2 * w + 1], den[2 * (w & 1) + 1]);
+          if constexpr (F16) asm("max.f16x2 %0, %1, %2;" : "=r"(q[w]) : "r"(q[w]), "r"(0u));
+          else asm("max.bf16x2 %0, %1, %2;" : "=r"(q[w]) : "r"(q[w]), "r"(0u));
+          den[2 * (w & 1)] = fmaf(lo16<F16>(q[w]), kk[2 * w], den[2 * (w & 1)]);
+          den[2 * (w & 1) + 1] = fmaf(hi16<F16>(q[w]), kk[2 * w + 1], den[2 * (w & 1) + 1]);
         }
         const float inv = __frcp_rn((den[0] + den[1]) + (den[2] + den[3]) + p.eps);
 #pragma unroll
-        for (int w = 0; w < D / 2; ++w) q[w] = pack2(__uint_as_float(q[w] << 16) * inv, __uint_as_float(q[w] & 0xffff0000u) * inv);
+        for (int w = 0; w < D / 2; ++w) q[w] = pack16<F16>(lo16<F16>(q[w]) * inv, hi16<F16>(q[w]) * inv);
 #pragma unroll
         for (int c = 0; c < PCS; ++c)
           asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(rbase + (((uint32_t)c ^ swz) << 4)), "r"(q[4 * c]), "r"(q[4 * c + 1]),
@@ -443,7 +469,7 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
     const uint32_t stage = staging + (uint32_t)(warp - 2 - O_XWARPS) * O_STAGING_WARP;
     const uint32_t my_row = stage + lane * 128, sw = (uint32_t)(lane & 7);
     const int row0 = (int)rank * OM + quarter * 32;
-    const float bias = (p.bias && row0 + lane < p.Cout) ? __bfloat162float(p.bias[row0 + lane]) : 0.f;
+    const float bias = !(p.bias && row0 + lane < p.Cout) ? 0.f : F16 ? __half2float(reinterpret_cast<const __half*>(p.bias)[row0 + lane]) : __bfloat162float(p.bias[row0 + lane]);
     const uint32_t tempty_remote = map_to_cta(tempty_bar, 0);
     // RES: the residual arrives by TMA, one 32-channel x 64-token block per warp and request, a block ahead of its use
     const uint32_t my_resid_bar = resid_bar + 8 * (uint32_t)(warp - 2 - O_XWARPS);
@@ -495,8 +521,8 @@ fused_out_kernel(const __grid_constant__ CUtensorMap tmM, const __grid_constant_
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             float f0 = __uint_as_float(rc[v * 8 + 2 * e]) + bias, f1 = __uint_as_float(rc[v * 8 + 2 * e + 1]) + bias;
-            if (RES) { f0 += __uint_as_float(rw[e] << 16); f1 += __uint_as_float(rw[e] & 0xffff0000u); }
-            w[e] = pack2(f0, f1);
+            if (RES) { f0 += lo16<F16>(rw[e]); f1 += hi16<F16>(rw[e]); }
+            w[e] = pack16<F16>(f0, f1);
           }
           asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(my_row + ((pc ^ sw) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]),
                        "r"(w[3]) : "memory");
@@ -552,9 +578,29 @@ size_t fused_out_scratch_bytes(int B, int Ht, int d, int Cout) { return fused_ou
 // state of (b, h) = sum over s < S of partial[(b * Ht + h) * S + s] ([d][d+1] fp32 each: KV, then the key sum in
 // column d).  q: planar bf16 query matrices [N][d], head h of image b at q + b*q_sb + h*q_sh (elements); y: NCHW
 // [B, Cout, N].
+namespace {
+template <int D, bool RES, bool F16>
+msla_status_t launch_fused(dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tmM, const CUtensorMap& tmQ, const CUtensorMap& tmO,
+                           const CUtensorMap& tmR, const OutParams& p) {
+  static std::atomic<unsigned long long> attr_done{0};
+  const msla_status_t s = ensure_smem_attr(attr_done, fused_out_kernel<D, RES, F16>, O_SMEM_LIMIT);
+  if (s != MSLA_OK) return s;
+  launch_pdl_cluster2(fused_out_kernel<D, RES, F16>, grid, dim3(O_THREADS), (size_t)smem, st, tmM, tmQ, tmO, tmR, p);
+  return MSLA_OK;
+}
+template <bool F16>
+msla_status_t launch_fused_for(int d, bool res, dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tmM, const CUtensorMap& tmQ,
+                               const CUtensorMap& tmO, const CUtensorMap& tmR, const OutParams& p) {
+  if (d == 32) return res ? launch_fused<32, true, F16>(grid, smem, st, tmM, tmQ, tmO, tmR, p) : launch_fused<32, false, F16>(grid, smem, st, tmM, tmQ, tmO, tmR, p);
+  return res ? launch_fused<16, true, F16>(grid, smem, st, tmM, tmQ, tmO, tmR, p) : launch_fused<16, false, F16>(grid, smem, st, tmM, tmQ, tmO, tmR, p);
+}
+}  // namespace
+
+// f16: queries, weights, bias, residual and output are IEEE binary16 instead of bfloat16; M, the key sums and eps are
+// scaled by the power of two just above 1 / N (N tokens' sums would leave binary16's range otherwise).
 msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, const float* partial, int S, void* scratch,
                                  const void* w, const void* bias, const void* residual, void* y, int B, int Ht, int d, int N, int Cout,
-                                 float eps, cudaStream_t st) {
+                                 float eps, cudaStream_t st, bool f16) {
   if (!fused_out_bf16_supported(Ht, d, Cout, N) || q_sb % 8 != 0 || q_sh % 8 != 0)
     return fail(MSLA_ERR_UNSUPPORTED, "fused apply + projection: %d heads of %d channels, %d output channels, %d tokens", Ht, d, Cout, N);
   if (S < 1 || S > 8 * FOLD_RUNS) return fail(MSLA_ERR_UNSUPPORTED, "fused apply + projection: %d partial states per head (1 .. %d)", S, 8 * FOLD_RUNS);
@@ -584,7 +630,10 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   }
   OutParams p{};
   p.ks = ks; p.bias = (const bf16*)bias; p.residual = (const bf16*)residual;
-  p.B = B; p.N = N; p.Cout = Cout; p.Ht = Ht; p.d = d; p.eps = eps;
+  float scale = 1.f;
+  if (f16)
+    for (long long n = 1; n < N; n <<= 1) scale *= 0.5f;
+  p.B = B; p.N = N; p.Cout = Cout; p.Ht = Ht; p.d = d; p.eps = eps * scale;
   p.kslices = (K + OKS - 1) / OKS;
   p.ot = ot;
   p.tiles_per_image = (N + 2 * ot - 1) / (2 * ot);
@@ -597,28 +646,22 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   if (p.stages > O_MAX_STAGES) p.stages = O_MAX_STAGES;
   if (p.stages < O_MIN_STAGES) return fail(MSLA_ERR_UNSUPPORTED, "fused apply + projection: no room for the query ring (%d slots)", p.stages);
   const int smem = smem_fixed + p.stages * slot;
-  static std::atomic<unsigned long long> attr_done{0}, attr_done16{0}, attr_res{0}, attr_res16{0};
-  constexpr int smem_max = O_SMEM_LIMIT;
-  msla_status_t s = ensure_smem_attr(attr_done, fused_out_kernel<32, false>, smem_max);
-  if (s == MSLA_OK) s = ensure_smem_attr(attr_done16, fused_out_kernel<16, false>, smem_max);
-  if (s == MSLA_OK && residual) s = ensure_smem_attr(attr_res, fused_out_kernel<32, true>, smem_max);
-  if (s == MSLA_OK && residual) s = ensure_smem_attr(attr_res16, fused_out_kernel<16, true>, smem_max);
-  if (s != MSLA_OK) return s;
   long long pairs = sms / 2;
   if (pairs > tiles) pairs = tiles;
   if (pairs < 1) pairs = 1;
   // about one CTA per SM: few heads -> up to four CTAs per head, each with a share of the head's key channels
   int fold_chunks = sms / (B * Ht);
   fold_chunks = fold_chunks >= 4 ? 4 : (fold_chunks >= 2 ? 2 : 1);
-  static std::atomic<unsigned long long> attr_fold{0};
-  if ((s = ensure_smem_attr(attr_fold, state_fold_kernel, FOLD_SMEM)) != MSLA_OK) return s;
-  launch_pdl(state_fold_kernel, dim3((unsigned)(B * Ht), (unsigned)fold_chunks), dim3(FOLD_THREADS), FOLD_SMEM, st, partial, S,
-             (const bf16*)w, M, ks, Ht, d, Cout, K, d / fold_chunks);
-  const dim3 grid((unsigned)(2 * pairs)), block(O_THREADS);
-  if (d == 32 && !residual) launch_pdl_cluster2(fused_out_kernel<32, false>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, tmR, p);
-  else if (d == 32) launch_pdl_cluster2(fused_out_kernel<32, true>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, tmR, p);
-  else if (!residual) launch_pdl_cluster2(fused_out_kernel<16, false>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, tmR, p);
-  else launch_pdl_cluster2(fused_out_kernel<16, true>, grid, block, (size_t)smem, st, tmM, tmQ, tmO, tmR, p);
+  static std::atomic<unsigned long long> attr_fold{0}, attr_fold16{0};
+  msla_status_t s = f16 ? ensure_smem_attr(attr_fold16, state_fold_kernel<true>, FOLD_SMEM) : ensure_smem_attr(attr_fold, state_fold_kernel<false>, FOLD_SMEM);
+  if (s != MSLA_OK) return s;
+  const dim3 fold_grid((unsigned)(B * Ht), (unsigned)fold_chunks);
+  if (f16) launch_pdl(state_fold_kernel<true>, fold_grid, dim3(FOLD_THREADS), FOLD_SMEM, st, partial, S, (const bf16*)w, M, ks, Ht, d, Cout, K, d / fold_chunks, scale);
+  else launch_pdl(state_fold_kernel<false>, fold_grid, dim3(FOLD_THREADS), FOLD_SMEM, st, partial, S, (const bf16*)w, M, ks, Ht, d, Cout, K, d / fold_chunks, scale);
+  const dim3 grid((unsigned)(2 * pairs));
+  s = f16 ? launch_fused_for<true>(d, residual != nullptr, grid, smem, st, tmM, tmQ, tmO, tmR, p)
+          : launch_fused_for<false>(d, residual != nullptr, grid, smem, st, tmM, tmQ, tmO, tmR, p);
+  if (s != MSLA_OK) return s;
   count_launches(2);
   return check_launch("fused apply + output projection (tcgen05, paired CTAs)");
 }

@@ -472,7 +472,7 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   const HeadView ov = att_planar ? HeadView{(long long)N * ld_att, (long long)N * 2 * d, 2 * d, 1}
                                  : HeadView{(long long)N * ld_att, d, ld_att, 0};
   // Steps 4 and 5 run as one kernel when it takes the shape: the head concat then stays in shared memory.
-  const bool fused = desc->dtype == MSLA_BF16 && fused_out_bf16_supported(Ht, d, desc->C_out, N);
+  const bool fused = desc->dtype != MSLA_F32 && fused_out_bf16_supported(Ht, d, desc->C_out, N);
   s = run_core(desc->dtype, ms, ms + (size_t)N * d * e, ms + (size_t)2 * N * d * e, att, in, ov, desc->B, Ht, N, d, desc->eps, p.core,
                ws + p.core_off, st, events ? (cudaEvent_t)events[3] : nullptr, fused ? CORE_STATE : CORE_ALL);
   if (s != MSLA_OK) return s;
@@ -480,7 +480,7 @@ static msla_status_t forward_impl(const msla_desc* desc, const void* x, const ms
   // 5. output projection back to NCHW
   if (fused)
     s = run_fused_out_bf16(ms, ms_sb, 3LL * N * d, reinterpret_cast<const float*>(ws + p.core_off + p.core.partial_off), p.core.S, att, w->w_proj,
-                           w->b_proj, residual, out_dev, desc->B, Ht, d, N, desc->C_out, desc->eps, st);
+                           w->b_proj, residual, out_dev, desc->B, Ht, d, N, desc->C_out, desc->eps, st, f16);
   else
     s = att_planar ? run_project_out_planar_bf16(att, w->w_proj, w->b_proj, residual, out_dev, desc->B, S * Cp, desc->C_out, N, st, f16)
                    : run_project_out(desc->dtype, att, w->w_proj, w->b_proj, out_dev, desc->B, S * Cp, desc->C_out, N, st, residual);
@@ -590,8 +590,9 @@ static msla_status_t band_output_impl(const msla_desc* desc, const msla_weights*
   count_launches(1);
   if ((s = check_launch("sum of the bands' states")) != MSLA_OK) return s;
   const char* q = ms + (size_t)b.tok_off * d * e;
-  if (desc->dtype == MSLA_BF16 && fused_out_bf16_supported(Ht, d, desc->C_out, Nb))
-    return run_fused_out_bf16(q, ms_sb, 3LL * N * d, state, 1, att, w->w_proj, w->b_proj, nullptr, out, desc->B, Ht, d, Nb, desc->C_out, desc->eps, st);
+  if (desc->dtype != MSLA_F32 && fused_out_bf16_supported(Ht, d, desc->C_out, Nb))
+    return run_fused_out_bf16(q, ms_sb, 3LL * N * d, state, 1, att, w->w_proj, w->b_proj, nullptr, out, desc->B, Ht, d, Nb, desc->C_out, desc->eps, st,
+                              desc->dtype == MSLA_F16);
   const HeadView in{ms_sb, 3LL * N * d, d};
   const bool att_planar = desc->dtype != MSLA_F32 && d == 32 && Ht % 2 == 0 && project_out_planar_bf16_supported(p.S * Cp, desc->C_out, Nb);
   const HeadView ov = att_planar ? HeadView{(long long)Nb * ld_att, (long long)Nb * 2 * d, 2 * d, 1}

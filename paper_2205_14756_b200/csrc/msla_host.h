@@ -119,7 +119,7 @@ bool fused_out_bf16_supported(int Ht, int d, int Cout, int N);
 size_t fused_out_scratch_bytes(int B, int Ht, int d, int Cout);
 msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, const float* partial, int S, void* scratch,
                                  const void* w, const void* bias, const void* residual, void* y, int B, int Ht, int d, int N, int Cout,
-                                 float eps, cudaStream_t st);
+                                 float eps, cudaStream_t st, bool f16 = false);
 int fused_timeout_flag();
 int dw_timeout_flag();
 

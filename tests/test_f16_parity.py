@@ -1,8 +1,8 @@
 """fp16 storage (the paper's deployment precision, Section 4.1's TensorRT fp16 runs) through the C ABI: every entry
 point with dtype MSLA_F16, element by element against the fp64 oracle on inputs rounded to fp16.  The projections, the
-aggregation, the attention core and the FFN (both linear layers, the depthwise convolution, the residual epilogues)
-run on their tensor-core kernels instantiated for f16 (steps 4 and 5 as two kernels); shapes those do not take run on
-the plain kernels.  fp32 accumulation and state throughout."""
+aggregation, the attention core, the fused apply + output projection and the FFN (both linear layers, the depthwise
+convolution, the residual epilogues) run on their tensor-core kernels instantiated for f16; shapes those do not take
+run on the plain kernels.  fp32 accumulation and state throughout."""
 import numpy as np
 import pytest
 
@@ -38,13 +38,15 @@ def test_module_f16(B, C, H, W, heads, d, n_scales, k1):
     util.assert_close(util.run_module(s, t), ref, "f16", "module fp16", block=util.MODULE_BLOCK)
 
 
-def test_many_tokens_do_not_overflow_f16():
-    """The state sums over all tokens (here 16 384 per head: entries of the order of 10^4) and stays in fp32; only
-    the quotient of Eq. 3, which is of the order of the values, is stored in 16 bits."""
-    s = inputs.ModuleShape("module_f16_128x128", "f16", 1, 32, 128, 128, 1, 32, seed=53)
+@pytest.mark.parametrize("side", [128, 512])
+def test_many_tokens_do_not_overflow_f16(side):
+    """The state sums over all tokens (16 384 and, at the benchmark's resolution, 262 144 per head: entries of the
+    order of 10^4 and 10^5) and stays in fp32; what is stored in 16 bits is scaled by a power of two near 1 / N (the
+    state folded into the projection weights, the key sums and eps alike), which leaves Eq. 3's quotient unchanged."""
+    s = inputs.ModuleShape(f"module_f16_{side}x{side}", "f16", 1, 32, side, side, 1, 32, seed=53)
     t = inputs.module_inputs(s)
     ref = oracle.msla_forward(t["x"], t["w_qkv"], t["w_dw"], t["w_pw"], t["w_proj"], heads=1, d=32)
-    util.assert_close(util.run_module(s, t), ref, "f16", "fp16, 16384 tokens", block=util.MODULE_BLOCK)
+    util.assert_close(util.run_module(s, t), ref, "f16", f"fp16, {side * side} tokens", block=util.MODULE_BLOCK)
 
 
 def test_ffn_and_block_f16():
