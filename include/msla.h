@@ -44,8 +44,9 @@ typedef enum {
 } msla_status_t;
 
 /* Storage type of activations and weights.  Arithmetic and the attention state are fp32 for all three.  MSLA_F16
- * (the paper's deployment precision, Section 4.1): projections, aggregation and attention core run on tensor cores as
- * for bf16 (steps 4 and 5 as two kernels); the FFN runs on the library's plain kernels.  MSLA_F16 is accepted wherever a dtype is taken (msla_linattn_relu_ws and _noalloc, msla_forward*, the band
+ * (the paper's deployment precision, Section 4.1): every tensor-core kernel of the bf16 path (projections, aggregation,
+ * attention core, fused apply + output projection, FFN) is instantiated for it; what is stored in 16 bits of the state
+ * is scaled by a power of two near 1 / N, which leaves Eq. 3's quotient unchanged.  MSLA_F16 is accepted wherever a dtype is taken (msla_linattn_relu_ws and _noalloc, msla_forward*, the band
  * pair, the stage entry points, msla_ffn_dwconv, msla_evit_block). */
 typedef enum { MSLA_F32 = 0, MSLA_BF16 = 1, MSLA_F16 = 2 } msla_dtype_t;
 
