@@ -588,8 +588,7 @@ def main() -> None:
         other["cfg4"] = time_module(inputs.CONFIG4)
         # a bf16, d = 16 sibling of config 1's width at 256 x 256 tokens, 384 channels
         other["d16_256x256_c384"] = time_module(inputs.ModuleShape("bf16_d16_256x256_c384", "bf16", 1, 384, 256, 256, 24, 16, seed=7))
-        # fp16 storage at the bench workload's shape: projections, aggregation and attention core on their f16
-        # tensor-core instantiations, steps 4 and 5 as two kernels
+        # fp16 storage at the bench workload's shape: the same tensor-core kernels instantiated for binary16
         other["cfg5_512x512_f16"] = time_module(inputs.ModuleShape(s.name.replace("bf16", "f16"), "f16", s.B, s.C, s.H, s.W, s.heads, s.d, seed=s.seed))
         # the token-sharded path's two band calls on one rank (no halo, one state): what the split itself costs
         band1 = time_token_sharded(s, 0, 1, steps=10, warmup=3, blocks=5)
