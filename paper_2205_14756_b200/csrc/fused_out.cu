@@ -51,7 +51,6 @@ constexpr int OM = 128;                  // output channels per CTA (256 per pai
 constexpr int OKS = 64;                  // k-extent of one resident slice of M (one 128-byte swizzle span)
 constexpr int O_A_SLICE = OM * OKS * 2;  // 16 KB: 128 rows of M x 64 k
 constexpr int O_MAX_KS = 8;              // K = 2C' <= 512
-constexpr int O_SLICE_MAX = OT * 32 * 2; // 8 KB: 128 tokens x 32 channels (d = 16: half of it is used)
 constexpr int O_MIN_STAGES = 2, O_MAX_STAGES = 16;  // query ring: as many slots (of two slices each) as shared memory holds (the host decides)
 constexpr int O_XWARPS = 12;             // transform warps: three groups of four, each taking every third slice
 constexpr int O_THREADS = 32 * (2 + O_XWARPS + 4);
