@@ -648,9 +648,10 @@ msla_status_t run_fused_out_bf16(const void* q, long long q_sb, long long q_sh, 
   long long pairs = sms / 2;
   if (pairs > tiles) pairs = tiles;
   if (pairs < 1) pairs = 1;
-  // about one CTA per SM: few heads -> up to four CTAs per head, each with a share of the head's key channels
+  // about one CTA per SM: few heads -> up to eight CTAs per head, each with a share of the head's key channels
+  // (a share's rows of the state, da * (d + 1) floats, must stay a whole number of 16-byte vectors: da >= 4)
   int fold_chunks = sms / (B * Ht);
-  fold_chunks = fold_chunks >= 4 ? 4 : (fold_chunks >= 2 ? 2 : 1);
+  fold_chunks = (fold_chunks >= 8 && d == 32) ? 8 : fold_chunks >= 4 ? 4 : (fold_chunks >= 2 ? 2 : 1);
   static std::atomic<unsigned long long> attr_fold{0}, attr_fold16{0};
   msla_status_t s = f16 ? ensure_smem_attr(attr_fold16, state_fold_kernel<true>, FOLD_SMEM) : ensure_smem_attr(attr_fold, state_fold_kernel<false>, FOLD_SMEM);
   if (s != MSLA_OK) return s;
